@@ -1,0 +1,18 @@
+"""B200-native kernel-halving compression + weighted attention (arXiv 2606.10944 hot path).
+
+``compress`` / ``attend`` and friends are thin argument-marshalling wrappers over the C-ABI
+CUDA library in ``csrc/``; they are loaded on first use so that the input generators in
+``workloads`` stay importable on machines without the built library.
+"""
+_BINDING_NAMES = {
+    "compress", "attend", "compress_attend_host", "workspace_bytes", "default_delta_levels",
+    "ElmParams", "ElmError", "library_path", "load_library", "make_params", "profile_enable",
+    "profile_read", "version", "EXPORTED_SYMBOLS", "STAGE_NAMES",
+}
+
+
+def __getattr__(name):
+    if name in _BINDING_NAMES:
+        from . import binding
+        return getattr(binding, name)
+    raise AttributeError(name)
