@@ -1,0 +1,353 @@
+#!/usr/bin/env python
+"""Benchmark: compress + attend tokens/s on one B200 (or N independent replicas).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg5] [--impl reference]
+
+A step is one pass of the whole hot path (elm_compress then elm_attend) over one batch of
+seeded synthetic input already resident in HBM.  Rank 0 prints one JSON line.  The path has no
+exchange step, so N > 1 runs N independent replicas ("replicas only") and adds their tokens.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "compress+attend tokens/sec per B200"
+UNIT = "tokens/s"
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            pk = json.load(f)
+        return {"hbm_gbs": pk["hbm_gbs"], "bf16_tflops": pk["bf16_tflops"],
+                "bf16_tflops_sustained": pk.get("bf16_tflops_sustained", pk["bf16_tflops"]),
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.rows = []
+        self._stop = threading.Event()
+        self._thr = None
+
+    def _run(self):
+        while not self._stop.is_set():
+            try:
+                out = subprocess.run(["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.FIELDS}",
+                                      "--format=csv,noheader,nounits"], capture_output=True, text=True,
+                                     timeout=5).stdout.strip()
+                if out:
+                    self.rows.append([c.strip() for c in out.splitlines()[0].split(",")])
+            except Exception:
+                pass
+            self._stop.wait(0.1)
+
+    def __enter__(self):
+        self._thr = threading.Thread(target=self._run, daemon=True)
+        self._thr.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        self._thr.join(timeout=10)
+
+    def summary(self):
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except (ValueError, IndexError):
+                continue
+            for name, val in zip(names, r[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": max(mx), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def algorithmic_counts(wl):
+    """Flops and bytes the method itself needs per step (not what exact attention would need)."""
+    es = 2 if wl.dtype == "bf16" else 4
+    attend_flops = wl.batch * wl.q_heads * wl.n_q * wl.n_out * 4 * wl.d
+    compress_flops = wl.batch * wl.kv_heads * wl.m * 8 * wl.d * wl.n_out ** 2
+    hbm_bytes = 2 * wl.batch * wl.q_heads * wl.n_q * wl.d * es + 2 * wl.batch * wl.kv_heads * wl.n * wl.d * es
+    return attend_flops, compress_flops, hbm_bytes
+
+
+def cpu_baseline(wl, Q, K, V, budget_heads=None):
+    """The oracle as it stands, timed on this machine's cores on a bounded sample of the workload."""
+    import numpy as np
+    import oracle
+    from paper_2606_10944_b200.workloads import as_f32_numpy
+    cores = oracle.num_threads()
+    problems = wl.batch * wl.kv_heads
+    # compression cost per problem ~ 3 m n_out^2 kernel evaluations of 2d MACs; aim for <= ~20 s
+    per_problem_s = 3.0 * wl.m * wl.n_out ** 2 * 2 * wl.d / 0.6e9
+    waves = max(1, int(20.0 / max(per_problem_s, 1e-3)))
+    heads = budget_heads or max(1, min(problems, cores * waves))
+    Kf = as_f32_numpy(K).reshape(problems, wl.n, wl.d)[:heads]
+    Vf = as_f32_numpy(V).reshape(problems, wl.n, wl.d)[:heads]
+    t0 = time.perf_counter()
+    idx, w, _ = oracle.compress2_batched(Kf, Vf, wl.log2_nout, wl.m, seed=1)
+    t_c = time.perf_counter() - t0
+    # attention: a fixed number of query rows of every query head (~0.5 us per coreset point)
+    per_query_s = wl.n_out * 2 * wl.d / 0.6e9
+    nq_s = int(max(8, min(wl.n_q, 8.0 * cores / (per_query_s * wl.batch * wl.q_heads))))
+    Qf = as_f32_numpy(Q[:, :, :nq_s])
+    Kall = as_f32_numpy(K)
+    Vall = as_f32_numpy(V)
+    # every query head needs a coreset for its KV head: reuse the sampled ones cyclically
+    full_idx = np.stack([idx[i % heads] for i in range(problems)]).reshape(wl.batch, wl.kv_heads, -1)
+    full_w = np.stack([w[i % heads] for i in range(problems)]).reshape(wl.batch, wl.kv_heads, -1)
+    t0 = time.perf_counter()
+    oracle.wtd_attention_batched(Qf, Kall, Vall, full_idx, full_w)
+    t_a = time.perf_counter() - t0
+    est = t_c * problems / heads + t_a * wl.n_q / nq_s
+    return {"value": wl.batch * wl.n / est, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"compress of {heads}/{problems} KV problems at full n={wl.n} ({t_c:.2f} s) + attend of "
+                      f"{nq_s}/{wl.n_q} query rows of all {wl.batch * wl.q_heads} query heads ({t_a:.2f} s), "
+                      f"scaled linearly to the full step ({est:.1f} s)"}, est
+
+
+def run_reference(args, wl):
+    """--impl reference: the CPU oracle timed on the host cores (rank 0 only)."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    from paper_2606_10944_b200.workloads import generate
+    Q, K, V = generate(wl, seed=args.data_seed)
+    times = []
+    base = None
+    for i in range(args.warmup + args.steps):
+        base, est = cpu_baseline(wl, Q, K, V, budget_heads=args.ref_heads)
+        if i >= args.warmup:
+            times.append(est)
+        if sum(times) > 0 and (time.perf_counter() - T_START) > 240:
+            break
+    est = sum(times) / len(times)
+    value = wl.batch * wl.n / est
+    base["value"] = value
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": len(times), "warmup": args.warmup, "ms_per_step": est * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(wl, args), "cpu_baseline": base,
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def workload_config(wl, args):
+    return {"workload": wl.name, "batch": wl.batch, "q_heads": wl.q_heads, "kv_heads": wl.kv_heads,
+            "seq_len": wl.n, "head_dim": wl.d, "n_out": wl.n_out, "compress2_depth": wl.m, "g": wl.g,
+            "storage": wl.dtype, "precision": args.precision, "recipe": wl.recipe,
+            "parallelism": "replicas only", "l2": "inputs (>= 2.6 GB per step) exceed the 126 MB L2"
+            if wl.name in ("cfg5", "cfg4") else "L2 flushed by a 256 MB write between steps"}
+
+
+T_START = time.perf_counter()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg5")
+    ap.add_argument("--precision", default="fp32", choices=["fp32", "fp64"])
+    ap.add_argument("--data-seed", type=int, default=1234)
+    ap.add_argument("--seed", type=int, default=1)
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--ref-heads", type=int, default=None)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+
+    from paper_2606_10944_b200.workloads import WORKLOADS, generate
+    wl = WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, wl)
+        return
+
+    import torch
+    import paper_2606_10944_b200 as elm
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU fallback")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    elm.load_library()
+    warmup = max(args.warmup, 3)
+
+    Q, K, V = generate(wl, seed=args.data_seed + rank)      # each replica has its own batch
+    Qd, Kd, Vd = Q.cuda(), K.cuda(), V.cuda()
+    dev = Qd.device
+    p, _ = elm.make_params(wl.batch, wl.q_heads, wl.kv_heads, wl.n, wl.n_q, wl.d, wl.log2_nout, wl.m,
+                           1 if wl.dtype == "bf16" else 0, args.precision)
+    cb, ab = elm.workspace_bytes(p)
+    ws_c = torch.empty(cb, dtype=torch.uint8, device=dev)
+    ws_a = torch.empty(ab, dtype=torch.uint8, device=dev)
+    O = torch.empty_like(Qd)
+    small_inputs = wl.name not in ("cfg4", "cfg5")
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev) if small_inputs else None
+
+    def step(seed):
+        if flush is not None:
+            flush.zero_()
+        idx, w = elm.compress(Kd, Vd, wl.log2_nout, wl.m, seed=seed, precision=args.precision, workspace=ws_c)
+        elm.attend(Qd, Kd, Vd, idx, w, precision=args.precision, workspace=ws_a, out=O)
+        return idx, w
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(warmup):
+        step(args.seed + i)
+    barrier()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    flush_ms = 0.0
+    if flush is not None:           # cost of the flush itself, subtracted below
+        f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        f0.record()
+        for _ in range(args.steps):
+            flush.zero_()
+        f1.record()
+        torch.cuda.synchronize()
+        flush_ms = f0.elapsed_time(f1)
+    launches0 = elm.launch_count()
+    elm.profile_enable(True)
+    with ClockSampler(local) as clocks:
+        barrier()
+        ev0.record()
+        for i in range(args.steps):
+            step(args.seed + i)
+        ev1.record()
+        barrier()
+    stage = elm.profile_read()
+    elm.profile_enable(False)
+    launches = elm.launch_count() - launches0
+    ms_total = ev0.elapsed_time(ev1) - flush_ms
+    t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_total = float(t.item())
+    ms_step = ms_total / args.steps
+    tokens_per_step = wl.batch * wl.n * world
+    value = tokens_per_step / (ms_step * 1e-3)
+
+    # end to end through the host-buffer entry point (pinned inputs, copies inside the timed region)
+    e2e = None
+    if not args.no_e2e:
+        Qp, Kp, Vp = Q.pin_memory(), K.pin_memory(), V.pin_memory()
+        Oh = torch.empty_like(Q).pin_memory()
+        scratch = torch.empty(elm.host_call_scratch_bytes(wl.batch, wl.q_heads, wl.kv_heads, wl.n, wl.n_q, wl.d,
+                                                          wl.log2_nout, wl.m, Q.dtype, args.precision),
+                              dtype=torch.uint8, device=dev)
+        elm.compress_attend_host(Qp, Kp, Vp, wl.log2_nout, wl.m, seed=args.seed, precision=args.precision,
+                                 scratch=scratch, out=Oh)
+        barrier()
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        g0.record()
+        for i in range(args.e2e_steps):
+            elm.compress_attend_host(Qp, Kp, Vp, wl.log2_nout, wl.m, seed=args.seed + i,
+                                     precision=args.precision, scratch=scratch, out=Oh)
+        g1.record()
+        barrier()
+        te = torch.tensor([g0.elapsed_time(g1)], dtype=torch.float64, device=dev)
+        if dist is not None:
+            dist.all_reduce(te, op=dist.ReduceOp.MAX)
+        e2e_ms = float(te.item()) / args.e2e_steps
+        e2e = {"value": tokens_per_step / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
+               "h2d_bytes_per_step": Q.numel() * Q.element_size() + 2 * K.numel() * K.element_size(),
+               "d2h_bytes_per_step": Q.numel() * Q.element_size(), "steps": args.e2e_steps}
+        del scratch
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peaks = load_peaks()
+    attend_flops, compress_flops, hbm_bytes = algorithmic_counts(wl)
+    stage_ms = {k: v[0] / args.steps for k, v in stage.items()}
+    att_ms = stage_ms["attend"]
+    tensor_peak = peaks["bf16_tflops_sustained"]
+    # the dominant kernel: weighted attention (dense contraction -> tensor roofline) unless the
+    # workload's coreset is so small that its Q/O traffic dominates
+    t_tensor = attend_flops / (tensor_peak * 1e12)
+    att_bytes = 2 * wl.batch * wl.q_heads * wl.n_q * wl.d * (2 if wl.dtype == "bf16" else 4)
+    t_hbm = att_bytes / (peaks["hbm_gbs"] * 1e9)
+    if wl.dtype == "bf16" and t_tensor >= t_hbm:
+        achieved = attend_flops / (att_ms * 1e-3) / 1e12
+        roofline = {"bound": "tensor", "kernel": "attend", "achieved": achieved, "peak": tensor_peak,
+                    "unit": "TFLOP/s", "frac": achieved / tensor_peak, "traffic": None,
+                    "peak_source": f"{peaks['source']} bf16 sustained", "ms_per_launch": att_ms}
+    else:
+        achieved = att_bytes / (att_ms * 1e-3) / 1e9
+        roofline = {"bound": "hbm", "kernel": "attend", "achieved": achieved, "peak": peaks["hbm_gbs"],
+                    "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "traffic": None,
+                    "peak_source": f"{peaks['source']} copy", "ms_per_launch": att_ms}
+    traffic_path = os.path.join(ROOT, "profiles", "attend_traffic.json")
+    if os.path.exists(traffic_path):
+        with open(traffic_path) as f:
+            tr = json.load(f)
+        if tr.get("workload") == wl.name:
+            roofline["traffic"] = tr.get("dram_bytes_per_launch")
+    whole_roof_s = max((attend_flops + compress_flops) / (tensor_peak * 1e12), hbm_bytes / (peaks["hbm_gbs"] * 1e9))
+
+    base = None
+    if not args.no_cpu_baseline:
+        base, _ = cpu_baseline(wl, Q, K, V)
+
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16" if wl.dtype == "bf16" else "f32", "data": "synthetic",
+        "config": workload_config(wl, args),
+        "roofline": roofline,
+        "whole_path_roofline": {"roofline_ms": whole_roof_s * 1e3, "frac": whole_roof_s * 1e3 / ms_step,
+                                "attend_flops": attend_flops, "compress_flops": compress_flops,
+                                "hbm_bytes": hbm_bytes},
+        "stage_ms": stage_ms,
+        "cpu_baseline": base,
+        "e2e": e2e,
+        "gpu_launches": launches,
+        "clocks": clocks.summary(),
+    }
+    print(json.dumps(out))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,159 @@
+/*
+ * elm.h -- C ABI of the B200 (sm_100a) kernel-halving compression + weighted attention library.
+ *
+ * The two main calls follow the problem statement of "Express Language Modeling"
+ * (arXiv 2606.10944):
+ *
+ *   elm_compress   a thinning algorithm in the sense of Definition 1: every attention problem
+ *                  (one batch entry, one KV head) with n key-value pairs is reduced to a coreset
+ *                  of n_out = 2^log2_nout of its own points with positive weights summing to 1.
+ *                  The thinning is Offline-Compress2 (the recursive form of Algorithm 2) with
+ *                  Halve = KH(delta) (Algorithm A.1) under the key-value attention kernel of
+ *                  Eq. (katt).
+ *   elm_attend     Eq. (def:att_approx) / the return line of Algorithm 5: every query attends
+ *                  over one weighted coreset with softmax weights w * exp(<q,k>/sqrt(d)).
+ *
+ * Conventions for every call
+ *   - All tensor pointers are DEVICE pointers unless the name ends in _host.  The caller owns
+ *     every buffer; the library allocates no device memory and keeps no pointer after return.
+ *   - Tensors are dense and row-major: Q, O [batch][q_heads][n_q][d]; K, V [batch][kv_heads][n_kv][d];
+ *     idx, w [batch][kv_heads][n_core].  Element type of Q, K, V, O is params->dtype.
+ *     Base pointers must be 16-byte aligned.
+ *   - Query head h of a batch entry reads KV head floor(h * kv_heads / q_heads) (grouped queries).
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Device calls
+ *     only enqueue work; they do not synchronise.
+ *   - The return value is ELM_OK (0) or a negative elm_status.  Argument errors are detected on
+ *     the host before anything is launched.  Nothing throws across this boundary.
+ */
+#ifndef ELM_H
+#define ELM_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum { ELM_F32 = 0, ELM_BF16 = 1 } elm_dtype;
+
+typedef enum {
+    ELM_PREC_FP64_DET = 0, /* all kernel-halving arithmetic in fp64: decisions reproduce an fp64
+                              CPU statement of Algorithm A.1 unless a uniform falls within
+                              rounding distance of its swap probability */
+    ELM_PREC_FP32 = 1      /* fp32 accumulation; bf16 inputs use the tensor cores */
+} elm_precision;
+
+typedef enum {
+    ELM_OK = 0,
+    ELM_ERR_NULL = -1,        /* a required pointer is NULL */
+    ELM_ERR_SHAPE = -2,       /* unsupported or inconsistent sizes */
+    ELM_ERR_DTYPE = -3,       /* unknown dtype / precision */
+    ELM_ERR_ALIGN = -4,       /* a pointer is not 16-byte aligned */
+    ELM_ERR_WORKSPACE = -5,   /* workspace too small */
+    ELM_ERR_DELTA = -6,       /* a failure parameter outside (0, 1) */
+    ELM_ERR_CUDA = -7,        /* a CUDA runtime call or launch failed */
+    ELM_ERR_UNAVAILABLE = -8  /* no usable CUDA device */
+} elm_status;
+
+typedef struct elm_params {
+    int32_t batch;       /* B >= 1 */
+    int32_t q_heads;     /* H_q, a multiple of kv_heads */
+    int32_t kv_heads;    /* H_kv */
+    int32_t n_kv;        /* n: key-value pairs per attention problem; must equal 2^m * 2^log2_nout */
+    int32_t n_q;         /* queries per head (any value >= 1) */
+    int32_t d;           /* head dimension: 64 or 128 */
+    int32_t log2_nout;   /* coreset size n_out = 2^log2_nout (Algorithm 4's h) */
+    int32_t m;           /* Compress2 depth (Algorithm 2); 0 returns every point; the level-0
+                            groups hold n_kv / 4^(m-1) points and must hold at least 2 */
+    int32_t dtype;       /* elm_dtype of Q, K, V, O */
+    int32_t precision;   /* elm_precision */
+    double delta;        /* failure budget delta in (0,1); the paper's experiments use 1/2 */
+    const double *delta_level; /* optional HOST array[m]: KH failure parameter of level i.  NULL
+                                  selects delta_i = 4^(i+1-m) * delta / (3m), the schedule of
+                                  Corollary 2 with this call's own depth */
+} elm_params;
+
+/* Bytes of device workspace elm_compress and elm_attend need for `params` (n_core taken as
+ * n_out).  Either output pointer may be NULL. */
+int elm_workspace_bytes(const elm_params *params, size_t *compress_bytes, size_t *attend_bytes);
+
+/* The default per-level failure parameters described at elm_params.delta_level; out[m] on the host. */
+int elm_default_delta_levels(int32_t m, double delta, double *out_host);
+
+/*
+ * Definition 1 + Offline-Compress2 + Algorithm A.1 under Eq. (katt).
+ *   K, V       [batch][kv_heads][n_kv][d], read only.
+ *   seed       selects the uniforms: pair i of Halve call g at level l of problem p uses the first
+ *              word of Philox4x32-10(counter = (i, g, l, p), key = (seed low, seed high)), top 24 bits.
+ *   idx_out    [batch][kv_heads][n_out] row numbers in [0, n_kv), in the order Algorithm A.1 appends
+ *              them (not sorted); all distinct.
+ *   w_out      [batch][kv_heads][n_out], every entry 1/n_out.
+ *   workspace  at least compress_bytes of elm_workspace_bytes, 256-byte aligned; contents are
+ *              scratch.  Two calls that overlap in time need separate workspaces.
+ * v_max of Eq. (katt) is taken per attention problem.  exp(<k,k'>/sqrt(d)) is evaluated with a
+ * running shift (the largest ||k||^2/sqrt(d) seen so far in the Halve call), which leaves every
+ * swap probability unchanged and keeps the arithmetic finite for any input.
+ */
+int elm_compress(const void *K, const void *V, const elm_params *params, uint64_t seed,
+                 int32_t *idx_out, float *w_out, void *workspace, size_t workspace_bytes,
+                 void *stream);
+
+/*
+ * Eq. (def:att_approx) with one coreset per attention problem (Algorithm 5's return line).
+ *   Q          [batch][q_heads][n_q][d]
+ *   K, V       the ORIGINAL [batch][kv_heads][n_kv][d] tensors; rows are gathered through idx.
+ *   idx, w     [batch][kv_heads][n_core]; any positive finite weights (they need not sum to 1),
+ *              1 <= n_core <= n_kv.
+ *   O          [batch][q_heads][n_q][d], same dtype as Q.
+ *   workspace  at least elm_attend_workspace_bytes(params, n_core), 256-byte aligned.
+ * precision FP64_DET accumulates in fp64, FP32 in fp32 (bf16 inputs: tensor cores).
+ */
+int elm_attend(const void *Q, const void *K, const void *V, const int32_t *idx, const float *w,
+               int32_t n_core, const elm_params *params, void *O, void *workspace,
+               size_t workspace_bytes, void *stream);
+
+/* Workspace of elm_attend for an explicit coreset size. */
+int elm_attend_workspace_bytes(const elm_params *params, int32_t n_core, size_t *bytes);
+
+/*
+ * End-to-end convenience call on HOST buffers: copies Q, K, V to the device, runs elm_compress and
+ * elm_attend, copies O (and, when non-NULL, idx and w) back, and synchronises `stream` before it
+ * returns.  Host buffers may be pageable or pinned.  `device_scratch` is a DEVICE buffer of at
+ * least elm_host_call_scratch_bytes(params) bytes, 256-byte aligned, owned by the caller.
+ */
+int elm_host_call_scratch_bytes(const elm_params *params, size_t *bytes);
+int elm_compress_attend_host(const void *Q_host, const void *K_host, const void *V_host,
+                             void *O_host, int32_t *idx_host, float *w_host,
+                             const elm_params *params, uint64_t seed, void *device_scratch,
+                             size_t device_scratch_bytes, void *stream);
+
+/*
+ * Per-stage device timing (off by default).  When enabled, every elm_compress / elm_attend call
+ * records CUDA events around each of its stages on the caller's stream; elm_profile_read
+ * synchronises those events and returns, for stage s < ELM_N_STAGES, the accumulated milliseconds
+ * and kernel launches since the last read, then resets them.  Not thread safe.
+ */
+enum {
+    ELM_STAGE_PREPASS = 0,  /* v_max, key norms, identity index list */
+    ELM_STAGE_LEVEL_PREP,   /* per-level running shifts */
+    ELM_STAGE_GRAM,         /* kernel evaluation -> pair Gram */
+    ELM_STAGE_WALK,         /* halving walk */
+    ELM_STAGE_EMIT,         /* weights */
+    ELM_STAGE_GATHER,       /* coreset rows -> contiguous operands */
+    ELM_STAGE_ATTEND,       /* weighted attention */
+    ELM_N_STAGES
+};
+int elm_profile_enable(int on);
+int elm_profile_read(float *ms_out, int64_t *launches_out, int32_t n_stages);
+
+/* Kernels launched by this library since it was loaded (all calls, all stages). */
+int64_t elm_launch_count(void);
+
+const char *elm_strerror(int status);
+int elm_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ELM_H */

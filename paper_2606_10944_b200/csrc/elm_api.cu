@@ -1,0 +1,208 @@
+// Host-side pieces of the C ABI that launch nothing themselves: argument validation, workspace
+// sizing, the host-buffer convenience call, per-stage timing and status text.
+#include <math.h>
+#include <stdio.h>
+
+#include <atomic>
+
+#include "elm_attend.cuh"
+#include "elm_common.cuh"
+#include "elm_compress.cuh"
+
+namespace elm {
+
+static std::atomic<int64_t> g_launches{0};
+static int64_t g_stage_launches[ELM_N_STAGES];
+
+Profiler &profiler()
+{
+    static Profiler p;
+    return p;
+}
+
+void count_launches(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+StageTimer::StageTimer(int stage, cudaStream_t stream, int launches) : stream_(stream)
+{
+    Profiler &pr = profiler();
+    g_stage_launches[stage] += launches;
+    if (!pr.enabled || pr.n_records >= Profiler::kMaxRecords) return;
+    rec_ = pr.n_records++;
+    if (rec_ >= pr.events_created) {
+        cudaEventCreate(&pr.ev_begin[rec_]);
+        cudaEventCreate(&pr.ev_end[rec_]);
+        pr.events_created = rec_ + 1;
+    }
+    pr.stage_of[rec_] = stage;
+    pr.launches_of[rec_] = launches;
+    cudaEventRecord(pr.ev_begin[rec_], stream_);
+}
+
+StageTimer::~StageTimer()
+{
+    if (rec_ >= 0) cudaEventRecord(profiler().ev_end[rec_], stream_);
+}
+
+int validate_params(const elm_params *p)
+{
+    if (p->batch < 1 || p->kv_heads < 1 || p->q_heads < 1 || p->n_q < 1) return ELM_ERR_SHAPE;
+    if (p->q_heads % p->kv_heads != 0) return ELM_ERR_SHAPE;
+    if (p->d != 64 && p->d != 128) return ELM_ERR_SHAPE;
+    if (p->log2_nout < 0 || p->log2_nout > 24 || p->m < 0 || p->m > 12) return ELM_ERR_SHAPE;
+    if (p->log2_nout + p->m > 30) return ELM_ERR_SHAPE;
+    if ((int64_t)p->n_kv != ((int64_t)1 << (p->log2_nout + p->m))) return ELM_ERR_SHAPE;
+    if (p->m >= 1 && p->log2_nout - p->m + 2 < 1) return ELM_ERR_SHAPE;      // level-0 groups >= 2 points
+    if ((int64_t)p->batch * p->q_heads > 65535) return ELM_ERR_SHAPE;
+    if (p->dtype != ELM_F32 && p->dtype != ELM_BF16) return ELM_ERR_DTYPE;
+    if (p->precision != ELM_PREC_FP64_DET && p->precision != ELM_PREC_FP32) return ELM_ERR_DTYPE;
+    if (!(p->delta > 0.0 && p->delta < 1.0)) return ELM_ERR_DELTA;
+    if (p->delta_level)
+        for (int i = 0; i < p->m; ++i)
+            if (!(p->delta_level[i] > 0.0 && p->delta_level[i] < 1.0)) return ELM_ERR_DELTA;
+    return ELM_OK;
+}
+
+}  // namespace elm
+
+using namespace elm;
+
+extern "C" int elm_workspace_bytes(const elm_params *params, size_t *compress_bytes, size_t *attend_bytes)
+{
+    if (!params) return ELM_ERR_NULL;
+    int rc = validate_params(params);
+    if (rc != ELM_OK) return rc;
+    if (compress_bytes) *compress_bytes = compress_layout(params).total;
+    if (attend_bytes) *attend_bytes = attend_layout(params, 1 << params->log2_nout).total;
+    return ELM_OK;
+}
+
+extern "C" int elm_default_delta_levels(int32_t m, double delta, double *out_host)
+{
+    if (!out_host && m > 0) return ELM_ERR_NULL;
+    if (m < 0 || m > 32) return ELM_ERR_SHAPE;
+    if (!(delta > 0.0 && delta < 1.0)) return ELM_ERR_DELTA;
+    // Corollary 2's delta_{m,i} = 4^(i+1-q) delta_m / (3q) with q = this call's depth and
+    // delta_m = the caller's budget.
+    for (int i = 0; i < m; ++i) out_host[i] = ldexp(delta, 2 * (i + 1 - m)) / (3.0 * (double)m);
+    return ELM_OK;
+}
+
+namespace {
+struct HostCallLayout {
+    size_t Q, K, V, O, idx, w, ws_compress, ws_attend, total;
+};
+HostCallLayout host_layout(const elm_params *p)
+{
+    HostCallLayout L;
+    const size_t es = elt_bytes(p->dtype);
+    const size_t qo = (size_t)p->batch * p->q_heads * p->n_q * p->d * es;
+    const size_t kv = (size_t)p->batch * p->kv_heads * p->n_kv * p->d * es;
+    const size_t core = (size_t)p->batch * p->kv_heads * ((size_t)1 << p->log2_nout);
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+    L.Q = take(qo);
+    L.K = take(kv);
+    L.V = take(kv);
+    L.O = take(qo);
+    L.idx = take(core * 4);
+    L.w = take(core * 4);
+    L.ws_compress = take(compress_layout(p).total);
+    L.ws_attend = take(attend_layout(p, 1 << p->log2_nout).total);
+    L.total = off;
+    return L;
+}
+}  // namespace
+
+extern "C" int elm_host_call_scratch_bytes(const elm_params *params, size_t *bytes)
+{
+    if (!params || !bytes) return ELM_ERR_NULL;
+    int rc = validate_params(params);
+    if (rc != ELM_OK) return rc;
+    *bytes = host_layout(params).total;
+    return ELM_OK;
+}
+
+extern "C" int elm_compress_attend_host(const void *Q_host, const void *K_host, const void *V_host,
+                                        void *O_host, int32_t *idx_host, float *w_host,
+                                        const elm_params *params, uint64_t seed, void *device_scratch,
+                                        size_t device_scratch_bytes, void *stream)
+{
+    if (!params) return ELM_ERR_NULL;
+    int rc = validate_params(params);
+    if (rc != ELM_OK) return rc;
+    if (!Q_host || !K_host || !V_host || !O_host || !device_scratch) return ELM_ERR_NULL;
+    if ((uintptr_t)device_scratch & 255) return ELM_ERR_ALIGN;
+    const HostCallLayout L = host_layout(params);
+    if (device_scratch_bytes < L.total) return ELM_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    unsigned char *base = (unsigned char *)device_scratch;
+    const size_t es = elt_bytes(params->dtype);
+    const size_t qo = (size_t)params->batch * params->q_heads * params->n_q * params->d * es;
+    const size_t kv = (size_t)params->batch * params->kv_heads * params->n_kv * params->d * es;
+    const size_t core = (size_t)params->batch * params->kv_heads * ((size_t)1 << params->log2_nout);
+    // K and V first: compression can start while Q is still in flight on a copy engine only if the
+    // caller splits streams; on one stream the order is simply K, V, Q.
+    ELM_CUDA_TRY(cudaMemcpyAsync(base + L.K, K_host, kv, cudaMemcpyHostToDevice, st));
+    ELM_CUDA_TRY(cudaMemcpyAsync(base + L.V, V_host, kv, cudaMemcpyHostToDevice, st));
+    ELM_CUDA_TRY(cudaMemcpyAsync(base + L.Q, Q_host, qo, cudaMemcpyHostToDevice, st));
+    rc = elm_compress(base + L.K, base + L.V, params, seed, (int32_t *)(base + L.idx), (float *)(base + L.w),
+                      base + L.ws_compress, compress_layout(params).total, stream);
+    if (rc != ELM_OK) return rc;
+    const int32_t n_core = 1 << params->log2_nout;
+    rc = elm_attend(base + L.Q, base + L.K, base + L.V, (const int32_t *)(base + L.idx),
+                    (const float *)(base + L.w), n_core, params, base + L.O, base + L.ws_attend,
+                    attend_layout(params, n_core).total, stream);
+    if (rc != ELM_OK) return rc;
+    ELM_CUDA_TRY(cudaMemcpyAsync(O_host, base + L.O, qo, cudaMemcpyDeviceToHost, st));
+    if (idx_host) ELM_CUDA_TRY(cudaMemcpyAsync(idx_host, base + L.idx, core * 4, cudaMemcpyDeviceToHost, st));
+    if (w_host) ELM_CUDA_TRY(cudaMemcpyAsync(w_host, base + L.w, core * 4, cudaMemcpyDeviceToHost, st));
+    ELM_CUDA_TRY(cudaStreamSynchronize(st));
+    return ELM_OK;
+}
+
+extern "C" int elm_profile_enable(int on)
+{
+    Profiler &pr = profiler();
+    pr.enabled = on != 0;
+    pr.n_records = 0;
+    for (int s = 0; s < ELM_N_STAGES; ++s) g_stage_launches[s] = 0;
+    return ELM_OK;
+}
+
+extern "C" int elm_profile_read(float *ms_out, int64_t *launches_out, int32_t n_stages)
+{
+    Profiler &pr = profiler();
+    if (!ms_out || n_stages < ELM_N_STAGES) return ELM_ERR_NULL;
+    for (int s = 0; s < ELM_N_STAGES; ++s) ms_out[s] = 0.f;
+    for (int r = 0; r < pr.n_records; ++r) {
+        if (cudaEventSynchronize(pr.ev_end[r]) != cudaSuccess) return ELM_ERR_CUDA;
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, pr.ev_begin[r], pr.ev_end[r]) != cudaSuccess) return ELM_ERR_CUDA;
+        ms_out[pr.stage_of[r]] += ms;
+    }
+    if (launches_out)
+        for (int s = 0; s < ELM_N_STAGES; ++s) launches_out[s] = g_stage_launches[s];
+    pr.n_records = 0;
+    for (int s = 0; s < ELM_N_STAGES; ++s) g_stage_launches[s] = 0;
+    return ELM_OK;
+}
+
+extern "C" int64_t elm_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+extern "C" const char *elm_strerror(int status)
+{
+    switch (status) {
+    case ELM_OK: return "ok";
+    case ELM_ERR_NULL: return "a required pointer is NULL";
+    case ELM_ERR_SHAPE: return "unsupported or inconsistent sizes";
+    case ELM_ERR_DTYPE: return "unknown dtype or precision";
+    case ELM_ERR_ALIGN: return "a pointer is not sufficiently aligned";
+    case ELM_ERR_WORKSPACE: return "workspace too small";
+    case ELM_ERR_DELTA: return "failure parameter outside (0, 1)";
+    case ELM_ERR_CUDA: return "a CUDA call or kernel launch failed";
+    case ELM_ERR_UNAVAILABLE: return "no usable CUDA device";
+    default: return "unknown status";
+    }
+}
+
+extern "C" int elm_version(void) { return 100; }

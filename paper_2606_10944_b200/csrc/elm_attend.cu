@@ -1,0 +1,252 @@
+// Weighted attention over a coreset, Eq. (def:att_approx):
+//   O[j,:] = sum_c w_c exp(<q_j,k_c>/sqrt(d)) v_c / sum_c w_c exp(<q_j,k_c>/sqrt(d)).
+// Stage gather copies the coreset rows of every attention problem into contiguous operands and
+// turns the weights into a base-2 logit bias log2(w_c); stage attend is an online-softmax pass.
+// This file holds the precision-generic SIMT kernel (fp64 mode and fp32 inputs); bf16 inputs in
+// fp32 mode take the tensor-core kernel in elm_attend_tc.cu.
+#include <math.h>
+
+#include "elm_attend.cuh"
+#include "elm_common.cuh"
+
+namespace elm {
+
+// ---------------------------------------------------------------------------------------------
+// Stage gather: Kc, Vc [problems][n_core][d] in the input dtype, bias [problems][n_core] fp32
+// ---------------------------------------------------------------------------------------------
+template <typename Tin>
+__global__ void __launch_bounds__(256) gather_kernel(const Tin *__restrict__ K,
+                                                     const Tin *__restrict__ V,
+                                                     const int32_t *__restrict__ idx,
+                                                     const float *__restrict__ w, int64_t n, int d,
+                                                     int n_core, Tin *__restrict__ Kc,
+                                                     Tin *__restrict__ Vc, float *__restrict__ bias)
+{
+    const int p = blockIdx.y;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int c = blockIdx.x * 8 + warp;
+    if (c >= n_core) return;
+    const int64_t row = idx[(int64_t)p * n_core + c];
+    const Tin *ks = K + ((int64_t)p * n + row) * d;
+    const Tin *vs = V + ((int64_t)p * n + row) * d;
+    Tin *kd = Kc + ((int64_t)p * n_core + c) * d;
+    Tin *vd = Vc + ((int64_t)p * n_core + c) * d;
+    for (int e = lane; e < d; e += 32) {
+        kd[e] = ks[e];
+        vd[e] = vs[e];
+    }
+    if (lane == 0) bias[(int64_t)p * n_core + c] = log2f(w[(int64_t)p * n_core + c]);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Stage attend (SIMT): one CTA = 64 queries of one head; coreset streamed in chunks of 32 points.
+// Logits are kept in base 2: s = <q,k> * log2(e)/sqrt(d) + log2(w).
+// ---------------------------------------------------------------------------------------------
+template <typename Tin, typename T, int D>
+__global__ void __launch_bounds__(128) attend_simt_kernel(const Tin *__restrict__ Q,
+                                                          const Tin *__restrict__ Kc,
+                                                          const Tin *__restrict__ Vc,
+                                                          const float *__restrict__ bias,
+                                                          Tin *__restrict__ O, int q_heads,
+                                                          int kv_heads, int64_t n_q, int n_core)
+{
+    constexpr int BM = 64, BN = 32;
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    T *Qt = reinterpret_cast<T *>(smem_raw);        // [D][BM]   transposed query tile
+    T *Kt = Qt + D * BM;                            // [D][BN]   transposed key chunk
+    T *Vs = Kt + D * BN;                            // [BN][D]
+    T *S = Vs + BN * D;                             // [BM][BN+1] logits, then probabilities
+    T *rowscale = S + BM * (BN + 1);                // [BM] factor applied to the old accumulator
+    T *rowsum = rowscale + BM;                      // [BM] running denominator
+    T *rowmax = rowsum + BM;                        // [BM] running maximum
+    T *sbias = rowmax + BM;                         // [BN]
+
+    const int tid = threadIdx.x;
+    const int bh = blockIdx.y;                      // batch * q_heads + head
+    const int b = bh / q_heads, h = bh % q_heads;
+    const int64_t prob = (int64_t)b * kv_heads + ((int64_t)h * kv_heads) / q_heads;
+    const int64_t q0 = (int64_t)blockIdx.x * BM;
+    const Tin *Qp = Q + ((int64_t)bh * n_q) * D;
+    const Tin *Kp = Kc + prob * n_core * D;
+    const Tin *Vp = Vc + prob * n_core * D;
+    const float *bp = bias + prob * n_core;
+    const T scale = (T)(1.4426950408889634 / sqrt((double)D));
+
+    for (int e = tid; e < BM * D; e += 128) {
+        int r = e / D, k = e % D;
+        Qt[k * BM + r] = (q0 + r < n_q) ? load_as<T>(Qp, (q0 + r) * D + k) : (T)0;
+    }
+    if (tid < BM) { rowsum[tid] = 0; rowmax[tid] = -INFINITY; }
+
+    const int ty = tid >> 3, tx = tid & 7;          // S tile: rows 4ty.., cols 4tx..
+    constexpr int OC = D / 8;                       // output columns per thread
+    T acc[4][OC];
+#pragma unroll
+    for (int r = 0; r < 4; ++r)
+#pragma unroll
+        for (int c = 0; c < OC; ++c) acc[r][c] = 0;
+
+    for (int c0 = 0; c0 < n_core; c0 += BN) {
+        __syncthreads();
+        for (int e = tid; e < BN * D; e += 128) {
+            int c = e / D, k = e % D;
+            bool ok = c0 + c < n_core;
+            Kt[k * BN + c] = ok ? load_as<T>(Kp, (int64_t)(c0 + c) * D + k) : (T)0;
+            Vs[c * D + k] = ok ? load_as<T>(Vp, (int64_t)(c0 + c) * D + k) : (T)0;
+        }
+        if (tid < BN) sbias[tid] = (c0 + tid < n_core) ? (T)bp[c0 + tid] : (T)0;
+        __syncthreads();
+        T s[4][4];
+#pragma unroll
+        for (int r = 0; r < 4; ++r)
+#pragma unroll
+            for (int c = 0; c < 4; ++c) s[r][c] = 0;
+        for (int k = 0; k < D; ++k) {
+            T qv[4], kv[4];
+#pragma unroll
+            for (int r = 0; r < 4; ++r) { qv[r] = Qt[k * BM + 4 * ty + r]; kv[r] = Kt[k * BN + 4 * tx + r]; }
+#pragma unroll
+            for (int r = 0; r < 4; ++r)
+#pragma unroll
+                for (int c = 0; c < 4; ++c) s[r][c] += qv[r] * kv[c];
+        }
+#pragma unroll
+        for (int r = 0; r < 4; ++r)
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                int col = 4 * tx + c;
+                S[(4 * ty + r) * (BN + 1) + col] = (c0 + col < n_core) ? s[r][c] * scale + sbias[col] : (T)-INFINITY;
+            }
+        __syncthreads();
+        if (tid < BM) {
+            T *row = S + tid * (BN + 1);
+            T mx = rowmax[tid];
+            for (int c = 0; c < BN; ++c) mx = row[c] > mx ? row[c] : mx;
+            T f = (rowmax[tid] == -INFINITY) ? (T)0 : (T)exp2((T)(rowmax[tid] - mx));
+            T sum = 0;
+            for (int c = 0; c < BN; ++c) {
+                T pr = (row[c] == -INFINITY) ? (T)0 : (T)exp2((T)(row[c] - mx));
+                row[c] = pr;
+                sum += pr;
+            }
+            rowscale[tid] = f;
+            rowsum[tid] = rowsum[tid] * f + sum;
+            rowmax[tid] = mx;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            T f = rowscale[4 * ty + r];
+#pragma unroll
+            for (int c = 0; c < OC; ++c) acc[r][c] *= f;
+        }
+        for (int c = 0; c < BN; ++c) {
+            T pr[4];
+#pragma unroll
+            for (int r = 0; r < 4; ++r) pr[r] = S[(4 * ty + r) * (BN + 1) + c];
+#pragma unroll
+            for (int o = 0; o < OC; ++o) {
+                T v = Vs[c * D + tx + 8 * o];
+#pragma unroll
+                for (int r = 0; r < 4; ++r) acc[r][o] += pr[r] * v;
+            }
+        }
+    }
+    Tin *Op = O + ((int64_t)bh * n_q) * D;
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+        int64_t q = q0 + 4 * ty + r;
+        if (q >= n_q) continue;
+        T inv = (T)1 / rowsum[4 * ty + r];
+#pragma unroll
+        for (int o = 0; o < OC; ++o) store_from(Op, q * D + tx + 8 * o, acc[r][o] * inv);
+    }
+}
+
+AttendLayout attend_layout(const elm_params *p, int32_t n_core)
+{
+    AttendLayout L;
+    const size_t problems = (size_t)p->batch * p->kv_heads;
+    const size_t es = elt_bytes(p->dtype);
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+    L.Kc = take(problems * (size_t)n_core * p->d * es);
+    L.Vc = take(problems * (size_t)n_core * p->d * es);
+    L.bias = take(problems * (size_t)n_core * 4);
+    L.total = off;
+    return L;
+}
+
+template <typename Tin, typename T, int D>
+static int launch_attend_simt(const Tin *Q, const Tin *Kc, const Tin *Vc, const float *bias, Tin *O,
+                              const elm_params *p, int n_core, cudaStream_t st)
+{
+    constexpr int BM = 64, BN = 32;
+    const size_t smem = sizeof(T) * (size_t)(D * BM + D * BN + BN * D + BM * (BN + 1) + 3 * BM + BN);
+    auto kern = attend_simt_kernel<Tin, T, D>;
+    ELM_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    dim3 grid((unsigned)((p->n_q + BM - 1) / BM), (unsigned)(p->batch * p->q_heads));
+    kern<<<grid, 128, smem, st>>>(Q, Kc, Vc, bias, O, p->q_heads, p->kv_heads, p->n_q, n_core);
+    count_launches(1);
+    return cuda_status(cudaGetLastError());
+}
+
+template <typename Tin, typename T>
+static int attend_impl(const Tin *Q, const Tin *K, const Tin *V, const int32_t *idx, const float *w,
+                       int n_core, const elm_params *p, Tin *O, unsigned char *ws, cudaStream_t st)
+{
+    const AttendLayout L = attend_layout(p, n_core);
+    Tin *Kc = reinterpret_cast<Tin *>(ws + L.Kc);
+    Tin *Vc = reinterpret_cast<Tin *>(ws + L.Vc);
+    float *bias = reinterpret_cast<float *>(ws + L.bias);
+    const int problems = p->batch * p->kv_heads;
+    {
+        StageTimer t(ELM_STAGE_GATHER, st, 1);
+        gather_kernel<Tin><<<dim3((unsigned)((n_core + 7) / 8), (unsigned)problems), 256, 0, st>>>(
+            K, V, idx, w, p->n_kv, p->d, n_core, Kc, Vc, bias);
+        count_launches(1);
+        ELM_CUDA_TRY(cudaGetLastError());
+    }
+    StageTimer t(ELM_STAGE_ATTEND, st, 1);
+    if (p->d == 64) return launch_attend_simt<Tin, T, 64>(Q, Kc, Vc, bias, O, p, n_core, st);
+    return launch_attend_simt<Tin, T, 128>(Q, Kc, Vc, bias, O, p, n_core, st);
+}
+
+}  // namespace elm
+
+extern "C" int elm_attend_workspace_bytes(const elm_params *params, int32_t n_core, size_t *bytes)
+{
+    using namespace elm;
+    if (!params || !bytes) return ELM_ERR_NULL;
+    int rc = validate_params(params);
+    if (rc != ELM_OK) return rc;
+    if (n_core < 1 || n_core > params->n_kv) return ELM_ERR_SHAPE;
+    *bytes = attend_layout(params, n_core).total;
+    return ELM_OK;
+}
+
+extern "C" int elm_attend(const void *Q, const void *K, const void *V, const int32_t *idx,
+                          const float *w, int32_t n_core, const elm_params *params, void *O,
+                          void *workspace, size_t workspace_bytes, void *stream)
+{
+    using namespace elm;
+    if (!params) return ELM_ERR_NULL;
+    int rc = validate_params(params);
+    if (rc != ELM_OK) return rc;
+    if (!Q || !K || !V || !idx || !w || !O || !workspace) return ELM_ERR_NULL;
+    if (n_core < 1 || n_core > params->n_kv) return ELM_ERR_SHAPE;
+    if (((uintptr_t)Q | (uintptr_t)K | (uintptr_t)V | (uintptr_t)idx | (uintptr_t)w | (uintptr_t)O) & 15)
+        return ELM_ERR_ALIGN;
+    if ((uintptr_t)workspace & 255) return ELM_ERR_ALIGN;
+    if (workspace_bytes < attend_layout(params, n_core).total) return ELM_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    unsigned char *ws = (unsigned char *)workspace;
+    const bool det = params->precision == ELM_PREC_FP64_DET;
+    if (params->dtype == ELM_F32) {
+        return det ? attend_impl<float, double>((const float *)Q, (const float *)K, (const float *)V, idx, w, n_core, params, (float *)O, ws, st)
+                   : attend_impl<float, float>((const float *)Q, (const float *)K, (const float *)V, idx, w, n_core, params, (float *)O, ws, st);
+    }
+    typedef __nv_bfloat16 bf;
+    return det ? attend_impl<bf, double>((const bf *)Q, (const bf *)K, (const bf *)V, idx, w, n_core, params, (bf *)O, ws, st)
+               : attend_impl<bf, float>((const bf *)Q, (const bf *)K, (const bf *)V, idx, w, n_core, params, (bf *)O, ws, st);
+}

@@ -1,0 +1,101 @@
+// Shared host/device helpers of the CUDA library (not used by, and sharing nothing with, the
+// CPU oracle).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/elm.h"
+
+namespace elm {
+
+// ---------------------------------------------------------------------------------------------
+// launch bookkeeping and per-stage timing
+// ---------------------------------------------------------------------------------------------
+struct Profiler {
+    bool enabled = false;
+    static constexpr int kMaxRecords = 4096;
+    int n_records = 0;
+    cudaEvent_t ev_begin[kMaxRecords];
+    cudaEvent_t ev_end[kMaxRecords];
+    int stage_of[kMaxRecords];
+    int launches_of[kMaxRecords];
+    int events_created = 0;
+};
+Profiler &profiler();
+void count_launches(int n);
+
+// RAII: times everything enqueued on `stream` during its lifetime as one record of `stage`.
+class StageTimer {
+  public:
+    StageTimer(int stage, cudaStream_t stream, int launches);
+    ~StageTimer();
+
+  private:
+    int rec_ = -1;
+    cudaStream_t stream_;
+};
+
+inline int cuda_status(cudaError_t e) { return e == cudaSuccess ? ELM_OK : ELM_ERR_CUDA; }
+
+#define ELM_CUDA_TRY(expr)                                \
+    do {                                                  \
+        cudaError_t _e = (expr);                          \
+        if (_e != cudaSuccess) return ELM_ERR_CUDA;       \
+    } while (0)
+
+int validate_params(const elm_params *p);
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+inline size_t elt_bytes(int dtype) { return dtype == ELM_BF16 ? 2 : 4; }
+
+// ---------------------------------------------------------------------------------------------
+// device helpers
+// ---------------------------------------------------------------------------------------------
+template <typename T> __device__ __forceinline__ T load_as(const float *p, int64_t i) { return (T)p[i]; }
+template <typename T> __device__ __forceinline__ T load_as(const __nv_bfloat16 *p, int64_t i)
+{
+    return (T)__bfloat162float(p[i]);
+}
+__device__ __forceinline__ void store_from(float *p, int64_t i, double v) { p[i] = (float)v; }
+__device__ __forceinline__ void store_from(float *p, int64_t i, float v) { p[i] = v; }
+__device__ __forceinline__ void store_from(__nv_bfloat16 *p, int64_t i, double v)
+{
+    p[i] = __float2bfloat16_rn((float)v);
+}
+__device__ __forceinline__ void store_from(__nv_bfloat16 *p, int64_t i, float v)
+{
+    p[i] = __float2bfloat16_rn(v);
+}
+
+// Philox4x32-10 (Salmon et al., SC'11), first output word only.
+__device__ __forceinline__ uint32_t philox4x32_10_word0(uint32_t c0, uint32_t c1, uint32_t c2,
+                                                        uint32_t c3, uint32_t k0, uint32_t k1)
+{
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
+        uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+        uint32_t n0 = hi1 ^ c1 ^ k0, n2 = hi0 ^ c3 ^ k1;
+        c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
+        k0 += 0x9E3779B9u;
+        k1 += 0xBB67AE85u;
+    }
+    return c0;
+}
+
+// The uniform of pair `pair` of Halve call `group` at `level` of attention problem `problem`:
+// top 24 bits of the first Philox word, so the value is exact in fp32 and fp64 alike.
+template <typename T>
+__device__ __forceinline__ T halving_uniform(uint64_t seed, uint32_t pair, uint32_t group,
+                                             uint32_t level, uint32_t problem)
+{
+    uint32_t w = philox4x32_10_word0(pair, group, level, problem, (uint32_t)seed, (uint32_t)(seed >> 32));
+    return (T)(w >> 8) * (T)(1.0 / 16777216.0);
+}
+
+// exp with the underflow floor used throughout the halving path: a shifted exponent below the
+// floor gives exactly 0, so no subnormal ever enters a difference of kernel values.
+__device__ __forceinline__ double floored_exp(double x) { return x < -700.0 ? 0.0 : exp(x); }
+__device__ __forceinline__ float floored_exp(float x) { return x < -80.0f ? 0.0f : __expf(x); }
+
+}  // namespace elm

@@ -1,0 +1,503 @@
+// Kernel-halving compression: Offline-Compress2 scheduled level by level, each level being
+//   (1) level_prep : running shifts M_i of the Halve calls of that level,
+//   (2) gram       : kernel evaluation of Eq. (katt) reduced to the pair Gram F = P G P^T,
+//   (3) walk       : the self-balancing signed walk of Algorithm A.1 on F.
+// This file holds the precision-generic SIMT kernels (fp64 deterministic mode, fp32 inputs) and
+// the host-side level scheduler.  The tensor-core Gram for bf16 inputs lives in elm_gram_tc.cu.
+#include <math.h>
+
+#include "elm_common.cuh"
+#include "elm_compress.cuh"
+
+namespace elm {
+
+// ---------------------------------------------------------------------------------------------
+// Stage S0: per attention problem v_max (Eq. katt), c_t = ||k_t||^2 / sqrt(d), identity index list
+// ---------------------------------------------------------------------------------------------
+template <typename Tin, typename T>
+__global__ void __launch_bounds__(256) prepass_kernel(const Tin *__restrict__ K,
+                                                      const Tin *__restrict__ V, int64_t n, int d,
+                                                      T *__restrict__ cnorm,
+                                                      unsigned *__restrict__ vmax_bits,
+                                                      int32_t *__restrict__ cur)
+{
+    const int p = blockIdx.y;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int64_t row0 = (int64_t)blockIdx.x * 64;
+    const Tin *Kp = K + (int64_t)p * n * d;
+    const Tin *Vp = V + (int64_t)p * n * d;
+    const T rsd = sqrt((T)d);
+    float vm = 0.f;
+    for (int r = warp; r < 64; r += 8) {
+        int64_t t = row0 + r;
+        if (t >= n) break;
+        T s = 0;
+        for (int e = lane; e < d; e += 32) {
+            T kv = load_as<T>(Kp, t * d + e);
+            s += kv * kv;
+            vm = fmaxf(vm, fabsf(load_as<float>(Vp, t * d + e)));
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        if (lane == 0) {
+            cnorm[(int64_t)p * n + t] = s / rsd;
+            cur[(int64_t)p * n + t] = (int32_t)t;
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) vm = fmaxf(vm, __shfl_xor_sync(0xffffffffu, vm, o));
+    if (lane == 0) atomicMax(vmax_bits + p, __float_as_uint(vm));   // non-negative floats order as uints
+}
+
+// ---------------------------------------------------------------------------------------------
+// Stage level_prep: for every Halve call of the level, M_i = max over the call's first 2i points
+// of c, and the factor exp(-(M_i - M_{i-1})/2) that carries b_max from one shift to the next.
+// One CTA per call.
+// ---------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(128) level_prep_kernel(const T *__restrict__ cnorm,
+                                                         const int32_t *__restrict__ cur, int64_t n,
+                                                         int P, T *__restrict__ Mpair,
+                                                         T *__restrict__ rdecay)
+{
+    __shared__ T warp_tot[4];
+    const int p = blockIdx.y, g = blockIdx.x;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const T *cp = cnorm + (int64_t)p * n;
+    const int32_t *curp = cur + (int64_t)p * n;
+    const int64_t base = (int64_t)g * P;
+    T carry = 0;            // c >= 0, so 0 is the identity of the running max
+    for (int c0 = 0; c0 < P; c0 += 128) {
+        int i = c0 + threadIdx.x;
+        T v = 0;
+        if (i < P) {
+            T a = cp[curp[2 * (base + i)]], b = cp[curp[2 * (base + i) + 1]];
+            v = a > b ? a : b;
+        }
+        T inc = v;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            T u = __shfl_up_sync(0xffffffffu, inc, o);
+            if (lane >= o) inc = inc > u ? inc : u;
+        }
+        if (lane == 31) warp_tot[warp] = inc;
+        __syncthreads();
+        T before = carry;
+        for (int w = 0; w < warp; ++w) before = before > warp_tot[w] ? before : warp_tot[w];
+        T prev_lane = __shfl_up_sync(0xffffffffu, inc, 1);
+        T excl = lane == 0 ? before : (before > prev_lane ? before : prev_lane);
+        T M = inc > before ? inc : before;
+        if (i < P) {
+            Mpair[(int64_t)p * (n / 2) + base + i] = M;
+            rdecay[(int64_t)p * (n / 2) + base + i] = (i == 0) ? (T)1 : (T)exp(-(double)(M - excl) * 0.5);
+        }
+        T tot = carry;
+        for (int w = 0; w < 4; ++w) tot = tot > warp_tot[w] ? tot : warp_tot[w];
+        __syncthreads();
+        carry = tot;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Stage gram (SIMT): one CTA computes a 32 x 32 tile of pair-Gram entries (64 x 64 points).
+//   G[a,b] = E(<k_a,k_b>/sqrt(d) - M_pair(b)) * (<v_a,v_b> + v_max^2)          Eq. (katt), shifted
+//   F[j,i] = G[2j,2i] - G[2j,2i+1] - G[2j+1,2i] + G[2j+1,2i+1] = <f_j, f_i>   Algorithm A.1's f_i
+// Only j <= i is produced (the walk needs j < i and the diagonal b_i^2 = F[i,i]).
+// Pairs are numbered along the problem's current sequence (J = g*P + j); when a call has fewer
+// than 32 pairs a tile holds several whole calls and only same-call entries are written.
+// ---------------------------------------------------------------------------------------------
+template <typename Tin, typename T, int D>
+__global__ void __launch_bounds__(256) gram_simt_kernel(const Tin *__restrict__ K,
+                                                        const Tin *__restrict__ V,
+                                                        const int32_t *__restrict__ cur,
+                                                        const T *__restrict__ Mpair,
+                                                        const unsigned *__restrict__ vmax_bits,
+                                                        int64_t n, int P, int64_t Ptotal,
+                                                        T *__restrict__ F, int64_t F_stride)
+{
+    constexpr int DC = 16, LD = 68;
+    __shared__ T Ak[DC][LD], Bk[DC][LD], Av[DC][LD], Bv[DC][LD];
+    __shared__ int32_t rowsA[64], rowsB[64];
+    const int p = blockIdx.y;
+    const int tid = threadIdx.x;
+    int64_t JR, JC;
+    if (P >= 32) {
+        const int Tg = P / 32, ntri = Tg * (Tg + 1) / 2;
+        const int g = blockIdx.x / ntri, local = blockIdx.x % ntri;
+        int tc = (int)((sqrtf(8.f * (float)local + 1.f) - 1.f) * 0.5f);
+        while ((tc + 1) * (tc + 2) / 2 <= local) ++tc;
+        while (tc * (tc + 1) / 2 > local) --tc;
+        const int tr = local - tc * (tc + 1) / 2;
+        JR = (int64_t)g * P + tr * 32;
+        JC = (int64_t)g * P + tc * 32;
+    } else {
+        JR = JC = (int64_t)blockIdx.x * 32;
+    }
+    const int32_t *curp = cur + (int64_t)p * n;
+    if (tid < 64) {
+        int64_t pt = 2 * JR + tid;
+        rowsA[tid] = pt < 2 * Ptotal ? curp[pt] : 0;
+    } else if (tid < 128) {
+        int64_t pt = 2 * JC + (tid - 64);
+        rowsB[tid - 64] = pt < 2 * Ptotal ? curp[pt] : 0;
+    }
+    __syncthreads();
+    const Tin *Kp = K + (int64_t)p * n * D;
+    const Tin *Vp = V + (int64_t)p * n * D;
+    const int ty = tid >> 4, tx = tid & 15;
+    T kk[4][4], vv[4][4];
+#pragma unroll
+    for (int r = 0; r < 4; ++r)
+#pragma unroll
+        for (int c = 0; c < 4; ++c) { kk[r][c] = 0; vv[r][c] = 0; }
+
+    for (int k0 = 0; k0 < D; k0 += DC) {
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            int e = tid + 256 * r;
+            int pt = e / DC, q = e % DC;
+            int64_t ra = (int64_t)rowsA[pt] * D + k0 + q, rb = (int64_t)rowsB[pt] * D + k0 + q;
+            Ak[q][pt] = load_as<T>(Kp, ra);
+            Av[q][pt] = load_as<T>(Vp, ra);
+            Bk[q][pt] = load_as<T>(Kp, rb);
+            Bv[q][pt] = load_as<T>(Vp, rb);
+        }
+        __syncthreads();
+#pragma unroll
+        for (int q = 0; q < DC; ++q) {
+            T a[4], b[4], av[4], bv[4];
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+                a[r] = Ak[q][4 * ty + r];
+                av[r] = Av[q][4 * ty + r];
+                b[r] = Bk[q][4 * tx + r];
+                bv[r] = Bv[q][4 * tx + r];
+            }
+#pragma unroll
+            for (int r = 0; r < 4; ++r)
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    kk[r][c] += a[r] * b[c];
+                    vv[r][c] += av[r] * bv[c];
+                }
+        }
+        __syncthreads();
+    }
+
+    const T vm = (T)__uint_as_float(vmax_bits[p]);
+    const T vm2 = vm * vm;
+    const T rsd = sqrt((T)D);
+    T *Fp = F + (int64_t)p * F_stride;
+#pragma unroll
+    for (int cp = 0; cp < 2; ++cp) {
+        const int64_t jc = JC + 2 * tx + cp;
+        if (jc >= Ptotal) continue;
+        const T M = Mpair[(int64_t)p * (n / 2) + jc];
+        const int64_t gc = jc / P;
+#pragma unroll
+        for (int rp = 0; rp < 2; ++rp) {
+            const int64_t jr = JR + 2 * ty + rp;
+            if (jr > jc || jr / P != gc) continue;
+            T g00 = floored_exp(kk[2 * rp][2 * cp] / rsd - M) * (vv[2 * rp][2 * cp] + vm2);
+            T g01 = floored_exp(kk[2 * rp][2 * cp + 1] / rsd - M) * (vv[2 * rp][2 * cp + 1] + vm2);
+            T g10 = floored_exp(kk[2 * rp + 1][2 * cp] / rsd - M) * (vv[2 * rp + 1][2 * cp] + vm2);
+            T g11 = floored_exp(kk[2 * rp + 1][2 * cp + 1] / rsd - M) * (vv[2 * rp + 1][2 * cp + 1] + vm2);
+            Fp[jr * P + (jc - gc * P)] = (g00 - g01) - (g10 - g11);
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Stage walk: Algorithm A.1 on the pair Gram.  With eta_j = +1 when x_{2j-1} stayed in S^(1) and
+// -1 when the pair was swapped, the balancing score is alpha_i = -sum_{j<i} eta_j F[j,i].
+// A warp resolves 32 consecutive pairs: lane i holds column i of the 32 x 32 diagonal tile and its
+// running alpha_i; each step publishes one decision with a ballot and every later lane folds it in.
+// ---------------------------------------------------------------------------------------------
+template <typename T> struct WalkState {
+    T bmax;   // b_{max,i-1} in the shift of the last pair seen (warp-uniform)
+};
+
+// swap iff U < min(1, (1/2)(1 - alpha/a)_+);  a == 0 (or not finite) => probability 1/2
+__device__ __forceinline__ bool swap_decision(double alpha, double a, double U)
+{
+    double p = 0.5;
+    if (a > 0.0 && isfinite(a)) {
+        double t = 1.0 - alpha / a;
+        t = t < 0.0 ? 0.0 : t;
+        p = 0.5 * t;
+        p = p > 1.0 ? 1.0 : p;
+    }
+    return U < p;
+}
+// fp32 mode: the same test with the division cleared, alpha < a (1 - 2U)
+__device__ __forceinline__ bool swap_decision(float alpha, float a, float U)
+{
+    if (a > 0.f && isfinite(a)) return alpha < a * (1.f - 2.f * U);
+    return U < 0.5f;
+}
+
+// Resolve pairs [i0, i0 + cnt) (cnt <= 32) of one call.  `alpha` is this lane's score from all
+// earlier blocks; Fg points at the call's P x P pair Gram; returns the 32-bit swap mask.
+template <typename T>
+__device__ __forceinline__ uint32_t walk_block(const T *__restrict__ Fg, int P, int i0, int cnt,
+                                               T alpha, T r, T U, T logfac, T &bmax, int lane)
+{
+    T Fd[32];
+    T b2 = 0;
+#pragma unroll
+    for (int t = 0; t < 32; ++t) {
+        T v = 0;
+        if (t <= lane && lane < cnt) v = Fg[(int64_t)(i0 + t) * P + i0 + lane];
+        Fd[t] = v;
+        if (t == lane) b2 = v;
+    }
+    T b = sqrt(b2 > 0 ? b2 : (T)0);
+    // b_{max,i} for every lane (independent of the decisions)
+    T my_bmax = 0;
+#pragma unroll
+    for (int t = 0; t < 32; ++t) {
+        T bt = __shfl_sync(0xffffffffu, b, t);
+        T rt = __shfl_sync(0xffffffffu, r, t);
+        if (t < cnt) {
+            T carried = bmax * rt;
+            bmax = bt > carried ? bt : carried;
+        }
+        if (t == lane) my_bmax = bmax;
+    }
+    const T a = b * my_bmax * logfac;
+    uint32_t swaps = 0;
+#pragma unroll
+    for (int t = 0; t < 32; ++t) {
+        bool mine = (lane == t) && (t < cnt) && swap_decision(alpha, a, U);
+        uint32_t sw = (__ballot_sync(0xffffffffu, mine) >> t) & 1u;
+        swaps |= sw << t;
+        // alpha_i = -sum_j eta_j F[j,i]: a kept pair (eta = +1) subtracts, a swapped one adds
+        alpha += sw ? Fd[t] : -Fd[t];
+    }
+    return swaps;
+}
+
+// Calls with at least 32 pairs: one CTA of 8 warps per call.
+template <typename T>
+__global__ void __launch_bounds__(256) walk_cta_kernel(const T *__restrict__ F, int64_t F_stride,
+                                                       const T *__restrict__ rdecay,
+                                                       const int32_t *__restrict__ cur,
+                                                       int32_t *__restrict__ out, int64_t out_stride,
+                                                       int64_t n, int P, int level, uint64_t seed,
+                                                       T logfac)
+{
+    extern __shared__ unsigned char smem_raw[];
+    T *eta = reinterpret_cast<T *>(smem_raw);      // [P]
+    T *part = eta + P;                             // [8][32]
+    const int p = blockIdx.y, g = blockIdx.x;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const T *Fg = F + (int64_t)p * F_stride + (int64_t)g * P * P;
+    const int64_t base = (int64_t)g * P;
+    T bmax = 0;
+    for (int c = 0; c < P / 32; ++c) {
+        const int i0 = 32 * c;
+        T acc = 0;
+        for (int j = warp; j < i0; j += 8) acc += eta[j] * Fg[(int64_t)j * P + i0 + lane];
+        part[warp * 32 + lane] = acc;
+        __syncthreads();
+        if (warp == 0) {
+            T alpha = 0;
+#pragma unroll
+            for (int w = 0; w < 8; ++w) alpha -= part[w * 32 + lane];
+            const T r = rdecay[(int64_t)p * (n / 2) + base + i0 + lane];
+            const T U = halving_uniform<T>(seed, (uint32_t)(i0 + lane), (uint32_t)g, (uint32_t)level, (uint32_t)p);
+            uint32_t swaps = walk_block<T>(Fg, P, i0, 32, alpha, r, U, logfac, bmax, lane);
+            const uint32_t sw = (swaps >> lane) & 1u;
+            eta[i0 + lane] = sw ? (T)-1 : (T)1;
+            out[(int64_t)p * out_stride + base + i0 + lane] = cur[(int64_t)p * n + 2 * (base + i0 + lane) + sw];
+        }
+        __syncthreads();
+    }
+}
+
+// Calls with fewer than 32 pairs: one warp per call, 8 calls per CTA.
+template <typename T>
+__global__ void __launch_bounds__(256) walk_warp_kernel(const T *__restrict__ F, int64_t F_stride,
+                                                        const T *__restrict__ rdecay,
+                                                        const int32_t *__restrict__ cur,
+                                                        int32_t *__restrict__ out, int64_t out_stride,
+                                                        int64_t n, int P, int groups, int level,
+                                                        uint64_t seed, T logfac)
+{
+    const int p = blockIdx.y;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int g = blockIdx.x * 8 + warp;
+    if (g >= groups) return;
+    const T *Fg = F + (int64_t)p * F_stride + (int64_t)g * P * P;
+    const int64_t base = (int64_t)g * P;
+    T bmax = 0;
+    const bool live = lane < P;
+    const T r = live ? rdecay[(int64_t)p * (n / 2) + base + lane] : (T)1;
+    const T U = halving_uniform<T>(seed, (uint32_t)lane, (uint32_t)g, (uint32_t)level, (uint32_t)p);
+    uint32_t swaps = walk_block<T>(Fg, P, 0, P, (T)0, r, U, logfac, bmax, lane);
+    if (live) {
+        const uint32_t sw = (swaps >> lane) & 1u;
+        out[(int64_t)p * out_stride + base + lane] = cur[(int64_t)p * n + 2 * (base + lane) + sw];
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Stage emit: weights 1/n_out (Definition 1: positive, summing to 1); identity list when m = 0
+// ---------------------------------------------------------------------------------------------
+__global__ void emit_kernel(float *__restrict__ w, int32_t *__restrict__ idx, int64_t total,
+                            int64_t n_out, int write_identity)
+{
+    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= total) return;
+    w[i] = 1.0f / (float)n_out;
+    if (write_identity) idx[i] = (int32_t)(i % n_out);
+}
+
+// ---------------------------------------------------------------------------------------------
+// workspace layout and the level scheduler
+// ---------------------------------------------------------------------------------------------
+CompressLayout compress_layout(const elm_params *p)
+{
+    CompressLayout L;
+    const size_t ts = p->precision == ELM_PREC_FP64_DET ? 8 : 4;
+    const size_t BH = (size_t)p->batch * p->kv_heads;
+    const size_t n = (size_t)p->n_kv;
+    const size_t n_out = (size_t)1 << p->log2_nout;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+    L.vmax_bits = take(BH * 4);
+    L.cnorm = take(BH * n * ts);
+    L.cur = take(BH * n * 4);
+    L.nxt = take(BH * n * 4);
+    L.Mpair = take(BH * (n / 2 + 1) * ts);
+    L.rdecay = take(BH * (n / 2 + 1) * ts);
+    L.F_stride = n_out * n_out;
+    L.F = take(p->m > 0 ? BH * L.F_stride * ts : 0);
+    L.total = off;
+    return L;
+}
+
+template <typename Tin, typename T>
+static int run_gram_simt(const Tin *K, const Tin *V, const elm_params *p, const int32_t *cur,
+                         const T *Mpair, const unsigned *vmax_bits, int P, int64_t Ptotal, int groups,
+                         T *F, int64_t F_stride, cudaStream_t st)
+{
+    const int BH = p->batch * p->kv_heads;
+    int64_t tiles;
+    if (P >= 32) {
+        const int Tg = P / 32;
+        tiles = (int64_t)groups * (Tg * (Tg + 1) / 2);
+    } else {
+        tiles = (Ptotal + 31) / 32;
+    }
+    dim3 grid((unsigned)tiles, (unsigned)BH);
+    if (p->d == 64)
+        gram_simt_kernel<Tin, T, 64><<<grid, 256, 0, st>>>(K, V, cur, Mpair, vmax_bits, p->n_kv, P, Ptotal, F, F_stride);
+    else
+        gram_simt_kernel<Tin, T, 128><<<grid, 256, 0, st>>>(K, V, cur, Mpair, vmax_bits, p->n_kv, P, Ptotal, F, F_stride);
+    count_launches(1);
+    return cuda_status(cudaGetLastError());
+}
+
+template <typename Tin, typename T>
+static int compress_impl(const Tin *K, const Tin *V, const elm_params *p, uint64_t seed,
+                         int32_t *idx_out, float *w_out, unsigned char *ws, cudaStream_t st)
+{
+    const CompressLayout L = compress_layout(p);
+    const int BH = p->batch * p->kv_heads;
+    const int64_t n = p->n_kv;
+    const int64_t n_out = (int64_t)1 << p->log2_nout;
+    const int m = p->m;
+    unsigned *vmax_bits = reinterpret_cast<unsigned *>(ws + L.vmax_bits);
+    T *cnorm = reinterpret_cast<T *>(ws + L.cnorm);
+    int32_t *cur = reinterpret_cast<int32_t *>(ws + L.cur);
+    int32_t *nxt = reinterpret_cast<int32_t *>(ws + L.nxt);
+    T *Mpair = reinterpret_cast<T *>(ws + L.Mpair);
+    T *rdecay = reinterpret_cast<T *>(ws + L.rdecay);
+    T *F = reinterpret_cast<T *>(ws + L.F);
+
+    double dl[32];
+    if (p->delta_level) {
+        for (int i = 0; i < m; ++i) dl[i] = p->delta_level[i];
+    } else {
+        elm_default_delta_levels(m, p->delta, dl);
+    }
+
+    if (m > 0) {
+        StageTimer t(ELM_STAGE_PREPASS, st, 1);
+        ELM_CUDA_TRY(cudaMemsetAsync(vmax_bits, 0, (size_t)BH * 4, st));
+        dim3 grid((unsigned)((n + 63) / 64), (unsigned)BH);
+        prepass_kernel<Tin, T><<<grid, 256, 0, st>>>(K, V, n, p->d, cnorm, vmax_bits, cur);
+        count_launches(1);
+        ELM_CUDA_TRY(cudaGetLastError());
+    }
+    for (int level = 0; level < m; ++level) {
+        const int64_t len = n >> level;                            // points alive
+        const int groups = 1 << (2 * (m - 1 - level));             // 4^(m-1-level) Halve calls
+        const int64_t s = len / groups;                            // points per call
+        const int P = (int)(s / 2);
+        const int64_t Ptotal = len / 2;
+        const T logfac = (T)(0.5 + log(2.0 * (double)s / dl[level]));
+        const bool last = level == m - 1;
+        int32_t *out = last ? idx_out : nxt;
+        const int64_t out_stride = last ? n_out : n;
+        {
+            StageTimer t(ELM_STAGE_LEVEL_PREP, st, 1);
+            level_prep_kernel<T><<<dim3((unsigned)groups, (unsigned)BH), 128, 0, st>>>(cnorm, cur, n, P, Mpair, rdecay);
+            count_launches(1);
+            ELM_CUDA_TRY(cudaGetLastError());
+        }
+        {
+            StageTimer t(ELM_STAGE_GRAM, st, 1);
+            int rc = run_gram_simt<Tin, T>(K, V, p, cur, Mpair, vmax_bits, P, Ptotal, groups, F, L.F_stride, st);
+            if (rc != ELM_OK) return rc;
+        }
+        {
+            StageTimer t(ELM_STAGE_WALK, st, 1);
+            if (P >= 32) {
+                size_t smem = ((size_t)P + 256) * sizeof(T);
+                walk_cta_kernel<T><<<dim3((unsigned)groups, (unsigned)BH), 256, smem, st>>>(
+                    F, L.F_stride, rdecay, cur, out, out_stride, n, P, level, seed, logfac);
+            } else {
+                walk_warp_kernel<T><<<dim3((unsigned)((groups + 7) / 8), (unsigned)BH), 256, 0, st>>>(
+                    F, L.F_stride, rdecay, cur, out, out_stride, n, P, groups, level, seed, logfac);
+            }
+            count_launches(1);
+            ELM_CUDA_TRY(cudaGetLastError());
+        }
+        int32_t *tmp = cur; cur = nxt; nxt = tmp;
+    }
+    {
+        StageTimer t(ELM_STAGE_EMIT, st, 1);
+        const int64_t total = (int64_t)BH * n_out;
+        emit_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(w_out, idx_out, total, n_out, m == 0);
+        count_launches(1);
+        ELM_CUDA_TRY(cudaGetLastError());
+    }
+    return ELM_OK;
+}
+
+}  // namespace elm
+
+extern "C" int elm_compress(const void *K, const void *V, const elm_params *params, uint64_t seed,
+                            int32_t *idx_out, float *w_out, void *workspace, size_t workspace_bytes,
+                            void *stream)
+{
+    using namespace elm;
+    if (!params) return ELM_ERR_NULL;
+    int rc = validate_params(params);
+    if (rc != ELM_OK) return rc;
+    if (!K || !V || !idx_out || !w_out || !workspace) return ELM_ERR_NULL;
+    if (((uintptr_t)K | (uintptr_t)V | (uintptr_t)idx_out | (uintptr_t)w_out) & 15) return ELM_ERR_ALIGN;
+    if ((uintptr_t)workspace & 255) return ELM_ERR_ALIGN;
+    if (workspace_bytes < compress_layout(params).total) return ELM_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    unsigned char *ws = (unsigned char *)workspace;
+    const bool det = params->precision == ELM_PREC_FP64_DET;
+    if (params->dtype == ELM_F32) {
+        return det ? compress_impl<float, double>((const float *)K, (const float *)V, params, seed, idx_out, w_out, ws, st)
+                   : compress_impl<float, float>((const float *)K, (const float *)V, params, seed, idx_out, w_out, ws, st);
+    }
+    return det ? compress_impl<__nv_bfloat16, double>((const __nv_bfloat16 *)K, (const __nv_bfloat16 *)V, params, seed, idx_out, w_out, ws, st)
+               : compress_impl<__nv_bfloat16, float>((const __nv_bfloat16 *)K, (const __nv_bfloat16 *)V, params, seed, idx_out, w_out, ws, st);
+}

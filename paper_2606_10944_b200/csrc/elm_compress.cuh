@@ -1,0 +1,23 @@
+// Workspace layout of elm_compress (byte offsets into the caller's workspace).
+#pragma once
+#include <stddef.h>
+#include <stdint.h>
+
+#include "../../include/elm.h"
+
+namespace elm {
+
+struct CompressLayout {
+    size_t vmax_bits;  // [BH] float bits of v_max per attention problem
+    size_t cnorm;      // [BH][n]   c_t = ||k_t||^2 / sqrt(d)
+    size_t cur;        // [BH][n]   current point sequence (row numbers)
+    size_t nxt;        // [BH][n]   next level's sequence
+    size_t Mpair;      // [BH][n/2] running shift of each pair
+    size_t rdecay;     // [BH][n/2] exp(-(M_i - M_{i-1})/2)
+    size_t F;          // [BH][n_out^2] pair Gram of the current level (all calls)
+    size_t F_stride;   // elements per problem
+    size_t total;
+};
+CompressLayout compress_layout(const elm_params *p);
+
+}  // namespace elm
