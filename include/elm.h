@@ -53,7 +53,8 @@ typedef enum {
     ELM_ERR_WORKSPACE = -5,   /* workspace too small */
     ELM_ERR_DELTA = -6,       /* a failure parameter outside (0, 1) */
     ELM_ERR_CUDA = -7,        /* a CUDA runtime call or launch failed */
-    ELM_ERR_UNAVAILABLE = -8  /* no usable CUDA device */
+    ELM_ERR_UNAVAILABLE = -8, /* no usable CUDA device */
+    ELM_ERR_STATIC_LIMIT = -9 /* elm_attend_static: the coreset does not fit the built-in scratch */
 } elm_status;
 
 typedef struct elm_params {
@@ -115,6 +116,36 @@ int elm_attend(const void *Q, const void *K, const void *V, const int32_t *idx, 
 
 /* Workspace of elm_attend for an explicit coreset size. */
 int elm_attend_workspace_bytes(const elm_params *params, int32_t n_core, size_t *bytes);
+
+/*
+ * elm_attend for callers that cannot hand over a workspace.  (The paper has no counterpart: this
+ * is a packaging variant of elm_attend, same arithmetic, same kernels.)
+ *
+ * Who needs it: code that runs after a serving process has given all device memory to its own
+ * pool, plug-ins that are forbidden to call the CUDA allocator on the request path (an allocation
+ * there can stall every stream of the process or fail outright when the pool owns the card), and
+ * embedders that only hold raw pointers to Q/K/V/O and have nowhere to carve a workspace from.
+ * This entry point calls no cudaMalloc, cudaFree or any other allocating routine, and takes no
+ * workspace argument.  The gathered coreset operands are staged in an array of
+ * ELM_ATTEND_STATIC_SCRATCH_BYTES that is compiled into the library as device global memory;
+ * every GPU that loads the library holds that array until the process exits.
+ *
+ * Arguments, layouts, dtype / precision handling and results are those of elm_attend.
+ * Limits and rules:
+ *   - elm_attend_workspace_bytes(params, n_core) must not exceed ELM_ATTEND_STATIC_SCRATCH_BYTES
+ *     (e.g. 8 KV problems x 2048 coreset points x d = 128 in bf16 needs about 8.1 MiB); larger
+ *     requests return ELM_ERR_STATIC_LIMIT before anything is launched.
+ *   - The first call on each device looks up the array's device address (once per device, with
+ *     that device current).  Make that first call outside any stream capture.
+ *   - All calls on a device share the one array and it keeps the previous call's contents.  Each
+ *     call rewrites every byte it later reads, so nothing needs clearing, but two calls whose
+ *     kernels can overlap on the GPU (different streams, no ordering between them) race on it:
+ *     order them, or use elm_attend with separate workspaces.
+ *   - Per-stage timing (elm_profile_enable) does not cover this entry point.
+ */
+#define ELM_ATTEND_STATIC_SCRATCH_BYTES (16u << 20)
+int elm_attend_static(const void *Q, const void *K, const void *V, const int32_t *idx, const float *w,
+                      int32_t n_core, const elm_params *params, void *O, void *stream);
 
 /*
  * End-to-end convenience call on HOST buffers: copies Q, K, V to the device, runs elm_compress and

@@ -20,7 +20,7 @@ STAGE_NAMES = ["prepass", "level_prep", "gram", "walk", "emit", "gather", "atten
 
 EXPORTED_SYMBOLS = [
     "elm_workspace_bytes", "elm_default_delta_levels", "elm_compress", "elm_attend",
-    "elm_attend_workspace_bytes", "elm_host_call_scratch_bytes", "elm_compress_attend_host",
+    "elm_attend_workspace_bytes", "elm_attend_static", "elm_host_call_scratch_bytes", "elm_compress_attend_host",
     "elm_profile_enable", "elm_profile_read", "elm_launch_count", "elm_strerror", "elm_version",
 ]
 
@@ -63,6 +63,7 @@ def load_library():
     lib.elm_compress.argtypes = [vp, vp, pp, ctypes.c_uint64, vp, vp, vp, sz, vp]
     lib.elm_attend.argtypes = [vp, vp, vp, vp, vp, ctypes.c_int32, pp, vp, vp, sz, vp]
     lib.elm_attend_workspace_bytes.argtypes = [pp, ctypes.c_int32, szp]
+    lib.elm_attend_static.argtypes = [vp, vp, vp, vp, vp, ctypes.c_int32, pp, vp, vp]
     lib.elm_host_call_scratch_bytes.argtypes = [pp, szp]
     lib.elm_compress_attend_host.argtypes = [vp, vp, vp, vp, vp, vp, pp, ctypes.c_uint64, vp, sz, vp]
     lib.elm_profile_enable.argtypes = [ctypes.c_int]
@@ -177,6 +178,31 @@ def attend(Q, K, V, idx, w, precision="fp32", workspace=None, out=None):
     _check(lib.elm_attend(Q.data_ptr(), K.data_ptr(), V.data_ptr(), idx.data_ptr(), w.data_ptr(),
                           n_core, ctypes.byref(p), O.data_ptr(), ws.data_ptr(), ws.numel(), _stream()),
            "elm_attend")
+    return O
+
+
+ATTEND_STATIC_SCRATCH_BYTES = 16 << 20
+
+
+def attend_static(Q, K, V, idx, w, precision="fp32", out=None):
+    """elm_attend_static: elm_attend without a workspace argument.
+
+    For callers that may not allocate device memory: the coreset operands are staged in a
+    fixed array inside the library (ATTEND_STATIC_SCRATCH_BYTES), so this wrapper allocates
+    nothing when ``out`` is supplied.  Calls on one device share that array; do not let two of
+    them overlap on the GPU.
+    """
+    lib = load_library()
+    _require_cuda(Q, K, V, idx, w)
+    B, Hq, nq, d = Q.shape
+    Hkv, n = K.shape[1], K.shape[2]
+    if idx.dtype != torch.int32 or w.dtype != torch.float32:
+        raise ElmError("idx must be int32 and w float32")
+    p, _ = make_params(B, Hq, Hkv, n, nq, d, n.bit_length() - 1, 0, _dtype_code(Q), precision)
+    O = out if out is not None else torch.empty_like(Q)
+    _check(lib.elm_attend_static(Q.data_ptr(), K.data_ptr(), V.data_ptr(), idx.data_ptr(), w.data_ptr(),
+                                 idx.shape[-1], ctypes.byref(p), O.data_ptr(), _stream()),
+           "elm_attend_static")
     return O
 
 

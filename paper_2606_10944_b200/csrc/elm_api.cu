@@ -201,6 +201,7 @@ extern "C" const char *elm_strerror(int status)
     case ELM_ERR_DELTA: return "failure parameter outside (0, 1)";
     case ELM_ERR_CUDA: return "a CUDA call or kernel launch failed";
     case ELM_ERR_UNAVAILABLE: return "no usable CUDA device";
+    case ELM_ERR_STATIC_LIMIT: return "coreset operands exceed the built-in static scratch (use elm_attend with a workspace)";
     default: return "unknown status";
     }
 }

@@ -6,6 +6,8 @@
 // fp32 mode take the tensor-core kernel in elm_attend_tc.cu.
 #include <math.h>
 
+#include <mutex>
+
 #include "elm_attend.cuh"
 #include "elm_common.cuh"
 
@@ -212,6 +214,57 @@ static int attend_impl(const Tin *Q, const Tin *K, const Tin *V, const int32_t *
     return launch_attend_simt<Tin, T, 128>(Q, Kc, Vc, bias, O, p, n_core, st);
 }
 
+
+// ---------------------------------------------------------------------------------------------
+// Built-in scratch for elm_attend_static.  The array lives in every GPU that loads this library
+// until the process exits.  Its name is only a host-side handle: the device address is looked
+// up once per device with cudaGetSymbolAddress and that address is what the kernels receive.
+// ---------------------------------------------------------------------------------------------
+}  // namespace elm
+
+static __device__ __align__(256) unsigned char g_attend_static_scratch[ELM_ATTEND_STATIC_SCRATCH_BYTES];
+
+namespace elm {
+
+static std::mutex g_static_mutex;
+static unsigned char *g_static_addr[64];    // device address of the array, per device ordinal
+
+static int static_scratch_address(unsigned char **out)
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return ELM_ERR_UNAVAILABLE;
+    if (dev < 0 || dev >= 64) return ELM_ERR_UNAVAILABLE;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_addr[dev]) {
+        void *addr = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(&addr, g_attend_static_scratch);
+        if (e != cudaSuccess || addr == nullptr) return ELM_ERR_CUDA;
+        g_static_addr[dev] = static_cast<unsigned char *>(addr);
+    }
+    *out = g_static_addr[dev];
+    return ELM_OK;
+}
+
+// Same two launches as attend_impl, without the event-based stage timers (creating an event may
+// allocate) and with the gathered operands placed in `scratch`.
+template <typename Tin, typename T>
+static int attend_enqueue_untimed(const Tin *Q, const Tin *K, const Tin *V, const int32_t *idx,
+                                  const float *w, int n_core, const elm_params *p, Tin *O,
+                                  unsigned char *scratch, cudaStream_t st)
+{
+    const AttendLayout L = attend_layout(p, n_core);
+    Tin *Kc = reinterpret_cast<Tin *>(scratch + L.Kc);
+    Tin *Vc = reinterpret_cast<Tin *>(scratch + L.Vc);
+    float *bias = reinterpret_cast<float *>(scratch + L.bias);
+    const int problems = p->batch * p->kv_heads;
+    gather_kernel<Tin><<<dim3((unsigned)((n_core + 7) / 8), (unsigned)problems), 256, 0, st>>>(
+        K, V, idx, w, p->n_kv, p->d, n_core, Kc, Vc, bias);
+    count_launches(1);
+    ELM_CUDA_TRY(cudaGetLastError());
+    if (p->d == 64) return launch_attend_simt<Tin, T, 64>(Q, Kc, Vc, bias, O, p, n_core, st);
+    return launch_attend_simt<Tin, T, 128>(Q, Kc, Vc, bias, O, p, n_core, st);
+}
+
 }  // namespace elm
 
 extern "C" int elm_attend_workspace_bytes(const elm_params *params, int32_t n_core, size_t *bytes)
@@ -249,4 +302,31 @@ extern "C" int elm_attend(const void *Q, const void *K, const void *V, const int
     typedef __nv_bfloat16 bf;
     return det ? attend_impl<bf, double>((const bf *)Q, (const bf *)K, (const bf *)V, idx, w, n_core, params, (bf *)O, ws, st)
                : attend_impl<bf, float>((const bf *)Q, (const bf *)K, (const bf *)V, idx, w, n_core, params, (bf *)O, ws, st);
+}
+
+extern "C" int elm_attend_static(const void *Q, const void *K, const void *V, const int32_t *idx,
+                                 const float *w, int32_t n_core, const elm_params *params, void *O,
+                                 void *stream)
+{
+    using namespace elm;
+    if (!params) return ELM_ERR_NULL;
+    int rc = validate_params(params);
+    if (rc != ELM_OK) return rc;
+    if (!Q || !K || !V || !idx || !w || !O) return ELM_ERR_NULL;
+    if (n_core < 1 || n_core > params->n_kv) return ELM_ERR_SHAPE;
+    if (((uintptr_t)Q | (uintptr_t)K | (uintptr_t)V | (uintptr_t)idx | (uintptr_t)w | (uintptr_t)O) & 15)
+        return ELM_ERR_ALIGN;
+    if (attend_layout(params, n_core).total > (size_t)ELM_ATTEND_STATIC_SCRATCH_BYTES) return ELM_ERR_STATIC_LIMIT;
+    unsigned char *scratch = nullptr;
+    rc = static_scratch_address(&scratch);
+    if (rc != ELM_OK) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    const bool det = params->precision == ELM_PREC_FP64_DET;
+    if (params->dtype == ELM_F32) {
+        return det ? attend_enqueue_untimed<float, double>((const float *)Q, (const float *)K, (const float *)V, idx, w, n_core, params, (float *)O, scratch, st)
+                   : attend_enqueue_untimed<float, float>((const float *)Q, (const float *)K, (const float *)V, idx, w, n_core, params, (float *)O, scratch, st);
+    }
+    typedef __nv_bfloat16 bf;
+    return det ? attend_enqueue_untimed<bf, double>((const bf *)Q, (const bf *)K, (const bf *)V, idx, w, n_core, params, (bf *)O, scratch, st)
+               : attend_enqueue_untimed<bf, float>((const bf *)Q, (const bf *)K, (const bf *)V, idx, w, n_core, params, (bf *)O, scratch, st);
 }
