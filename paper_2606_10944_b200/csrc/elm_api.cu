@@ -24,6 +24,7 @@ void count_launches(int n) { g_launches.fetch_add(n, std::memory_order_relaxed);
 
 StageTimer::StageTimer(int stage, cudaStream_t stream, int launches) : stream_(stream)
 {
+    if (stage < 0) return;      // untimed caller
     Profiler &pr = profiler();
     g_stage_launches[stage] += launches;
     if (!pr.enabled || pr.n_records >= Profiler::kMaxRecords) return;

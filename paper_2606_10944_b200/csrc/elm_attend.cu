@@ -7,6 +7,7 @@
 #include <math.h>
 
 #include <mutex>
+#include <type_traits>
 
 #include "elm_attend.cuh"
 #include "elm_common.cuh"
@@ -172,9 +173,11 @@ AttendLayout attend_layout(const elm_params *p, int32_t n_core)
     const size_t es = elt_bytes(p->dtype);
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
-    L.Kc = take(problems * (size_t)n_core * p->d * es);
-    L.Vc = take(problems * (size_t)n_core * p->d * es);
-    L.bias = take(problems * (size_t)n_core * 4);
+    const size_t n_pad = ((size_t)n_core + 127) / 128 * 128;      // the tensor-core path pads to its block size
+    L.Kc = take(problems * n_pad * p->d * es);
+    L.Vc = take(problems * n_pad * p->d * es);
+    L.bias = take(problems * n_pad * 4);
+    L.flags = take((problems + 1) * 4);
     L.total = off;
     return L;
 }
@@ -197,6 +200,8 @@ template <typename Tin, typename T>
 static int attend_impl(const Tin *Q, const Tin *K, const Tin *V, const int32_t *idx, const float *w,
                        int n_core, const elm_params *p, Tin *O, unsigned char *ws, cudaStream_t st)
 {
+    if constexpr (std::is_same<Tin, __nv_bfloat16>::value && std::is_same<T, float>::value)
+        return attend_tc(Q, K, V, idx, w, n_core, p, O, ws, st, true);
     const AttendLayout L = attend_layout(p, n_core);
     Tin *Kc = reinterpret_cast<Tin *>(ws + L.Kc);
     Tin *Vc = reinterpret_cast<Tin *>(ws + L.Vc);
@@ -252,6 +257,8 @@ static int attend_enqueue_untimed(const Tin *Q, const Tin *K, const Tin *V, cons
                                   const float *w, int n_core, const elm_params *p, Tin *O,
                                   unsigned char *scratch, cudaStream_t st)
 {
+    if constexpr (std::is_same<Tin, __nv_bfloat16>::value && std::is_same<T, float>::value)
+        return attend_tc(Q, K, V, idx, w, n_core, p, O, scratch, st, false);
     const AttendLayout L = attend_layout(p, n_core);
     Tin *Kc = reinterpret_cast<Tin *>(scratch + L.Kc);
     Tin *Vc = reinterpret_cast<Tin *>(scratch + L.Vc);

@@ -1,0 +1,567 @@
+// Weighted attention over a coreset on the sm_100a tensor cores (bf16 inputs, fp32 accumulation).
+//
+//   O[j,:] = sum_c w_c exp(<q_j,k_c>/sqrt(d)) v_c / sum_c w_c exp(<q_j,k_c>/sqrt(d))      Eq. (def:att_approx)
+//
+// One CTA owns two tiles of 128 queries of one head and streams the head's coreset in blocks of
+// 128 points.  Roles (320 threads):
+//   warps 0-3 / 4-7  softmax of query tile 0 / 1: read the logits from TMEM (one row per thread),
+//                    keep a running row maximum and denominator, write the probabilities back to
+//                    TMEM as packed bf16 (they overwrite the logits), rescale the output
+//                    accumulator only when the maximum grew by more than 2^8, and run the epilogue
+//   warp 8           TMA producer: Q tiles once, then K / V^T blocks through a 2-stage ring
+//   warp 9           tcgen05.mma issuer: S = Q K^T (operands in shared memory), O += P V (P read
+//                    from TMEM, V^T from shared memory); owns the TMEM allocation
+// TMEM columns: [0,128) S/P of tile 0, [128,256) S/P of tile 1, [256,256+D) O of tile 0,
+// [384,384+D) O of tile 1.  Every mbarrier wait is bounded; on expiry the CTA records a status
+// word and leaves through the common exit, which frees the TMEM it holds.
+#include <cuda.h>
+#include <math.h>
+
+#include "elm_attend.cuh"
+#include "elm_common.cuh"
+
+namespace elm {
+namespace tc {
+
+constexpr int BM = 128;          // query rows per tile (= TMEM lanes)
+constexpr int BN = 128;          // coreset points per block
+constexpr int STAGES = 2;
+constexpr int NTHREADS = 320;
+constexpr uint32_t TMEM_COLS = 512;
+constexpr float RESCALE_TAU = 8.0f;      // rescale the accumulator only if the max grew by > 2^8
+
+// ---- PTX wrappers ---------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.b32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait: gives up after ~2 s of wall time.
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    uint64_t t0;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t0));
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 2048; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+        uint64_t t1;
+        asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t1));
+        if (t1 - t0 > 2000000000ull) return false;
+    }
+}
+__device__ __forceinline__ void fence_barrier_init()
+{
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void tma_load_3d(void *dst, const CUtensorMap *map, uint64_t *bar, int c0, int c1, int c2)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2)
+        : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint64_t *bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]^T, both operands K-major
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem]^T
+__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// 32 lanes x 32 consecutive 32-bit columns: thread i of the warp gets lane (base + i)
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31};"
+        ::"r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+          "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+          "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+          "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31]),
+          "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ float fast_exp2(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
+{
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
+// Shared-memory operand descriptor: K-major tile of rows x 64 bf16 (128 B per row), 128-byte
+// swizzle as written by TMA; 8-row groups are 1024 B apart.
+__device__ __forceinline__ uint64_t umma_desc_k128(uint32_t smem_addr)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3FFFF) >> 4);       // start address
+    d |= (uint64_t)1 << 16;                            // leading byte offset (unused for swizzled K-major)
+    d |= (uint64_t)(1024 >> 4) << 32;                  // stride byte offset
+    d |= (uint64_t)1 << 46;                            // descriptor version (sm_100)
+    d |= (uint64_t)2 << 61;                            // SWIZZLE_128B
+    return d;
+}
+// kind::f16 instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M x N tile
+__host__ __device__ constexpr uint32_t umma_idesc_bf16(int M, int N)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
+struct __align__(8) Barriers {
+    uint64_t q_full;
+    uint64_t k_full[STAGES], v_full[STAGES], k_empty[STAGES], v_empty[STAGES];
+    uint64_t s_full[2], p_ready[2], o_done[2];
+    uint32_t tmem_base;
+    uint32_t abort_flag;
+};
+
+template <int D> struct Smem {
+    static constexpr int KH = D / 64;                       // 64-element halves of the head dimension
+    static constexpr int Q_TILE = BM * D * 2;               // bytes
+    static constexpr int K_BLOCK = BN * D * 2;
+    static constexpr int V_BLOCK = D * BN * 2;
+    static constexpr int OFF_Q = 0;
+    static constexpr int OFF_K = OFF_Q + 2 * Q_TILE;
+    static constexpr int OFF_V = OFF_K + STAGES * K_BLOCK;
+    static constexpr int OFF_BAR = OFF_V + STAGES * V_BLOCK;
+    static constexpr int TOTAL = OFF_BAR + 256 + 1024;      // + slack for 1024-byte alignment
+};
+
+// ---------------------------------------------------------------------------------------------
+// gather for the tensor-core path: Kc [p][n_pad][D] (zero rows beyond n_core), Vt [p][D][n_pad]
+// (transposed, zero columns beyond n_core), bias = log2 w, and a per-problem flag that says
+// whether all weights of the problem are equal (then the bias cancels in the ratio).
+// ---------------------------------------------------------------------------------------------
+template <int D>
+__global__ void __launch_bounds__(256) gather_tc_kernel(const __nv_bfloat16 *__restrict__ K,
+                                                        const __nv_bfloat16 *__restrict__ V,
+                                                        const int32_t *__restrict__ idx,
+                                                        const float *__restrict__ w, int64_t n, int n_core,
+                                                        int n_pad, __nv_bfloat16 *__restrict__ Kc,
+                                                        __nv_bfloat16 *__restrict__ Vt,
+                                                        float *__restrict__ bias, int *__restrict__ nonuniform)
+{
+    __shared__ __nv_bfloat16 tile[32][D + 2];
+    const int p = blockIdx.y;
+    const int c0 = blockIdx.x * 32;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const float w0 = w[(int64_t)p * n_core];
+    bool differs = false;
+    for (int r = warp; r < 32; r += 8) {
+        const int c = c0 + r;
+        const bool ok = c < n_core;
+        const int64_t row = ok ? idx[(int64_t)p * n_core + c] : 0;
+        const __nv_bfloat16 *ks = K + ((int64_t)p * n + row) * D;
+        const __nv_bfloat16 *vs = V + ((int64_t)p * n + row) * D;
+        __nv_bfloat16 *kd = Kc + ((int64_t)p * n_pad + c) * D;
+        for (int e = lane; e < D; e += 32) {
+            kd[e] = ok ? ks[e] : __float2bfloat16(0.f);
+            tile[r][e] = ok ? vs[e] : __float2bfloat16(0.f);
+        }
+        if (lane == 0) {
+            float wc = ok ? w[(int64_t)p * n_core + c] : 0.f;
+            bias[(int64_t)p * n_pad + c] = ok ? log2f(wc) : -INFINITY;
+            if (ok && wc != w0) differs = true;
+        }
+    }
+    if (differs) atomicOr(nonuniform + p, 1);
+    __syncthreads();
+    // transposed write: thread -> (dimension e, point r) with r fastest
+    for (int i = threadIdx.x; i < 32 * D; i += 256) {
+        const int e = i >> 5, r = i & 31;
+        Vt[((int64_t)p * D + e) * n_pad + c0 + r] = tile[r][e];
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// the attention kernel
+// ---------------------------------------------------------------------------------------------
+template <int D>
+__global__ void __launch_bounds__(NTHREADS, 1)
+attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
+                 const __grid_constant__ CUtensorMap mapV, const float *__restrict__ bias,
+                 const int *__restrict__ nonuniform, __nv_bfloat16 *__restrict__ O, int q_heads,
+                 int kv_heads, int n_q, int n_core, int n_pad, float scale_log2, int *__restrict__ status)
+{
+    using SM = Smem<D>;
+    constexpr int KH = SM::KH;
+    extern __shared__ unsigned char smem_dyn[];
+    unsigned char *smem = reinterpret_cast<unsigned char *>(((uintptr_t)smem_dyn + 1023) & ~(uintptr_t)1023);
+    Barriers *bar = reinterpret_cast<Barriers *>(smem + SM::OFF_BAR);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int bh = blockIdx.y;
+    const int b = bh / q_heads, h = bh % q_heads;
+    const int prob = b * kv_heads + (int)(((int64_t)h * kv_heads) / q_heads);
+    const int q0 = blockIdx.x * (2 * BM);
+    const int nblk = n_pad / BN;
+
+    // a CTA that gave up on a wait poisons the launch: the remaining CTAs leave at once
+    if (*reinterpret_cast<volatile int *>(status) != 0) return;
+
+    if (threadIdx.x == 0) {
+        mbar_init(&bar->q_full, 1);
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(&bar->k_full[s], 1);
+            mbar_init(&bar->v_full[s], 1);
+            mbar_init(&bar->k_empty[s], 1);
+            mbar_init(&bar->v_empty[s], 1);
+        }
+        for (int t = 0; t < 2; ++t) {
+            mbar_init(&bar->s_full[t], 1);
+            mbar_init(&bar->p_ready[t], 128);
+            mbar_init(&bar->o_done[t], 1);
+        }
+        bar->abort_flag = 0;
+        fence_barrier_init();
+    }
+    if (warp == 9) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&bar->tmem_base)), "r"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = bar->tmem_base;
+
+    if (warp == 8) {
+        // ------------------------------ TMA producer ------------------------------
+        if (lane == 0) {
+            mbar_expect_tx(&bar->q_full, 2 * SM::Q_TILE);
+            for (int t = 0; t < 2; ++t)
+                for (int kh = 0; kh < KH; ++kh)
+                    tma_load_3d(smem + SM::OFF_Q + t * SM::Q_TILE + kh * (BM * 128), &mapQ, &bar->q_full, kh * 64, q0 + t * BM, bh);
+            bool ok = true;
+            for (int j = 0; j < nblk && ok; ++j) {
+                const int s = j % STAGES;
+                const uint32_t ph = (uint32_t)(j / STAGES) & 1u;
+                ok = mbar_wait(&bar->k_empty[s], ph ^ 1u);
+                if (!ok) break;
+                mbar_expect_tx(&bar->k_full[s], SM::K_BLOCK);
+                for (int kh = 0; kh < KH; ++kh)
+                    tma_load_3d(smem + SM::OFF_K + s * SM::K_BLOCK + kh * (BN * 128), &mapK, &bar->k_full[s], kh * 64, j * BN, prob);
+                ok = mbar_wait(&bar->v_empty[s], ph ^ 1u);
+                if (!ok) break;
+                mbar_expect_tx(&bar->v_full[s], SM::V_BLOCK);
+                for (int hh = 0; hh < 2; ++hh)
+                    tma_load_3d(smem + SM::OFF_V + s * SM::V_BLOCK + hh * (D * 128), &mapV, &bar->v_full[s], j * BN + hh * 64, 0, prob);
+            }
+            if (!ok) { atomicExch(status, 1); bar->abort_flag = 1; }
+        }
+    } else if (warp == 9) {
+        // ------------------------------ MMA issuer ------------------------------
+        if (lane == 0) {
+            constexpr uint32_t IDESC_QK = umma_idesc_bf16(BM, BN);
+            constexpr uint32_t IDESC_PV = umma_idesc_bf16(BM, D);
+            const uint32_t sQ = smem_u32(smem + SM::OFF_Q), sK = smem_u32(smem + SM::OFF_K), sV = smem_u32(smem + SM::OFF_V);
+            auto issue_qk = [&](int t, int s) {
+#pragma unroll
+                for (int kh = 0; kh < KH; ++kh)
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks)
+                        mma_ss(tmem + t * 128, umma_desc_k128(sQ + t * SM::Q_TILE + kh * (BM * 128) + ks * 32),
+                               umma_desc_k128(sK + s * SM::K_BLOCK + kh * (BN * 128) + ks * 32), IDESC_QK, (kh | ks) != 0);
+            };
+            auto issue_pv = [&](int t, int s, bool acc) {
+#pragma unroll
+                for (int hh = 0; hh < 2; ++hh)
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks)
+                        mma_ts(tmem + 256 + t * 128, tmem + t * 128 + hh * 32 + ks * 8,
+                               umma_desc_k128(sV + s * SM::V_BLOCK + hh * (D * 128) + ks * 32), IDESC_PV,
+                               (acc || (hh | ks) != 0) ? 1u : 0u);
+            };
+            bool ok = mbar_wait(&bar->q_full, 0) && mbar_wait(&bar->k_full[0], 0);
+            if (ok) {
+                tc_fence_after();
+                for (int t = 0; t < 2; ++t) { issue_qk(t, 0); tc_commit(&bar->s_full[t]); }
+                tc_commit(&bar->k_empty[0]);
+            }
+            for (int j = 0; j < nblk && ok; ++j) {
+                const int s = j % STAGES;
+                const bool more = j + 1 < nblk;
+                const int sn = (j + 1) % STAGES;
+                if (more) ok = mbar_wait(&bar->k_full[sn], (uint32_t)((j + 1) / STAGES) & 1u);
+                ok = ok && mbar_wait(&bar->v_full[s], (uint32_t)(j / STAGES) & 1u);
+                for (int t = 0; t < 2 && ok; ++t) {
+                    ok = mbar_wait(&bar->p_ready[t], (uint32_t)j & 1u);
+                    if (!ok) break;
+                    tc_fence_after();
+                    issue_pv(t, s, j > 0);
+                    tc_commit(&bar->o_done[t]);
+                    if (more) { issue_qk(t, sn); tc_commit(&bar->s_full[t]); }
+                }
+                if (!ok) break;
+                tc_commit(&bar->v_empty[s]);
+                if (more) tc_commit(&bar->k_empty[sn]);
+            }
+            if (!ok) { atomicExch(status, 2); bar->abort_flag = 1; }
+        }
+    } else {
+        // ------------------------------ softmax + epilogue ------------------------------
+        const int t = warp >> 2;                                   // query tile of this warpgroup
+        const int row = (warp & 3) * 32 + lane;                    // row in the tile = TMEM lane
+        const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t tS = tmem + lane_addr + t * 128;            // logits / probabilities
+        const uint32_t tO = tmem + lane_addr + 256 + t * 128;      // output accumulator
+        const bool use_bias = nonuniform[prob] != 0;
+        const float *bp = bias + (int64_t)prob * n_pad;
+        float m_ref = -INFINITY, l = 0.f;
+        bool ok = true;
+        for (int j = 0; j < nblk; ++j) {
+            ok = mbar_wait(&bar->s_full[t], (uint32_t)j & 1u);
+            if (!ok) break;
+            tc_fence_after();
+            uint32_t sraw[4][32];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) tmem_ld32(tS + q * 32, sraw[q]);
+            tmem_wait_ld();
+            const int valid = n_core - j * BN;                     // columns of this block that exist
+            float mx = -INFINITY;
+            if (use_bias || valid < BN) {
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) {
+                        float v = __uint_as_float(sraw[q][c]) * scale_log2;
+                        if (use_bias) v += __ldg(bp + j * BN + q * 32 + c);
+                        if (q * 32 + c >= valid) v = -INFINITY;
+                        sraw[q][c] = __float_as_uint(v);
+                        mx = fmaxf(mx, v);
+                    }
+            } else {
+                float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
+#pragma unroll
+                for (int c = 0; c < 32; ++c) {
+                    m0 = fmaxf(m0, __uint_as_float(sraw[0][c]));
+                    m1 = fmaxf(m1, __uint_as_float(sraw[1][c]));
+                    m2 = fmaxf(m2, __uint_as_float(sraw[2][c]));
+                    m3 = fmaxf(m3, __uint_as_float(sraw[3][c]));
+                }
+                mx = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3)) * scale_log2;
+            }
+            // lazy rescale: keep the old reference unless the maximum grew by more than 2^TAU
+            const bool grow = mx > m_ref + RESCALE_TAU;
+            if (__any_sync(0xffffffffu, grow)) {
+                if (j > 0) {
+                    ok = mbar_wait(&bar->o_done[t], (uint32_t)(j - 1) & 1u);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const float alpha = grow ? fast_exp2(m_ref - mx) : 1.f;
+#pragma unroll
+                    for (int q = 0; q < D / 32; ++q) {
+                        uint32_t o[32];
+                        tmem_ld32(tO + q * 32, o);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
+                        tmem_st32(tO + q * 32, o);
+                    }
+                    l *= alpha;
+                }
+                if (grow) m_ref = mx;
+            }
+            float sum0 = 0.f, sum1 = 0.f;
+            const bool prescaled = use_bias || valid < BN;
+            const float neg_m = -m_ref;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                uint32_t pk[16];
+#pragma unroll
+                for (int c = 0; c < 32; c += 2) {
+                    float x0 = __uint_as_float(sraw[q][c]), x1 = __uint_as_float(sraw[q][c + 1]);
+                    float p0 = prescaled ? fast_exp2(x0 + neg_m) : fast_exp2(fmaf(x0, scale_log2, neg_m));
+                    float p1 = prescaled ? fast_exp2(x1 + neg_m) : fast_exp2(fmaf(x1, scale_log2, neg_m));
+                    sum0 += p0;
+                    sum1 += p1;
+                    pk[c >> 1] = pack_bf16x2(p0, p1);
+                }
+                // 16 packed columns: probabilities of points 32q .. 32q+31 of this block
+                asm volatile(
+                    "tcgen05.st.sync.aligned.32x32b.x16.b32 [%16], {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15};"
+                    ::"r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3]), "r"(pk[4]), "r"(pk[5]), "r"(pk[6]), "r"(pk[7]),
+                      "r"(pk[8]), "r"(pk[9]), "r"(pk[10]), "r"(pk[11]), "r"(pk[12]), "r"(pk[13]), "r"(pk[14]), "r"(pk[15]),
+                      "r"(tS + q * 16)
+                    : "memory");
+            }
+            l += sum0 + sum1;
+            tmem_wait_st();
+            tc_fence_before();
+            mbar_arrive(&bar->p_ready[t]);
+        }
+        if (ok) ok = mbar_wait(&bar->o_done[t], (uint32_t)(nblk - 1) & 1u);
+        if (ok) {
+            tc_fence_after();
+            const float inv = 1.f / l;
+            const int64_t qrow = (int64_t)q0 + t * BM + row;
+            __nv_bfloat16 *dst = O + ((int64_t)bh * n_q + qrow) * D;
+#pragma unroll
+            for (int q = 0; q < D / 32; ++q) {
+                uint32_t o[32];
+                tmem_ld32(tO + q * 32, o);
+                tmem_wait_ld();
+                if (qrow < n_q) {
+#pragma unroll
+                    for (int c = 0; c < 32; c += 8) {
+                        uint4 v;
+                        v.x = pack_bf16x2(__uint_as_float(o[c]) * inv, __uint_as_float(o[c + 1]) * inv);
+                        v.y = pack_bf16x2(__uint_as_float(o[c + 2]) * inv, __uint_as_float(o[c + 3]) * inv);
+                        v.z = pack_bf16x2(__uint_as_float(o[c + 4]) * inv, __uint_as_float(o[c + 5]) * inv);
+                        v.w = pack_bf16x2(__uint_as_float(o[c + 6]) * inv, __uint_as_float(o[c + 7]) * inv);
+                        *reinterpret_cast<uint4 *>(dst + q * 32 + c) = v;
+                    }
+                }
+            }
+        } else if (lane == 0) {
+            atomicExch(status, 3);
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 9) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// host side
+// ---------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// 3-D bf16 tensor [d2][d1][d0] (d0 contiguous), box {64, box_rows, 1}, 128-byte swizzle
+static bool make_map(CUtensorMap *map, const void *base, uint64_t d0, uint64_t d1, uint64_t d2, uint32_t box_rows)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[3] = {d0, d1, d2};
+    cuuint64_t strides[2] = {d0 * 2, d0 * d1 * 2};
+    cuuint32_t box[3] = {64, box_rows, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int D>
+static int launch(const __nv_bfloat16 *Q, const __nv_bfloat16 *K, const __nv_bfloat16 *V, const int32_t *idx,
+                  const float *w, int n_core, const elm_params *p, __nv_bfloat16 *O, unsigned char *ws,
+                  cudaStream_t st, bool timed)
+{
+    const AttendLayout L = attend_layout(p, n_core);
+    const int n_pad = (n_core + BN - 1) / BN * BN;
+    const int problems = p->batch * p->kv_heads;
+    __nv_bfloat16 *Kc = reinterpret_cast<__nv_bfloat16 *>(ws + L.Kc);
+    __nv_bfloat16 *Vt = reinterpret_cast<__nv_bfloat16 *>(ws + L.Vc);
+    float *bias = reinterpret_cast<float *>(ws + L.bias);
+    int *flags = reinterpret_cast<int *>(ws + L.flags);
+    int *status = flags + problems;
+    CUtensorMap mQ, mK, mV;
+    if (!make_map(&mQ, Q, D, (uint64_t)p->n_q, (uint64_t)p->batch * p->q_heads, BM) ||
+        !make_map(&mK, Kc, D, (uint64_t)n_pad, (uint64_t)problems, BN) ||
+        !make_map(&mV, Vt, (uint64_t)n_pad, D, (uint64_t)problems, D))
+        return ELM_ERR_CUDA;
+    {
+        StageTimer t(timed ? ELM_STAGE_GATHER : -1, st, 1);
+        ELM_CUDA_TRY(cudaMemsetAsync(flags, 0, sizeof(int) * (size_t)(problems + 1), st));
+        gather_tc_kernel<D><<<dim3((unsigned)(n_pad / 32), (unsigned)problems), 256, 0, st>>>(
+            K, V, idx, w, p->n_kv, n_core, n_pad, Kc, Vt, bias, flags);
+        count_launches(1);
+        ELM_CUDA_TRY(cudaGetLastError());
+    }
+    StageTimer t(timed ? ELM_STAGE_ATTEND : -1, st, 1);
+    auto kern = attend_tc_kernel<D>;
+    ELM_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<D>::TOTAL));
+    dim3 grid((unsigned)((p->n_q + 2 * BM - 1) / (2 * BM)), (unsigned)(p->batch * p->q_heads));
+    const float scale_log2 = (float)(1.4426950408889634 / sqrt((double)D));
+    kern<<<grid, NTHREADS, Smem<D>::TOTAL, st>>>(mQ, mK, mV, bias, flags, O, p->q_heads, p->kv_heads, p->n_q,
+                                                 n_core, n_pad, scale_log2, status);
+    count_launches(1);
+    return cuda_status(cudaGetLastError());
+}
+
+}  // namespace tc
+
+int attend_tc(const __nv_bfloat16 *Q, const __nv_bfloat16 *K, const __nv_bfloat16 *V, const int32_t *idx,
+              const float *w, int n_core, const elm_params *p, __nv_bfloat16 *O, unsigned char *ws,
+              cudaStream_t st, bool timed)
+{
+    if (p->d == 64) return tc::launch<64>(Q, K, V, idx, w, n_core, p, O, ws, st, timed);
+    return tc::launch<128>(Q, K, V, idx, w, n_core, p, O, ws, st, timed);
+}
+
+}  // namespace elm
