@@ -6,6 +6,8 @@
 // the host-side level scheduler.  The tensor-core Gram for bf16 inputs lives in elm_gram_tc.cu.
 #include <math.h>
 
+#include <type_traits>
+
 #include "elm_common.cuh"
 #include "elm_compress.cuh"
 
@@ -365,7 +367,7 @@ CompressLayout compress_layout(const elm_params *p)
     const size_t n_out = (size_t)1 << p->log2_nout;
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
-    L.vmax_bits = take(BH * 4);
+    L.vmax_bits = take((BH + 1) * 4);      // + one device status word
     L.cnorm = take(BH * n * ts);
     L.cur = take(BH * n * 4);
     L.nxt = take(BH * n * 4);
@@ -425,7 +427,7 @@ static int compress_impl(const Tin *K, const Tin *V, const elm_params *p, uint64
 
     if (m > 0) {
         StageTimer t(ELM_STAGE_PREPASS, st, 1);
-        ELM_CUDA_TRY(cudaMemsetAsync(vmax_bits, 0, (size_t)BH * 4, st));
+        ELM_CUDA_TRY(cudaMemsetAsync(vmax_bits, 0, (size_t)(BH + 1) * 4, st));
         dim3 grid((unsigned)((n + 63) / 64), (unsigned)BH);
         prepass_kernel<Tin, T><<<grid, 256, 0, st>>>(K, V, n, p->d, cnorm, vmax_bits, cur);
         count_launches(1);
@@ -449,7 +451,15 @@ static int compress_impl(const Tin *K, const Tin *V, const elm_params *p, uint64
         }
         {
             StageTimer t(ELM_STAGE_GRAM, st, 1);
-            int rc = run_gram_simt<Tin, T>(K, V, p, cur, Mpair, vmax_bits, P, Ptotal, groups, F, L.F_stride, st);
+            int rc;
+            if constexpr (std::is_same<Tin, __nv_bfloat16>::value && std::is_same<T, float>::value) {
+                // tensor cores once a Halve call fills at least a quarter of a 64-pair tile side
+                rc = P >= 16 ? gram_tc(K, V, p, cur, Mpair, vmax_bits, P, Ptotal, groups, F, L.F_stride,
+                                       reinterpret_cast<int *>(vmax_bits + BH), st)
+                             : run_gram_simt<Tin, T>(K, V, p, cur, Mpair, vmax_bits, P, Ptotal, groups, F, L.F_stride, st);
+            } else {
+                rc = run_gram_simt<Tin, T>(K, V, p, cur, Mpair, vmax_bits, P, Ptotal, groups, F, L.F_stride, st);
+            }
             if (rc != ELM_OK) return rc;
         }
         {

@@ -3,6 +3,9 @@
 #include <stddef.h>
 #include <stdint.h>
 
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
 #include "../../include/elm.h"
 
 namespace elm {
@@ -19,5 +22,11 @@ struct CompressLayout {
     size_t total;
 };
 CompressLayout compress_layout(const elm_params *p);
+
+// Tensor-core pair Gram of one level (bf16 storage, fp32 arithmetic); same output layout as the
+// generic kernel.  `status` is a device word that a timed-out wait sets to a non-zero code.
+int gram_tc(const __nv_bfloat16 *K, const __nv_bfloat16 *V, const elm_params *p, const int32_t *cur,
+            const float *Mpair, const unsigned *vmax_bits, int P, int64_t Ptotal, int groups, float *F,
+            int64_t F_stride, int *status, cudaStream_t st);
 
 }  // namespace elm

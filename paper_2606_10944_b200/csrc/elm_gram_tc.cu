@@ -1,0 +1,238 @@
+// Kernel evaluation for one Compress2 level on the sm_100a tensor cores (bf16 inputs, fp32 mode).
+//
+// A CTA produces one 64 x 64 tile of the pair Gram F = P G P^T, i.e. a 128 x 128 tile of
+//   G[a,b] = exp(<k_a,k_b>/sqrt(d) - M_pair(b)) * (<v_a,v_b> + v_max^2)                Eq. (katt), shifted
+// The 128 row points and 128 column points are gathered through the level's index list straight
+// into the 128-byte-swizzled K-major layout tcgen05.mma reads (rows are never copied in HBM).
+// Two accumulators in TMEM hold K K^T and V V^T; the epilogue applies the exponential, the
+// product and the +/- pair combination F[j,i] = G[2j,2i] - G[2j,2i+1] - G[2j+1,2i] + G[2j+1,2i+1]
+// (Algorithm A.1's <f_j, f_i>) and stores only j <= i within one Halve call.
+#include <math.h>
+
+#include "elm_common.cuh"
+#include "elm_compress.cuh"
+#include "elm_sm100.cuh"
+
+namespace elm {
+namespace gramtc {
+
+using namespace sm100;
+
+constexpr int TP = 64;            // pairs per tile side
+constexpr int TR = 128;           // points per tile side
+constexpr int NTHREADS = 256;
+constexpr uint32_t TMEM_COLS = 256;
+
+template <int D> struct Smem {
+    static constexpr int KH = D / 64;
+    static constexpr int OPERAND = TR * D * 2;                 // one 128-row operand tile, bytes
+    static constexpr int OFF_AK = 0, OFF_AV = OPERAND, OFF_BK = 2 * OPERAND, OFF_BV = 3 * OPERAND;
+    static constexpr int OFF_MISC = 4 * OPERAND;
+    static constexpr int TOTAL = OFF_MISC + 2048 + 1024;       // misc block + alignment slack
+};
+
+struct Misc {
+    uint64_t mma_done;
+    uint32_t tmem_base;
+    uint32_t pad;
+    float colshift[TP];          // M of each pair column, in log2 units
+    int32_t rowsA[TR], rowsB[TR];
+};
+
+// Gather 128 rows of X (row-major [n][D] bf16) into a swizzled K-major operand tile.
+template <int D>
+__device__ __forceinline__ void gather_operand(unsigned char *dst, const __nv_bfloat16 *__restrict__ X,
+                                               const int32_t *rows, int tid)
+{
+    constexpr int CHUNKS = D / 8;                              // 16-byte chunks per row
+    const uint32_t dst_s = smem_u32(dst);
+#pragma unroll
+    for (int q = tid; q < TR * CHUNKS; q += NTHREADS) {
+        const int r = q / CHUNKS, ch = q % CHUNKS;
+        const int kh = ch >> 3, c = ch & 7;
+        // asynchronous 16-byte copies: all of a thread's chunks are in flight at once
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst_s + kh * (TR * 128) + (r >> 3) * 1024 +
+                                                                        (r & 7) * 128 + ((c ^ (r & 7)) << 4)),
+                     "l"(X + (int64_t)rows[r] * D + ch * 8)
+                     : "memory");
+    }
+}
+
+template <int D>
+__global__ void __launch_bounds__(NTHREADS, 1)
+gram_tc_kernel(const __nv_bfloat16 *__restrict__ K, const __nv_bfloat16 *__restrict__ V,
+               const int32_t *__restrict__ cur, const float *__restrict__ Mpair,
+               const unsigned *__restrict__ vmax_bits, int64_t n, int P, int64_t Ptotal,
+               float *__restrict__ F, int64_t F_stride, int *__restrict__ status)
+{
+    using SM = Smem<D>;
+    constexpr int KH = SM::KH;
+    extern __shared__ unsigned char smem_dyn[];
+    unsigned char *smem = reinterpret_cast<unsigned char *>(((uintptr_t)smem_dyn + 1023) & ~(uintptr_t)1023);
+    Misc *misc = reinterpret_cast<Misc *>(smem + SM::OFF_MISC);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int p = blockIdx.y;
+
+    if (*reinterpret_cast<volatile int *>(status) != 0) return;
+
+    int64_t JR, JC;
+    if (P >= TP) {
+        const int Tg = P / TP, ntri = Tg * (Tg + 1) / 2;
+        const int g = blockIdx.x / ntri, local = blockIdx.x % ntri;
+        int tc = (int)((sqrtf(8.f * (float)local + 1.f) - 1.f) * 0.5f);
+        while ((tc + 1) * (tc + 2) / 2 <= local) ++tc;
+        while (tc * (tc + 1) / 2 > local) --tc;
+        const int tr = local - tc * (tc + 1) / 2;
+        JR = (int64_t)g * P + tr * TP;
+        JC = (int64_t)g * P + tc * TP;
+    } else {
+        JR = JC = (int64_t)blockIdx.x * TP;
+    }
+    const bool diagonal = JR == JC;
+    const int32_t *curp = cur + (int64_t)p * n;
+    const float LOG2E = 1.4426950408889634f;
+    if (tid < TR) {
+        const int64_t pt = 2 * JR + tid;
+        misc->rowsA[tid] = pt < 2 * Ptotal ? curp[pt] : 0;
+    } else {
+        const int64_t pt = 2 * JC + (tid - TR);
+        misc->rowsB[tid - TR] = pt < 2 * Ptotal ? curp[pt] : 0;
+    }
+    if (tid < TP) {
+        const int64_t jc = JC + tid;
+        misc->colshift[tid] = jc < Ptotal ? Mpair[(int64_t)p * (n / 2) + jc] * LOG2E : 0.f;
+    }
+    if (tid == 0) {
+        mbar_init(&misc->mma_done, 1);
+        fence_barrier_init();
+    }
+    if (warp == 1) tmem_alloc(&misc->tmem_base, TMEM_COLS);
+    __syncthreads();
+
+    const __nv_bfloat16 *Kp = K + (int64_t)p * n * D;
+    const __nv_bfloat16 *Vp = V + (int64_t)p * n * D;
+    gather_operand<D>(smem + SM::OFF_AK, Kp, misc->rowsA, tid);
+    gather_operand<D>(smem + SM::OFF_AV, Vp, misc->rowsA, tid);
+    if (!diagonal) {
+        gather_operand<D>(smem + SM::OFF_BK, Kp, misc->rowsB, tid);
+        gather_operand<D>(smem + SM::OFF_BV, Vp, misc->rowsB, tid);
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = misc->tmem_base;
+
+    if (tid == 0) {
+        constexpr uint32_t IDESC = umma_idesc_bf16(TR, TR);
+        const uint32_t sAK = smem_u32(smem + SM::OFF_AK), sAV = smem_u32(smem + SM::OFF_AV);
+        const uint32_t sBK = diagonal ? sAK : smem_u32(smem + SM::OFF_BK);
+        const uint32_t sBV = diagonal ? sAV : smem_u32(smem + SM::OFF_BV);
+#pragma unroll
+        for (int kh = 0; kh < KH; ++kh)
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks)
+                mma_ss(tmem, umma_desc_k128(sAK + kh * (TR * 128) + ks * 32),
+                       umma_desc_k128(sBK + kh * (TR * 128) + ks * 32), IDESC, (kh | ks) != 0);
+#pragma unroll
+        for (int kh = 0; kh < KH; ++kh)
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks)
+                mma_ss(tmem + 128, umma_desc_k128(sAV + kh * (TR * 128) + ks * 32),
+                       umma_desc_k128(sBV + kh * (TR * 128) + ks * 32), IDESC, (kh | ks) != 0);
+        tc_commit(&misc->mma_done);
+    }
+
+    // epilogue: warp w owns TMEM lanes 32 (w % 4) .. +31 (tile rows) and the column half w / 4
+    const bool ok = mbar_wait(&misc->mma_done, 0);
+    if (ok) {
+        tc_fence_after();
+        const int r = (warp & 3) * 32 + lane;                 // point row in the tile
+        const int ch = warp >> 2;                             // columns [64 ch, 64 ch + 64)
+        const uint32_t taddr = tmem + ((uint32_t)((warp & 3) * 32) << 16) + ch * 64;
+        const float vm = __uint_as_float(vmax_bits[p]);
+        const float vm2 = vm * vm;
+        const float qscale = LOG2E / sqrtf((float)D);
+        float h[32];                                          // G[r,2i] - G[r,2i+1] for the 32 pair columns
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+            uint32_t kk[32], vv[32];
+            tmem_ld32(taddr + q * 32, kk);
+            tmem_ld32(taddr + 128 + q * 32, vv);
+            tmem_wait_ld();
+#pragma unroll
+            for (int c = 0; c < 32; c += 2) {
+                const float sh = misc->colshift[ch * 32 + q * 16 + (c >> 1)];
+                float e0 = fmaf(__uint_as_float(kk[c]), qscale, -sh);
+                float e1 = fmaf(__uint_as_float(kk[c + 1]), qscale, -sh);
+                float g0 = e0 < -115.f ? 0.f : fast_exp2(e0) * (__uint_as_float(vv[c]) + vm2);
+                float g1 = e1 < -115.f ? 0.f : fast_exp2(e1) * (__uint_as_float(vv[c + 1]) + vm2);
+                h[q * 16 + (c >> 1)] = g0 - g1;
+            }
+        }
+        // pair rows are adjacent lanes: the even lane finishes pair columns 0..15 of its 32, the odd
+        // lane columns 16..31
+        const bool odd = lane & 1;
+        float f[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const float send = odd ? h[i] : h[i + 16];
+            const float recv = __shfl_xor_sync(0xffffffffu, send, 1);
+            f[i] = odd ? recv - h[i + 16] : h[i] - recv;
+        }
+        const int64_t jr = JR + (r >> 1);
+        const int64_t jc0 = JC + ch * 32 + (odd ? 16 : 0);
+        float *Fp = F + (int64_t)p * F_stride;
+        if (jr < Ptotal) {
+            const int64_t gr = jr / P;
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const int64_t jc = jc0 + i;
+                if (jc < Ptotal && jr <= jc && jc / P == gr) Fp[jr * P + (jc - gr * P)] = f[i];
+            }
+        }
+    } else if (lane == 0) {
+        atomicExch(status, 4);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem, TMEM_COLS);
+    }
+}
+
+template <int D>
+static int launch(const __nv_bfloat16 *K, const __nv_bfloat16 *V, const elm_params *p, const int32_t *cur,
+                  const float *Mpair, const unsigned *vmax_bits, int P, int64_t Ptotal, int groups, float *F,
+                  int64_t F_stride, int *status, cudaStream_t st)
+{
+    const int BH = p->batch * p->kv_heads;
+    int64_t tiles;
+    if (P >= TP) {
+        const int Tg = P / TP;
+        tiles = (int64_t)groups * (Tg * (Tg + 1) / 2);
+    } else {
+        tiles = (Ptotal + TP - 1) / TP;
+    }
+    auto kern = gram_tc_kernel<D>;
+    ELM_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<D>::TOTAL));
+    kern<<<dim3((unsigned)tiles, (unsigned)BH), NTHREADS, Smem<D>::TOTAL, st>>>(K, V, cur, Mpair, vmax_bits, p->n_kv, P,
+                                                                                 Ptotal, F, F_stride, status);
+    count_launches(1);
+    return cuda_status(cudaGetLastError());
+}
+
+}  // namespace gramtc
+
+int gram_tc(const __nv_bfloat16 *K, const __nv_bfloat16 *V, const elm_params *p, const int32_t *cur,
+            const float *Mpair, const unsigned *vmax_bits, int P, int64_t Ptotal, int groups, float *F,
+            int64_t F_stride, int *status, cudaStream_t st)
+{
+    if (p->d == 64) return gramtc::launch<64>(K, V, p, cur, Mpair, vmax_bits, P, Ptotal, groups, F, F_stride, status, st);
+    return gramtc::launch<128>(K, V, p, cur, Mpair, vmax_bits, P, Ptotal, groups, F, F_stride, status, st);
+}
+
+}  // namespace elm
