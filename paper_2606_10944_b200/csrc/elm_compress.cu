@@ -279,9 +279,44 @@ __device__ __forceinline__ uint32_t walk_block(const T *__restrict__ Fg, int P, 
     return swaps;
 }
 
-// Calls with at least 32 pairs: one CTA of 8 warps per call.
+// The serial part of a 32-pair block with the diagonal tile already in registers: Fd[t] is
+// F[i0 + t, i0 + lane] for t <= lane (anything for t > lane), b2 = F[i0 + lane, i0 + lane].
 template <typename T>
-__global__ void __launch_bounds__(256) walk_cta_kernel(const T *__restrict__ F, int64_t F_stride,
+__device__ __forceinline__ uint32_t walk_block_regs(const T (&Fd)[32], T b2, T alpha, T r, T U, T logfac,
+                                                    T &bmax, int lane)
+{
+    T b = sqrt(b2 > 0 ? b2 : (T)0);
+    T my_bmax = 0;
+#pragma unroll
+    for (int t = 0; t < 32; ++t) {
+        T bt = __shfl_sync(0xffffffffu, b, t);
+        T rt = __shfl_sync(0xffffffffu, r, t);
+        T carried = bmax * rt;
+        bmax = bt > carried ? bt : carried;
+        if (t == lane) my_bmax = bmax;
+    }
+    const T a = b * my_bmax * logfac;
+    uint32_t swaps = 0;
+#pragma unroll
+    for (int t = 0; t < 32; ++t) {
+        bool mine = (lane == t) && swap_decision(alpha, a, U);
+        uint32_t sw = (__ballot_sync(0xffffffffu, mine) >> t) & 1u;
+        swaps |= sw << t;
+        T f = t < lane ? Fd[t] : (T)0;
+        alpha += sw ? f : -f;
+    }
+    return swaps;
+}
+
+// Calls with at least 32 pairs: one CTA per call, warp 0 walks, the other warps fold finished
+// blocks into the scores of later columns one block behind the walker:
+//   iteration c   walker : alpha(block c) = alpha_smem + contribution of block c-1 taken from a
+//                          prefetched 32 x 32 tile, then the 32 serial steps of block c, while the
+//                          tiles it needs for block c+1 are already in flight;
+//                 others : alpha_smem[i] -= sum_t eta_{c-1,t} F[32(c-1)+t, i] for all i >= 32(c+1).
+// One __syncthreads per block separates the iterations.
+template <typename T, bool PREFETCH>
+__global__ void __launch_bounds__(512) walk_cta_kernel(const T *__restrict__ F, int64_t F_stride,
                                                        const T *__restrict__ rdecay,
                                                        const int32_t *__restrict__ cur,
                                                        int32_t *__restrict__ out, int64_t out_stride,
@@ -289,29 +324,79 @@ __global__ void __launch_bounds__(256) walk_cta_kernel(const T *__restrict__ F, 
                                                        T logfac)
 {
     extern __shared__ unsigned char smem_raw[];
-    T *eta = reinterpret_cast<T *>(smem_raw);      // [P]
-    T *part = eta + P;                             // [8][32]
+    T *alpha_s = reinterpret_cast<T *>(smem_raw);                    // [P] scores from finished rounds
+    uint32_t *mask_s = reinterpret_cast<uint32_t *>(alpha_s + P);    // [P/32] swap masks
     const int p = blockIdx.y, g = blockIdx.x;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int nthr = blockDim.x;
     const T *Fg = F + (int64_t)p * F_stride + (int64_t)g * P * P;
     const int64_t base = (int64_t)g * P;
+    const int nb = P / 32;
+    for (int i = threadIdx.x; i < P; i += nthr) alpha_s[i] = 0;
+
+    T Fd[32], Fx[32], b2 = 0;
     T bmax = 0;
-    for (int c = 0; c < P / 32; ++c) {
-        const int i0 = 32 * c;
-        T acc = 0;
-        for (int j = warp; j < i0; j += 8) acc += eta[j] * Fg[(int64_t)j * P + i0 + lane];
-        part[warp * 32 + lane] = acc;
-        __syncthreads();
-        if (warp == 0) {
-            T alpha = 0;
+    if (warp == 0) {
 #pragma unroll
-            for (int w = 0; w < 8; ++w) alpha -= part[w * 32 + lane];
+        for (int t = 0; t < 32; ++t) {
+            Fd[t] = t <= lane ? Fg[(int64_t)t * P + lane] : (T)0;
+            Fx[t] = 0;
+            if (t == lane) b2 = Fd[t];
+        }
+    }
+    __syncthreads();
+    for (int c = 0; c < nb; ++c) {
+        const int i0 = 32 * c;
+        if (warp == 0) {
+            T alpha = alpha_s[i0 + lane];
+            if (c > 0) {
+                const uint32_t pm = mask_s[c - 1];
+#pragma unroll
+                for (int t = 0; t < 32; ++t) alpha += ((pm >> t) & 1u) ? Fx[t] : -Fx[t];
+            }
             const T r = rdecay[(int64_t)p * (n / 2) + base + i0 + lane];
             const T U = halving_uniform<T>(seed, (uint32_t)(i0 + lane), (uint32_t)g, (uint32_t)level, (uint32_t)p);
-            uint32_t swaps = walk_block<T>(Fg, P, i0, 32, alpha, r, U, logfac, bmax, lane);
+            // tiles for the next block: diagonal (c+1, c+1) and the one that couples it to block c
+            T Fd_n[32], Fx_n[32], b2_n = 0;
+            const bool more = c + 1 < nb;
+            if (PREFETCH && more) {
+#pragma unroll
+                for (int t = 0; t < 32; ++t) {
+                    Fd_n[t] = t <= lane ? Fg[(int64_t)(i0 + 32 + t) * P + i0 + 32 + lane] : (T)0;
+                    Fx_n[t] = Fg[(int64_t)(i0 + t) * P + i0 + 32 + lane];
+                    if (t == lane) b2_n = Fd_n[t];
+                }
+            }
+            const uint32_t swaps = walk_block_regs<T>(Fd, b2, alpha, r, U, logfac, bmax, lane);
             const uint32_t sw = (swaps >> lane) & 1u;
-            eta[i0 + lane] = sw ? (T)-1 : (T)1;
+            if (lane == 0) mask_s[c] = swaps;
             out[(int64_t)p * out_stride + base + i0 + lane] = cur[(int64_t)p * n + 2 * (base + i0 + lane) + sw];
+            if (!PREFETCH && more) {
+#pragma unroll
+                for (int t = 0; t < 32; ++t) {
+                    Fd_n[t] = t <= lane ? Fg[(int64_t)(i0 + 32 + t) * P + i0 + 32 + lane] : (T)0;
+                    Fx_n[t] = Fg[(int64_t)(i0 + t) * P + i0 + 32 + lane];
+                    if (t == lane) b2_n = Fd_n[t];
+                }
+            }
+            if (more) {
+#pragma unroll
+                for (int t = 0; t < 32; ++t) { Fd[t] = Fd_n[t]; Fx[t] = Fx_n[t]; }
+                b2 = b2_n;
+            }
+        } else if (c > 0) {
+            // round c-1: rows of block c-1 into every column from block c+1 on
+            const uint32_t pm = mask_s[c - 1];
+            const T *rows = Fg + (int64_t)(i0 - 32) * P;
+            for (int i = i0 + 32 + (threadIdx.x - 32); i < P; i += nthr - 32) {
+                T acc = 0;
+#pragma unroll
+                for (int t = 0; t < 32; ++t) {
+                    const T f = rows[(int64_t)t * P + i];
+                    acc += ((pm >> t) & 1u) ? f : -f;
+                }
+                alpha_s[i] += acc;
+            }
         }
         __syncthreads();
     }
@@ -465,8 +550,13 @@ static int compress_impl(const Tin *K, const Tin *V, const elm_params *p, uint64
         {
             StageTimer t(ELM_STAGE_WALK, st, 1);
             if (P >= 32) {
-                size_t smem = ((size_t)P + 256) * sizeof(T);
-                walk_cta_kernel<T><<<dim3((unsigned)groups, (unsigned)BH), 256, smem, st>>>(
+                // one walker warp plus enough warps to sweep the remaining columns once per block
+                int warps = P / 64 + 1;
+                warps = warps < 1 ? 1 : (warps > 16 ? 16 : warps);
+                if (P >= 64 && warps < 2) warps = 2;
+                const size_t smem = (size_t)P * sizeof(T) + (size_t)(P / 32) * 4;
+                constexpr bool kPrefetch = std::is_same<T, float>::value;
+                walk_cta_kernel<T, kPrefetch><<<dim3((unsigned)groups, (unsigned)BH), warps * 32, smem, st>>>(
                     F, L.F_stride, rdecay, cur, out, out_stride, n, P, level, seed, logfac);
             } else {
                 walk_warp_kernel<T><<<dim3((unsigned)((groups + 7) / 8), (unsigned)BH), 256, 0, st>>>(
