@@ -162,7 +162,7 @@ def workload_config(wl, args):
             "seq_len": wl.n, "head_dim": wl.d, "n_out": wl.n_out, "compress2_depth": wl.m, "g": wl.g,
             "storage": wl.dtype, "precision": args.precision, "recipe": wl.recipe,
             "parallelism": "replicas only", "l2": "inputs (>= 2.6 GB per step) exceed the 126 MB L2"
-            if wl.name in ("cfg5", "cfg4") else "L2 flushed by a 256 MB write between steps"}
+            if wl.name.startswith(("cfg5", "cfg4")) else "L2 flushed by a 256 MB write between steps"}
 
 
 T_START = time.perf_counter()
@@ -180,12 +180,19 @@ def main():
     ap.add_argument("--seed", type=int, default=1)
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--ref-heads", type=int, default=None)
+    ap.add_argument("--override", default="", help="comma list of Workload fields for small profiling "
+                    "captures, e.g. q_heads=8,kv_heads=2,n=32768,n_q=32768 (the line then names the scaled case)")
+    ap.add_argument("--only", default="both", choices=["both", "compress", "attend"],
+                    help="run one half of the step (profiling captures only)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
 
     from paper_2606_10944_b200.workloads import WORKLOADS, generate
     wl = WORKLOADS[args.workload]
+    if args.override:
+        kv = dict(item.split("=") for item in args.override.split(","))
+        wl = wl.scaled(name=f"{wl.name}[{args.override}]", **{k: int(v) for k, v in kv.items()})
     if args.impl == "reference":
         run_reference(args, wl)
         return
@@ -215,15 +222,19 @@ def main():
     ws_c = torch.empty(cb, dtype=torch.uint8, device=dev)
     ws_a = torch.empty(ab, dtype=torch.uint8, device=dev)
     O = torch.empty_like(Qd)
-    small_inputs = wl.name not in ("cfg4", "cfg5")
+    small_inputs = not wl.name.startswith(("cfg4", "cfg5"))
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev) if small_inputs else None
+
+    state = {}
 
     def step(seed):
         if flush is not None:
             flush.zero_()
-        idx, w = elm.compress(Kd, Vd, wl.log2_nout, wl.m, seed=seed, precision=args.precision, workspace=ws_c)
-        elm.attend(Qd, Kd, Vd, idx, w, precision=args.precision, workspace=ws_a, out=O)
-        return idx, w
+        if args.only != "attend" or "idx" not in state:
+            state["idx"], state["w"] = elm.compress(Kd, Vd, wl.log2_nout, wl.m, seed=seed, precision=args.precision,
+                                                    workspace=ws_c)
+        if args.only != "compress":
+            elm.attend(Qd, Kd, Vd, state["idx"], state["w"], precision=args.precision, workspace=ws_a, out=O)
 
     def barrier():
         torch.cuda.synchronize()
@@ -300,7 +311,7 @@ def main():
     peaks = load_peaks()
     attend_flops, compress_flops, hbm_bytes = algorithmic_counts(wl)
     stage_ms = {k: v[0] / args.steps for k, v in stage.items()}
-    att_ms = stage_ms["attend"]
+    att_ms = stage_ms["attend"] or float("nan")     # zero only under --only compress
     tensor_peak = peaks["bf16_tflops_sustained"]
     # the dominant kernel: weighted attention (dense contraction -> tensor roofline) unless the
     # workload's coreset is so small that its Q/O traffic dominates

@@ -21,6 +21,13 @@
 #include "elm_common.cuh"
 #include "elm_sm100.cuh"
 
+#ifdef ELM_TRACE
+__device__ long long g_trace_buf[8192];
+#define TRACE(slot) do { if (trace_on) g_trace_buf[(slot)] = clock64(); } while (0)
+#else
+#define TRACE(slot) do { } while (0)
+#endif
+
 namespace elm {
 namespace tc {
 
@@ -197,6 +204,9 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                                umma_desc_k128(sV + s * SM::V_BLOCK + hh * (D * 128) + ks * 32), IDESC_PV,
                                (acc || (hh | ks) != 0) ? 1u : 0u);
             };
+#ifdef ELM_TRACE
+            const bool trace_on = blockIdx.x == 3 && blockIdx.y == 0;
+#endif
             bool ok = mbar_wait(&bar->q_full, 0) && mbar_wait(&bar->k_full[0], 0);
             if (ok) {
                 tc_fence_after();
@@ -209,13 +219,16 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                 const int sn = (j + 1) % STAGES;
                 if (more) ok = mbar_wait(&bar->k_full[sn], (uint32_t)((j + 1) / STAGES) & 1u);
                 ok = ok && mbar_wait(&bar->v_full[s], (uint32_t)(j / STAGES) & 1u);
+                TRACE(4096 + j * 8 + 0);
                 for (int t = 0; t < 2 && ok; ++t) {
                     ok = mbar_wait(&bar->p_ready[t], (uint32_t)j & 1u);
                     if (!ok) break;
+                    TRACE(4096 + j * 8 + 1 + 2 * t);
                     tc_fence_after();
                     issue_pv(t, s, j > 0);
                     tc_commit(&bar->o_done[t]);
                     if (more) { issue_qk(t, sn); tc_commit(&bar->s_full[t]); }
+                    TRACE(4096 + j * 8 + 2 + 2 * t);
                 }
                 if (!ok) break;
                 tc_commit(&bar->v_empty[s]);
@@ -234,38 +247,47 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
         const float *bp = bias + (int64_t)prob * n_pad;
         float m_ref = -INFINITY, l = 0.f;
         bool ok = true;
+#ifdef ELM_TRACE
+        const bool trace_on = blockIdx.x == 3 && blockIdx.y == 0 && (warp & 3) == ELM_TRACE_WARP && lane == 0;
+        const int tb = t * 2048;
+#endif
         for (int j = 0; j < nblk; ++j) {
+            TRACE(tb + j * 8 + 0);
             ok = mbar_wait(&bar->s_full[t], (uint32_t)j & 1u);
             if (!ok) break;
             tc_fence_after();
-            uint32_t sraw[4][32];
-#pragma unroll
-            for (int q = 0; q < 4; ++q) tmem_ld32(tS + q * 32, sraw[q]);
-            tmem_wait_ld();
+            TRACE(tb + j * 8 + 1);
             const int valid = n_core - j * BN;                     // columns of this block that exist
-            float mx = -INFINITY;
-            if (use_bias || valid < BN) {
+            const bool special = use_bias || valid < BN;           // per-column bias and/or a ragged tail
+            // ---- pass 1: row maximum (the logits stay in TMEM and are read again in pass 2) ----
+            float mx;
+            {
+                float m0 = -INFINITY, m1 = -INFINITY;
+                uint32_t a[2][32];
+                tmem_ld32(tS, a[0]);
 #pragma unroll
-                for (int q = 0; q < 4; ++q)
+                for (int q = 0; q < 4; ++q) {
+                    tmem_wait_ld();
+                    if (q < 3) tmem_ld32(tS + (q + 1) * 32, a[(q + 1) & 1]);
+                    if (!special) {
 #pragma unroll
-                    for (int c = 0; c < 32; ++c) {
-                        float v = __uint_as_float(sraw[q][c]) * scale_log2;
-                        if (use_bias) v += __ldg(bp + j * BN + q * 32 + c);
-                        if (q * 32 + c >= valid) v = -INFINITY;
-                        sraw[q][c] = __float_as_uint(v);
-                        mx = fmaxf(mx, v);
+                        for (int c = 0; c < 32; c += 4) {
+                            m0 = max3(m0, __uint_as_float(a[q & 1][c]), __uint_as_float(a[q & 1][c + 1]));
+                            m1 = max3(m1, __uint_as_float(a[q & 1][c + 2]), __uint_as_float(a[q & 1][c + 3]));
+                        }
+                    } else {
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) {
+                            float v = __uint_as_float(a[q & 1][c]) * scale_log2;
+                            if (use_bias) v += __ldg(bp + j * BN + q * 32 + c);
+                            if (q * 32 + c >= valid) v = -INFINITY;
+                            m0 = fmaxf(m0, v);
+                        }
                     }
-            } else {
-                float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
-#pragma unroll
-                for (int c = 0; c < 32; ++c) {
-                    m0 = fmaxf(m0, __uint_as_float(sraw[0][c]));
-                    m1 = fmaxf(m1, __uint_as_float(sraw[1][c]));
-                    m2 = fmaxf(m2, __uint_as_float(sraw[2][c]));
-                    m3 = fmaxf(m3, __uint_as_float(sraw[3][c]));
                 }
-                mx = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3)) * scale_log2;
+                mx = special ? m0 : fmaxf(m0, m1) * scale_log2;
             }
+            TRACE(tb + j * 8 + 2);
             // lazy rescale: keep the old reference unless the maximum grew by more than 2^TAU
             const bool grow = mx > m_ref + RESCALE_TAU;
             if (__any_sync(0xffffffffu, grow)) {
@@ -287,33 +309,79 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                 }
                 if (grow) m_ref = mx;
             }
-            float sum0 = 0.f, sum1 = 0.f;
-            const bool prescaled = use_bias || valid < BN;
+            TRACE(tb + j * 8 + 3);
+            // ---- pass 2: p = 2^(s - m_ref), running denominator, bf16 probabilities back to TMEM ----
             const float neg_m = -m_ref;
+            const uint64_t scale2 = pack2(scale_log2, scale_log2), negm2 = pack2(neg_m, neg_m);
+            uint64_t sum2 = pack2(0.f, 0.f), sum2b = pack2(0.f, 0.f);
+            float sum0 = 0.f;
+            {
+                uint32_t a[2][32];
+                tmem_ld32(tS, a[0]);
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                uint32_t pk[16];
+                for (int q = 0; q < 4; ++q) {
+                    tmem_wait_ld();
+                    if (q < 3) tmem_ld32(tS + (q + 1) * 32, a[(q + 1) & 1]);
+                    uint32_t pk[16];
+                    if (!special) {
+                        // staged over the 16 pairs of the chunk so that independent work interleaves
+                        uint64_t x2[16];
 #pragma unroll
-                for (int c = 0; c < 32; c += 2) {
-                    float x0 = __uint_as_float(sraw[q][c]), x1 = __uint_as_float(sraw[q][c + 1]);
-                    float p0 = prescaled ? fast_exp2(x0 + neg_m) : fast_exp2(fmaf(x0, scale_log2, neg_m));
-                    float p1 = prescaled ? fast_exp2(x1 + neg_m) : fast_exp2(fmaf(x1, scale_log2, neg_m));
-                    sum0 += p0;
-                    sum1 += p1;
-                    pk[c >> 1] = pack_bf16x2(p0, p1);
+                        for (int i = 0; i < 16; ++i)
+                            x2[i] = fma2(pack2(__uint_as_float(a[q & 1][2 * i]), __uint_as_float(a[q & 1][2 * i + 1])), scale2, negm2);
+                        float pe[32];
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) {
+                            float x0, x1;
+                            unpack2(x2[i], x0, x1);
+                            pe[2 * i] = fast_exp2(x0);
+                            pe[2 * i + 1] = fast_exp2(x1);
+                        }
+#pragma unroll
+                        for (int i = 0; i < 16; i += 2) {
+                            sum2 = add2(sum2, pack2(pe[2 * i], pe[2 * i + 1]));
+                            sum2b = add2(sum2b, pack2(pe[2 * i + 2], pe[2 * i + 3]));
+                        }
+#pragma unroll
+                        for (int i = 0; i < 16; ++i)
+                            pk[i] = __byte_perm(__float_as_uint(pe[2 * i]) + 0x8000u, __float_as_uint(pe[2 * i + 1]) + 0x8000u, 0x7632);
+                    } else {
+#pragma unroll
+                        for (int c = 0; c < 32; c += 2) {
+                            float v0 = __uint_as_float(a[q & 1][c]) * scale_log2, v1 = __uint_as_float(a[q & 1][c + 1]) * scale_log2;
+                            if (use_bias) { v0 += __ldg(bp + j * BN + q * 32 + c); v1 += __ldg(bp + j * BN + q * 32 + c + 1); }
+                            const float p0 = (q * 32 + c < valid) ? fast_exp2(v0 + neg_m) : 0.f;
+                            const float p1 = (q * 32 + c + 1 < valid) ? fast_exp2(v1 + neg_m) : 0.f;
+                            sum0 += p0 + p1;
+                            // round to bf16 on the integer pipe: add half an ulp, keep the upper halves
+                            pk[c >> 1] = __byte_perm(__float_as_uint(p0) + 0x8000u, __float_as_uint(p1) + 0x8000u, 0x7632);
+                        }
+                    }
+                    // 16 packed columns: probabilities of points 32q .. 32q+31 of this block
+#ifdef ELM_NOST
+                    if (pk[0] == 0x12345678u && pk[7] == 0x9abcdef0u && pk[15] == 77u)
+#endif
+                    asm volatile(
+                        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%16], {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15};"
+                        ::"r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3]), "r"(pk[4]), "r"(pk[5]), "r"(pk[6]), "r"(pk[7]),
+                          "r"(pk[8]), "r"(pk[9]), "r"(pk[10]), "r"(pk[11]), "r"(pk[12]), "r"(pk[13]), "r"(pk[14]), "r"(pk[15]),
+                          "r"(tS + q * 16)
+                        : "memory");
                 }
-                // 16 packed columns: probabilities of points 32q .. 32q+31 of this block
-                asm volatile(
-                    "tcgen05.st.sync.aligned.32x32b.x16.b32 [%16], {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15};"
-                    ::"r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3]), "r"(pk[4]), "r"(pk[5]), "r"(pk[6]), "r"(pk[7]),
-                      "r"(pk[8]), "r"(pk[9]), "r"(pk[10]), "r"(pk[11]), "r"(pk[12]), "r"(pk[13]), "r"(pk[14]), "r"(pk[15]),
-                      "r"(tS + q * 16)
-                    : "memory");
             }
+            {
+                float s_lo, s_hi;
+                unpack2(add2(sum2, sum2b), s_lo, s_hi);
+                sum0 += s_lo + s_hi;
+            }
+            const float sum1 = 0.f;
             l += sum0 + sum1;
+            TRACE(tb + j * 8 + 4);
             tmem_wait_st();
             tc_fence_before();
+            TRACE(tb + j * 8 + 5);
             mbar_arrive(&bar->p_ready[t]);
+            TRACE(tb + j * 8 + 6);
         }
         if (ok) ok = mbar_wait(&bar->o_done[t], (uint32_t)(nblk - 1) & 1u);
         if (ok) {
@@ -432,3 +500,10 @@ int attend_tc(const __nv_bfloat16 *Q, const __nv_bfloat16 *K, const __nv_bfloat1
 }
 
 }  // namespace elm
+
+#ifdef ELM_TRACE
+extern "C" int elm_debug_read_trace(long long *host, int n)
+{
+    return cudaMemcpyFromSymbol(host, g_trace_buf, sizeof(long long) * (size_t)n) == cudaSuccess ? 0 : -7;
+}
+#endif
