@@ -24,12 +24,14 @@ __device__ __forceinline__ void mbar_arrive(uint64_t *bar)
 __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
 {
     uint32_t ok;
+    // the last operand is a suspend-time hint: the thread sleeps in hardware until the phase
+    // completes or the hint expires, instead of spinning on issue slots other warps need
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.b32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
+        : "r"(smem_u32(bar)), "r"(parity), "r"(0x989680u)
         : "memory");
     return ok != 0;
 }
@@ -41,7 +43,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity)
     asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t0));
     for (;;) {
 #pragma unroll 1
-        for (int i = 0; i < 2048; ++i)
+        for (int i = 0; i < 64; ++i)
             if (mbar_try_wait(bar, parity)) return true;
         uint64_t t1;
         asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t1));
