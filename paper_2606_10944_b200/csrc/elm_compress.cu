@@ -279,13 +279,12 @@ __device__ __forceinline__ uint32_t walk_block(const T *__restrict__ Fg, int P, 
     return swaps;
 }
 
-// The serial part of a 32-pair block with the diagonal tile already in registers: Fd[t] is
-// F[i0 + t, i0 + lane] for t <= lane (anything for t > lane), b2 = F[i0 + lane, i0 + lane].
+// The serial part of a 32-pair block with everything in registers: Fd[t] = F[i0 + t, i0 + lane]
+// (used for t < lane), b = b_i of this lane's pair.  No memory operation inside.
 template <typename T>
-__device__ __forceinline__ uint32_t walk_block_regs(const T (&Fd)[32], T b2, T alpha, T r, T U, T logfac,
+__device__ __forceinline__ uint32_t walk_block_regs(const T (&Fd)[32], T b, T alpha, T r, T U, T logfac,
                                                     T &bmax, int lane)
 {
-    T b = sqrt(b2 > 0 ? b2 : (T)0);
     T my_bmax = 0;
 #pragma unroll
     for (int t = 0; t < 32; ++t) {
@@ -308,95 +307,127 @@ __device__ __forceinline__ uint32_t walk_block_regs(const T (&Fd)[32], T b2, T a
     return swaps;
 }
 
-// Calls with at least 32 pairs: one CTA per call, warp 0 walks, the other warps fold finished
-// blocks into the scores of later columns one block behind the walker:
-//   iteration c   walker : alpha(block c) = alpha_smem + contribution of block c-1 taken from a
-//                          prefetched 32 x 32 tile, then the 32 serial steps of block c, while the
-//                          tiles it needs for block c+1 are already in flight;
-//                 others : alpha_smem[i] -= sum_t eta_{c-1,t} F[32(c-1)+t, i] for all i >= 32(c+1).
-// One __syncthreads per block separates the iterations.
-template <typename T, bool PREFETCH>
-__global__ void __launch_bounds__(512) walk_cta_kernel(const T *__restrict__ F, int64_t F_stride,
-                                                       const T *__restrict__ rdecay,
-                                                       const int32_t *__restrict__ cur,
-                                                       int32_t *__restrict__ out, int64_t out_stride,
-                                                       int64_t n, int P, int level, uint64_t seed,
-                                                       T logfac)
+// 16-byte asynchronous copy global -> shared
+__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gsrc)
 {
-    extern __shared__ unsigned char smem_raw[];
-    T *alpha_s = reinterpret_cast<T *>(smem_raw);                    // [P] scores from finished rounds
-    uint32_t *mask_s = reinterpret_cast<uint32_t *>(alpha_s + P);    // [P/32] swap masks
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc) : "memory");
+}
+
+__device__ __forceinline__ void load4(const float *p, float (&f)[4])
+{
+    const float4 v = __ldg(reinterpret_cast<const float4 *>(p));
+    f[0] = v.x; f[1] = v.y; f[2] = v.z; f[3] = v.w;
+}
+__device__ __forceinline__ void load4(const double *p, double (&f)[4])
+{
+    const double2 a = __ldg(reinterpret_cast<const double2 *>(p));
+    const double2 b = __ldg(reinterpret_cast<const double2 *>(p) + 1);
+    f[0] = a.x; f[1] = a.y; f[2] = b.x; f[3] = b.y;
+}
+
+// Calls with at least 32 pairs: one CTA per call.
+//   setup      all threads: b_i = sqrt(F[i,i]), the decay factors and the uniforms of every pair
+//              into shared memory; scores alpha = 0.
+//   warp 0     the walker: for block c it adds block c-1's contribution from a 32 x 32 tile that
+//              was copied to shared memory during the previous block, takes the diagonal tile
+//              (c, c) into registers and runs the 32 serial steps without touching memory.
+//   warp 1     also copies the two tiles the walker needs for block c+1 (asynchronous copies).
+//   warps 1..  fold block c-1 into the scores of all columns from block c+1 on, one block behind
+//              the walker (16-byte loads, four adjacent columns per thread).
+// One __syncthreads per block separates the iterations.
+template <typename T>
+__global__ void __launch_bounds__(1024) walk_cta_kernel(const T *__restrict__ F, int64_t F_stride,
+                                                        const T *__restrict__ rdecay,
+                                                        const int32_t *__restrict__ cur,
+                                                        int32_t *__restrict__ out, int64_t out_stride,
+                                                        int64_t n, int P, int level, uint64_t seed,
+                                                        T logfac)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    T *tiles = reinterpret_cast<T *>(smem_raw);                      // [2][2][32][32]: buffer, (diag, cross)
+    T *alpha_s = tiles + 4 * 1024;                                   // [P] scores from finished rounds
+    T *b_s = alpha_s + P;                                            // [P]
+    T *r_s = b_s + P;                                                // [P]
+    T *U_s = r_s + P;                                                // [P]
+    uint32_t *mask_s = reinterpret_cast<uint32_t *>(U_s + P);        // [P/32] swap masks
     const int p = blockIdx.y, g = blockIdx.x;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int nthr = blockDim.x;
     const T *Fg = F + (int64_t)p * F_stride + (int64_t)g * P * P;
     const int64_t base = (int64_t)g * P;
     const int nb = P / 32;
-    for (int i = threadIdx.x; i < P; i += nthr) alpha_s[i] = 0;
+    constexpr int CH = 16 / sizeof(T);                               // elements per 16-byte chunk
+    constexpr int CPR = 32 / CH;                                     // chunks per 32-element tile row
 
-    T Fd[32], Fx[32], b2 = 0;
-    T bmax = 0;
-    if (warp == 0) {
-#pragma unroll
-        for (int t = 0; t < 32; ++t) {
-            Fd[t] = t <= lane ? Fg[(int64_t)t * P + lane] : (T)0;
-            Fx[t] = 0;
-            if (t == lane) b2 = Fd[t];
+    // copies tile (rows r0.., cols c0..) of the call's pair Gram into `dst` [32][32]
+    auto copy_tile = [&](T *dst, int r0, int c0) {
+        for (int q = lane; q < 32 * CPR; q += 32) {
+            const int t = q / CPR, k = q % CPR;
+            cp_async16(dst + t * 32 + k * CH, Fg + (int64_t)(r0 + t) * P + c0 + k * CH);
         }
+    };
+    if (warp == (nthr > 32 ? 1 : 0)) {
+        copy_tile(tiles, 0, 0);
+        asm volatile("cp.async.commit_group;" ::: "memory");
     }
+    for (int i = threadIdx.x; i < P; i += nthr) {
+        alpha_s[i] = 0;
+        const T d = Fg[(int64_t)i * P + i];
+        b_s[i] = sqrt(d > 0 ? d : (T)0);
+        r_s[i] = rdecay[(int64_t)p * (n / 2) + base + i];
+        U_s[i] = halving_uniform<T>(seed, (uint32_t)i, (uint32_t)g, (uint32_t)level, (uint32_t)p);
+    }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
     __syncthreads();
+
+    T bmax = 0;
     for (int c = 0; c < nb; ++c) {
         const int i0 = 32 * c;
+        T *tdiag = tiles + (c & 1) * 2048, *tcross = tdiag + 1024;
+        T *ndiag = tiles + ((c + 1) & 1) * 2048, *ncross = ndiag + 1024;
         if (warp == 0) {
             T alpha = alpha_s[i0 + lane];
             if (c > 0) {
                 const uint32_t pm = mask_s[c - 1];
 #pragma unroll
-                for (int t = 0; t < 32; ++t) alpha += ((pm >> t) & 1u) ? Fx[t] : -Fx[t];
-            }
-            const T r = rdecay[(int64_t)p * (n / 2) + base + i0 + lane];
-            const T U = halving_uniform<T>(seed, (uint32_t)(i0 + lane), (uint32_t)g, (uint32_t)level, (uint32_t)p);
-            // tiles for the next block: diagonal (c+1, c+1) and the one that couples it to block c
-            T Fd_n[32], Fx_n[32], b2_n = 0;
-            const bool more = c + 1 < nb;
-            if (PREFETCH && more) {
-#pragma unroll
                 for (int t = 0; t < 32; ++t) {
-                    Fd_n[t] = t <= lane ? Fg[(int64_t)(i0 + 32 + t) * P + i0 + 32 + lane] : (T)0;
-                    Fx_n[t] = Fg[(int64_t)(i0 + t) * P + i0 + 32 + lane];
-                    if (t == lane) b2_n = Fd_n[t];
+                    const T f = tcross[t * 32 + lane];
+                    alpha += ((pm >> t) & 1u) ? f : -f;
                 }
             }
-            const uint32_t swaps = walk_block_regs<T>(Fd, b2, alpha, r, U, logfac, bmax, lane);
+            T Fd[32];
+#pragma unroll
+            for (int t = 0; t < 32; ++t) Fd[t] = tdiag[t * 32 + lane];
+            const uint32_t swaps = walk_block_regs<T>(Fd, b_s[i0 + lane], alpha, r_s[i0 + lane], U_s[i0 + lane],
+                                                      logfac, bmax, lane);
             const uint32_t sw = (swaps >> lane) & 1u;
             if (lane == 0) mask_s[c] = swaps;
             out[(int64_t)p * out_stride + base + i0 + lane] = cur[(int64_t)p * n + 2 * (base + i0 + lane) + sw];
-            if (!PREFETCH && more) {
+        } else {
+            if (warp == 1 && c + 1 < nb) {
+                copy_tile(ndiag, i0 + 32, i0 + 32);
+                copy_tile(ncross, i0, i0 + 32);
+                asm volatile("cp.async.commit_group;" ::: "memory");
+            }
+            if (c > 0) {
+                // round c-1: rows of block c-1 into every column from block c+1 on
+                const uint32_t pm = mask_s[c - 1];
+                const T *rows = Fg + (int64_t)(i0 - 32) * P;
+                for (int i = i0 + 32 + 4 * (threadIdx.x - 32); i < P; i += 4 * (nthr - 32)) {
+                    T acc[4] = {0, 0, 0, 0};
+#pragma unroll 8
+                    for (int t = 0; t < 32; ++t) {
+                        T f[4];
+                        load4(rows + (int64_t)t * P + i, f);
+                        const bool sw = (pm >> t) & 1u;
 #pragma unroll
-                for (int t = 0; t < 32; ++t) {
-                    Fd_n[t] = t <= lane ? Fg[(int64_t)(i0 + 32 + t) * P + i0 + 32 + lane] : (T)0;
-                    Fx_n[t] = Fg[(int64_t)(i0 + t) * P + i0 + 32 + lane];
-                    if (t == lane) b2_n = Fd_n[t];
+                        for (int k = 0; k < 4; ++k) acc[k] += sw ? f[k] : -f[k];
+                    }
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) alpha_s[i + k] += acc[k];
                 }
             }
-            if (more) {
-#pragma unroll
-                for (int t = 0; t < 32; ++t) { Fd[t] = Fd_n[t]; Fx[t] = Fx_n[t]; }
-                b2 = b2_n;
-            }
-        } else if (c > 0) {
-            // round c-1: rows of block c-1 into every column from block c+1 on
-            const uint32_t pm = mask_s[c - 1];
-            const T *rows = Fg + (int64_t)(i0 - 32) * P;
-            for (int i = i0 + 32 + (threadIdx.x - 32); i < P; i += nthr - 32) {
-                T acc = 0;
-#pragma unroll
-                for (int t = 0; t < 32; ++t) {
-                    const T f = rows[(int64_t)t * P + i];
-                    acc += ((pm >> t) & 1u) ? f : -f;
-                }
-                alpha_s[i] += acc;
-            }
+            if (warp == 1) asm volatile("cp.async.wait_group 0;" ::: "memory");
         }
         __syncthreads();
     }
@@ -551,12 +582,14 @@ static int compress_impl(const Tin *K, const Tin *V, const elm_params *p, uint64
             StageTimer t(ELM_STAGE_WALK, st, 1);
             if (P >= 32) {
                 // one walker warp plus enough warps to sweep the remaining columns once per block
-                int warps = P / 64 + 1;
-                warps = warps < 1 ? 1 : (warps > 16 ? 16 : warps);
+                // four columns per updater thread cover the call's remaining columns in one sweep
+                int warps = P / 128 + 1;
+                warps = warps > 32 ? 32 : warps;
                 if (P >= 64 && warps < 2) warps = 2;
-                const size_t smem = (size_t)P * sizeof(T) + (size_t)(P / 32) * 4;
-                constexpr bool kPrefetch = std::is_same<T, float>::value;
-                walk_cta_kernel<T, kPrefetch><<<dim3((unsigned)groups, (unsigned)BH), warps * 32, smem, st>>>(
+                const size_t smem = (size_t)(4 * 1024 + 4 * P) * sizeof(T) + (size_t)(P / 32) * 4;
+                auto kern = walk_cta_kernel<T>;
+                ELM_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+                kern<<<dim3((unsigned)groups, (unsigned)BH), warps * 32, smem, st>>>(
                     F, L.F_stride, rdecay, cur, out, out_stride, n, P, level, seed, logfac);
             } else {
                 walk_warp_kernel<T><<<dim3((unsigned)((groups + 7) / 8), (unsigned)BH), 256, 0, st>>>(

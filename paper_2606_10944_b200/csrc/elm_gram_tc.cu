@@ -23,16 +23,19 @@ constexpr int TR = 128;           // points per tile side
 constexpr int NTHREADS = 256;
 constexpr uint32_t TMEM_COLS = 256;
 
+// Shared memory holds ONE pair of operand tiles (row points, column points): the keys first, then,
+// once K K^T has been consumed, the values in the same place.  64 KB (d = 128) lets two CTAs share
+// an SM, so one CTA's gather overlaps the other's MMAs and epilogue.
 template <int D> struct Smem {
     static constexpr int KH = D / 64;
     static constexpr int OPERAND = TR * D * 2;                 // one 128-row operand tile, bytes
-    static constexpr int OFF_AK = 0, OFF_AV = OPERAND, OFF_BK = 2 * OPERAND, OFF_BV = 3 * OPERAND;
-    static constexpr int OFF_MISC = 4 * OPERAND;
+    static constexpr int OFF_A = 0, OFF_B = OPERAND;
+    static constexpr int OFF_MISC = 2 * OPERAND;
     static constexpr int TOTAL = OFF_MISC + 2048 + 1024;       // misc block + alignment slack
 };
 
 struct Misc {
-    uint64_t mma_done;
+    uint64_t mma_done[2];        // K K^T done, V V^T done
     uint32_t tmem_base;
     uint32_t pad;
     float colshift[TP];          // M of each pair column, in log2 units
@@ -59,7 +62,7 @@ __device__ __forceinline__ void gather_operand(unsigned char *dst, const __nv_bf
 }
 
 template <int D>
-__global__ void __launch_bounds__(NTHREADS, 1)
+__global__ void __launch_bounds__(NTHREADS, 2)
 gram_tc_kernel(const __nv_bfloat16 *__restrict__ K, const __nv_bfloat16 *__restrict__ V,
                const int32_t *__restrict__ cur, const float *__restrict__ Mpair,
                const unsigned *__restrict__ vmax_bits, int64_t n, int P, int64_t Ptotal,
@@ -103,7 +106,8 @@ gram_tc_kernel(const __nv_bfloat16 *__restrict__ K, const __nv_bfloat16 *__restr
         misc->colshift[tid] = jc < Ptotal ? Mpair[(int64_t)p * (n / 2) + jc] * LOG2E : 0.f;
     }
     if (tid == 0) {
-        mbar_init(&misc->mma_done, 1);
+        mbar_init(&misc->mma_done[0], 1);
+        mbar_init(&misc->mma_done[1], 1);
         fence_barrier_init();
     }
     if (warp == 1) tmem_alloc(&misc->tmem_base, TMEM_COLS);
@@ -111,42 +115,37 @@ gram_tc_kernel(const __nv_bfloat16 *__restrict__ K, const __nv_bfloat16 *__restr
 
     const __nv_bfloat16 *Kp = K + (int64_t)p * n * D;
     const __nv_bfloat16 *Vp = V + (int64_t)p * n * D;
-    gather_operand<D>(smem + SM::OFF_AK, Kp, misc->rowsA, tid);
-    gather_operand<D>(smem + SM::OFF_AV, Vp, misc->rowsA, tid);
-    if (!diagonal) {
-        gather_operand<D>(smem + SM::OFF_BK, Kp, misc->rowsB, tid);
-        gather_operand<D>(smem + SM::OFF_BV, Vp, misc->rowsB, tid);
-    }
-    asm volatile("cp.async.commit_group;" ::: "memory");
-    asm volatile("cp.async.wait_group 0;" ::: "memory");
-    fence_proxy_async();
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem = misc->tmem_base;
-
-    if (tid == 0) {
-        constexpr uint32_t IDESC = umma_idesc_bf16(TR, TR);
-        const uint32_t sAK = smem_u32(smem + SM::OFF_AK), sAV = smem_u32(smem + SM::OFF_AV);
-        const uint32_t sBK = diagonal ? sAK : smem_u32(smem + SM::OFF_BK);
-        const uint32_t sBV = diagonal ? sAV : smem_u32(smem + SM::OFF_BV);
+    constexpr uint32_t IDESC = umma_idesc_bf16(TR, TR);
+    const uint32_t sA = smem_u32(smem + SM::OFF_A);
+    const uint32_t sB = diagonal ? sA : smem_u32(smem + SM::OFF_B);
+    uint32_t tmem = 0;
+    bool ok = true;
 #pragma unroll
-        for (int kh = 0; kh < KH; ++kh)
+    for (int phase = 0; phase < 2; ++phase) {                  // 0: keys -> K K^T, 1: values -> V V^T
+        const __nv_bfloat16 *X = phase == 0 ? Kp : Vp;
+        gather_operand<D>(smem + SM::OFF_A, X, misc->rowsA, tid);
+        if (!diagonal) gather_operand<D>(smem + SM::OFF_B, X, misc->rowsB, tid);
+        asm volatile("cp.async.commit_group;" ::: "memory");
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        fence_proxy_async();
+        tc_fence_before();
+        __syncthreads();
+        tc_fence_after();
+        tmem = misc->tmem_base;
+        if (tid == 0) {
 #pragma unroll
-            for (int ks = 0; ks < 4; ++ks)
-                mma_ss(tmem, umma_desc_k128(sAK + kh * (TR * 128) + ks * 32),
-                       umma_desc_k128(sBK + kh * (TR * 128) + ks * 32), IDESC, (kh | ks) != 0);
+            for (int kh = 0; kh < KH; ++kh)
 #pragma unroll
-        for (int kh = 0; kh < KH; ++kh)
-#pragma unroll
-            for (int ks = 0; ks < 4; ++ks)
-                mma_ss(tmem + 128, umma_desc_k128(sAV + kh * (TR * 128) + ks * 32),
-                       umma_desc_k128(sBV + kh * (TR * 128) + ks * 32), IDESC, (kh | ks) != 0);
-        tc_commit(&misc->mma_done);
+                for (int ks = 0; ks < 4; ++ks)
+                    mma_ss(tmem + phase * 128, umma_desc_k128(sA + kh * (TR * 128) + ks * 32),
+                           umma_desc_k128(sB + kh * (TR * 128) + ks * 32), IDESC, (kh | ks) != 0);
+            tc_commit(&misc->mma_done[phase]);
+        }
+        // the operand tiles are reused by the next phase only after the MMAs have read them
+        ok = ok && mbar_wait(&misc->mma_done[phase], 0);
     }
 
     // epilogue: warp w owns TMEM lanes 32 (w % 4) .. +31 (tile rows) and the column half w / 4
-    const bool ok = mbar_wait(&misc->mma_done, 0);
     if (ok) {
         tc_fence_after();
         const int r = (warp & 3) * 32 + lane;                 // point row in the tile
