@@ -307,6 +307,43 @@ __device__ __forceinline__ uint32_t walk_block_regs(const T (&Fd)[32], T b, T al
     return swaps;
 }
 
+// fp32 walker: the 32 serial steps of a block run in ONE thread with the diagonal tile in shared
+// memory.  Thread-local state d[u] = alpha_u - a_u (1 - 2 U_u) makes "swap pair u" the sign test
+// d[u] < 0; a decision then updates the later d[u] with independent FMAs, so a step costs one
+// compare-select-FMA chain instead of a warp vote.  b_u = 0 (a_u = 0) needs no special case in the
+// updates because then F[., u] = 0 (Cauchy-Schwarz in the RKHS); its decision is U_u < 1/2.
+__device__ __forceinline__ uint32_t walk_block_thread(const float *__restrict__ tile, const float *__restrict__ alpha32,
+                                                      const float *__restrict__ b32, const float *__restrict__ r32,
+                                                      const float *__restrict__ U32, float logfac, float &bmax)
+{
+    float d[32];
+#pragma unroll
+    for (int t = 0; t < 32; ++t) {
+        const float bt = b32[t], carried = bmax * r32[t];
+        bmax = bt > carried ? bt : carried;
+        const float a = bt * bmax * logfac;
+        const float U = U32[t];
+        d[t] = (a > 0.f && isfinite(a)) ? alpha32[t] - a * (1.f - 2.f * U) : (U < 0.5f ? -1.f : 1.f);
+    }
+    uint32_t swaps = 0;
+#pragma unroll
+    for (int t = 0; t < 32; ++t) {
+        const bool sw = d[t] < 0.f;
+        swaps |= (sw ? 1u : 0u) << t;
+        const float s = sw ? 1.f : -1.f;          // alpha_u = -sum_j eta_j F[j,u]: kept pair subtracts
+        const float4 *row = reinterpret_cast<const float4 *>(tile + t * 32);
+#pragma unroll
+        for (int g4 = (t + 1) / 4; g4 < 8; ++g4) {
+            const float4 v = row[g4];
+            if (4 * g4 + 0 > t) d[4 * g4 + 0] = fmaf(s, v.x, d[4 * g4 + 0]);
+            if (4 * g4 + 1 > t) d[4 * g4 + 1] = fmaf(s, v.y, d[4 * g4 + 1]);
+            if (4 * g4 + 2 > t) d[4 * g4 + 2] = fmaf(s, v.z, d[4 * g4 + 2]);
+            if (4 * g4 + 3 > t) d[4 * g4 + 3] = fmaf(s, v.w, d[4 * g4 + 3]);
+        }
+    }
+    return swaps;
+}
+
 // 16-byte asynchronous copy global -> shared
 __device__ __forceinline__ void cp_async16(void *smem_dst, const void *gsrc)
 {
@@ -329,27 +366,33 @@ __device__ __forceinline__ void load4(const double *p, double (&f)[4])
 //   setup      all threads: b_i = sqrt(F[i,i]), the decay factors and the uniforms of every pair
 //              into shared memory; scores alpha = 0.
 //   warp 0     the walker: for block c it adds block c-1's contribution from a 32 x 32 tile that
-//              was copied to shared memory during the previous block, takes the diagonal tile
-//              (c, c) into registers and runs the 32 serial steps without touching memory.
-//   warp 1     also copies the two tiles the walker needs for block c+1 (asynchronous copies).
-//   warps 1..  fold block c-1 into the scores of all columns from block c+1 on, one block behind
-//              the walker (16-byte loads, four adjacent columns per thread).
+//              was copied to shared memory during the previous block and runs the 32 serial steps
+//              on the diagonal tile (c, c) without touching global memory.
+//   warp 1     copies the two tiles the walker needs for block c+1 (asynchronous copies).
+//   warps 2..  the updaters fold block c-1 into the scores of all columns from block c+1 on, one
+//              block behind the walker.  The rows of a block are streamed through two shared-memory
+//              panels with asynchronous copies; F does not depend on the decisions, so the first
+//              panel of the next round is already in flight when its swap mask becomes known.
 // One __syncthreads per block separates the iterations.
 template <typename T>
-__global__ void __launch_bounds__(1024) walk_cta_kernel(const T *__restrict__ F, int64_t F_stride,
-                                                        const T *__restrict__ rdecay,
-                                                        const int32_t *__restrict__ cur,
-                                                        int32_t *__restrict__ out, int64_t out_stride,
-                                                        int64_t n, int P, int level, uint64_t seed,
-                                                        T logfac)
+__global__ void __launch_bounds__(576) walk_cta_kernel(const T *__restrict__ F, int64_t F_stride,
+                                                       const T *__restrict__ rdecay,
+                                                       const int32_t *__restrict__ cur,
+                                                       int32_t *__restrict__ out, int64_t out_stride,
+                                                       int64_t n, int P, int level, uint64_t seed,
+                                                       T logfac)
 {
+    constexpr int PW = 2048 / sizeof(T);                             // panel width in columns (64 KB / 2 buffers... per 32 rows)
     extern __shared__ __align__(16) unsigned char smem_raw[];
     T *tiles = reinterpret_cast<T *>(smem_raw);                      // [2][2][32][32]: buffer, (diag, cross)
     T *alpha_s = tiles + 4 * 1024;                                   // [P] scores from finished rounds
     T *b_s = alpha_s + P;                                            // [P]
     T *r_s = b_s + P;                                                // [P]
     T *U_s = r_s + P;                                                // [P]
-    uint32_t *mask_s = reinterpret_cast<uint32_t *>(U_s + P);        // [P/32] swap masks
+    T *a32_s = U_s + P;                                              // [32] the walker's scores of the block
+    T *panels = a32_s + 32;                                          // [2][32][pw_alloc]
+    const int pw_alloc = P - 64 < PW ? (P - 64 > 0 ? P - 64 : 32) : PW;
+    uint32_t *mask_s = reinterpret_cast<uint32_t *>(panels + 2 * 32 * pw_alloc);   // [P/32] swap masks
     const int p = blockIdx.y, g = blockIdx.x;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int nthr = blockDim.x;
@@ -377,7 +420,27 @@ __global__ void __launch_bounds__(1024) walk_cta_kernel(const T *__restrict__ F,
         r_s[i] = rdecay[(int64_t)p * (n / 2) + base + i];
         U_s[i] = halving_uniform<T>(seed, (uint32_t)i, (uint32_t)g, (uint32_t)level, (uint32_t)p);
     }
-    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    if (warp <= 1) asm volatile("cp.async.wait_group 0;" ::: "memory");
+
+    // ---- updater streaming state ----
+    const int NU = nthr - 64;                                        // updater threads (warps 2..)
+    const int u = threadIdx.x - 64;
+    // panel `pi` of round `r` (rows of block r): columns [32 (r + 2) + pi * PW, ...)
+    auto panels_of = [&](int r) { const int cols = P - 32 * (r + 2); return cols > 0 ? (cols + PW - 1) / PW : 0; };
+    auto issue_panel = [&](int r, int pi, int buf) {
+        const int col0 = 32 * (r + 2) + pi * PW;
+        const int pw = P - col0 < PW ? P - col0 : PW;
+        const int cpr = pw / CH;
+        const T *rows = Fg + (int64_t)(32 * r) * P + col0;
+        T *dst = panels + (size_t)buf * 32 * pw_alloc;
+        for (int q = u; q < 32 * cpr; q += NU) {
+            const int t = q / cpr, k = q % cpr;
+            cp_async16(dst + t * pw_alloc + k * CH, rows + (int64_t)t * P + k * CH);
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    int stream = 0;                                                  // panels consumed so far (buffer parity)
+    if (warp >= 2 && panels_of(0) > 0) issue_panel(0, 0, 0);
     __syncthreads();
 
     T bmax = 0;
@@ -395,41 +458,62 @@ __global__ void __launch_bounds__(1024) walk_cta_kernel(const T *__restrict__ F,
                     alpha += ((pm >> t) & 1u) ? f : -f;
                 }
             }
-            T Fd[32];
+            if constexpr (std::is_same<T, float>::value) {
+                a32_s[lane] = alpha;
+                __syncwarp();
+                if (lane == 0)
+                    mask_s[c] = walk_block_thread(tdiag, a32_s, b_s + i0, r_s + i0, U_s + i0, logfac, bmax);
+            } else {
+                T Fd[32];
 #pragma unroll
-            for (int t = 0; t < 32; ++t) Fd[t] = tdiag[t * 32 + lane];
-            const uint32_t swaps = walk_block_regs<T>(Fd, b_s[i0 + lane], alpha, r_s[i0 + lane], U_s[i0 + lane],
-                                                      logfac, bmax, lane);
-            const uint32_t sw = (swaps >> lane) & 1u;
-            if (lane == 0) mask_s[c] = swaps;
-            out[(int64_t)p * out_stride + base + i0 + lane] = cur[(int64_t)p * n + 2 * (base + i0 + lane) + sw];
-        } else {
-            if (warp == 1 && c + 1 < nb) {
+                for (int t = 0; t < 32; ++t) Fd[t] = tdiag[t * 32 + lane];
+                const uint32_t swaps = walk_block_regs<T>(Fd, b_s[i0 + lane], alpha, r_s[i0 + lane], U_s[i0 + lane],
+                                                          logfac, bmax, lane);
+                if (lane == 0) mask_s[c] = swaps;
+            }
+        } else if (warp == 1) {
+            if (c + 1 < nb) {
                 copy_tile(ndiag, i0 + 32, i0 + 32);
                 copy_tile(ncross, i0, i0 + 32);
                 asm volatile("cp.async.commit_group;" ::: "memory");
+                asm volatile("cp.async.wait_group 0;" ::: "memory");
             }
-            if (c > 0) {
-                // round c-1: rows of block c-1 into every column from block c+1 on
-                const uint32_t pm = mask_s[c - 1];
-                const T *rows = Fg + (int64_t)(i0 - 32) * P;
-                for (int i = i0 + 32 + 4 * (threadIdx.x - 32); i < P; i += 4 * (nthr - 32)) {
-                    T acc[4] = {0, 0, 0, 0};
-#pragma unroll 8
+        } else if (c > 0) {
+            // round r = c-1: rows of block r into every column from block r+2 on
+            const int r = c - 1;
+            const uint32_t pm = mask_s[r];
+            const int np = panels_of(r);
+            for (int pi = 0; pi < np; ++pi, ++stream) {
+                const int buf = stream & 1;
+                bool issued = true;
+                if (pi + 1 < np) issue_panel(r, pi + 1, buf ^ 1);
+                else if (panels_of(c) > 0) issue_panel(c, 0, buf ^ 1);       // first panel of the next round
+                else issued = false;
+                if (issued) asm volatile("cp.async.wait_group 1;" ::: "memory");
+                else asm volatile("cp.async.wait_group 0;" ::: "memory");
+                asm volatile("bar.sync 1, %0;" ::"r"(NU) : "memory");
+                const int col0 = 32 * (r + 2) + pi * PW;
+                const int pw = P - col0 < PW ? P - col0 : PW;
+                const T *src = panels + (size_t)buf * 32 * pw_alloc;
+                for (int j = u; j < pw; j += NU) {
+                    T acc = 0;
+#pragma unroll
                     for (int t = 0; t < 32; ++t) {
-                        T f[4];
-                        load4(rows + (int64_t)t * P + i, f);
-                        const bool sw = (pm >> t) & 1u;
-#pragma unroll
-                        for (int k = 0; k < 4; ++k) acc[k] += sw ? f[k] : -f[k];
+                        const T f = src[t * pw_alloc + j];
+                        acc += ((pm >> t) & 1u) ? f : -f;
                     }
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) alpha_s[i + k] += acc[k];
+                    alpha_s[col0 + j] += acc;
                 }
+                asm volatile("bar.sync 1, %0;" ::"r"(NU) : "memory");
             }
-            if (warp == 1) asm volatile("cp.async.wait_group 0;" ::: "memory");
         }
         __syncthreads();
+    }
+    // survivors: pair i keeps its second point when it was swapped (kept out of the walker's loop,
+    // where a dependent global load would stall the one warp everything waits for)
+    for (int i = threadIdx.x; i < P; i += nthr) {
+        const uint32_t sw = (mask_s[i >> 5] >> (i & 31)) & 1u;
+        out[(int64_t)p * out_stride + base + i] = cur[(int64_t)p * n + 2 * (base + i) + sw];
     }
 }
 
@@ -582,14 +666,16 @@ static int compress_impl(const Tin *K, const Tin *V, const elm_params *p, uint64
             StageTimer t(ELM_STAGE_WALK, st, 1);
             if (P >= 32) {
                 // one walker warp plus enough warps to sweep the remaining columns once per block
-                // four columns per updater thread cover the call's remaining columns in one sweep
-                int warps = P / 128 + 1;
-                warps = warps > 32 ? 32 : warps;
-                if (P >= 64 && warps < 2) warps = 2;
-                const size_t smem = (size_t)(4 * 1024 + 4 * P) * sizeof(T) + (size_t)(P / 32) * 4;
+                // walker warp + tile-copy warp + updaters (one per two pairs, at most 512 threads)
+                int upd = P / 2;
+                upd = upd < 32 ? 32 : (upd > 512 ? 512 : upd);
+                const int threads = P == 32 ? 32 : 64 + upd;
+                constexpr int PW = 2048 / sizeof(T);
+                const int pw_alloc = P - 64 < PW ? (P - 64 > 0 ? P - 64 : 32) : PW;
+                const size_t smem = (size_t)(4 * 1024 + 4 * P + 32 + 2 * 32 * pw_alloc) * sizeof(T) + (size_t)(P / 32) * 4;
                 auto kern = walk_cta_kernel<T>;
                 ELM_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-                kern<<<dim3((unsigned)groups, (unsigned)BH), warps * 32, smem, st>>>(
+                kern<<<dim3((unsigned)groups, (unsigned)BH), threads, smem, st>>>(
                     F, L.F_stride, rdecay, cur, out, out_stride, n, P, level, seed, logfac);
             } else {
                 walk_warp_kernel<T><<<dim3((unsigned)((groups + 7) / 8), (unsigned)BH), 256, 0, st>>>(
