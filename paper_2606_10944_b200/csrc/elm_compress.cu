@@ -16,6 +16,32 @@ namespace elm {
 // ---------------------------------------------------------------------------------------------
 // Stage S0: per attention problem v_max (Eq. katt), c_t = ||k_t||^2 / sqrt(d), identity index list
 // ---------------------------------------------------------------------------------------------
+// 16-byte row chunks: 8 bf16 or 4 fp32 elements
+template <typename T> __device__ __forceinline__ void chunk_sq_absmax(const __nv_bfloat16 *kp, const __nv_bfloat16 *vp, T &sq, float &vm)
+{
+    const uint4 kq = __ldg(reinterpret_cast<const uint4 *>(kp));
+    const uint4 vq = __ldg(reinterpret_cast<const uint4 *>(vp));
+    const uint32_t kw[4] = {kq.x, kq.y, kq.z, kq.w}, vw[4] = {vq.x, vq.y, vq.z, vq.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const T a = (T)__uint_as_float(kw[i] << 16), b = (T)__uint_as_float(kw[i] & 0xffff0000u);
+        sq += a * a;
+        sq += b * b;
+        vm = fmaxf(vm, fmaxf(fabsf(__uint_as_float(vw[i] << 16)), fabsf(__uint_as_float(vw[i] & 0xffff0000u))));
+    }
+}
+template <typename T> __device__ __forceinline__ void chunk_sq_absmax(const float *kp, const float *vp, T &sq, float &vm)
+{
+    const float4 kq = __ldg(reinterpret_cast<const float4 *>(kp));
+    const float4 vq = __ldg(reinterpret_cast<const float4 *>(vp));
+    sq += (T)kq.x * (T)kq.x;
+    sq += (T)kq.y * (T)kq.y;
+    sq += (T)kq.z * (T)kq.z;
+    sq += (T)kq.w * (T)kq.w;
+    vm = fmaxf(vm, fmaxf(fmaxf(fabsf(vq.x), fabsf(vq.y)), fmaxf(fabsf(vq.z), fabsf(vq.w))));
+}
+
+// One pass over K and V with 16-byte loads: a group of (row bytes / 16) lanes owns a row.
 template <typename Tin, typename T>
 __global__ void __launch_bounds__(256) prepass_kernel(const Tin *__restrict__ K,
                                                       const Tin *__restrict__ V, int64_t n, int d,
@@ -23,32 +49,29 @@ __global__ void __launch_bounds__(256) prepass_kernel(const Tin *__restrict__ K,
                                                       unsigned *__restrict__ vmax_bits,
                                                       int32_t *__restrict__ cur)
 {
+    constexpr int EPC = 16 / sizeof(Tin);                 // elements per 16-byte chunk
     const int p = blockIdx.y;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int64_t row0 = (int64_t)blockIdx.x * 64;
+    const int lpr = d / EPC;                              // lanes per row: 8, 16 or 32
+    const int rows_per_pass = 256 / lpr;
+    const int sub = threadIdx.x % lpr, rloc = threadIdx.x / lpr;
+    const int64_t row0 = (int64_t)blockIdx.x * 256;       // 256 rows per CTA
     const Tin *Kp = K + (int64_t)p * n * d;
     const Tin *Vp = V + (int64_t)p * n * d;
     const T rsd = sqrt((T)d);
     float vm = 0.f;
-    for (int r = warp; r < 64; r += 8) {
-        int64_t t = row0 + r;
-        if (t >= n) break;
+    for (int r = rloc; r < 256; r += rows_per_pass) {
+        const int64_t t = row0 + r;
         T s = 0;
-        for (int e = lane; e < d; e += 32) {
-            T kv = load_as<T>(Kp, t * d + e);
-            s += kv * kv;
-            vm = fmaxf(vm, fabsf(load_as<float>(Vp, t * d + e)));
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-        if (lane == 0) {
+        if (t < n) chunk_sq_absmax<T>(Kp + t * d + sub * EPC, Vp + t * d + sub * EPC, s, vm);
+        for (int o = lpr >> 1; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        if (sub == 0 && t < n) {
             cnorm[(int64_t)p * n + t] = s / rsd;
             cur[(int64_t)p * n + t] = (int32_t)t;
         }
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) vm = fmaxf(vm, __shfl_xor_sync(0xffffffffu, vm, o));
-    if (lane == 0) atomicMax(vmax_bits + p, __float_as_uint(vm));   // non-negative floats order as uints
+    if ((threadIdx.x & 31) == 0) atomicMax(vmax_bits + p, __float_as_uint(vm));   // non-negative floats order as uints
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -57,19 +80,20 @@ __global__ void __launch_bounds__(256) prepass_kernel(const Tin *__restrict__ K,
 // One CTA per call.
 // ---------------------------------------------------------------------------------------------
 template <typename T>
-__global__ void __launch_bounds__(128) level_prep_kernel(const T *__restrict__ cnorm,
+__global__ void __launch_bounds__(1024) level_prep_kernel(const T *__restrict__ cnorm,
                                                          const int32_t *__restrict__ cur, int64_t n,
                                                          int P, T *__restrict__ Mpair,
                                                          T *__restrict__ rdecay)
 {
-    __shared__ T warp_tot[4];
+    __shared__ T warp_tot[32];
     const int p = blockIdx.y, g = blockIdx.x;
+    const int nthr = blockDim.x, nwarp = nthr >> 5;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const T *cp = cnorm + (int64_t)p * n;
     const int32_t *curp = cur + (int64_t)p * n;
     const int64_t base = (int64_t)g * P;
     T carry = 0;            // c >= 0, so 0 is the identity of the running max
-    for (int c0 = 0; c0 < P; c0 += 128) {
+    for (int c0 = 0; c0 < P; c0 += nthr) {
         int i = c0 + threadIdx.x;
         T v = 0;
         if (i < P) {
@@ -94,7 +118,7 @@ __global__ void __launch_bounds__(128) level_prep_kernel(const T *__restrict__ c
             rdecay[(int64_t)p * (n / 2) + base + i] = (i == 0) ? (T)1 : (T)exp(-(double)(M - excl) * 0.5);
         }
         T tot = carry;
-        for (int w = 0; w < 4; ++w) tot = tot > warp_tot[w] ? tot : warp_tot[w];
+        for (int w = 0; w < nwarp; ++w) tot = tot > warp_tot[w] ? tot : warp_tot[w];
         __syncthreads();
         carry = tot;
     }
@@ -628,7 +652,7 @@ static int compress_impl(const Tin *K, const Tin *V, const elm_params *p, uint64
     if (m > 0) {
         StageTimer t(ELM_STAGE_PREPASS, st, 1);
         ELM_CUDA_TRY(cudaMemsetAsync(vmax_bits, 0, (size_t)(BH + 1) * 4, st));
-        dim3 grid((unsigned)((n + 63) / 64), (unsigned)BH);
+        dim3 grid((unsigned)((n + 255) / 256), (unsigned)BH);
         prepass_kernel<Tin, T><<<grid, 256, 0, st>>>(K, V, n, p->d, cnorm, vmax_bits, cur);
         count_launches(1);
         ELM_CUDA_TRY(cudaGetLastError());
@@ -645,7 +669,8 @@ static int compress_impl(const Tin *K, const Tin *V, const elm_params *p, uint64
         const int64_t out_stride = last ? n_out : n;
         {
             StageTimer t(ELM_STAGE_LEVEL_PREP, st, 1);
-            level_prep_kernel<T><<<dim3((unsigned)groups, (unsigned)BH), 128, 0, st>>>(cnorm, cur, n, P, Mpair, rdecay);
+            const int lp_threads = P >= 1024 ? 1024 : (P <= 32 ? 32 : (P + 31) / 32 * 32);
+            level_prep_kernel<T><<<dim3((unsigned)groups, (unsigned)BH), lp_threads, 0, st>>>(cnorm, cur, n, P, Mpair, rdecay);
             count_launches(1);
             ELM_CUDA_TRY(cudaGetLastError());
         }
