@@ -3,13 +3,14 @@
 //   O[j,:] = sum_c w_c exp(<q_j,k_c>/sqrt(d)) v_c / sum_c w_c exp(<q_j,k_c>/sqrt(d))      Eq. (def:att_approx)
 //
 // One CTA owns two tiles of 128 queries of one head and streams the head's coreset in blocks of
-// 128 points.  Roles (320 threads):
-//   warps 0-3 / 4-7  softmax of query tile 0 / 1: read the logits from TMEM (one row per thread),
-//                    keep a running row maximum and denominator, write the probabilities back to
-//                    TMEM as packed bf16 (they overwrite the logits), rescale the output
-//                    accumulator only when the maximum grew by more than 2^8, and run the epilogue
-//   warp 8           TMA producer: Q tiles once, then K / V^T blocks through a 2-stage ring
-//   warp 9           tcgen05.mma issuer: S = Q K^T (operands in shared memory), O += P V (P read
+// 128 points.  Roles (576 threads):
+//   warps 0-7 / 8-15 softmax of query tile 0 / 1, two passes over the logits in TMEM (row maximum,
+//                    then probabilities).  A thread owns one row and half of the block's columns;
+//                    the two halves exchange row maxima through shared memory.  Probabilities go
+//                    back to TMEM as packed bf16 (over the logits); the output accumulator is
+//                    rescaled only when the maximum grew by more than 2^8.  Same warps: epilogue.
+//   warp 16          TMA producer: Q tiles once, then K / V^T blocks through a 2-stage ring
+//   warp 17          tcgen05.mma issuer: S = Q K^T (operands in shared memory), O += P V (P read
 //                    from TMEM, V^T from shared memory); owns the TMEM allocation
 // TMEM columns: [0,128) S/P of tile 0, [128,256) S/P of tile 1, [256,256+D) O of tile 0,
 // [384,384+D) O of tile 1.  Every mbarrier wait is bounded; on expiry the CTA records a status
@@ -21,20 +22,14 @@
 #include "elm_common.cuh"
 #include "elm_sm100.cuh"
 
-#ifdef ELM_TRACE
-__device__ long long g_trace_buf[8192];
-#define TRACE(slot) do { if (trace_on) g_trace_buf[(slot)] = clock64(); } while (0)
-#else
-#define TRACE(slot) do { } while (0)
-#endif
-
 namespace elm {
 namespace tc {
 
 constexpr int BM = 128;          // query rows per tile (= TMEM lanes)
 constexpr int BN = 128;          // coreset points per block
 constexpr int STAGES = 2;
-constexpr int NTHREADS = 320;
+constexpr int NTHREADS = 576;          // 16 softmax warps + TMA producer + MMA issuer
+constexpr int TMA_WARP = 16, MMA_WARP = 17;
 constexpr uint32_t TMEM_COLS = 512;
 constexpr float RESCALE_TAU = 8.0f;      // rescale the accumulator only if the max grew by > 2^8
 
@@ -46,6 +41,7 @@ struct __align__(8) Barriers {
     uint64_t s_full[2], p_ready[2], o_done[2];
     uint32_t tmem_base;
     uint32_t abort_flag;
+    float xchg[2][2][BM];        // per tile, per column half: row maxima / denominators being exchanged
 };
 
 template <int D> struct Smem {
@@ -57,7 +53,7 @@ template <int D> struct Smem {
     static constexpr int OFF_K = OFF_Q + 2 * Q_TILE;
     static constexpr int OFF_V = OFF_K + STAGES * K_BLOCK;
     static constexpr int OFF_BAR = OFF_V + STAGES * V_BLOCK;
-    static constexpr int TOTAL = OFF_BAR + 256 + 1024;      // + slack for 1024-byte alignment
+    static constexpr int TOTAL = OFF_BAR + 4096 + 1024;     // barrier block + slack for 1024-byte alignment
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -107,6 +103,101 @@ __global__ void __launch_bounds__(256) gather_tc_kernel(const __nv_bfloat16 *__r
 }
 
 // ---------------------------------------------------------------------------------------------
+// softmax helpers: a thread owns one row (TMEM lane) and NCH chunks of 32 logit columns
+// ---------------------------------------------------------------------------------------------
+// Row maximum in base-2 units (bias and tail mask applied when SPECIAL); the logits stay in TMEM.
+template <bool SPECIAL, int NCH>
+__device__ __forceinline__ float row_max(uint32_t tS, float scale_log2, const float *bias_cols, int valid)
+{
+    float m0 = -INFINITY, m1 = -INFINITY;
+    uint32_t a[2][32];
+    tmem_ld32(tS, a[0]);
+#pragma unroll
+    for (int q = 0; q < NCH; ++q) {
+        tmem_wait_ld();
+        if (q + 1 < NCH) tmem_ld32(tS + (q + 1) * 32, a[(q + 1) & 1]);
+        if (!SPECIAL) {
+#pragma unroll
+            for (int c = 0; c < 32; c += 4) {
+                m0 = max3(m0, __uint_as_float(a[q & 1][c]), __uint_as_float(a[q & 1][c + 1]));
+                m1 = max3(m1, __uint_as_float(a[q & 1][c + 2]), __uint_as_float(a[q & 1][c + 3]));
+            }
+        } else {
+#pragma unroll
+            for (int c = 0; c < 32; ++c) {
+                float v = __uint_as_float(a[q & 1][c]) * scale_log2;
+                if (bias_cols) v += __ldg(bias_cols + q * 32 + c);
+                if (q * 32 + c >= valid) v = -INFINITY;
+                m0 = fmaxf(m0, v);
+            }
+        }
+    }
+    return SPECIAL ? m0 : fmaxf(m0, m1) * scale_log2;
+}
+
+// p = 2^(logit - reference): reads the logits, writes the probabilities as packed bf16 to tP
+// (16 columns per chunk) and returns their fp32 row sum.  Each chunk is staged (all scalings, then
+// all exponentials, ...) so that independent operations interleave.
+template <bool SPECIAL, int NCH>
+__device__ __forceinline__ float exp_pass(uint32_t tS, uint32_t tP, float scale_log2, float neg_m,
+                                          const float *bias_cols, int valid)
+{
+    const uint64_t scale2 = pack2(scale_log2, scale_log2), negm2 = pack2(neg_m, neg_m);
+    uint64_t sum2 = pack2(0.f, 0.f), sum2b = pack2(0.f, 0.f);
+    float sum0 = 0.f;
+    uint32_t a[2][32];
+    tmem_ld32(tS, a[0]);
+#pragma unroll
+    for (int q = 0; q < NCH; ++q) {
+        tmem_wait_ld();
+        if (q + 1 < NCH) tmem_ld32(tS + (q + 1) * 32, a[(q + 1) & 1]);
+        uint32_t pk[16];
+        if (!SPECIAL) {
+            uint64_t x2[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i)
+                x2[i] = fma2(pack2(__uint_as_float(a[q & 1][2 * i]), __uint_as_float(a[q & 1][2 * i + 1])), scale2, negm2);
+            float pe[32];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                float x0, x1;
+                unpack2(x2[i], x0, x1);
+                pe[2 * i] = fast_exp2(x0);
+                pe[2 * i + 1] = fast_exp2(x1);
+            }
+#pragma unroll
+            for (int i = 0; i < 16; i += 2) {
+                sum2 = add2(sum2, pack2(pe[2 * i], pe[2 * i + 1]));
+                sum2b = add2(sum2b, pack2(pe[2 * i + 2], pe[2 * i + 3]));
+            }
+            // round to bf16 on the integer pipe: add half an ulp, keep the upper halves
+#pragma unroll
+            for (int i = 0; i < 16; ++i)
+                pk[i] = __byte_perm(__float_as_uint(pe[2 * i]) + 0x8000u, __float_as_uint(pe[2 * i + 1]) + 0x8000u, 0x7632);
+        } else {
+#pragma unroll
+            for (int c = 0; c < 32; c += 2) {
+                float v0 = __uint_as_float(a[q & 1][c]) * scale_log2, v1 = __uint_as_float(a[q & 1][c + 1]) * scale_log2;
+                if (bias_cols) { v0 += __ldg(bias_cols + q * 32 + c); v1 += __ldg(bias_cols + q * 32 + c + 1); }
+                const float p0 = (q * 32 + c < valid) ? fast_exp2(v0 + neg_m) : 0.f;
+                const float p1 = (q * 32 + c + 1 < valid) ? fast_exp2(v1 + neg_m) : 0.f;
+                sum0 += p0 + p1;
+                pk[c >> 1] = __byte_perm(__float_as_uint(p0) + 0x8000u, __float_as_uint(p1) + 0x8000u, 0x7632);
+            }
+        }
+        asm volatile(
+            "tcgen05.st.sync.aligned.32x32b.x16.b32 [%16], {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15};"
+            ::"r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3]), "r"(pk[4]), "r"(pk[5]), "r"(pk[6]), "r"(pk[7]),
+              "r"(pk[8]), "r"(pk[9]), "r"(pk[10]), "r"(pk[11]), "r"(pk[12]), "r"(pk[13]), "r"(pk[14]), "r"(pk[15]),
+              "r"(tP + q * 16)
+            : "memory");
+    }
+    float s_lo, s_hi;
+    unpack2(add2(sum2, sum2b), s_lo, s_hi);
+    return sum0 + s_lo + s_hi;
+}
+
+// ---------------------------------------------------------------------------------------------
 // the attention kernel
 // ---------------------------------------------------------------------------------------------
 template <int D>
@@ -142,22 +233,19 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
         }
         for (int t = 0; t < 2; ++t) {
             mbar_init(&bar->s_full[t], 1);
-            mbar_init(&bar->p_ready[t], 128);
+            mbar_init(&bar->p_ready[t], 256);
             mbar_init(&bar->o_done[t], 1);
         }
         bar->abort_flag = 0;
         fence_barrier_init();
     }
-    if (warp == 9) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&bar->tmem_base)), "r"(TMEM_COLS) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
+    if (warp == MMA_WARP) tmem_alloc(&bar->tmem_base, TMEM_COLS);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = bar->tmem_base;
 
-    if (warp == 8) {
+    if (warp == TMA_WARP) {
         // ------------------------------ TMA producer ------------------------------
         if (lane == 0) {
             mbar_expect_tx(&bar->q_full, 2 * SM::Q_TILE);
@@ -181,32 +269,34 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
             }
             if (!ok) { atomicExch(status, 1); bar->abort_flag = 1; }
         }
-    } else if (warp == 9) {
+    } else if (warp == MMA_WARP) {
         // ------------------------------ MMA issuer ------------------------------
         if (lane == 0) {
             constexpr uint32_t IDESC_QK = umma_idesc_bf16(BM, BN);
             constexpr uint32_t IDESC_PV = umma_idesc_bf16(BM, D);
-            const uint32_t sQ = smem_u32(smem + SM::OFF_Q), sK = smem_u32(smem + SM::OFF_K), sV = smem_u32(smem + SM::OFF_V);
+            // descriptors differ only in the 14-bit start-address field (address / 16)
+            const uint64_t dQ = umma_desc_k128(smem_u32(smem + SM::OFF_Q));
+            const uint64_t dK = umma_desc_k128(smem_u32(smem + SM::OFF_K));
+            const uint64_t dV = umma_desc_k128(smem_u32(smem + SM::OFF_V));
             auto issue_qk = [&](int t, int s) {
+                const uint64_t a0 = dQ + (uint64_t)(t * (SM::Q_TILE >> 4));
+                const uint64_t b0 = dK + (uint64_t)(s * (SM::K_BLOCK >> 4));
 #pragma unroll
                 for (int kh = 0; kh < KH; ++kh)
 #pragma unroll
                     for (int ks = 0; ks < 4; ++ks)
-                        mma_ss(tmem + t * 128, umma_desc_k128(sQ + t * SM::Q_TILE + kh * (BM * 128) + ks * 32),
-                               umma_desc_k128(sK + s * SM::K_BLOCK + kh * (BN * 128) + ks * 32), IDESC_QK, (kh | ks) != 0);
+                        mma_ss(tmem + t * 128, a0 + (uint64_t)(kh * (BM * 128 >> 4) + ks * 2),
+                               b0 + (uint64_t)(kh * (BN * 128 >> 4) + ks * 2), IDESC_QK, (kh | ks) != 0);
             };
             auto issue_pv = [&](int t, int s, bool acc) {
+                const uint64_t b0 = dV + (uint64_t)(s * (SM::V_BLOCK >> 4));
 #pragma unroll
                 for (int hh = 0; hh < 2; ++hh)
 #pragma unroll
                     for (int ks = 0; ks < 4; ++ks)
                         mma_ts(tmem + 256 + t * 128, tmem + t * 128 + hh * 32 + ks * 8,
-                               umma_desc_k128(sV + s * SM::V_BLOCK + hh * (D * 128) + ks * 32), IDESC_PV,
-                               (acc || (hh | ks) != 0) ? 1u : 0u);
+                               b0 + (uint64_t)(hh * (D * 128 >> 4) + ks * 2), IDESC_PV, (acc || (hh | ks) != 0) ? 1u : 0u);
             };
-#ifdef ELM_TRACE
-            const bool trace_on = blockIdx.x == 3 && blockIdx.y == 0;
-#endif
             bool ok = mbar_wait(&bar->q_full, 0) && mbar_wait(&bar->k_full[0], 0);
             if (ok) {
                 tc_fence_after();
@@ -219,16 +309,13 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                 const int sn = (j + 1) % STAGES;
                 if (more) ok = mbar_wait(&bar->k_full[sn], (uint32_t)((j + 1) / STAGES) & 1u);
                 ok = ok && mbar_wait(&bar->v_full[s], (uint32_t)(j / STAGES) & 1u);
-                TRACE(4096 + j * 8 + 0);
                 for (int t = 0; t < 2 && ok; ++t) {
                     ok = mbar_wait(&bar->p_ready[t], (uint32_t)j & 1u);
                     if (!ok) break;
-                    TRACE(4096 + j * 8 + 1 + 2 * t);
                     tc_fence_after();
                     issue_pv(t, s, j > 0);
                     tc_commit(&bar->o_done[t]);
                     if (more) { issue_qk(t, sn); tc_commit(&bar->s_full[t]); }
-                    TRACE(4096 + j * 8 + 2 + 2 * t);
                 }
                 if (!ok) break;
                 tc_commit(&bar->v_empty[s]);
@@ -238,56 +325,34 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
         }
     } else {
         // ------------------------------ softmax + epilogue ------------------------------
-        const int t = warp >> 2;                                   // query tile of this warpgroup
+        // 8 warps per query tile: warps with the same (warp % 4) share 32 rows (TMEM lanes) and split
+        // the block's 128 columns in two halves; the halves exchange their row maxima (and, at the
+        // end, their denominators) through shared memory.
+        const int t = warp >> 3;                                   // query tile
+        const int hh = (warp >> 2) & 1;                            // column half
         const int row = (warp & 3) * 32 + lane;                    // row in the tile = TMEM lane
         const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
-        const uint32_t tS = tmem + lane_addr + t * 128;            // logits / probabilities
-        const uint32_t tO = tmem + lane_addr + 256 + t * 128;      // output accumulator
+        const uint32_t tS = tmem + lane_addr + t * 128 + hh * 64;  // this thread's 64 logit columns
+        const uint32_t tP = tmem + lane_addr + t * 128 + hh * 32;  // ... and where their bf16 probabilities go
+        const uint32_t tO = tmem + lane_addr + 256 + t * 128 + hh * (D / 2);   // its half of the accumulator
+        float *xmine = bar->xchg[t][hh], *xother = bar->xchg[t][hh ^ 1];
         const bool use_bias = nonuniform[prob] != 0;
-        const float *bp = bias + (int64_t)prob * n_pad;
+        const float *bp = bias + (int64_t)prob * n_pad + hh * 64;
         float m_ref = -INFINITY, l = 0.f;
         bool ok = true;
-#ifdef ELM_TRACE
-        const bool trace_on = blockIdx.x == 3 && blockIdx.y == 0 && (warp & 3) == ELM_TRACE_WARP && lane == 0;
-        const int tb = t * 2048;
-#endif
         for (int j = 0; j < nblk; ++j) {
-            TRACE(tb + j * 8 + 0);
             ok = mbar_wait(&bar->s_full[t], (uint32_t)j & 1u);
             if (!ok) break;
             tc_fence_after();
-            TRACE(tb + j * 8 + 1);
-            const int valid = n_core - j * BN;                     // columns of this block that exist
-            const bool special = use_bias || valid < BN;           // per-column bias and/or a ragged tail
-            // ---- pass 1: row maximum (the logits stay in TMEM and are read again in pass 2) ----
-            float mx;
-            {
-                float m0 = -INFINITY, m1 = -INFINITY;
-                uint32_t a[2][32];
-                tmem_ld32(tS, a[0]);
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    tmem_wait_ld();
-                    if (q < 3) tmem_ld32(tS + (q + 1) * 32, a[(q + 1) & 1]);
-                    if (!special) {
-#pragma unroll
-                        for (int c = 0; c < 32; c += 4) {
-                            m0 = max3(m0, __uint_as_float(a[q & 1][c]), __uint_as_float(a[q & 1][c + 1]));
-                            m1 = max3(m1, __uint_as_float(a[q & 1][c + 2]), __uint_as_float(a[q & 1][c + 3]));
-                        }
-                    } else {
-#pragma unroll
-                        for (int c = 0; c < 32; ++c) {
-                            float v = __uint_as_float(a[q & 1][c]) * scale_log2;
-                            if (use_bias) v += __ldg(bp + j * BN + q * 32 + c);
-                            if (q * 32 + c >= valid) v = -INFINITY;
-                            m0 = fmaxf(m0, v);
-                        }
-                    }
-                }
-                mx = special ? m0 : fmaxf(m0, m1) * scale_log2;
-            }
-            TRACE(tb + j * 8 + 2);
+            const int valid = n_core - j * BN - hh * 64;           // of this thread's 64 columns, how many exist
+            const bool special = use_bias || valid < 64;           // per-column bias and/or a ragged tail
+            const float *bcols = use_bias ? bp + j * BN : nullptr;
+            // ---- pass 1: row maximum over both halves ----
+            const float mh = special ? row_max<true, 2>(tS, scale_log2, bcols, valid)
+                                     : row_max<false, 2>(tS, scale_log2, bcols, valid);
+            xmine[row] = mh;
+            asm volatile("bar.sync %0, 256;" ::"r"(1 + t) : "memory");
+            const float mx = fmaxf(mh, xother[row]);
             // lazy rescale: keep the old reference unless the maximum grew by more than 2^TAU
             const bool grow = mx > m_ref + RESCALE_TAU;
             if (__any_sync(0xffffffffu, grow)) {
@@ -297,7 +362,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                     tc_fence_after();
                     const float alpha = grow ? fast_exp2(m_ref - mx) : 1.f;
 #pragma unroll
-                    for (int q = 0; q < D / 32; ++q) {
+                    for (int q = 0; q < D / 64; ++q) {
                         uint32_t o[32];
                         tmem_ld32(tO + q * 32, o);
                         tmem_wait_ld();
@@ -309,88 +374,23 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                 }
                 if (grow) m_ref = mx;
             }
-            TRACE(tb + j * 8 + 3);
-            // ---- pass 2: p = 2^(s - m_ref), running denominator, bf16 probabilities back to TMEM ----
-            const float neg_m = -m_ref;
-            const uint64_t scale2 = pack2(scale_log2, scale_log2), negm2 = pack2(neg_m, neg_m);
-            uint64_t sum2 = pack2(0.f, 0.f), sum2b = pack2(0.f, 0.f);
-            float sum0 = 0.f;
-            {
-                uint32_t a[2][32];
-                tmem_ld32(tS, a[0]);
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    tmem_wait_ld();
-                    if (q < 3) tmem_ld32(tS + (q + 1) * 32, a[(q + 1) & 1]);
-                    uint32_t pk[16];
-                    if (!special) {
-                        // staged over the 16 pairs of the chunk so that independent work interleaves
-                        uint64_t x2[16];
-#pragma unroll
-                        for (int i = 0; i < 16; ++i)
-                            x2[i] = fma2(pack2(__uint_as_float(a[q & 1][2 * i]), __uint_as_float(a[q & 1][2 * i + 1])), scale2, negm2);
-                        float pe[32];
-#pragma unroll
-                        for (int i = 0; i < 16; ++i) {
-                            float x0, x1;
-                            unpack2(x2[i], x0, x1);
-                            pe[2 * i] = fast_exp2(x0);
-                            pe[2 * i + 1] = fast_exp2(x1);
-                        }
-#pragma unroll
-                        for (int i = 0; i < 16; i += 2) {
-                            sum2 = add2(sum2, pack2(pe[2 * i], pe[2 * i + 1]));
-                            sum2b = add2(sum2b, pack2(pe[2 * i + 2], pe[2 * i + 3]));
-                        }
-#pragma unroll
-                        for (int i = 0; i < 16; ++i)
-                            pk[i] = __byte_perm(__float_as_uint(pe[2 * i]) + 0x8000u, __float_as_uint(pe[2 * i + 1]) + 0x8000u, 0x7632);
-                    } else {
-#pragma unroll
-                        for (int c = 0; c < 32; c += 2) {
-                            float v0 = __uint_as_float(a[q & 1][c]) * scale_log2, v1 = __uint_as_float(a[q & 1][c + 1]) * scale_log2;
-                            if (use_bias) { v0 += __ldg(bp + j * BN + q * 32 + c); v1 += __ldg(bp + j * BN + q * 32 + c + 1); }
-                            const float p0 = (q * 32 + c < valid) ? fast_exp2(v0 + neg_m) : 0.f;
-                            const float p1 = (q * 32 + c + 1 < valid) ? fast_exp2(v1 + neg_m) : 0.f;
-                            sum0 += p0 + p1;
-                            // round to bf16 on the integer pipe: add half an ulp, keep the upper halves
-                            pk[c >> 1] = __byte_perm(__float_as_uint(p0) + 0x8000u, __float_as_uint(p1) + 0x8000u, 0x7632);
-                        }
-                    }
-                    // 16 packed columns: probabilities of points 32q .. 32q+31 of this block
-#ifdef ELM_NOST
-                    if (pk[0] == 0x12345678u && pk[7] == 0x9abcdef0u && pk[15] == 77u)
-#endif
-                    asm volatile(
-                        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%16], {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15};"
-                        ::"r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3]), "r"(pk[4]), "r"(pk[5]), "r"(pk[6]), "r"(pk[7]),
-                          "r"(pk[8]), "r"(pk[9]), "r"(pk[10]), "r"(pk[11]), "r"(pk[12]), "r"(pk[13]), "r"(pk[14]), "r"(pk[15]),
-                          "r"(tS + q * 16)
-                        : "memory");
-                }
-            }
-            {
-                float s_lo, s_hi;
-                unpack2(add2(sum2, sum2b), s_lo, s_hi);
-                sum0 += s_lo + s_hi;
-            }
-            const float sum1 = 0.f;
-            l += sum0 + sum1;
-            TRACE(tb + j * 8 + 4);
+            // ---- pass 2: probabilities and running denominator ----
+            l += special ? exp_pass<true, 2>(tS, tP, scale_log2, -m_ref, bcols, valid)
+                         : exp_pass<false, 2>(tS, tP, scale_log2, -m_ref, bcols, valid);
             tmem_wait_st();
             tc_fence_before();
-            TRACE(tb + j * 8 + 5);
             mbar_arrive(&bar->p_ready[t]);
-            TRACE(tb + j * 8 + 6);
         }
         if (ok) ok = mbar_wait(&bar->o_done[t], (uint32_t)(nblk - 1) & 1u);
         if (ok) {
             tc_fence_after();
-            const float inv = 1.f / l;
+            xmine[row] = l;
+            asm volatile("bar.sync %0, 256;" ::"r"(1 + t) : "memory");
+            const float inv = 1.f / (l + xother[row]);
             const int64_t qrow = (int64_t)q0 + t * BM + row;
-            __nv_bfloat16 *dst = O + ((int64_t)bh * n_q + qrow) * D;
+            __nv_bfloat16 *dst = O + ((int64_t)bh * n_q + qrow) * D + hh * (D / 2);
 #pragma unroll
-            for (int q = 0; q < D / 32; ++q) {
+            for (int q = 0; q < D / 64; ++q) {
                 uint32_t o[32];
                 tmem_ld32(tO + q * 32, o);
                 tmem_wait_ld();
@@ -412,9 +412,9 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 9) {
+    if (warp == MMA_WARP) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");
+        tmem_dealloc(tmem, TMEM_COLS);
     }
 }
 
@@ -501,9 +501,3 @@ int attend_tc(const __nv_bfloat16 *Q, const __nv_bfloat16 *K, const __nv_bfloat1
 
 }  // namespace elm
 
-#ifdef ELM_TRACE
-extern "C" int elm_debug_read_trace(long long *host, int n)
-{
-    return cudaMemcpyFromSymbol(host, g_trace_buf, sizeof(long long) * (size_t)n) == cudaSuccess ? 0 : -7;
-}
-#endif
