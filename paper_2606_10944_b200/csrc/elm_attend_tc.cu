@@ -12,8 +12,10 @@
 //   warp 16          TMA producer: Q tiles once, then K / V^T blocks through a 2-stage ring
 //   warp 17          tcgen05.mma issuer: S = Q K^T (operands in shared memory), O += P V (P read
 //                    from TMEM, V^T from shared memory); owns the TMEM allocation
-// TMEM columns: [0,128) S/P of tile 0, [128,256) S/P of tile 1, [256,256+D) O of tile 0,
-// [384,384+D) O of tile 1.  Every mbarrier wait is bounded; on expiry the CTA records a status
+// TMEM columns: [0,128) S of tile 0, [128,256) S of tile 1, [256,256+D) O of tile 0, [384,384+D) O of
+// tile 1.  The probabilities of points 0-63 / 64-127 of a block are written over the first 32
+// columns of the logits of the same points ([0,32) / [64,96) of the tile's S region), so a thread
+// only ever overwrites logits it has already read itself.  Every mbarrier wait is bounded; on expiry the CTA records a status
 // word and leaves through the common exit, which frees the TMEM it holds.
 #include <cuda.h>
 #include <math.h>
@@ -294,7 +296,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                 for (int hh = 0; hh < 2; ++hh)
 #pragma unroll
                     for (int ks = 0; ks < 4; ++ks)
-                        mma_ts(tmem + 256 + t * 128, tmem + t * 128 + hh * 32 + ks * 8,
+                        mma_ts(tmem + 256 + t * 128, tmem + t * 128 + hh * 64 + ks * 8,
                                b0 + (uint64_t)(hh * (D * 128 >> 4) + ks * 2), IDESC_PV, (acc || (hh | ks) != 0) ? 1u : 0u);
             };
             bool ok = mbar_wait(&bar->q_full, 0) && mbar_wait(&bar->k_full[0], 0);
@@ -333,7 +335,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
         const int row = (warp & 3) * 32 + lane;                    // row in the tile = TMEM lane
         const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
         const uint32_t tS = tmem + lane_addr + t * 128 + hh * 64;  // this thread's 64 logit columns
-        const uint32_t tP = tmem + lane_addr + t * 128 + hh * 32;  // ... and where their bf16 probabilities go
+        const uint32_t tP = tS;                                    // their bf16 probabilities overwrite the first 32 of them
         const uint32_t tO = tmem + lane_addr + 256 + t * 128 + hh * (D / 2);   // its half of the accumulator
         float *xmine = bar->xchg[t][hh], *xother = bar->xchg[t][hh ^ 1];
         const bool use_bias = nonuniform[prob] != 0;
