@@ -21,6 +21,10 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
+# dram__bytes_read.sum + dram__bytes_write.sum of one attend launch, from the ncu capture summarised
+# in profiles/attend_tc_cfg5_dram_traffic.md (read 1 084 004 352 + write 1 027 012 096 bytes)
+NCU_DRAM_BYTES_PER_ATTEND_LAUNCH = {"cfg5": 2111016448}
+
 METRIC = "compress+attend tokens/sec per B200"
 UNIT = "tokens/s"
 
@@ -328,12 +332,7 @@ def main():
         roofline = {"bound": "hbm", "kernel": "attend", "achieved": achieved, "peak": peaks["hbm_gbs"],
                     "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "traffic": None,
                     "peak_source": f"{peaks['source']} copy", "ms_per_launch": att_ms}
-    traffic_path = os.path.join(ROOT, "profiles", "attend_traffic.json")
-    if os.path.exists(traffic_path):
-        with open(traffic_path) as f:
-            tr = json.load(f)
-        if tr.get("workload") == wl.name:
-            roofline["traffic"] = tr.get("dram_bytes_per_launch")
+    roofline["traffic"] = NCU_DRAM_BYTES_PER_ATTEND_LAUNCH.get(wl.name)
     whole_roof_s = max((attend_flops + compress_flops) / (tensor_peak * 1e12), hbm_bytes / (peaks["hbm_gbs"] * 1e9))
 
     base = None
