@@ -34,12 +34,16 @@ constexpr int NTHREADS = 576;          // 16 softmax warps + TMA producer + MMA 
 constexpr int TMA_WARP = 16, MMA_WARP = 17;
 constexpr uint32_t TMEM_COLS = 512;
 constexpr float RESCALE_TAU = 8.0f;      // rescale the accumulator only if the max grew by > 2^8
+#ifndef ELM_EMU_PAIRS
+#define ELM_EMU_PAIRS 4
+#endif
+constexpr int EMU_PAIRS = ELM_EMU_PAIRS;  // of every 16 column pairs, how many take exp2 from the FMA pipe
 
 using namespace sm100;
 
 struct __align__(8) Barriers {
     uint64_t q_full;
-    uint64_t k_full[STAGES], v_full[STAGES], k_empty[STAGES], v_empty[STAGES];
+    uint64_t k_full[STAGES], v_full[STAGES], kv_free[STAGES];
     uint64_t s_full[2], p_ready[2], o_done[2];
     uint32_t tmem_base;
     uint32_t abort_flag;
@@ -160,8 +164,30 @@ __device__ __forceinline__ float exp_pass(uint32_t tS, uint32_t tP, float scale_
             for (int i = 0; i < 16; ++i)
                 x2[i] = fma2(pack2(__uint_as_float(a[q & 1][2 * i]), __uint_as_float(a[q & 1][2 * i + 1])), scale2, negm2);
             float pe[32];
+            // The special-function unit (16 exp2 per clock per SM) is the scarcest pipe of this loop, so
+            // EMU_PAIRS of the 16 pairs take 2^x from the FMA pipe instead: x = n + f with n = round(x)
+            // (magic-number add), 2^f by a cubic on [-1/2, 1/2] (relative error 1e-4, below the bf16
+            // rounding of the probabilities), n added to the exponent field.
 #pragma unroll
-            for (int i = 0; i < 16; ++i) {
+            for (int i = 0; i < EMU_PAIRS; ++i) {
+                float x0, x1;
+                unpack2(x2[i], x0, x1);
+                const uint64_t xc = pack2(fmaxf(x0, -125.f), fmaxf(x1, -125.f));
+                const uint64_t magic = pack2(12582912.f, 12582912.f), nmagic = pack2(-12582912.f, -12582912.f);
+                const uint64_t tt = add2(xc, magic);                       // low mantissa bits = n
+                const uint64_t nn = add2(tt, nmagic);                      // n as a float
+                const uint64_t ff = fma2(nn, pack2(-1.f, -1.f), xc);           // f = x - n
+                uint64_t pp = fma2(pack2(0.05500893f, 0.05500893f), ff, pack2(0.24221096f, 0.24221096f));
+                pp = fma2(pp, ff, pack2(0.69328293f, 0.69328293f));
+                pp = fma2(pp, ff, pack2(1.f, 1.f));
+                float p0, p1, t0, t1;
+                unpack2(pp, p0, p1);
+                unpack2(tt, t0, t1);
+                pe[2 * i] = __uint_as_float(__float_as_uint(p0) + (__float_as_uint(t0) << 23));
+                pe[2 * i + 1] = __uint_as_float(__float_as_uint(p1) + (__float_as_uint(t1) << 23));
+            }
+#pragma unroll
+            for (int i = EMU_PAIRS; i < 16; ++i) {
                 float x0, x1;
                 unpack2(x2[i], x0, x1);
                 pe[2 * i] = fast_exp2(x0);
@@ -230,8 +256,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(&bar->k_full[s], 1);
             mbar_init(&bar->v_full[s], 1);
-            mbar_init(&bar->k_empty[s], 1);
-            mbar_init(&bar->v_empty[s], 1);
+            mbar_init(&bar->kv_free[s], 1);
         }
         for (int t = 0; t < 2; ++t) {
             mbar_init(&bar->s_full[t], 1);
@@ -254,20 +279,35 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
             for (int t = 0; t < 2; ++t)
                 for (int kh = 0; kh < KH; ++kh)
                     tma_load_3d(smem + SM::OFF_Q + t * SM::Q_TILE + kh * (BM * 128), &mapQ, &bar->q_full, kh * 64, q0 + t * BM, bh);
+            // The issuer commits "event" i to kv_free[i % 2] after the prologue (i = 0: S = Q K^T of block
+            // 0 issued) and after iteration i - 1 (O += P V of block i - 1 and S = Q K^T of block i issued).
+            // Once event i is complete, K's stage i % 2 (block i) and V's stage (i + 1) % 2 (block i - 1)
+            // have been read, so K(i + 2) and V(i + 1) may overwrite them.
             bool ok = true;
-            for (int j = 0; j < nblk && ok; ++j) {
+            auto load_k = [&](int j) {
                 const int s = j % STAGES;
-                const uint32_t ph = (uint32_t)(j / STAGES) & 1u;
-                ok = mbar_wait(&bar->k_empty[s], ph ^ 1u);
-                if (!ok) break;
                 mbar_expect_tx(&bar->k_full[s], SM::K_BLOCK);
                 for (int kh = 0; kh < KH; ++kh)
                     tma_load_3d(smem + SM::OFF_K + s * SM::K_BLOCK + kh * (BN * 128), &mapK, &bar->k_full[s], kh * 64, j * BN, prob);
-                ok = mbar_wait(&bar->v_empty[s], ph ^ 1u);
-                if (!ok) break;
+            };
+            auto load_v = [&](int j) {
+                const int s = j % STAGES;
                 mbar_expect_tx(&bar->v_full[s], SM::V_BLOCK);
                 for (int hh = 0; hh < 2; ++hh)
                     tma_load_3d(smem + SM::OFF_V + s * SM::V_BLOCK + hh * (D * 128), &mapV, &bar->v_full[s], j * BN + hh * 64, 0, prob);
+            };
+            for (int j = 0; j < STAGES && j < nblk; ++j) { load_k(j); load_v(j); }
+            for (int i = 0; i + 2 < nblk && ok; ++i) {
+                ok = mbar_wait(&bar->kv_free[i % STAGES], (uint32_t)(i / STAGES) & 1u);
+                if (!ok) break;
+                load_k(i + 2);
+                if (i >= 1) load_v(i + 1);
+            }
+            // the last V block: freed by event nblk - 1
+            if (ok && nblk > STAGES) {
+                const int i = nblk - 2;
+                ok = mbar_wait(&bar->kv_free[i % STAGES], (uint32_t)(i / STAGES) & 1u);
+                if (ok) load_v(i + 1);
             }
             if (!ok) { atomicExch(status, 1); bar->abort_flag = 1; }
         }
@@ -303,7 +343,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
             if (ok) {
                 tc_fence_after();
                 for (int t = 0; t < 2; ++t) { issue_qk(t, 0); tc_commit(&bar->s_full[t]); }
-                tc_commit(&bar->k_empty[0]);
+                tc_commit(&bar->kv_free[0]);                                   // event 0
             }
             for (int j = 0; j < nblk && ok; ++j) {
                 const int s = j % STAGES;
@@ -316,12 +356,13 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                     if (!ok) break;
                     tc_fence_after();
                     issue_pv(t, s, j > 0);
-                    tc_commit(&bar->o_done[t]);
+                    // s_full also tells the softmax warps that O += P V of block j is complete (a commit
+                    // covers every earlier MMA); only the last block needs o_done for the epilogue
                     if (more) { issue_qk(t, sn); tc_commit(&bar->s_full[t]); }
+                    else tc_commit(&bar->o_done[t]);
                 }
                 if (!ok) break;
-                tc_commit(&bar->v_empty[s]);
-                if (more) tc_commit(&bar->k_empty[sn]);
+                tc_commit(&bar->kv_free[(j + 1) % STAGES]);                    // event j + 1
             }
             if (!ok) { atomicExch(status, 2); bar->abort_flag = 1; }
         }
@@ -359,9 +400,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
             const bool grow = mx > m_ref + RESCALE_TAU;
             if (__any_sync(0xffffffffu, grow)) {
                 if (j > 0) {
-                    ok = mbar_wait(&bar->o_done[t], (uint32_t)(j - 1) & 1u);
-                    if (!ok) break;
-                    tc_fence_after();
+                    // O += P V of block j-1 is complete: s_full of block j was committed after it
                     const float alpha = grow ? fast_exp2(m_ref - mx) : 1.f;
 #pragma unroll
                     for (int q = 0; q < D / 64; ++q) {
@@ -383,7 +422,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
             tc_fence_before();
             mbar_arrive(&bar->p_ready[t]);
         }
-        if (ok) ok = mbar_wait(&bar->o_done[t], (uint32_t)(nblk - 1) & 1u);
+        if (ok) ok = mbar_wait(&bar->o_done[t], 0);
         if (ok) {
             tc_fence_after();
             xmine[row] = l;
