@@ -117,14 +117,18 @@ gram_tc_kernel(const __nv_bfloat16 *__restrict__ K, const __nv_bfloat16 *__restr
     const __nv_bfloat16 *Vp = V + (int64_t)p * n * D;
     constexpr uint32_t IDESC = umma_idesc_bf16(TR, TR);
     const uint32_t sA = smem_u32(smem + SM::OFF_A);
-    const uint32_t sB = diagonal ? sA : smem_u32(smem + SM::OFF_B);
+    const uint32_t sB = smem_u32(smem + SM::OFF_B);
     uint32_t tmem = 0;
     bool ok = true;
+    auto issue = [&](int acc, uint32_t a_addr, uint32_t b_addr) {     // one 128 x 128 x D product into accumulator `acc`
 #pragma unroll
-    for (int phase = 0; phase < 2; ++phase) {                  // 0: keys -> K K^T, 1: values -> V V^T
-        const __nv_bfloat16 *X = phase == 0 ? Kp : Vp;
-        gather_operand<D>(smem + SM::OFF_A, X, misc->rowsA, tid);
-        if (!diagonal) gather_operand<D>(smem + SM::OFF_B, X, misc->rowsB, tid);
+        for (int kh = 0; kh < KH; ++kh)
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks)
+                mma_ss(tmem + acc * 128, umma_desc_k128(a_addr + kh * (TR * 128) + ks * 32),
+                       umma_desc_k128(b_addr + kh * (TR * 128) + ks * 32), IDESC, (kh | ks) != 0);
+    };
+    auto publish = [&]() {                                            // make the gathered tiles visible to the MMAs
         asm volatile("cp.async.commit_group;" ::: "memory");
         asm volatile("cp.async.wait_group 0;" ::: "memory");
         fence_proxy_async();
@@ -132,17 +136,33 @@ gram_tc_kernel(const __nv_bfloat16 *__restrict__ K, const __nv_bfloat16 *__restr
         __syncthreads();
         tc_fence_after();
         tmem = misc->tmem_base;
+    };
+    if (diagonal) {
+        // row points = column points: keys in the first slot, values in the second, one gather round
+        gather_operand<D>(smem + SM::OFF_A, Kp, misc->rowsA, tid);
+        gather_operand<D>(smem + SM::OFF_B, Vp, misc->rowsA, tid);
+        publish();
         if (tid == 0) {
-#pragma unroll
-            for (int kh = 0; kh < KH; ++kh)
-#pragma unroll
-                for (int ks = 0; ks < 4; ++ks)
-                    mma_ss(tmem + phase * 128, umma_desc_k128(sA + kh * (TR * 128) + ks * 32),
-                           umma_desc_k128(sB + kh * (TR * 128) + ks * 32), IDESC, (kh | ks) != 0);
-            tc_commit(&misc->mma_done[phase]);
+            const uint32_t sV = smem_u32(smem + SM::OFF_B);
+            issue(0, sA, sA);
+            issue(1, sV, sV);
+            tc_commit(&misc->mma_done[1]);
         }
-        // the operand tiles are reused by the next phase only after the MMAs have read them
-        ok = ok && mbar_wait(&misc->mma_done[phase], 0);
+        ok = mbar_wait(&misc->mma_done[1], 0);
+    } else {
+#pragma unroll
+        for (int phase = 0; phase < 2; ++phase) {              // 0: keys -> K K^T, 1: values -> V V^T
+            const __nv_bfloat16 *X = phase == 0 ? Kp : Vp;
+            gather_operand<D>(smem + SM::OFF_A, X, misc->rowsA, tid);
+            gather_operand<D>(smem + SM::OFF_B, X, misc->rowsB, tid);
+            publish();
+            if (tid == 0) {
+                issue(phase, sA, sB);
+                tc_commit(&misc->mma_done[phase]);
+            }
+            // the operand tiles are reused by the next phase only after the MMAs have read them
+            ok = ok && mbar_wait(&misc->mma_done[phase], 0);
+        }
     }
 
     // epilogue: warp w owns TMEM lanes 32 (w % 4) .. +31 (tile rows) and the column half w / 4
