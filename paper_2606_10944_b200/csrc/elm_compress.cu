@@ -10,6 +10,7 @@
 
 #include "elm_common.cuh"
 #include "elm_compress.cuh"
+#include "elm_walk.cuh"
 
 namespace elm {
 
@@ -243,25 +244,6 @@ template <typename T> struct WalkState {
     T bmax;   // b_{max,i-1} in the shift of the last pair seen (warp-uniform)
 };
 
-// swap iff U < min(1, (1/2)(1 - alpha/a)_+);  a == 0 (or not finite) => probability 1/2
-__device__ __forceinline__ bool swap_decision(double alpha, double a, double U)
-{
-    double p = 0.5;
-    if (a > 0.0 && isfinite(a)) {
-        double t = 1.0 - alpha / a;
-        t = t < 0.0 ? 0.0 : t;
-        p = 0.5 * t;
-        p = p > 1.0 ? 1.0 : p;
-    }
-    return U < p;
-}
-// fp32 mode: the same test with the division cleared, alpha < a (1 - 2U)
-__device__ __forceinline__ bool swap_decision(float alpha, float a, float U)
-{
-    if (a > 0.f && isfinite(a)) return alpha < a * (1.f - 2.f * U);
-    return U < 0.5f;
-}
-
 // Resolve pairs [i0, i0 + cnt) (cnt <= 32) of one call.  `alpha` is this lane's score from all
 // earlier blocks; Fg points at the call's P x P pair Gram; returns the 32-bit swap mask.
 template <typename T>
@@ -327,43 +309,6 @@ __device__ __forceinline__ uint32_t walk_block_regs(const T (&Fd)[32], T b, T al
         swaps |= sw << t;
         T f = t < lane ? Fd[t] : (T)0;
         alpha += sw ? f : -f;
-    }
-    return swaps;
-}
-
-// fp32 walker: the 32 serial steps of a block run in ONE thread with the diagonal tile in shared
-// memory.  Thread-local state d[u] = alpha_u - a_u (1 - 2 U_u) makes "swap pair u" the sign test
-// d[u] < 0; a decision then updates the later d[u] with independent FMAs, so a step costs one
-// compare-select-FMA chain instead of a warp vote.  b_u = 0 (a_u = 0) needs no special case in the
-// updates because then F[., u] = 0 (Cauchy-Schwarz in the RKHS); its decision is U_u < 1/2.
-__device__ __forceinline__ uint32_t walk_block_thread(const float *__restrict__ tile, const float *__restrict__ alpha32,
-                                                      const float *__restrict__ b32, const float *__restrict__ r32,
-                                                      const float *__restrict__ U32, float logfac, float &bmax)
-{
-    float d[32];
-#pragma unroll
-    for (int t = 0; t < 32; ++t) {
-        const float bt = b32[t], carried = bmax * r32[t];
-        bmax = bt > carried ? bt : carried;
-        const float a = bt * bmax * logfac;
-        const float U = U32[t];
-        d[t] = (a > 0.f && isfinite(a)) ? alpha32[t] - a * (1.f - 2.f * U) : (U < 0.5f ? -1.f : 1.f);
-    }
-    uint32_t swaps = 0;
-#pragma unroll
-    for (int t = 0; t < 32; ++t) {
-        const bool sw = d[t] < 0.f;
-        swaps |= (sw ? 1u : 0u) << t;
-        const float s = sw ? 1.f : -1.f;          // alpha_u = -sum_j eta_j F[j,u]: kept pair subtracts
-        const float4 *row = reinterpret_cast<const float4 *>(tile + t * 32);
-#pragma unroll
-        for (int g4 = (t + 1) / 4; g4 < 8; ++g4) {
-            const float4 v = row[g4];
-            if (4 * g4 + 0 > t) d[4 * g4 + 0] = fmaf(s, v.x, d[4 * g4 + 0]);
-            if (4 * g4 + 1 > t) d[4 * g4 + 1] = fmaf(s, v.y, d[4 * g4 + 1]);
-            if (4 * g4 + 2 > t) d[4 * g4 + 2] = fmaf(s, v.z, d[4 * g4 + 2]);
-            if (4 * g4 + 3 > t) d[4 * g4 + 3] = fmaf(s, v.w, d[4 * g4 + 3]);
-        }
     }
     return swaps;
 }
@@ -486,7 +431,7 @@ __global__ void __launch_bounds__(576) walk_cta_kernel(const T *__restrict__ F, 
                 a32_s[lane] = alpha;
                 __syncwarp();
                 if (lane == 0)
-                    mask_s[c] = walk_block_thread(tdiag, a32_s, b_s + i0, r_s + i0, U_s + i0, logfac, bmax);
+                    mask_s[c] = walk_block_thread<32>(tdiag, a32_s, b_s + i0, r_s + i0, U_s + i0, logfac, bmax);
             } else {
                 T Fd[32];
 #pragma unroll
@@ -674,23 +619,36 @@ static int compress_impl(const Tin *K, const Tin *V, const elm_params *p, uint64
             count_launches(1);
             ELM_CUDA_TRY(cudaGetLastError());
         }
+        bool walked = false;                                       // the Gram kernel walked the level itself
         {
             StageTimer t(ELM_STAGE_GRAM, st, 1);
             int rc;
             if constexpr (std::is_same<Tin, __nv_bfloat16>::value && std::is_same<T, float>::value) {
-                // tensor cores once a Halve call fills at least a quarter of a 64-pair tile side
-                rc = P >= 16 ? gram_tc(K, V, p, cur, Mpair, vmax_bits, P, Ptotal, groups, F, L.F_stride,
-                                       reinterpret_cast<int *>(vmax_bits + BH), st)
-                             : run_gram_simt<Tin, T>(K, V, p, cur, Mpair, vmax_bits, P, Ptotal, groups, F, L.F_stride, st);
+                // tensor cores once a Halve call fills at least a quarter of a 64-pair tile side; calls
+                // that fit a tile (<= 64 pairs) are also walked inside the Gram kernel
+                if (P >= 16) {
+                    WalkArgs wk;
+                    wk.fused = P <= 64;
+                    wk.level = level;
+                    wk.seed = seed;
+                    wk.logfac = logfac;
+                    wk.rdecay = rdecay;
+                    wk.out = out;
+                    wk.out_stride = out_stride;
+                    walked = wk.fused;
+                    rc = gram_tc(K, V, p, cur, Mpair, vmax_bits, P, Ptotal, groups, F, L.F_stride,
+                                 reinterpret_cast<int *>(vmax_bits + BH), wk, st);
+                } else {
+                    rc = run_gram_simt<Tin, T>(K, V, p, cur, Mpair, vmax_bits, P, Ptotal, groups, F, L.F_stride, st);
+                }
             } else {
                 rc = run_gram_simt<Tin, T>(K, V, p, cur, Mpair, vmax_bits, P, Ptotal, groups, F, L.F_stride, st);
             }
             if (rc != ELM_OK) return rc;
         }
-        {
+        if (!walked) {
             StageTimer t(ELM_STAGE_WALK, st, 1);
             if (P >= 32) {
-                // one walker warp plus enough warps to sweep the remaining columns once per block
                 // walker warp + tile-copy warp + updaters (one per two pairs, at most 512 threads)
                 int upd = P / 2;
                 upd = upd < 32 ? 32 : (upd > 512 ? 512 : upd);

@@ -23,10 +23,23 @@ struct CompressLayout {
 };
 CompressLayout compress_layout(const elm_params *p);
 
+// What the Gram kernel needs to also run the halving walk of calls that fit one of its tiles
+// (at most 64 pairs): with `fused` set the pair Gram of the level never leaves shared memory and
+// the survivors go straight to `out`.
+struct WalkArgs {
+    int fused;
+    int level;
+    uint64_t seed;
+    float logfac;
+    const float *rdecay;     // [BH][n/2]
+    int32_t *out;            // next level's sequence (or the final coreset)
+    int64_t out_stride;
+};
+
 // Tensor-core pair Gram of one level (bf16 storage, fp32 arithmetic); same output layout as the
 // generic kernel.  `status` is a device word that a timed-out wait sets to a non-zero code.
 int gram_tc(const __nv_bfloat16 *K, const __nv_bfloat16 *V, const elm_params *p, const int32_t *cur,
             const float *Mpair, const unsigned *vmax_bits, int P, int64_t Ptotal, int groups, float *F,
-            int64_t F_stride, int *status, cudaStream_t st);
+            int64_t F_stride, int *status, const WalkArgs &wk, cudaStream_t st);
 
 }  // namespace elm

@@ -12,6 +12,7 @@
 #include "elm_common.cuh"
 #include "elm_compress.cuh"
 #include "elm_sm100.cuh"
+#include "elm_walk.cuh"
 
 namespace elm {
 namespace gramtc {
@@ -39,8 +40,57 @@ struct Misc {
     uint32_t tmem_base;
     uint32_t pad;
     float colshift[TP];          // M of each pair column, in log2 units
+    float rdec[TP], unif[TP];    // fused walk: decay factor and uniform of each pair of the tile
     int32_t rowsA[TR], rowsB[TR];
 };
+
+constexpr int FS_LD = 68;         // row stride of the shared-memory pair Gram of a fused tile (floats)
+
+// Halving walk (Algorithm A.1) of the calls that lie inside one 64-pair tile, on the tile's pair
+// Gram in shared memory: warp w walks call w of the tile (P = 16, 32 or 64 pairs per call) in blocks
+// of 32 pairs, the serial steps in one thread, the coupling between the two blocks of a 64-pair
+// call lane-parallel.  `scratch` provides 4 x 32 floats per warp (placed after the 64 x 68 floats of Fs).
+__device__ __forceinline__ void walk_in_tile(const float *Fs, float *scratch, const float *rdec, const float *unif, int p,
+                                             int64_t JR, int P, int64_t Ptotal, int64_t n,
+                                             const int32_t *__restrict__ cur, const WalkArgs &wk, int warp, int lane)
+{
+    const int calls = TP / P;
+    if (warp >= calls) return;
+    const int64_t J0 = JR + (int64_t)warp * P;                 // first pair of this call along the level's sequence
+    if (J0 >= Ptotal) return;
+    float *a32 = scratch + warp * 128, *b32 = a32 + 32, *r32 = a32 + 64, *U32 = a32 + 96;
+    const float *Fc = Fs + (warp * P) * FS_LD + warp * P;      // the call's P x P block
+    float bmax = 0.f;
+    uint32_t mask_prev = 0;
+    for (int blk = 0; blk * 32 < P; ++blk) {
+        const int i = blk * 32 + lane;                         // pair within the call
+        const bool live = i < P;
+        float alpha = 0.f;
+        if (blk > 0) {
+#pragma unroll
+            for (int t = 0; t < 32; ++t) {
+                const float fv = Fc[t * FS_LD + i];
+                alpha += ((mask_prev >> t) & 1u) ? fv : -fv;
+            }
+        }
+        const float dgn = live ? Fc[i * FS_LD + i] : 0.f;
+        a32[lane] = alpha;
+        b32[lane] = sqrtf(dgn > 0.f ? dgn : 0.f);
+        r32[lane] = live ? rdec[warp * P + i] : 1.f;
+        U32[lane] = live ? unif[warp * P + i] : 1.f;
+        __syncwarp();
+        uint32_t swaps = 0;
+        if (lane == 0) swaps = walk_block_thread<FS_LD>(Fc + (blk * 32) * FS_LD + blk * 32, a32, b32, r32, U32, wk.logfac, bmax);
+        swaps = __shfl_sync(0xffffffffu, swaps, 0);
+        bmax = __shfl_sync(0xffffffffu, bmax, 0);
+        if (live) {
+            const uint32_t sw = (swaps >> lane) & 1u;
+            wk.out[(int64_t)p * wk.out_stride + J0 + i] = cur[(int64_t)p * n + 2 * (J0 + i) + sw];
+        }
+        mask_prev = swaps;
+        __syncwarp();
+    }
+}
 
 // Gather 128 rows of X (row-major [n][D] bf16) into a swizzled K-major operand tile.
 template <int D>
@@ -66,7 +116,7 @@ __global__ void __launch_bounds__(NTHREADS, 2)
 gram_tc_kernel(const __nv_bfloat16 *__restrict__ K, const __nv_bfloat16 *__restrict__ V,
                const int32_t *__restrict__ cur, const float *__restrict__ Mpair,
                const unsigned *__restrict__ vmax_bits, int64_t n, int P, int64_t Ptotal,
-               float *__restrict__ F, int64_t F_stride, int *__restrict__ status)
+               float *__restrict__ F, int64_t F_stride, int *__restrict__ status, WalkArgs wk)
 {
     using SM = Smem<D>;
     constexpr int KH = SM::KH;
@@ -104,6 +154,11 @@ gram_tc_kernel(const __nv_bfloat16 *__restrict__ K, const __nv_bfloat16 *__restr
     if (tid < TP) {
         const int64_t jc = JC + tid;
         misc->colshift[tid] = jc < Ptotal ? Mpair[(int64_t)p * (n / 2) + jc] * LOG2E : 0.f;
+        if (wk.fused) {
+            // everything the in-tile walk needs from global memory, fetched while the tile is built
+            misc->rdec[tid] = jc < Ptotal ? wk.rdecay[(int64_t)p * (n / 2) + jc] : 1.f;
+            misc->unif[tid] = halving_uniform<float>(wk.seed, (uint32_t)(jc % P), (uint32_t)(jc / P), (uint32_t)wk.level, (uint32_t)p);
+        }
     }
     if (tid == 0) {
         mbar_init(&misc->mma_done[0], 1);
@@ -203,13 +258,21 @@ gram_tc_kernel(const __nv_bfloat16 *__restrict__ K, const __nv_bfloat16 *__restr
         }
         const int64_t jr = JR + (r >> 1);
         const int64_t jc0 = JC + ch * 32 + (odd ? 16 : 0);
-        float *Fp = F + (int64_t)p * F_stride;
-        if (jr < Ptotal) {
-            const int64_t gr = jr / P;
+        if (wk.fused) {
+            // calls of at most 64 pairs lie inside this (diagonal) tile: keep the pair Gram in shared
+            // memory (over the operand tiles, which the MMAs have finished reading) and walk here
+            float *Fs = reinterpret_cast<float *>(smem + SM::OFF_A);
 #pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                const int64_t jc = jc0 + i;
-                if (jc < Ptotal && jr <= jc && jc / P == gr) Fp[jr * P + (jc - gr * P)] = f[i];
+            for (int i = 0; i < 16; ++i) Fs[(r >> 1) * FS_LD + ch * 32 + (odd ? 16 : 0) + i] = f[i];
+        } else {
+            float *Fp = F + (int64_t)p * F_stride;
+            if (jr < Ptotal) {
+                const int64_t gr = jr / P;
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    const int64_t jc = jc0 + i;
+                    if (jc < Ptotal && jr <= jc && jc / P == gr) Fp[jr * P + (jc - gr * P)] = f[i];
+                }
             }
         }
     } else if (lane == 0) {
@@ -221,12 +284,14 @@ gram_tc_kernel(const __nv_bfloat16 *__restrict__ K, const __nv_bfloat16 *__restr
         tc_fence_after();
         tmem_dealloc(tmem, TMEM_COLS);
     }
+    if (wk.fused && ok) walk_in_tile(reinterpret_cast<float *>(smem + SM::OFF_A), reinterpret_cast<float *>(smem + SM::OFF_A + 20480),
+                                     misc->rdec, misc->unif, p, JR, P, Ptotal, n, cur, wk, warp, lane);
 }
 
 template <int D>
 static int launch(const __nv_bfloat16 *K, const __nv_bfloat16 *V, const elm_params *p, const int32_t *cur,
                   const float *Mpair, const unsigned *vmax_bits, int P, int64_t Ptotal, int groups, float *F,
-                  int64_t F_stride, int *status, cudaStream_t st)
+                  int64_t F_stride, int *status, const WalkArgs &wk, cudaStream_t st)
 {
     const int BH = p->batch * p->kv_heads;
     int64_t tiles;
@@ -239,7 +304,7 @@ static int launch(const __nv_bfloat16 *K, const __nv_bfloat16 *V, const elm_para
     auto kern = gram_tc_kernel<D>;
     ELM_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<D>::TOTAL));
     kern<<<dim3((unsigned)tiles, (unsigned)BH), NTHREADS, Smem<D>::TOTAL, st>>>(K, V, cur, Mpair, vmax_bits, p->n_kv, P,
-                                                                                 Ptotal, F, F_stride, status);
+                                                                                 Ptotal, F, F_stride, status, wk);
     count_launches(1);
     return cuda_status(cudaGetLastError());
 }
@@ -248,10 +313,10 @@ static int launch(const __nv_bfloat16 *K, const __nv_bfloat16 *V, const elm_para
 
 int gram_tc(const __nv_bfloat16 *K, const __nv_bfloat16 *V, const elm_params *p, const int32_t *cur,
             const float *Mpair, const unsigned *vmax_bits, int P, int64_t Ptotal, int groups, float *F,
-            int64_t F_stride, int *status, cudaStream_t st)
+            int64_t F_stride, int *status, const WalkArgs &wk, cudaStream_t st)
 {
-    if (p->d == 64) return gramtc::launch<64>(K, V, p, cur, Mpair, vmax_bits, P, Ptotal, groups, F, F_stride, status, st);
-    return gramtc::launch<128>(K, V, p, cur, Mpair, vmax_bits, P, Ptotal, groups, F, F_stride, status, st);
+    if (p->d == 64) return gramtc::launch<64>(K, V, p, cur, Mpair, vmax_bits, P, Ptotal, groups, F, F_stride, status, wk, st);
+    return gramtc::launch<128>(K, V, p, cur, Mpair, vmax_bits, P, Ptotal, groups, F, F_stride, status, wk, st);
 }
 
 }  // namespace elm
