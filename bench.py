@@ -91,6 +91,20 @@ class ClockSampler:
                 "samples": len(sm)}
 
 
+def max_over_ranks(ms_local: float, dist, device) -> float:
+    """The slowest rank's time (every rank gets it); `dist` is None for a single process."""
+    import torch
+    t = torch.tensor([ms_local], dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_tokens_per_s(tokens_per_rank_step: int, world: int, ms_per_step: float) -> float:
+    """Replicas only: every rank processes its own batch, the job's tokens add up."""
+    return tokens_per_rank_step * world / (ms_per_step * 1e-3)
+
+
 def algorithmic_counts(wl):
     """Flops and bytes the method itself needs per step (not what exact attention would need)."""
     es = 2 if wl.dtype == "bf16" else 4
@@ -271,14 +285,10 @@ def main():
     stage = elm.profile_read()
     elm.profile_enable(False)
     launches = elm.launch_count() - launches0
-    ms_total = ev0.elapsed_time(ev1) - flush_ms
-    t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
-    if dist is not None:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_total = float(t.item())
+    ms_total = max_over_ranks(ev0.elapsed_time(ev1) - flush_ms, dist, dev)
     ms_step = ms_total / args.steps
     tokens_per_step = wl.batch * wl.n * world
-    value = tokens_per_step / (ms_step * 1e-3)
+    value = whole_job_tokens_per_s(wl.batch * wl.n, world, ms_step)
 
     # end to end through the host-buffer entry point (pinned inputs, copies inside the timed region)
     e2e = None
@@ -298,10 +308,7 @@ def main():
                                      precision=args.precision, scratch=scratch, out=Oh)
         g1.record()
         barrier()
-        te = torch.tensor([g0.elapsed_time(g1)], dtype=torch.float64, device=dev)
-        if dist is not None:
-            dist.all_reduce(te, op=dist.ReduceOp.MAX)
-        e2e_ms = float(te.item()) / args.e2e_steps
+        e2e_ms = max_over_ranks(g0.elapsed_time(g1), dist, dev) / args.e2e_steps
         e2e = {"value": tokens_per_step / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
                "h2d_bytes_per_step": Q.numel() * Q.element_size() + 2 * K.numel() * K.element_size(),
                "d2h_bytes_per_step": Q.numel() * Q.element_size(), "steps": args.e2e_steps}

@@ -178,6 +178,17 @@ enum {
 int elm_profile_enable(int on);
 int elm_profile_read(float *ms_out, int64_t *launches_out, int32_t n_stages);
 
+/*
+ * Device-side health of the last elm_compress / elm_attend call that used `workspace`.  Every wait
+ * inside the tensor-core kernels (on an mbarrier) is bounded; a wait that expires (about 2 s)
+ * records a non-zero code in a status word inside the workspace and the launch winds down instead
+ * of hanging, leaving its outputs undefined.  These calls copy that word to *status_host (0 = every
+ * wait completed) after synchronising `stream`.  `params` / `n_core` must be those of the call.
+ */
+int elm_compress_status(const void *workspace, const elm_params *params, int32_t *status_host, void *stream);
+int elm_attend_status(const void *workspace, const elm_params *params, int32_t n_core, int32_t *status_host,
+                      void *stream);
+
 /* Kernels launched by this library since it was loaded (all calls, all stages). */
 int64_t elm_launch_count(void);
 

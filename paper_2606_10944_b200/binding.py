@@ -21,7 +21,7 @@ STAGE_NAMES = ["prepass", "level_prep", "gram", "walk", "emit", "gather", "atten
 EXPORTED_SYMBOLS = [
     "elm_workspace_bytes", "elm_default_delta_levels", "elm_compress", "elm_attend",
     "elm_attend_workspace_bytes", "elm_attend_static", "elm_host_call_scratch_bytes", "elm_compress_attend_host",
-    "elm_profile_enable", "elm_profile_read", "elm_launch_count", "elm_strerror", "elm_version",
+    "elm_compress_status", "elm_attend_status", "elm_profile_enable", "elm_profile_read", "elm_launch_count", "elm_strerror", "elm_version",
 ]
 
 
@@ -66,6 +66,8 @@ def load_library():
     lib.elm_attend_static.argtypes = [vp, vp, vp, vp, vp, ctypes.c_int32, pp, vp, vp]
     lib.elm_host_call_scratch_bytes.argtypes = [pp, szp]
     lib.elm_compress_attend_host.argtypes = [vp, vp, vp, vp, vp, vp, pp, ctypes.c_uint64, vp, sz, vp]
+    lib.elm_compress_status.argtypes = [vp, pp, ctypes.POINTER(ctypes.c_int32), vp]
+    lib.elm_attend_status.argtypes = [vp, pp, ctypes.c_int32, ctypes.POINTER(ctypes.c_int32), vp]
     lib.elm_profile_enable.argtypes = [ctypes.c_int]
     lib.elm_profile_read.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int64), ctypes.c_int32]
     lib.elm_launch_count.argtypes = []
@@ -241,6 +243,22 @@ def host_call_scratch_bytes(B, Hq, Hkv, n, nq, d, log2_nout, m, dtype, precision
     _check(load_library().elm_host_call_scratch_bytes(ctypes.byref(p), ctypes.byref(need)),
            "elm_host_call_scratch_bytes")
     return int(need.value)
+
+
+def compress_status(workspace, params: ElmParams) -> int:
+    """elm_compress_status: 0 unless a bounded device wait expired during the last compress call."""
+    out = ctypes.c_int32(-1)
+    _check(load_library().elm_compress_status(workspace.data_ptr(), ctypes.byref(params), ctypes.byref(out), _stream()),
+           "elm_compress_status")
+    return int(out.value)
+
+
+def attend_status(workspace, params: ElmParams, n_core: int) -> int:
+    """elm_attend_status: 0 unless a bounded device wait expired during the last attend call."""
+    out = ctypes.c_int32(-1)
+    _check(load_library().elm_attend_status(workspace.data_ptr(), ctypes.byref(params), n_core, ctypes.byref(out),
+                                            _stream()), "elm_attend_status")
+    return int(out.value)
 
 
 def profile_enable(on: bool = True):

@@ -161,6 +161,34 @@ extern "C" int elm_compress_attend_host(const void *Q_host, const void *K_host, 
     return ELM_OK;
 }
 
+extern "C" int elm_compress_status(const void *workspace, const elm_params *params, int32_t *status_host, void *stream)
+{
+    if (!workspace || !params || !status_host) return ELM_ERR_NULL;
+    int rc = validate_params(params);
+    if (rc != ELM_OK) return rc;
+    // the status word follows the per-problem v_max words at the head of the compress workspace
+    const unsigned char *word = (const unsigned char *)workspace + compress_layout(params).vmax_bits +
+                                4 * (size_t)params->batch * params->kv_heads;
+    ELM_CUDA_TRY(cudaMemcpyAsync(status_host, word, 4, cudaMemcpyDeviceToHost, (cudaStream_t)stream));
+    ELM_CUDA_TRY(cudaStreamSynchronize((cudaStream_t)stream));
+    return ELM_OK;
+}
+
+extern "C" int elm_attend_status(const void *workspace, const elm_params *params, int32_t n_core,
+                                 int32_t *status_host, void *stream)
+{
+    if (!workspace || !params || !status_host) return ELM_ERR_NULL;
+    int rc = validate_params(params);
+    if (rc != ELM_OK) return rc;
+    if (n_core < 1 || n_core > params->n_kv) return ELM_ERR_SHAPE;
+    // the status word follows the per-problem "weights differ" flags
+    const unsigned char *word = (const unsigned char *)workspace + attend_layout(params, n_core).flags +
+                                4 * (size_t)params->batch * params->kv_heads;
+    ELM_CUDA_TRY(cudaMemcpyAsync(status_host, word, 4, cudaMemcpyDeviceToHost, (cudaStream_t)stream));
+    ELM_CUDA_TRY(cudaStreamSynchronize((cudaStream_t)stream));
+    return ELM_OK;
+}
+
 extern "C" int elm_profile_enable(int on)
 {
     Profiler &pr = profiler();

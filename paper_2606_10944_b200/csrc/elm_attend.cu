@@ -209,6 +209,8 @@ static int attend_impl(const Tin *Q, const Tin *K, const Tin *V, const int32_t *
     const int problems = p->batch * p->kv_heads;
     {
         StageTimer t(ELM_STAGE_GATHER, st, 1);
+        // this path has no bounded waits: its status word reads 0
+        ELM_CUDA_TRY(cudaMemsetAsync(ws + L.flags, 0, sizeof(int) * (size_t)(problems + 1), st));
         gather_kernel<Tin><<<dim3((unsigned)((n_core + 7) / 8), (unsigned)problems), 256, 0, st>>>(
             K, V, idx, w, p->n_kv, p->d, n_core, Kc, Vc, bias);
         count_launches(1);

@@ -1,0 +1,74 @@
+"""The benchmark's launch configuration (cfg5 at full size, fp32 mode) against the oracle on
+sampled outputs: the coreset of every KV head, attention rows sampled from every query head, the
+end-to-end error on those rows, and the device status words."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2606_10944_b200 as elm
+from paper_2606_10944_b200.workloads import WORKLOADS, as_f32_numpy, generate
+
+from _util import check_coreset_structure, e_max, max_rel_err, mismatch_rate
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def cfg5():
+    wl = WORKLOADS["cfg5"]
+    Q, K, V = generate(wl, seed=1234)
+    return wl, Q, K, V
+
+
+def test_cfg5_full_size_fp32_mode_sampled_parity(cfg5):
+    wl, Q, K, V = cfg5
+    Qd, Kd, Vd = Q.cuda(), K.cuda(), V.cuda()
+    p, _ = elm.make_params(wl.batch, wl.q_heads, wl.kv_heads, wl.n, wl.n_q, wl.d, wl.log2_nout, wl.m, 1, "fp32")
+    cb, ab = elm.workspace_bytes(p)
+    ws_c = torch.empty(cb, dtype=torch.uint8, device="cuda")
+    ws_a = torch.empty(ab, dtype=torch.uint8, device="cuda")
+    idx, w = elm.compress(Kd, Vd, wl.log2_nout, wl.m, seed=1, precision="fp32", workspace=ws_c)
+    O = elm.attend(Qd, Kd, Vd, idx, w, precision="fp32", workspace=ws_a)
+    assert elm.compress_status(ws_c, p) == 0 and elm.attend_status(ws_a, p, wl.n_out) == 0
+    idx_h, w_h = idx.cpu().numpy(), w.cpu().numpy()
+    check_coreset_structure(idx_h, wl.n, wl.m)
+    assert np.allclose(w_h, 1.0 / wl.n_out)
+
+    # the oracle's coreset of every KV head (fp64), for the mismatch rate and for the error budget
+    Kf = as_f32_numpy(K)[0]
+    Vf = as_f32_numpy(V)[0]
+    ref_idx, ref_w, _ = oracle.compress2_batched(Kf, Vf, wl.log2_nout, wl.m, seed=1)
+    rate = mismatch_rate(idx_h[0], ref_idx)
+    print(f"[cfg5 full size, fp32 mode] index mismatch rate vs fp64 oracle = {rate:.4f}")
+    assert rate < 0.5
+
+    # sampled query rows of every query head: attention on the GPU's own coreset, recomputed by the oracle
+    rng = np.random.default_rng(0)
+    rows = np.sort(rng.choice(wl.n_q, size=48, replace=False))
+    rows[-1] = wl.n_q - 1                                      # the last row of the last tile
+    Qs = as_f32_numpy(Q[:, :, rows])
+    Og = O[:, :, rows].float().cpu().numpy()
+    ref = oracle.wtd_attention_batched(Qs, Kf[None], Vf[None], idx_h, w_h.astype(np.float64))
+    err = max_rel_err(Og, ref)
+    print(f"[cfg5 full size] attend on sampled rows: max rel err {err:.3e}")
+    assert err <= 2e-2
+
+    # end-to-end error on the sampled rows against exact attention, GPU pipeline vs oracle pipeline
+    exact = oracle.exact_attention_batched(Qs, Kf[None], Vf[None])
+    ref_pipe = oracle.wtd_attention_batched(Qs, Kf[None], Vf[None], ref_idx[None], ref_w[None])
+    e_gpu, e_ref = e_max(Og, exact), e_max(ref_pipe, exact)
+    print(f"[cfg5 full size] E_max on sampled rows: gpu {e_gpu:.4e} oracle {e_ref:.4e}")
+    assert e_gpu <= 1.05 * e_ref + 2e-2 * np.abs(exact).max()   # + the bf16 output rounding the oracle does not have
+
+
+def test_status_words_after_generic_kernels():
+    wl = WORKLOADS["cfg2"].scaled(batch=1, q_heads=2, kv_heads=2)
+    Q, K, V = (t.cuda() for t in generate(wl, seed=3))
+    p, _ = elm.make_params(1, 2, 2, wl.n, wl.n_q, wl.d, wl.log2_nout, wl.m, 0, "fp64")
+    cb, ab = elm.workspace_bytes(p)
+    ws_c = torch.full((cb,), 255, dtype=torch.uint8, device="cuda")
+    ws_a = torch.full((ab,), 255, dtype=torch.uint8, device="cuda")
+    idx, w = elm.compress(K, V, wl.log2_nout, wl.m, precision="fp64", workspace=ws_c)
+    elm.attend(Q, K, V, idx, w, precision="fp64", workspace=ws_a)
+    assert elm.compress_status(ws_c, p) == 0 and elm.attend_status(ws_a, p, wl.n_out) == 0

@@ -55,6 +55,7 @@ SMALL_CASES = {
     "cfg5_n8192": WORKLOADS["cfg5"].scaled(q_heads=4, kv_heads=2, n=8192, n_q=8192),
     "cfg5_n2048_g4": WORKLOADS["cfg5"].scaled(q_heads=2, kv_heads=2, n=2048, n_q=64, g=4),
     "mixture_d128_f32": WORKLOADS["cfg2"].scaled(batch=1, q_heads=2, kv_heads=2, n=4096, d=128, g=1),
+    "lowrank_d64_bf16": WORKLOADS["cfg3"].scaled(batch=1, q_heads=4, kv_heads=2, n=4096, n_q=700, d=64, g=1),
 }
 
 
@@ -132,7 +133,8 @@ def test_compress_fp64_full_size_heads(name, heads):
 # ----------------------------------------------------------------------------------------------
 # compress, fp32 mode: valid structure, mismatch rate reported
 # ----------------------------------------------------------------------------------------------
-@pytest.mark.parametrize("name", ["cfg1_full", "cfg2_two_batches", "cfg3_four_heads", "cfg5_n8192"])
+@pytest.mark.parametrize("name", ["cfg1_full", "cfg2_two_batches", "cfg3_four_heads", "cfg5_n8192", "cfg4_n8192",
+                                  "lowrank_d64_bf16"])
 def test_compress_fp32_structure_and_mismatch_rate(name):
     wl = SMALL_CASES[name]
     idx, w, ref_idx, ref_w, _ = _compress_both(wl, precision="fp32")
@@ -166,7 +168,7 @@ def _attend_case(wl, precision, weights="uniform", n_core=None, data_seed=99):
 
 
 @pytest.mark.parametrize("precision", ["fp32", "fp64"])
-@pytest.mark.parametrize("name", ["cfg1_full", "cfg2_two_batches", "cfg3_four_heads", "cfg5_n8192"])
+@pytest.mark.parametrize("name", ["cfg1_full", "cfg2_two_batches", "cfg3_four_heads", "cfg5_n8192", "lowrank_d64_bf16"])
 def test_attend_on_oracle_coreset(name, precision):
     wl = SMALL_CASES[name]
     wl = wl.scaled(n_q=min(wl.n_q, 1000))            # ragged last query tile
