@@ -288,6 +288,222 @@ gram_tc_kernel(const __nv_bfloat16 *__restrict__ K, const __nv_bfloat16 *__restr
                                      misc->rdec, misc->unif, p, JR, P, Ptotal, n, cur, wk, warp, lane);
 }
 
+// ---------------------------------------------------------------------------------------------
+// Persistent, pipelined variant for levels whose calls span several tiles (P > 64 pairs).
+// One CTA per SM walks the level's tile list (tile, problem) round-robin.  Roles:
+//   warps 0-3   loaders: gather the tile's row and column points with 16-byte cp.async into a ring
+//               of three 64 KB operand buffers -- one "job" for the keys, one for the values of each
+//               tile -- and let the copies' completion arrive on the job's mbarrier, so up to three
+//               jobs are in flight while earlier ones are multiplied
+//   warp 4      issues the tcgen05.mma of each job into one of two TMEM accumulator slots
+//               (K K^T | V V^T, 256 columns each); its commits free the operand buffers
+//   warps 5-12  epilogue of the previous tile (exp2, product, pair combination, stores) while the
+//               next tile is gathered and multiplied
+// ---------------------------------------------------------------------------------------------
+constexpr int PNS = 3;                       // operand ring depth (jobs)
+constexpr int PTHREADS = 13 * 32;
+
+struct PBarriers {
+    uint64_t full[PNS], empty[PNS], accfull[2], accempty[2];
+    uint32_t tmem_base;
+    uint32_t pad;
+};
+
+template <int D> struct PSmem {
+    static constexpr int JOB = 2 * TR * D * 2;                // row tile + column tile of one operand type
+    static constexpr int OFF_BAR = PNS * JOB;
+    static constexpr int TOTAL = OFF_BAR + 1024 + 1024;
+};
+
+__device__ __forceinline__ void decode_tile(int tile, int P, int64_t &JR, int64_t &JC)
+{
+    const int Tg = P / TP, ntri = Tg * (Tg + 1) / 2;
+    const int g = tile / ntri, local = tile % ntri;
+    int tc = (int)((sqrtf(8.f * (float)local + 1.f) - 1.f) * 0.5f);
+    while ((tc + 1) * (tc + 2) / 2 <= local) ++tc;
+    while (tc * (tc + 1) / 2 > local) --tc;
+    const int tr = local - tc * (tc + 1) / 2;
+    JR = (int64_t)g * P + tr * TP;
+    JC = (int64_t)g * P + tc * TP;
+}
+
+template <int D>
+__global__ void __launch_bounds__(PTHREADS, 1)
+gram_tc_persistent_kernel(const __nv_bfloat16 *__restrict__ K, const __nv_bfloat16 *__restrict__ V,
+                          const int32_t *__restrict__ cur, const float *__restrict__ Mpair,
+                          const unsigned *__restrict__ vmax_bits, int64_t n, int P, int tiles_per_problem,
+                          int total_items, float *__restrict__ F, int64_t F_stride, int *__restrict__ status)
+{
+    using SM = PSmem<D>;
+    constexpr int KH = D / 64;
+    constexpr int CHUNKS = D / 8;                             // 16-byte chunks per row
+    extern __shared__ unsigned char smem_dyn[];
+    unsigned char *smem = reinterpret_cast<unsigned char *>(((uintptr_t)smem_dyn + 1023) & ~(uintptr_t)1023);
+    PBarriers *bar = reinterpret_cast<PBarriers *>(smem + SM::OFF_BAR);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+    if (*reinterpret_cast<volatile int *>(status) != 0) return;
+    if (tid == 0) {
+        for (int b = 0; b < PNS; ++b) { mbar_init(&bar->full[b], 128); mbar_init(&bar->empty[b], 1); }
+        for (int s = 0; s < 2; ++s) { mbar_init(&bar->accfull[s], 1); mbar_init(&bar->accempty[s], 256); }
+        fence_barrier_init();
+    }
+    if (warp == 4) tmem_alloc(&bar->tmem_base, 512);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = bar->tmem_base;
+    bool ok = true;
+
+    if (warp < 4) {
+        // ------------------------------ loaders ------------------------------
+        int job = 0;
+        for (int it = blockIdx.x; it < total_items && ok; it += gridDim.x) {
+            const int p = it / tiles_per_problem, tile = it % tiles_per_problem;
+            int64_t JR, JC;
+            decode_tile(tile, P, JR, JC);
+            const bool diagonal = JR == JC;
+            const int32_t *curp = cur + (int64_t)p * n;
+            // chunk q = tid + 128 i of a 128-row tile lies in row tid / CHUNKS + (128 / CHUNKS) i
+            constexpr int RPT = TR * CHUNKS / 128;            // chunks (= distinct rows) per thread and tile
+            int32_t ra[RPT], rb[RPT];
+#pragma unroll
+            for (int i = 0; i < RPT; ++i) {
+                const int r = tid / CHUNKS + (128 / CHUNKS) * i;
+                ra[i] = __ldg(curp + 2 * JR + r);
+                rb[i] = diagonal ? 0 : __ldg(curp + 2 * JC + r);
+            }
+            const int ch = tid % CHUNKS, kh = ch >> 3, c = ch & 7;
+            for (int op = 0; op < 2 && ok; ++op, ++job) {     // 0: keys, 1: values
+                const int b = job % PNS;
+                ok = mbar_wait(&bar->empty[b], ((uint32_t)(job / PNS) & 1u) ^ 1u);
+                if (!ok) break;
+                const __nv_bfloat16 *X = (op == 0 ? K : V) + (int64_t)p * n * D;
+                const uint32_t dstA = smem_u32(smem + b * SM::JOB), dstB = dstA + TR * D * 2;
+#pragma unroll
+                for (int i = 0; i < RPT; ++i) {
+                    const int r = tid / CHUNKS + (128 / CHUNKS) * i;
+                    const uint32_t off = kh * (TR * 128) + (r >> 3) * 1024 + (r & 7) * 128 + ((c ^ (r & 7)) << 4);
+                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dstA + off), "l"(X + (int64_t)ra[i] * D + ch * 8) : "memory");
+                    if (!diagonal)
+                        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dstB + off), "l"(X + (int64_t)rb[i] * D + ch * 8) : "memory");
+                }
+                // the job's barrier completes when every loader thread's copies have landed
+                asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(&bar->full[b])) : "memory");
+            }
+        }
+        asm volatile("cp.async.wait_all;" ::: "memory");
+        if (!ok && lane == 0) atomicExch(status, 5);
+    } else if (warp == 4) {
+        // ------------------------------ MMA issuer ------------------------------
+        if (lane == 0) {
+            constexpr uint32_t IDESC = umma_idesc_bf16(TR, TR);
+            int job = 0, k = 0;
+            for (int it = blockIdx.x; it < total_items && ok; it += gridDim.x, ++k) {
+                const int tile = it % tiles_per_problem;
+                int64_t JR, JC;
+                decode_tile(tile, P, JR, JC);
+                const bool diagonal = JR == JC;
+                const int slot = k & 1;
+                ok = mbar_wait(&bar->accempty[slot], ((uint32_t)(k >> 1) & 1u) ^ 1u);
+                if (!ok) break;
+                tc_fence_after();
+                for (int op = 0; op < 2 && ok; ++op, ++job) {
+                    const int b = job % PNS;
+                    ok = mbar_wait(&bar->full[b], (uint32_t)(job / PNS) & 1u);
+                    if (!ok) break;
+                    fence_proxy_async();                       // the gathered bytes were written by generic-proxy copies
+                    tc_fence_after();
+                    const uint32_t sA = smem_u32(smem + b * SM::JOB), sB = diagonal ? sA : sA + TR * D * 2;
+#pragma unroll
+                    for (int kh = 0; kh < KH; ++kh)
+#pragma unroll
+                        for (int ks = 0; ks < 4; ++ks)
+                            mma_ss(tmem + slot * 256 + op * 128, umma_desc_k128(sA + kh * (TR * 128) + ks * 32),
+                                   umma_desc_k128(sB + kh * (TR * 128) + ks * 32), IDESC, (kh | ks) != 0);
+                    tc_commit(&bar->empty[b]);
+                }
+                if (ok) tc_commit(&bar->accfull[slot]);
+            }
+            if (!ok) atomicExch(status, 6);
+        }
+    } else {
+        // ------------------------------ epilogue ------------------------------
+        const int e = warp - 5;                               // 0..7
+        const int q4 = warp & 3;                              // TMEM lane quarter this warp may access
+        const int ch = e >> 2;                                // column half
+        const int r = q4 * 32 + lane;                         // point row in the tile
+        const float LOG2E = 1.4426950408889634f;
+        const float qscale = LOG2E / sqrtf((float)D);
+        int k = 0;
+        for (int it = blockIdx.x; it < total_items && ok; it += gridDim.x, ++k) {
+            const int p = it / tiles_per_problem, tile = it % tiles_per_problem;
+            int64_t JR, JC;
+            decode_tile(tile, P, JR, JC);
+            const int slot = k & 1;
+            const float vm = __uint_as_float(vmax_bits[p]);
+            const float vm2 = vm * vm;
+            // running shifts of this thread's 32 pair columns (in log2 units), fetched while the MMAs run
+            float sh[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) sh[i] = __ldg(Mpair + (int64_t)p * (n / 2) + JC + ch * 32 + i) * LOG2E;
+            ok = mbar_wait(&bar->accfull[slot], (uint32_t)(k >> 1) & 1u);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t taddr = tmem + ((uint32_t)(q4 * 32) << 16) + slot * 256 + ch * 64;
+            float h[32];
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                uint32_t kk[32], vv[32];
+                tmem_ld32(taddr + q * 32, kk);
+                tmem_ld32(taddr + 128 + q * 32, vv);
+                tmem_wait_ld();
+#pragma unroll
+                for (int c = 0; c < 32; c += 2) {
+                    const float shc = sh[q * 16 + (c >> 1)];
+                    float e0 = fmaf(__uint_as_float(kk[c]), qscale, -shc);
+                    float e1 = fmaf(__uint_as_float(kk[c + 1]), qscale, -shc);
+                    float g0 = e0 < -115.f ? 0.f : fast_exp2(e0) * (__uint_as_float(vv[c]) + vm2);
+                    float g1 = e1 < -115.f ? 0.f : fast_exp2(e1) * (__uint_as_float(vv[c + 1]) + vm2);
+                    h[q * 16 + (c >> 1)] = g0 - g1;
+                }
+            }
+            // the accumulator slot is free as soon as its values are in registers
+            tc_fence_before();
+            mbar_arrive(&bar->accempty[slot]);
+            const bool odd = lane & 1;
+            float f[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const float send = odd ? h[i] : h[i + 16];
+                const float recv = __shfl_xor_sync(0xffffffffu, send, 1);
+                f[i] = odd ? recv - h[i + 16] : h[i] - recv;
+            }
+            const int64_t jr = JR + (r >> 1);
+            const int64_t jc0 = JC + ch * 32 + (odd ? 16 : 0);
+            const int64_t gr = jr / P;
+            float *Fp = F + (int64_t)p * F_stride + jr * P - gr * P;
+            if (JR < JC) {
+                // a tile above the diagonal of its call: every entry is wanted, 64 contiguous bytes per thread
+#pragma unroll
+                for (int i = 0; i < 16; i += 4)
+                    *reinterpret_cast<float4 *>(Fp + jc0 + i) = make_float4(f[i], f[i + 1], f[i + 2], f[i + 3]);
+            } else {
+#pragma unroll
+                for (int i = 0; i < 16; ++i)
+                    if (jr <= jc0 + i) Fp[jc0 + i] = f[i];
+            }
+        }
+        if (!ok && lane == 0) atomicExch(status, 7);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 4) {
+        tc_fence_after();
+        tmem_dealloc(tmem, 512);
+    }
+}
+
 template <int D>
 static int launch(const __nv_bfloat16 *K, const __nv_bfloat16 *V, const elm_params *p, const int32_t *cur,
                   const float *Mpair, const unsigned *vmax_bits, int P, int64_t Ptotal, int groups, float *F,
@@ -300,6 +516,23 @@ static int launch(const __nv_bfloat16 *K, const __nv_bfloat16 *V, const elm_para
         tiles = (int64_t)groups * (Tg * (Tg + 1) / 2);
     } else {
         tiles = (Ptotal + TP - 1) / TP;
+    }
+    if (P > TP) {
+        // calls that span several tiles: persistent, pipelined kernel, one CTA per SM
+        static int sm_count = 0;
+        if (sm_count == 0) {
+            int dev = 0;
+            ELM_CUDA_TRY(cudaGetDevice(&dev));
+            ELM_CUDA_TRY(cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev));
+        }
+        const int64_t total = tiles * BH;
+        const int grid = (int)(total < sm_count ? total : sm_count);
+        auto pk = gram_tc_persistent_kernel<D>;
+        ELM_CUDA_TRY(cudaFuncSetAttribute(pk, cudaFuncAttributeMaxDynamicSharedMemorySize, PSmem<D>::TOTAL));
+        pk<<<grid, PTHREADS, PSmem<D>::TOTAL, st>>>(K, V, cur, Mpair, vmax_bits, p->n_kv, P, (int)tiles, (int)total, F,
+                                                   F_stride, status);
+        count_launches(1);
+        return cuda_status(cudaGetLastError());
     }
     auto kern = gram_tc_kernel<D>;
     ELM_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<D>::TOTAL));
