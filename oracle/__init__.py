@@ -84,6 +84,13 @@ def _load():
     lib.oracle_mmd2.argtypes = [_f32p, _f32p, ctypes.c_int, ctypes.c_double, _i32p, ctypes.c_int,
                                 _i32p, _f64p, ctypes.c_int, ctypes.c_double]
     lib.oracle_mmd2.restype = ctypes.c_double
+    _i64p = ctypes.POINTER(ctypes.c_int64)
+    lib.oracle_thinformer_express.argtypes = [_f32p, _f32p, _f32p, ctypes.c_int64, ctypes.c_int, ctypes.c_int,
+                                              ctypes.c_int, ctypes.c_double, ctypes.c_uint64, ctypes.c_uint32,
+                                              _f64p, _i32p, _i32p, _f64p, _i32p, _i64p]
+    lib.oracle_thinformer_express.restype = ctypes.c_int
+    lib.oracle_exact_causal_attention.argtypes = [_f32p, _f32p, _f32p, ctypes.c_int64, ctypes.c_int, _f64p]
+    lib.oracle_exact_causal_attention.restype = ctypes.c_int
     lib.oracle_num_threads.argtypes = []
     lib.oracle_num_threads.restype = ctypes.c_int
     _lib = lib
@@ -270,3 +277,42 @@ def mmd2(K, V, vmax_: float, in_idx, out_idx, w, shift: float = 0.0) -> float:
     w, wp = _f64(w)
     return float(_load().oracle_mmd2(kp, vp, K.shape[1], vmax_, ap, a.shape[0], op, wp,
                                      o.shape[0], shift))
+
+
+def thinformer_express(Q, K, V, log2_nout: int, mbar: int, delta: float = 0.5, seed: int = 1, head: int = 0,
+                       want_outputs: bool = True):
+    """Algorithms 1-5 streaming over one attention problem (Q, K, V are [n, d]).
+
+    Returns a dict: O [n, d] (or None), cache_size [n] (points in wtd_cache() when token t arrives),
+    final_idx / final_w (wtd_cache() after the last update), halve_calls."""
+    Q, qp = _f32(Q)
+    K, kp = _f32(K)
+    V, vp = _f32(V)
+    n, d = K.shape
+    n_out = 1 << log2_nout
+    O = np.zeros((n, d), dtype=np.float64) if want_outputs else None
+    cache = np.zeros(n, dtype=np.int32)
+    fidx = np.zeros(6 * n_out + 1, dtype=np.int32)
+    fw = np.zeros(6 * n_out + 1, dtype=np.float64)
+    fc = ctypes.c_int32(0)
+    hc = ctypes.c_int64(0)
+    rc = _load().oracle_thinformer_express(qp, kp, vp, n, d, log2_nout, mbar, delta, seed, head,
+                                           O.ctypes.data_as(_f64p) if want_outputs else None,
+                                           cache.ctypes.data_as(_i32p), fidx.ctypes.data_as(_i32p),
+                                           fw.ctypes.data_as(_f64p), ctypes.byref(fc), ctypes.byref(hc))
+    if rc != 0:
+        raise ValueError(f"oracle_thinformer_express failed with {rc}")
+    c = int(fc.value)
+    return {"O": O, "cache_size": cache, "final_idx": fidx[:c].copy(), "final_w": fw[:c].copy(),
+            "halve_calls": int(hc.value)}
+
+
+def exact_causal_attention(Q, K, V):
+    Q, qp = _f32(Q)
+    K, kp = _f32(K)
+    V, vp = _f32(V)
+    O = np.zeros(Q.shape, dtype=np.float64)
+    rc = _load().oracle_exact_causal_attention(qp, kp, vp, K.shape[0], K.shape[1], O.ctypes.data_as(_f64p))
+    if rc != 0:
+        raise ValueError(f"oracle_exact_causal_attention failed with {rc}")
+    return O

@@ -13,6 +13,8 @@
  *   oracle_wtd_attention      Algorithm 5 / Eq. (def:att_approx): weighted attention
  *   oracle_exact_attention    Eq. (unmaskedatt): exact unmasked attention
  *   oracle_mmd2               squared kernel MMD between a point set and a weighted subset
+ *   oracle_thinformer_express Algorithms 1-5 + Corollary 2: streaming Express cache with KH, per-token attention
+ *   oracle_exact_causal_attention  Eq. (def:att)
  *   oracle_philox4x32_10      the counter-based generator the uniforms come from
  *
  * Inputs are float arrays (bf16 and fp32 tensors are both exactly representable there);
@@ -433,6 +435,219 @@ double oracle_mmd2(const float *K, const float *V, int d, double vmax, const int
         for (int e = 0; e < n_out; ++e)
             t_out += w[c] * w[e] * oracle_katt(K, V, d, vmax, out[c], out[e], shift, 0);
     return t_in / ((double)n_in * (double)n_in) - 2.0 * t_x / (double)n_in + t_out;
+}
+
+/* ------------------------------------------------------------------------------------ */
+/* Express / KH-Express / Thinformer Express: Algorithms 1-5 and Corollary 2, streaming.   */
+/* One update per point, exactly in the order the algorithms state.                        */
+/*                                                                                          */
+/* Readings (beyond those at the top of this file):                                        */
+/*   R-vmax-causal  v_max of Eq. (katt) is taken over the whole observed sequence (the      */
+/*                  prefill setting: every token is known in advance).                     */
+/*   R-ctr          uniforms: Philox counter (pair, call number at that level of the       */
+/*                  current Compress2 instance, code, problem) with                        */
+/*                    code = level i + 64 (4 r + j)   Halve_i of sibling j in {1,2,3} of     */
+/*                                                    round r = m/2,                        */
+/*                    code = 62 + h + 64 (4 r)        h-th of the two E halvings of round r, */
+/*                    code = 61 + 64 (4 r + j)        Subsample of sibling j, counter word 0 */
+/*                                                    = stratum number.                    */
+/*   R-unif-int     Unif([n, n + 2^(m-mbar))) = n + floor(U 2^(m-mbar)), U the 24-bit uniform. */
+/* ------------------------------------------------------------------------------------ */
+typedef struct {
+    /* problem */
+    const float *K, *V;
+    int d;
+    double vmax, delta;
+    uint64_t seed;
+    uint32_t head;
+    int64_t n_out;
+    int mbar;
+    /* Express state (Algorithm 1) */
+    int m;              /* thinning factor */
+    int64_t n, ell;
+    int32_t *E;
+    int64_t nE;
+    int b;              /* completed thin phases since the last halve phase */
+    /* Subsample(m, mbar) state (Algorithm 3) */
+    int64_t s_n, s_i;
+    /* Compress2(q, 2^q n_out, Halve_m) state (Algorithm 2) */
+    int q;
+    int32_t *S[40];
+    int64_t nS[40];
+    int64_t calls[40];
+    int64_t halve_calls;   /* total KH calls made (cost accounting) */
+} express_state;
+
+static double kh_express_delta_m(double delta, int m)
+{
+    return 0.5 * delta * (1.0 / log2(0.5 * m + 2.0) - 1.0 / log2(0.5 * m + 3.0));
+}
+
+static void express_reset_thin(express_state *st)
+{
+    st->s_n = 0;
+    st->s_i = 0;
+    st->q = st->m < st->mbar ? st->m : st->mbar;
+    for (int i = 0; i <= st->q; ++i) { st->nS[i] = 0; st->calls[i] = 0; }
+}
+
+static int express_halve(express_state *st, int32_t *x, int64_t s, double dlt, uint32_t code, uint32_t call,
+                         int32_t *out)
+{
+    double *U = (double *)malloc(sizeof(double) * (size_t)(s / 2));
+    if (!U) return -2;
+    for (int64_t i = 0; i < s / 2; ++i) U[i] = oracle_uniform(st->seed, (uint32_t)i, call, code, st->head);
+    int rc = oracle_kh(st->K, st->V, st->d, st->vmax, x, (int)s, dlt, 1, U, out, NULL, NULL);
+    free(U);
+    st->halve_calls += 1;
+    return rc;
+}
+
+/* Compress2.update(x) with Halve_i = KH(delta_{m,i}) */
+static int express_compress2_update(express_state *st, int32_t x)
+{
+    const int q = st->q;
+    const int64_t n_in = st->n_out << q;
+    st->S[0][st->nS[0]++] = x;
+    for (int i = 0; i < q; ++i) {
+        const int64_t thresh = (n_in << i) >> (2 * (q - 1));            /* n_in 2^i / 4^(q-1) */
+        if (st->nS[i] == thresh) {
+            const double dm = kh_express_delta_m(st->delta, st->m);
+            const double dlt = pow(4.0, (double)(i + 1 - q)) * dm / (3.0 * (double)q);
+            const uint32_t code = (uint32_t)i + 64u * (uint32_t)(4 * (st->m / 2) + st->b + 1);
+            int rc = express_halve(st, st->S[i], thresh, dlt, code, (uint32_t)st->calls[i], st->S[i + 1] + st->nS[i + 1]);
+            if (rc != 0) return rc;
+            st->calls[i] += 1;
+            st->nS[i + 1] += thresh / 2;
+            st->nS[i] = 0;
+        }
+    }
+    return 0;
+}
+
+/* Subsample.keep(x) */
+static int express_subsample_keep(express_state *st)
+{
+    st->s_n += 1;
+    if (st->m <= st->mbar) return 1;
+    const int64_t w = (int64_t)1 << (st->m - st->mbar);
+    if ((st->s_n - 1) % w == 0) {
+        const uint32_t code = 61u + 64u * (uint32_t)(4 * (st->m / 2) + st->b + 1);
+        const double U = oracle_uniform(st->seed, (uint32_t)((st->s_n - 1) / w), 0u, code, st->head);
+        st->s_i = st->s_n + (int64_t)floor(U * (double)w);
+    }
+    return st->s_n == st->s_i;
+}
+
+/* Express.update(x) */
+static int express_update(express_state *st, int32_t x)
+{
+    st->n += 1;
+    if (st->n <= st->n_out) { st->E[st->nE++] = x; return 0; }          /* exact phase */
+    st->ell += 1;                                                        /* thin phase */
+    if (express_subsample_keep(st)) {
+        int rc = express_compress2_update(st, x);
+        if (rc != 0) return rc;
+    }
+    if (st->ell == (st->n_out << st->m)) {
+        for (int64_t i = 0; i < st->nS[st->q]; ++i) st->E[st->nE++] = st->S[st->q][i];
+        st->nS[st->q] = 0;
+        st->ell = 0;
+        st->b += 1;
+    }
+    if (st->n == 4 * (st->n_out << st->m)) {                             /* halve phase */
+        const double dm = kh_express_delta_m(st->delta, st->m);
+        int32_t *tmp = (int32_t *)malloc(sizeof(int32_t) * (size_t)(2 * st->n_out));
+        if (!tmp) return -2;
+        int rc = express_halve(st, st->E, 4 * st->n_out, 0.5 * dm, 62u + 64u * (uint32_t)(4 * (st->m / 2)), 0u, tmp);
+        if (rc == 0) rc = express_halve(st, tmp, 2 * st->n_out, 0.5 * dm, 63u + 64u * (uint32_t)(4 * (st->m / 2)), 0u, st->E);
+        free(tmp);
+        if (rc != 0) return rc;
+        st->nE = st->n_out;
+        st->m += 2;
+        st->b = 0;
+    }
+    if (st->ell == 0) express_reset_thin(st);
+    return 0;
+}
+
+/*
+ * Thinformer Express over one attention problem: for t = 1..n
+ *     o_t = WtdAttention((q_t, k_t, v_t), C)   then   C.update((k_t, v_t)).
+ * Outputs (each may be NULL):
+ *   O[n][d]          the attention outputs
+ *   cache_size[n]    points in wtd_cache() when token t arrives (the input token not counted)
+ *   final_idx/final_w/final_count  wtd_cache() after the last update (capacity 6 n_out)
+ *   halve_calls      number of KH calls made
+ */
+int oracle_thinformer_express(const float *Q, const float *K, const float *V, int64_t n, int d, int log2_nout,
+                              int mbar, double delta, uint64_t seed, uint32_t head, double *O,
+                              int32_t *cache_size, int32_t *final_idx, double *final_w, int32_t *final_count,
+                              int64_t *halve_calls)
+{
+    if (log2_nout < 0 || mbar < 0 || !(delta > 0.0 && delta < 1.0)) return -1;
+    express_state st;
+    memset(&st, 0, sizeof(st));
+    st.K = K; st.V = V; st.d = d; st.delta = delta; st.seed = seed; st.head = head;
+    st.n_out = (int64_t)1 << log2_nout;
+    st.mbar = mbar;
+    st.vmax = oracle_vmax(V, n, d);                                       /* R-vmax-causal */
+    st.E = (int32_t *)malloc(sizeof(int32_t) * (size_t)(4 * st.n_out));
+    int rc = st.E ? 0 : -2;
+    for (int i = 0; i <= mbar && rc == 0; ++i) {
+        /* level i of any Compress2(q <= mbar) holds at most max(n_out 2^(2-q+i), n_out) points */
+        st.S[i] = (int32_t *)malloc(sizeof(int32_t) * (size_t)(4 * st.n_out));
+        if (!st.S[i]) rc = -2;
+    }
+    const int64_t cap = 6 * st.n_out + 1;
+    int32_t *cidx = (int32_t *)malloc(sizeof(int32_t) * (size_t)cap);
+    double *cw = (double *)malloc(sizeof(double) * (size_t)cap);
+    float *qrow = NULL;
+    if (!cidx || !cw) rc = -2;
+    if (rc == 0) express_reset_thin(&st);
+    for (int64_t t = 0; t < n && rc == 0; ++t) {
+        /* wtd_cache(): [(S_i, 2^(i-q))]_{i=0..q} then (E, 1) */
+        int64_t c = 0;
+        for (int i = 0; i <= st.q; ++i)
+            for (int64_t a = 0; a < st.nS[i]; ++a) { cidx[c] = st.S[i][a]; cw[c] = ldexp(1.0, i - st.q); ++c; }
+        for (int64_t a = 0; a < st.nE; ++a) { cidx[c] = st.E[a]; cw[c] = 1.0; ++c; }
+        if (cache_size) cache_size[t] = (int32_t)c;
+        if (O) {
+            /* incorporate the input token into S_0 (weight 2^(-q)) and attend */
+            cidx[c] = (int32_t)t; cw[c] = ldexp(1.0, -st.q); ++c;
+            rc = oracle_wtd_attention(Q + t * d, K, V, cidx, cw, (int)c, 1, d, O + t * d);
+            if (rc != 0) break;
+        }
+        rc = express_update(&st, (int32_t)t);
+    }
+    if (rc == 0) {
+        int64_t c = 0;
+        for (int i = 0; i <= st.q; ++i)
+            for (int64_t a = 0; a < st.nS[i]; ++a) {
+                if (final_idx) final_idx[c] = st.S[i][a];
+                if (final_w) final_w[c] = ldexp(1.0, i - st.q);
+                ++c;
+            }
+        for (int64_t a = 0; a < st.nE; ++a) {
+            if (final_idx) final_idx[c] = st.E[a];
+            if (final_w) final_w[c] = 1.0;
+            ++c;
+        }
+        if (final_count) *final_count = (int32_t)c;
+        if (halve_calls) *halve_calls = st.halve_calls;
+    }
+    free(st.E);
+    for (int i = 0; i <= mbar; ++i) free(st.S[i]);
+    free(cidx); free(cw); free(qrow);
+    return rc;
+}
+
+/* Exact causal attention, Eq. (def:att): query t over the pairs 1..t. */
+int oracle_exact_causal_attention(const float *Q, const float *K, const float *V, int64_t n, int d, double *O)
+{
+    int rc = 0;
+    for (int64_t t = 0; t < n && rc == 0; ++t) rc = oracle_exact_attention(Q + t * d, K, V, t + 1, 1, d, O + t * d);
+    return rc;
 }
 
 int oracle_num_threads(void)
