@@ -276,6 +276,23 @@ static int attend_enqueue_untimed(const Tin *Q, const Tin *K, const Tin *V, cons
 
 }  // namespace elm
 
+namespace elm {
+// elm_attend after argument validation
+int attend_enqueue(const void *Q, const void *K, const void *V, const int32_t *idx, const float *w, int32_t n_core,
+                   const elm_params *params, void *O, void *workspace, cudaStream_t st)
+{
+    unsigned char *ws = (unsigned char *)workspace;
+    const bool det = params->precision == ELM_PREC_FP64_DET;
+    if (params->dtype == ELM_F32) {
+        return det ? attend_impl<float, double>((const float *)Q, (const float *)K, (const float *)V, idx, w, n_core, params, (float *)O, ws, st)
+                   : attend_impl<float, float>((const float *)Q, (const float *)K, (const float *)V, idx, w, n_core, params, (float *)O, ws, st);
+    }
+    typedef __nv_bfloat16 bf;
+    return det ? attend_impl<bf, double>((const bf *)Q, (const bf *)K, (const bf *)V, idx, w, n_core, params, (bf *)O, ws, st)
+               : attend_impl<bf, float>((const bf *)Q, (const bf *)K, (const bf *)V, idx, w, n_core, params, (bf *)O, ws, st);
+}
+}  // namespace elm
+
 extern "C" int elm_attend_workspace_bytes(const elm_params *params, int32_t n_core, size_t *bytes)
 {
     using namespace elm;
@@ -301,16 +318,7 @@ extern "C" int elm_attend(const void *Q, const void *K, const void *V, const int
         return ELM_ERR_ALIGN;
     if ((uintptr_t)workspace & 255) return ELM_ERR_ALIGN;
     if (workspace_bytes < attend_layout(params, n_core).total) return ELM_ERR_WORKSPACE;
-    cudaStream_t st = (cudaStream_t)stream;
-    unsigned char *ws = (unsigned char *)workspace;
-    const bool det = params->precision == ELM_PREC_FP64_DET;
-    if (params->dtype == ELM_F32) {
-        return det ? attend_impl<float, double>((const float *)Q, (const float *)K, (const float *)V, idx, w, n_core, params, (float *)O, ws, st)
-                   : attend_impl<float, float>((const float *)Q, (const float *)K, (const float *)V, idx, w, n_core, params, (float *)O, ws, st);
-    }
-    typedef __nv_bfloat16 bf;
-    return det ? attend_impl<bf, double>((const bf *)Q, (const bf *)K, (const bf *)V, idx, w, n_core, params, (bf *)O, ws, st)
-               : attend_impl<bf, float>((const bf *)Q, (const bf *)K, (const bf *)V, idx, w, n_core, params, (bf *)O, ws, st);
+    return attend_enqueue(Q, K, V, idx, w, n_core, params, O, workspace, (cudaStream_t)stream);
 }
 
 extern "C" int elm_attend_static(const void *Q, const void *K, const void *V, const int32_t *idx,

@@ -19,6 +19,10 @@ struct AttendLayout {
 };
 AttendLayout attend_layout(const elm_params *p, int32_t n_core);
 
+// elm_attend after argument validation
+int attend_enqueue(const void *Q, const void *K, const void *V, const int32_t *idx, const float *w, int32_t n_core,
+                   const elm_params *params, void *O, void *workspace, cudaStream_t st);
+
 // Tensor-core path (bf16 storage, fp32 accumulation): gather + attention, enqueued on `st`.
 // `timed` selects whether the per-stage event timers are used.
 int attend_tc(const __nv_bfloat16 *Q, const __nv_bfloat16 *K, const __nv_bfloat16 *V, const int32_t *idx,

@@ -349,7 +349,7 @@ __global__ void __launch_bounds__(576) walk_cta_kernel(const T *__restrict__ F, 
                                                        const int32_t *__restrict__ cur,
                                                        int32_t *__restrict__ out, int64_t out_stride,
                                                        int64_t n, int P, int level, uint64_t seed,
-                                                       T logfac)
+                                                       T logfac, uint32_t pbase)
 {
     constexpr int PW = 2048 / sizeof(T);                             // panel width in columns (64 KB / 2 buffers... per 32 rows)
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -387,7 +387,7 @@ __global__ void __launch_bounds__(576) walk_cta_kernel(const T *__restrict__ F, 
         const T d = Fg[(int64_t)i * P + i];
         b_s[i] = sqrt(d > 0 ? d : (T)0);
         r_s[i] = rdecay[(int64_t)p * (n / 2) + base + i];
-        U_s[i] = halving_uniform<T>(seed, (uint32_t)i, (uint32_t)g, (uint32_t)level, (uint32_t)p);
+        U_s[i] = halving_uniform<T>(seed, (uint32_t)i, (uint32_t)g, (uint32_t)level, (uint32_t)p + pbase);
     }
     if (warp <= 1) asm volatile("cp.async.wait_group 0;" ::: "memory");
 
@@ -493,7 +493,7 @@ __global__ void __launch_bounds__(256) walk_warp_kernel(const T *__restrict__ F,
                                                         const int32_t *__restrict__ cur,
                                                         int32_t *__restrict__ out, int64_t out_stride,
                                                         int64_t n, int P, int groups, int level,
-                                                        uint64_t seed, T logfac)
+                                                        uint64_t seed, T logfac, uint32_t pbase)
 {
     const int p = blockIdx.y;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -504,7 +504,7 @@ __global__ void __launch_bounds__(256) walk_warp_kernel(const T *__restrict__ F,
     T bmax = 0;
     const bool live = lane < P;
     const T r = live ? rdecay[(int64_t)p * (n / 2) + base + lane] : (T)1;
-    const T U = halving_uniform<T>(seed, (uint32_t)lane, (uint32_t)g, (uint32_t)level, (uint32_t)p);
+    const T U = halving_uniform<T>(seed, (uint32_t)lane, (uint32_t)g, (uint32_t)level, (uint32_t)p + pbase);
     uint32_t swaps = walk_block<T>(Fg, P, 0, P, (T)0, r, U, logfac, bmax, lane);
     if (live) {
         const uint32_t sw = (swaps >> lane) & 1u;
@@ -572,7 +572,7 @@ static int run_gram_simt(const Tin *K, const Tin *V, const elm_params *p, const 
 
 template <typename Tin, typename T>
 static int compress_impl(const Tin *K, const Tin *V, const elm_params *p, uint64_t seed,
-                         int32_t *idx_out, float *w_out, unsigned char *ws, cudaStream_t st)
+                         int32_t *idx_out, float *w_out, unsigned char *ws, cudaStream_t st, uint32_t pbase)
 {
     const CompressLayout L = compress_layout(p);
     const int BH = p->batch * p->kv_heads;
@@ -635,6 +635,7 @@ static int compress_impl(const Tin *K, const Tin *V, const elm_params *p, uint64
                     wk.rdecay = rdecay;
                     wk.out = out;
                     wk.out_stride = out_stride;
+                    wk.pbase = pbase;
                     walked = wk.fused;
                     rc = gram_tc(K, V, p, cur, Mpair, vmax_bits, P, Ptotal, groups, F, L.F_stride,
                                  reinterpret_cast<int *>(vmax_bits + BH), wk, st);
@@ -659,10 +660,10 @@ static int compress_impl(const Tin *K, const Tin *V, const elm_params *p, uint64
                 auto kern = walk_cta_kernel<T>;
                 ELM_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
                 kern<<<dim3((unsigned)groups, (unsigned)BH), threads, smem, st>>>(
-                    F, L.F_stride, rdecay, cur, out, out_stride, n, P, level, seed, logfac);
+                    F, L.F_stride, rdecay, cur, out, out_stride, n, P, level, seed, logfac, pbase);
             } else {
                 walk_warp_kernel<T><<<dim3((unsigned)((groups + 7) / 8), (unsigned)BH), 256, 0, st>>>(
-                    F, L.F_stride, rdecay, cur, out, out_stride, n, P, groups, level, seed, logfac);
+                    F, L.F_stride, rdecay, cur, out, out_stride, n, P, groups, level, seed, logfac, pbase);
             }
             count_launches(1);
             ELM_CUDA_TRY(cudaGetLastError());
@@ -681,6 +682,23 @@ static int compress_impl(const Tin *K, const Tin *V, const elm_params *p, uint64
 
 }  // namespace elm
 
+namespace elm {
+// Validated arguments -> launches.  `pbase` numbers the call's first attention problem in the
+// uniforms' counter, so that a batch processed in several slices draws the same uniforms as one call.
+int compress_enqueue(const void *K, const void *V, const elm_params *params, uint64_t seed, int32_t *idx_out,
+                     float *w_out, void *workspace, cudaStream_t st, uint32_t pbase)
+{
+    unsigned char *ws = (unsigned char *)workspace;
+    const bool det = params->precision == ELM_PREC_FP64_DET;
+    if (params->dtype == ELM_F32) {
+        return det ? compress_impl<float, double>((const float *)K, (const float *)V, params, seed, idx_out, w_out, ws, st, pbase)
+                   : compress_impl<float, float>((const float *)K, (const float *)V, params, seed, idx_out, w_out, ws, st, pbase);
+    }
+    return det ? compress_impl<__nv_bfloat16, double>((const __nv_bfloat16 *)K, (const __nv_bfloat16 *)V, params, seed, idx_out, w_out, ws, st, pbase)
+               : compress_impl<__nv_bfloat16, float>((const __nv_bfloat16 *)K, (const __nv_bfloat16 *)V, params, seed, idx_out, w_out, ws, st, pbase);
+}
+}  // namespace elm
+
 extern "C" int elm_compress(const void *K, const void *V, const elm_params *params, uint64_t seed,
                             int32_t *idx_out, float *w_out, void *workspace, size_t workspace_bytes,
                             void *stream)
@@ -693,13 +711,5 @@ extern "C" int elm_compress(const void *K, const void *V, const elm_params *para
     if (((uintptr_t)K | (uintptr_t)V | (uintptr_t)idx_out | (uintptr_t)w_out) & 15) return ELM_ERR_ALIGN;
     if ((uintptr_t)workspace & 255) return ELM_ERR_ALIGN;
     if (workspace_bytes < compress_layout(params).total) return ELM_ERR_WORKSPACE;
-    cudaStream_t st = (cudaStream_t)stream;
-    unsigned char *ws = (unsigned char *)workspace;
-    const bool det = params->precision == ELM_PREC_FP64_DET;
-    if (params->dtype == ELM_F32) {
-        return det ? compress_impl<float, double>((const float *)K, (const float *)V, params, seed, idx_out, w_out, ws, st)
-                   : compress_impl<float, float>((const float *)K, (const float *)V, params, seed, idx_out, w_out, ws, st);
-    }
-    return det ? compress_impl<__nv_bfloat16, double>((const __nv_bfloat16 *)K, (const __nv_bfloat16 *)V, params, seed, idx_out, w_out, ws, st)
-               : compress_impl<__nv_bfloat16, float>((const __nv_bfloat16 *)K, (const __nv_bfloat16 *)V, params, seed, idx_out, w_out, ws, st);
+    return compress_enqueue(K, V, params, seed, idx_out, w_out, workspace, (cudaStream_t)stream, 0u);
 }

@@ -23,6 +23,10 @@ struct CompressLayout {
 };
 CompressLayout compress_layout(const elm_params *p);
 
+// elm_compress after argument validation; `pbase` = number of the call's first attention problem.
+int compress_enqueue(const void *K, const void *V, const elm_params *params, uint64_t seed, int32_t *idx_out,
+                     float *w_out, void *workspace, cudaStream_t st, uint32_t pbase);
+
 // What the Gram kernel needs to also run the halving walk of calls that fit one of its tiles
 // (at most 64 pairs): with `fused` set the pair Gram of the level never leaves shared memory and
 // the survivors go straight to `out`.
@@ -34,6 +38,7 @@ struct WalkArgs {
     const float *rdecay;     // [BH][n/2]
     int32_t *out;            // next level's sequence (or the final coreset)
     int64_t out_stride;
+    uint32_t pbase;          // number of the first attention problem of this call (uniforms' counter)
 };
 
 // Tensor-core pair Gram of one level (bf16 storage, fp32 arithmetic); same output layout as the
