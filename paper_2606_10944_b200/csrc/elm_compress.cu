@@ -5,6 +5,7 @@
 // This file holds the precision-generic SIMT kernels (fp64 deterministic mode, fp32 inputs) and
 // the host-side level scheduler.  The tensor-core Gram for bf16 inputs lives in elm_gram_tc.cu.
 #include <math.h>
+#include <stdlib.h>
 
 #include <type_traits>
 
@@ -285,34 +286,6 @@ __device__ __forceinline__ uint32_t walk_block(const T *__restrict__ Fg, int P, 
     return swaps;
 }
 
-// The serial part of a 32-pair block with everything in registers: Fd[t] = F[i0 + t, i0 + lane]
-// (used for t < lane), b = b_i of this lane's pair.  No memory operation inside.
-template <typename T>
-__device__ __forceinline__ uint32_t walk_block_regs(const T (&Fd)[32], T b, T alpha, T r, T U, T logfac,
-                                                    T &bmax, int lane)
-{
-    T my_bmax = 0;
-#pragma unroll
-    for (int t = 0; t < 32; ++t) {
-        T bt = __shfl_sync(0xffffffffu, b, t);
-        T rt = __shfl_sync(0xffffffffu, r, t);
-        T carried = bmax * rt;
-        bmax = bt > carried ? bt : carried;
-        if (t == lane) my_bmax = bmax;
-    }
-    const T a = b * my_bmax * logfac;
-    uint32_t swaps = 0;
-#pragma unroll
-    for (int t = 0; t < 32; ++t) {
-        bool mine = (lane == t) && swap_decision(alpha, a, U);
-        uint32_t sw = (__ballot_sync(0xffffffffu, mine) >> t) & 1u;
-        swaps |= sw << t;
-        T f = t < lane ? Fd[t] : (T)0;
-        alpha += sw ? f : -f;
-    }
-    return swaps;
-}
-
 // 16-byte asynchronous copy global -> shared
 __device__ __forceinline__ void cp_async16(void *smem_dst, const void *gsrc)
 {
@@ -486,6 +459,21 @@ __global__ void __launch_bounds__(576) walk_cta_kernel(const T *__restrict__ F, 
     }
 }
 
+// Smallest call (in pairs) that goes to the chain kernel of elm_walk_chain.cu.  From about a
+// thousand pairs on, a call is worth a cluster of CTAs; below that one CTA per call (walk_cta_kernel)
+// already fills the GPU with calls.  The environment variable exists for tests, which push small
+// calls through the chain kernel.
+static int walk_chain_min_pairs()
+{
+    static int v = -1;
+    if (v < 0) {
+        const char *e = getenv("ELM_WALK_CHAIN_MIN_PAIRS");
+        v = e ? atoi(e) : 1024;
+        if (v < 32) v = 32;
+    }
+    return v;
+}
+
 // Calls with fewer than 32 pairs: one warp per call, 8 calls per CTA.
 template <typename T>
 __global__ void __launch_bounds__(256) walk_warp_kernel(const T *__restrict__ F, int64_t F_stride,
@@ -649,7 +637,11 @@ static int compress_impl(const Tin *K, const Tin *V, const elm_params *p, uint64
         }
         if (!walked) {
             StageTimer t(ELM_STAGE_WALK, st, 1);
-            if (P >= 32) {
+            if (P >= walk_chain_min_pairs() && walk_chain_covers<T>(P)) {
+                const int rc = walk_chain<T>(F, L.F_stride, rdecay, cur, out, out_stride, n, P, groups, (int)BH, level,
+                                             seed, logfac, pbase, reinterpret_cast<int *>(vmax_bits + BH), st);
+                if (rc != ELM_OK) return rc;
+            } else if (P >= 32) {
                 // walker warp + tile-copy warp + updaters (one per two pairs, at most 512 threads)
                 int upd = P / 2;
                 upd = upd < 32 ? 32 : (upd > 512 ? 512 : upd);

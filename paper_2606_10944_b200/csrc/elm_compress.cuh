@@ -47,4 +47,12 @@ int gram_tc(const __nv_bfloat16 *K, const __nv_bfloat16 *V, const elm_params *p,
             const float *Mpair, const unsigned *vmax_bits, int P, int64_t Ptotal, int groups, float *F,
             int64_t F_stride, int *status, const WalkArgs &wk, cudaStream_t st);
 
+// The halving walk of one level for calls of at least 32 pairs (one CTA or one cluster per call).
+// walk_chain_covers says whether a call size fits its shared-memory plan; `status` as above.
+template <typename T> bool walk_chain_covers(int P);
+template <typename T>
+int walk_chain(const T *F, int64_t F_stride, const T *rdecay, const int32_t *cur, int32_t *out, int64_t out_stride,
+               int64_t n, int P, int groups, int problems, int level, uint64_t seed, T logfac, uint32_t pbase,
+               int *status, cudaStream_t st);
+
 }  // namespace elm

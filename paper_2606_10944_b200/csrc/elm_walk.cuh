@@ -30,10 +30,10 @@ __device__ __forceinline__ bool swap_decision(float alpha, float a, float U)
 // d[u] < 0; a decision then updates the later d[u] with independent FMAs, so a step costs one
 // compare-select-FMA chain instead of a warp vote.  b_u = 0 (a_u = 0) needs no special case in the
 // updates because then F[., u] = 0 (Cauchy-Schwarz in the RKHS); its decision is U_u < 1/2.
-template <int LD>
-__device__ __forceinline__ uint32_t walk_block_thread(const float *__restrict__ tile, const float *__restrict__ alpha32,
-                                                      const float *__restrict__ b32, const float *__restrict__ r32,
-                                                      const float *__restrict__ U32, float logfac, float &bmax)
+__device__ __forceinline__ uint32_t walk_block_thread_ld(const float *__restrict__ tile, const int LD,
+                                                         const float *__restrict__ alpha32,
+                                                         const float *__restrict__ b32, const float *__restrict__ r32,
+                                                         const float *__restrict__ U32, float logfac, float &bmax)
 {
     float d[32];
 #pragma unroll
@@ -59,6 +59,41 @@ __device__ __forceinline__ uint32_t walk_block_thread(const float *__restrict__ 
             if (4 * g4 + 2 > t) d[4 * g4 + 2] = fmaf(s, v.z, d[4 * g4 + 2]);
             if (4 * g4 + 3 > t) d[4 * g4 + 3] = fmaf(s, v.w, d[4 * g4 + 3]);
         }
+    }
+    return swaps;
+}
+template <int LD>
+__device__ __forceinline__ uint32_t walk_block_thread(const float *__restrict__ tile, const float *__restrict__ alpha32,
+                                                      const float *__restrict__ b32, const float *__restrict__ r32,
+                                                      const float *__restrict__ U32, float logfac, float &bmax)
+{
+    return walk_block_thread_ld(tile, LD, alpha32, b32, r32, U32, logfac, bmax);
+}
+
+// The serial part of a 32-pair block with everything in registers: Fd[t] = F[i0 + t, i0 + lane]
+// (used for t < lane), b = b_i of this lane's pair.  No memory operation inside.
+template <typename T>
+__device__ __forceinline__ uint32_t walk_block_regs(const T (&Fd)[32], T b, T alpha, T r, T U, T logfac,
+                                                    T &bmax, int lane)
+{
+    T my_bmax = 0;
+#pragma unroll
+    for (int t = 0; t < 32; ++t) {
+        T bt = __shfl_sync(0xffffffffu, b, t);
+        T rt = __shfl_sync(0xffffffffu, r, t);
+        T carried = bmax * rt;
+        bmax = bt > carried ? bt : carried;
+        if (t == lane) my_bmax = bmax;
+    }
+    const T a = b * my_bmax * logfac;
+    uint32_t swaps = 0;
+#pragma unroll
+    for (int t = 0; t < 32; ++t) {
+        bool mine = (lane == t) && swap_decision(alpha, a, U);
+        uint32_t sw = (__ballot_sync(0xffffffffu, mine) >> t) & 1u;
+        swaps |= sw << t;
+        T f = t < lane ? Fd[t] : (T)0;
+        alpha += sw ? f : -f;
     }
     return swaps;
 }

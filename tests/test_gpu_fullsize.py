@@ -72,3 +72,23 @@ def test_status_words_after_generic_kernels():
     idx, w = elm.compress(K, V, wl.log2_nout, wl.m, precision="fp64", workspace=ws_c)
     elm.attend(Q, K, V, idx, w, precision="fp64", workspace=ws_a)
     assert elm.compress_status(ws_c, p) == 0 and elm.attend_status(ws_a, p, wl.n_out) == 0
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("min_pairs", ["32", "256"])
+def test_chain_walk_on_short_calls_matches_oracle(min_pairs):
+    """The chain walk kernel (one CTA or one cluster per call) normally takes only calls of >= 1024
+    pairs.  With the threshold lowered the small oracle-parity cases run through it, with one CTA per
+    call (calls of up to 256 pairs) and with clusters of 2 to 8 CTAs: same indices as the oracle in
+    fp64 mode, same structure / mismatch bounds in fp32 mode."""
+    import os
+    import subprocess
+    import sys
+    env = dict(os.environ, ELM_WALK_CHAIN_MIN_PAIRS=min_pairs)
+    here = os.path.dirname(os.path.abspath(__file__))
+    r = subprocess.run([sys.executable, "-m", "pytest", os.path.join(here, "test_gpu_parity.py"), "-q", "-x", "-m", "gpu",
+                        "-k", "fp64_indices_identical or fp64_edge_shapes or fp32_structure or full_pipeline_fp64 "
+                              "or fp64_full_size_heads"],
+                       env=env, capture_output=True, text=True, timeout=1500)
+    assert r.returncode == 0, r.stdout[-3000:] + r.stderr[-2000:]
+    assert " passed" in r.stdout
