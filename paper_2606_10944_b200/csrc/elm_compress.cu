@@ -307,10 +307,12 @@ __device__ __forceinline__ void load4(const double *p, double (&f)[4])
 // Calls with at least 32 pairs: one CTA per call.
 //   setup      all threads: b_i = sqrt(F[i,i]), the decay factors and the uniforms of every pair
 //              into shared memory; scores alpha = 0.
-//   warp 0     the walker: for block c it adds block c-1's contribution from a 32 x 32 tile that
-//              was copied to shared memory during the previous block and runs the 32 serial steps
-//              on the diagonal tile (c, c) without touching global memory.
-//   warp 1     copies the two tiles the walker needs for block c+1 (asynchronous copies).
+//   warp 0     the walker: the 32 serial steps of block c on a tile copied to shared memory during the
+//              previous block.  fp32: the warp-cooperative walker on rows of block c x columns of
+//              blocks c and c+1, so block c+1's scores are complete when block c ends; fp64: one
+//              vote per pair on the diagonal tile (c, c) after adding block c-1's contribution
+//              from the cross tile (c-1, c).
+//   warp 1     copies the tiles the walker needs for block c+1 (asynchronous copies).
 //   warps 2..  the updaters fold block c-1 into the scores of all columns from block c+1 on, one
 //              block behind the walker.  The rows of a block are streamed through two shared-memory
 //              panels with asynchronous copies; F does not depend on the decisions, so the first
@@ -351,8 +353,18 @@ __global__ void __launch_bounds__(576) walk_cta_kernel(const T *__restrict__ F, 
             cp_async16(dst + t * 32 + k * CH, Fg + (int64_t)(r0 + t) * P + c0 + k * CH);
         }
     };
+    // fp32: rows of a block x the columns of that block and of the next one, [32][64]
+    auto copy_tile64 = [&](T *dst, int r0) {
+        const int ncols = P - r0 < 64 ? P - r0 : 64, cpr = ncols / CH;
+        for (int q = lane; q < 32 * cpr; q += 32) {
+            const int t = q / cpr, k = q % cpr;
+            cp_async16(dst + t * 64 + k * CH, Fg + (int64_t)(r0 + t) * P + r0 + k * CH);
+        }
+    };
+    constexpr bool WARP_WALK = std::is_same<T, float>::value;
     if (warp == (nthr > 32 ? 1 : 0)) {
-        copy_tile(tiles, 0, 0);
+        if constexpr (WARP_WALK) copy_tile64(tiles, 0);
+        else copy_tile(tiles, 0, 0);
         asm volatile("cp.async.commit_group;" ::: "memory");
     }
     for (int i = threadIdx.x; i < P; i += nthr) {
@@ -386,26 +398,29 @@ __global__ void __launch_bounds__(576) walk_cta_kernel(const T *__restrict__ F, 
     __syncthreads();
 
     T bmax = 0;
+    float dn = 0.f;                                                  // fp32 walker: the next block's scores from the current block
     for (int c = 0; c < nb; ++c) {
         const int i0 = 32 * c;
         T *tdiag = tiles + (c & 1) * 2048, *tcross = tdiag + 1024;
         T *ndiag = tiles + ((c + 1) & 1) * 2048, *ncross = ndiag + 1024;
         if (warp == 0) {
-            T alpha = alpha_s[i0 + lane];
-            if (c > 0) {
-                const uint32_t pm = mask_s[c - 1];
-#pragma unroll
-                for (int t = 0; t < 32; ++t) {
-                    const T f = tcross[t * 32 + lane];
-                    alpha += ((pm >> t) & 1u) ? f : -f;
-                }
-            }
-            if constexpr (std::is_same<T, float>::value) {
-                a32_s[lane] = alpha;
-                __syncwarp();
-                if (lane == 0)
-                    mask_s[c] = walk_block_thread<32>(tdiag, a32_s, b_s + i0, r_s + i0, U_s + i0, logfac, bmax);
+            if constexpr (WARP_WALK) {
+                // the previous block folded its decisions into this block's scores as it went (dn)
+                const float a = walk_block_thresholds(b_s[i0 + lane], r_s[i0 + lane], bmax, logfac, lane);
+                const float d = walk_sign_score(alpha_s[i0 + lane] + dn, a, U_s[i0 + lane]);
+                dn = 0.f;
+                const uint32_t swaps = walk_block_warp(tiles + (c & 1) * 2048, 64, d, dn, lane);
+                if (lane == 0) mask_s[c] = swaps;
             } else {
+                T alpha = alpha_s[i0 + lane];
+                if (c > 0) {
+                    const uint32_t pm = mask_s[c - 1];
+#pragma unroll
+                    for (int t = 0; t < 32; ++t) {
+                        const T f = tcross[t * 32 + lane];
+                        alpha += ((pm >> t) & 1u) ? f : -f;
+                    }
+                }
                 T Fd[32];
 #pragma unroll
                 for (int t = 0; t < 32; ++t) Fd[t] = tdiag[t * 32 + lane];
@@ -415,8 +430,12 @@ __global__ void __launch_bounds__(576) walk_cta_kernel(const T *__restrict__ F, 
             }
         } else if (warp == 1) {
             if (c + 1 < nb) {
-                copy_tile(ndiag, i0 + 32, i0 + 32);
-                copy_tile(ncross, i0, i0 + 32);
+                if constexpr (WARP_WALK) {
+                    copy_tile64(tiles + ((c + 1) & 1) * 2048, i0 + 32);
+                } else {
+                    copy_tile(ndiag, i0 + 32, i0 + 32);
+                    copy_tile(ncross, i0, i0 + 32);
+                }
                 asm volatile("cp.async.commit_group;" ::: "memory");
                 asm volatile("cp.async.wait_group 0;" ::: "memory");
             }

@@ -48,9 +48,9 @@ constexpr int FS_LD = 68;         // row stride of the shared-memory pair Gram o
 
 // Halving walk (Algorithm A.1) of the calls that lie inside one 64-pair tile, on the tile's pair
 // Gram in shared memory: warp w walks call w of the tile (P = 16, 32 or 64 pairs per call) in blocks
-// of 32 pairs, the serial steps in one thread, the coupling between the two blocks of a 64-pair
-// call lane-parallel.  `scratch` provides 4 x 32 floats per warp (placed after the 64 x 68 floats of Fs).
-__device__ __forceinline__ void walk_in_tile(const float *Fs, float *scratch, const float *rdec, const float *unif, int p,
+// of 32 pairs with the warp-cooperative block walker; the first block of a 64-pair call folds its
+// decisions into the second block's scores as it goes.
+__device__ __forceinline__ void walk_in_tile(const float *Fs, const float *rdec, const float *unif, int p,
                                              int64_t JR, int P, int64_t Ptotal, int64_t n,
                                              const int32_t *__restrict__ cur, const WalkArgs &wk, int warp, int lane)
 {
@@ -58,37 +58,23 @@ __device__ __forceinline__ void walk_in_tile(const float *Fs, float *scratch, co
     if (warp >= calls) return;
     const int64_t J0 = JR + (int64_t)warp * P;                 // first pair of this call along the level's sequence
     if (J0 >= Ptotal) return;
-    float *a32 = scratch + warp * 128, *b32 = a32 + 32, *r32 = a32 + 64, *U32 = a32 + 96;
     const float *Fc = Fs + (warp * P) * FS_LD + warp * P;      // the call's P x P block
-    float bmax = 0.f;
-    uint32_t mask_prev = 0;
+    float bmax = 0.f, dn = 0.f;
     for (int blk = 0; blk * 32 < P; ++blk) {
         const int i = blk * 32 + lane;                         // pair within the call
         const bool live = i < P;
-        float alpha = 0.f;
-        if (blk > 0) {
-#pragma unroll
-            for (int t = 0; t < 32; ++t) {
-                const float fv = Fc[t * FS_LD + i];
-                alpha += ((mask_prev >> t) & 1u) ? fv : -fv;
-            }
-        }
         const float dgn = live ? Fc[i * FS_LD + i] : 0.f;
-        a32[lane] = alpha;
-        b32[lane] = sqrtf(dgn > 0.f ? dgn : 0.f);
-        r32[lane] = live ? rdec[warp * P + i] : 1.f;
-        U32[lane] = live ? unif[warp * P + i] : 1.f;
-        __syncwarp();
-        uint32_t swaps = 0;
-        if (lane == 0) swaps = walk_block_thread<FS_LD>(Fc + (blk * 32) * FS_LD + blk * 32, a32, b32, r32, U32, wk.logfac, bmax);
-        swaps = __shfl_sync(0xffffffffu, swaps, 0);
-        bmax = __shfl_sync(0xffffffffu, bmax, 0);
+        const float a = walk_block_thresholds(sqrtf(dgn > 0.f ? dgn : 0.f), live ? rdec[warp * P + i] : 1.f, bmax,
+                                              wk.logfac, lane);
+        // the previous block already folded its decisions into this block's scores (dn); pairs
+        // past the end of a short call come after the live ones and decide nothing
+        const float d = walk_sign_score(dn, a, live ? unif[warp * P + i] : 1.f);
+        dn = 0.f;
+        const uint32_t swaps = walk_block_warp(Fc + (blk * 32) * FS_LD + blk * 32, FS_LD, d, dn, lane);
         if (live) {
             const uint32_t sw = (swaps >> lane) & 1u;
             wk.out[(int64_t)p * wk.out_stride + J0 + i] = cur[(int64_t)p * n + 2 * (J0 + i) + sw];
         }
-        mask_prev = swaps;
-        __syncwarp();
     }
 }
 
@@ -284,7 +270,7 @@ gram_tc_kernel(const __nv_bfloat16 *__restrict__ K, const __nv_bfloat16 *__restr
         tc_fence_after();
         tmem_dealloc(tmem, TMEM_COLS);
     }
-    if (wk.fused && ok) walk_in_tile(reinterpret_cast<float *>(smem + SM::OFF_A), reinterpret_cast<float *>(smem + SM::OFF_A + 20480),
+    if (wk.fused && ok) walk_in_tile(reinterpret_cast<float *>(smem + SM::OFF_A),
                                      misc->rdec, misc->unif, p, JR, P, Ptotal, n, cur, wk, warp, lane);
 }
 

@@ -91,7 +91,7 @@ struct ChainSmem {
     size_t panels, alpha, a, U, ball, rall, xnext, mask, ctl, total;
     int NB;   // ring depth; < 3 means the call does not fit
 };
-__host__ __device__ inline ChainSmem chain_smem(int P, int C, int es)
+__host__ __device__ inline ChainSmem chain_smem(int P, int C, int es, int nb_cap)
 {
     ChainSmem s{};
     const int W = P / C;
@@ -101,7 +101,7 @@ __host__ __device__ inline ChainSmem chain_smem(int P, int C, int es)
     const size_t budget = 227 * 1024;
     int NB = budget > fixed ? (int)((budget - fixed) / panel) : 0;
     const int blocks = P / 32;
-    const int want = blocks < 3 ? 3 : (blocks < 6 ? blocks : 6);   // 4 panels ahead of the chain are enough
+    int want = blocks < 3 ? 3 : (blocks < nb_cap ? blocks : nb_cap);
     if (NB > want) NB = want;
     s.NB = NB;
     s.panels = 0;
@@ -115,92 +115,6 @@ __host__ __device__ inline ChainSmem chain_smem(int P, int C, int es)
     s.ctl = (s.mask + (size_t)(P / 32) * 4 + 15) / 16 * 16;          // progress word, then the mbarriers
     s.total = s.ctl + 16 + 8 * 8;
     return s;
-}
-
-// ---------------------------------------------------------------------------------------------
-// fp32 block walker: the serial chain itself, run redundantly by every lane so that
-// nothing is communicated inside it.  Every lane keeps broadcast copies x[0..8) of the scores of the
-// eight pairs being decided (as four packed pairs); a decision is one sign-bit operation on x[t],
-// followed by packed fused multiply-adds that fold it into the later x and into the lane's own
-// column d and (NEXT) the same column of the next block, dn.  The scores of the next eight pairs
-// are fetched from the lanes that own those columns two decisions before they are needed - hiding
-// the shuffle latency - and the two decisions taken meanwhile are folded into the copies.
-// A score of -0.0 counts as negative (the test reads the sign bit).  A single warp issues roughly
-// one instruction every third cycle on this part, so the instruction count per pair is what this
-// form keeps low.  The rows of F are fetched from shared memory three pairs ahead of their use.
-struct WalkRow {
-    float4 lo, hi, g0, g1;   // columns [t0, t0+4), [t0+4, t0+8) of the current eight, [t0+8, t0+16) of the next eight
-    float own, nxt;          // the lane's own column, and the same column of the next block
-};
-__device__ __forceinline__ void walk_row_load(const float *__restrict__ tile, const int ld, const int r, const int lane,
-                                              WalkRow &q)
-{
-    const float *row = tile + r * ld;
-    const int t0 = r & ~7, t = r & 7;
-    if (t < 3) q.lo = *reinterpret_cast<const float4 *>(row + t0);
-    if (t < 7) q.hi = *reinterpret_cast<const float4 *>(row + t0 + 4);
-    if (t0 < 24 && t >= 6) {
-        q.g0 = *reinterpret_cast<const float4 *>(row + t0 + 8);
-        q.g1 = *reinterpret_cast<const float4 *>(row + t0 + 12);
-    }
-    q.own = row[lane];
-    q.nxt = row[32 + lane];
-}
-// dn is meaningful only when the tile has 32 further columns of the same rows (otherwise the
-// loads read neighbouring shared memory and the caller ignores dn).
-__device__ __forceinline__ uint32_t walk_block_sub8(const float *__restrict__ tile, const int ld, float d, float &dn,
-                                                    const int lane)
-{
-    using sm100::fma2;
-    using sm100::pack2;
-    using sm100::unpack2;
-    uint32_t mask = 0;
-    uint64_t X[4], XN[4];
-    uint64_t DD = pack2(d, dn);
-    WalkRow q[4];
-    walk_row_load(tile, ld, 0, lane, q[0]);
-    walk_row_load(tile, ld, 1, lane, q[1]);
-    walk_row_load(tile, ld, 2, lane, q[2]);
-#pragma unroll
-    for (int j = 0; j < 4; ++j)
-        X[j] = pack2(__shfl_sync(FULL, d, 2 * j), __shfl_sync(FULL, d, 2 * j + 1));
-#pragma unroll
-    for (int r = 0; r < 32; ++r) {
-        const int t0 = r & ~7, t = r & 7;
-        const bool more = t0 < 24;
-        if (r + 3 < 32) walk_row_load(tile, ld, r + 3, lane, q[(r + 3) & 3]);
-        if (t == 6 && more) {
-            // the lanes' own scores hold every decision before pair t0 + 6
-            float dcur, dnx;
-            unpack2(DD, dcur, dnx);
-#pragma unroll
-            for (int j = 0; j < 4; ++j)
-                XN[j] = pack2(__shfl_sync(FULL, dcur, t0 + 8 + 2 * j), __shfl_sync(FULL, dcur, t0 + 9 + 2 * j));
-        }
-        const WalkRow &c = q[r & 3];
-        float xlo, xhi;
-        unpack2(X[t >> 1], xlo, xhi);
-        const uint32_t xb = __float_as_uint((t & 1) ? xhi : xlo);
-        const float s = __uint_as_float((~xb & 0x80000000u) | 0x3f800000u);   // swapped (negative) +1, kept -1
-        const uint64_t S2 = pack2(s, s);
-        mask = __funnelshift_l(xb, mask, 1);                         // decisions enter at bit 0, first one ends at bit 31
-        const uint64_t F2[4] = {pack2(c.lo.x, c.lo.y), pack2(c.lo.z, c.lo.w), pack2(c.hi.x, c.hi.y), pack2(c.hi.z, c.hi.w)};
-#pragma unroll
-        for (int v = (t + 1) >> 1; v < 4; ++v) X[v] = fma2(S2, F2[v], X[v]);
-        DD = fma2(S2, pack2(c.own, c.nxt), DD);
-        if (more && t >= 6) {
-            const uint64_t G2[4] = {pack2(c.g0.x, c.g0.y), pack2(c.g0.z, c.g0.w), pack2(c.g1.x, c.g1.y), pack2(c.g1.z, c.g1.w)};
-#pragma unroll
-            for (int j = 0; j < 4; ++j) XN[j] = fma2(S2, G2[j], XN[j]);
-        }
-        if (t == 7 && more) {
-#pragma unroll
-            for (int j = 0; j < 4; ++j) X[j] = XN[j];
-        }
-    }
-    float dcur;
-    unpack2(DD, dcur, dn);
-    return __brev(mask);
 }
 
 // sum over the 32 rows of a panel of eta_t F[t, column], eta = +1 for a swapped pair (bit set in pm):
@@ -241,13 +155,13 @@ __global__ void __launch_bounds__(96 + UPD_THREADS_MAX)
 walk_chain_kernel(const __grid_constant__ CUtensorMap mapF, const T *__restrict__ F, int64_t F_stride,
                   const T *__restrict__ rdecay,
                   const int32_t *__restrict__ cur, int32_t *__restrict__ out, int64_t out_stride,
-                  int64_t n, int P, int level, uint64_t seed, T logfac, uint32_t pbase, int *status)
+                  int64_t n, int P, int level, uint64_t seed, T logfac, uint32_t pbase, int nb_cap, int *status)
 {
     using namespace sm100;
     constexpr bool EAGER = std::is_same<T, float>::value;            // the fp32 walker also scores the next block
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const int C = (int)cluster_nctarank(), k = (int)cluster_ctarank();
-    const ChainSmem S = chain_smem(P, C, (int)sizeof(T));
+    const ChainSmem S = chain_smem(P, C, (int)sizeof(T), nb_cap);
     const int NB = S.NB;
     const int W = P / C, nbw = W / 32;
     T *panels = reinterpret_cast<T *>(smem_raw + S.panels);          // [NB][32][W]
@@ -389,7 +303,7 @@ walk_chain_kernel(const __grid_constant__ CUtensorMap mapF, const T *__restrict_
                         d = xnext_s[(lb & 1) * 32 + lane] + dn;          // warp 2 prepared all but this block's part
                     }
                     dn = 0.f;
-                    swaps = walk_block_sub8(pan + 32 * lb, W, d, dn, lane);
+                    swaps = walk_block_warp(pan + 32 * lb, W, d, dn, lane);
                 } else {
                     T alpha = alpha_s[c];
                     if (lb > 0) alpha += fold32(prev + c, W, mask_s[R - 1]);
@@ -469,7 +383,7 @@ template <typename T> bool walk_chain_covers(int P)
     if (P < 32 || P % 32 != 0) return false;
     const int C = chain_cluster_size(P);
     if (P % (32 * C) != 0 || P / C > 256) return false;               // a copy box is at most 256 elements wide
-    return chain_smem(P, C, (int)sizeof(T)).NB >= 3;
+    return chain_smem(P, C, (int)sizeof(T), 3).NB >= 3;
 }
 
 template <typename T>
@@ -478,7 +392,8 @@ int walk_chain(const T *F, int64_t F_stride, const T *rdecay, const int32_t *cur
                int *status, cudaStream_t st)
 {
     const int C = chain_cluster_size(P);
-    const ChainSmem S = chain_smem(P, C, (int)sizeof(T));
+    const int nb_cap = 6;                                            // four panels ahead of the chain are enough
+    const ChainSmem S = chain_smem(P, C, (int)sizeof(T), nb_cap);
     const int W = P / C;
     const int threads = 96 + (W > UPD_THREADS_MAX ? UPD_THREADS_MAX : W);
     CUtensorMap mapF;
@@ -509,7 +424,7 @@ int walk_chain(const T *F, int64_t F_stride, const T *rdecay, const int32_t *cur
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     ELM_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, mapF, F, F_stride, rdecay, cur, out, out_stride, n, P, level, seed, logfac,
-                                    pbase, status));
+                                    pbase, nb_cap, status));
     return ELM_OK;
 }
 
