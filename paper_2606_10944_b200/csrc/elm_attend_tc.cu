@@ -2,21 +2,28 @@
 //
 //   O[j,:] = sum_c w_c exp(<q_j,k_c>/sqrt(d)) v_c / sum_c w_c exp(<q_j,k_c>/sqrt(d))      Eq. (def:att_approx)
 //
-// One CTA owns two tiles of 128 queries of one head and streams the head's coreset in blocks of
-// 128 points.  Roles (576 threads):
-//   warps 0-7 / 8-15 softmax of query tile 0 / 1, two passes over the logits in TMEM (row maximum,
-//                    then probabilities).  A thread owns one row and half of the block's columns;
-//                    the two halves exchange row maxima through shared memory.  Probabilities go
-//                    back to TMEM as packed bf16 (over the logits); the output accumulator is
-//                    rescaled only when the maximum grew by more than 2^8.  Same warps: epilogue.
-//   warp 16          TMA producer: Q tiles once, then K / V^T blocks through a 2-stage ring
+// One persistent CTA per SM takes every gridDim.x-th pair of 128-query tiles (numbered with the head
+// slowest, so that the CTAs running at one time share one head's coreset in L2) and streams the
+// head's coreset in blocks of 128 points for each pair.  Roles (576 threads):
+//   warps 0-15       softmax: all 16 warps serve the tile whose logits are ready, tile 0 and tile 1
+//                    in turn, while the tensor pipe works on the other tile.  A thread owns one row
+//                    and a quarter of the block's columns; two passes over the logits in TMEM (row
+//                    maximum, then probabilities); the quarters exchange row maxima through shared
+//                    memory.  Probabilities go back to TMEM as packed bf16 (over the logits); the
+//                    output accumulator is rescaled only when the maximum grew by more than 2^8.
+//                    Same warps: epilogue of each pair of tiles.
+//   warp 16          TMA producer: the queries of each pair, K / V^T blocks through a 2-stage ring
+//                    that runs on across pairs
 //   warp 17          tcgen05.mma issuer: S = Q K^T (operands in shared memory), O += P V (P read
-//                    from TMEM, V^T from shared memory); owns the TMEM allocation
+//                    from TMEM, V^T from shared memory); owns the TMEM allocation.  The logits of the
+//                    next pair's first block are issued right behind the last O += P V of the
+//                    current pair, so the tensor pipe does not drain while a pair is normalised and
+//                    stored.
 // TMEM columns: [0,128) S of tile 0, [128,256) S of tile 1, [256,256+D) O of tile 0, [384,384+D) O of
-// tile 1.  The probabilities of points 0-63 / 64-127 of a block are written over the first 32
-// columns of the logits of the same points ([0,32) / [64,96) of the tile's S region), so a thread
-// only ever overwrites logits it has already read itself.  Every mbarrier wait is bounded; on expiry the CTA records a status
-// word and leaves through the common exit, which frees the TMEM it holds.
+// tile 1.  The probabilities of the points of column quarter c are written over the first 16 columns
+// of that quarter's logits, so a thread only ever overwrites logits it has already read itself.
+// Every mbarrier wait is bounded; on expiry the CTA records a status word and leaves through the
+// common exit, which frees the TMEM it holds.
 #include <cuda.h>
 #include <math.h>
 
@@ -42,12 +49,12 @@ constexpr int EMU_PAIRS = ELM_EMU_PAIRS;  // of every 16 column pairs, how many 
 using namespace sm100;
 
 struct __align__(8) Barriers {
-    uint64_t q_full;
+    uint64_t q_full, q_free;
     uint64_t k_full[STAGES], v_full[STAGES], kv_free[STAGES];
-    uint64_t s_full[2], p_ready[2], o_done[2];
+    uint64_t s_full[2], p_ready[2], o_done[2], o_free[2];
     uint32_t tmem_base;
     uint32_t abort_flag;
-    float xchg[2][2][BM];        // per tile, per column half: row maxima / denominators being exchanged
+    float xchg[2][4][BM];        // per tile, per column quarter: row maxima / denominators being exchanged
 };
 
 template <int D> struct Smem {
@@ -59,7 +66,7 @@ template <int D> struct Smem {
     static constexpr int OFF_K = OFF_Q + 2 * Q_TILE;
     static constexpr int OFF_V = OFF_K + STAGES * K_BLOCK;
     static constexpr int OFF_BAR = OFF_V + STAGES * V_BLOCK;
-    static constexpr int TOTAL = OFF_BAR + 4096 + 1024;     // barrier block + slack for 1024-byte alignment
+    static constexpr int TOTAL = OFF_BAR + 5120 + 1024;     // barrier block + slack for 1024-byte alignment
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -233,7 +240,8 @@ __global__ void __launch_bounds__(NTHREADS, 1)
 attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
                  const __grid_constant__ CUtensorMap mapV, const float *__restrict__ bias,
                  const int *__restrict__ nonuniform, __nv_bfloat16 *__restrict__ O, int q_heads,
-                 int kv_heads, int n_q, int n_core, int n_pad, float scale_log2, int *__restrict__ status)
+                 int kv_heads, int n_q, int n_core, int n_pad, float scale_log2, int tiles_x, int n_items_total,
+                 int *__restrict__ status)
 {
     using SM = Smem<D>;
     constexpr int KH = SM::KH;
@@ -242,17 +250,21 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
     Barriers *bar = reinterpret_cast<Barriers *>(smem + SM::OFF_BAR);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int bh = blockIdx.y;
-    const int b = bh / q_heads, h = bh % q_heads;
-    const int prob = b * kv_heads + (int)(((int64_t)h * kv_heads) / q_heads);
-    const int q0 = blockIdx.x * (2 * BM);
     const int nblk = n_pad / BN;
+    // Persistent CTA: work item k of this CTA is pair-of-query-tiles number blockIdx.x + k gridDim.x,
+    // numbered with the head slowest, so that at any time the CTAs share one head's coreset in L2.
+    const int n_items = (n_items_total - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+    const int total = n_items * nblk;                              // coreset blocks this CTA streams, over all items
+    auto item_bh = [&](int k) { return ((int)blockIdx.x + k * (int)gridDim.x) / tiles_x; };
+    auto item_q0 = [&](int k) { return (((int)blockIdx.x + k * (int)gridDim.x) % tiles_x) * (2 * BM); };
+    auto prob_of = [&](int bh) { return (bh / q_heads) * kv_heads + (int)(((int64_t)(bh % q_heads) * kv_heads) / q_heads); };
 
     // a CTA that gave up on a wait poisons the launch: the remaining CTAs leave at once
     if (*reinterpret_cast<volatile int *>(status) != 0) return;
 
     if (threadIdx.x == 0) {
         mbar_init(&bar->q_full, 1);
+        mbar_init(&bar->q_free, 1);
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(&bar->k_full[s], 1);
             mbar_init(&bar->v_full[s], 1);
@@ -260,8 +272,9 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
         }
         for (int t = 0; t < 2; ++t) {
             mbar_init(&bar->s_full[t], 1);
-            mbar_init(&bar->p_ready[t], 256);
+                        mbar_init(&bar->p_ready[t], 512);
             mbar_init(&bar->o_done[t], 1);
+            mbar_init(&bar->o_free[t], 16);
         }
         bar->abort_flag = 0;
         fence_barrier_init();
@@ -275,37 +288,55 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
     if (warp == TMA_WARP) {
         // ------------------------------ TMA producer ------------------------------
         if (lane == 0) {
-            mbar_expect_tx(&bar->q_full, 2 * SM::Q_TILE);
-            for (int t = 0; t < 2; ++t)
+            auto load_q = [&](int k) {
+                const int bh = item_bh(k), q0 = item_q0(k);
+                mbar_expect_tx(&bar->q_full, 2 * SM::Q_TILE);
+                for (int t = 0; t < 2; ++t)
+                    for (int kh = 0; kh < KH; ++kh)
+                        tma_load_3d(smem + SM::OFF_Q + t * SM::Q_TILE + kh * (BM * 128), &mapQ, &bar->q_full, kh * 64, q0 + t * BM, bh);
+            };
+            // Blocks are numbered G = k nblk + j along the CTA's whole stream (item k, block j).
+            auto load_k = [&](int G) {
+                const int s = G % STAGES, prob = prob_of(item_bh(G / nblk));
+                mbar_expect_tx(&bar->k_full[s], SM::K_BLOCK);
                 for (int kh = 0; kh < KH; ++kh)
-                    tma_load_3d(smem + SM::OFF_Q + t * SM::Q_TILE + kh * (BM * 128), &mapQ, &bar->q_full, kh * 64, q0 + t * BM, bh);
+                    tma_load_3d(smem + SM::OFF_K + s * SM::K_BLOCK + kh * (BN * 128), &mapK, &bar->k_full[s], kh * 64, (G % nblk) * BN, prob);
+            };
+            auto load_v = [&](int G) {
+                const int s = G % STAGES, prob = prob_of(item_bh(G / nblk));
+                mbar_expect_tx(&bar->v_full[s], SM::V_BLOCK);
+                for (int hh = 0; hh < 2; ++hh)
+                    tma_load_3d(smem + SM::OFF_V + s * SM::V_BLOCK + hh * (D * 128), &mapV, &bar->v_full[s], (G % nblk) * BN + hh * 64, 0, prob);
+            };
+            bool ok = true;
+            // The queries of item k may replace those of item k - 1 once every S = Q K^T of item k - 1
+            // has been computed (q_free); they are fetched right after the keys of the item's first block.
+            int next_q = 1, k_loaded = -1;
+            auto feed_q = [&]() {
+                while (ok && next_q < n_items && next_q * nblk <= k_loaded) {
+                    ok = mbar_wait(&bar->q_free, (uint32_t)(next_q - 1) & 1u);
+                    if (ok) load_q(next_q);
+                    ++next_q;
+                }
+            };
+            load_q(0);
             // The issuer commits "event" i to kv_free[i % 2] after the prologue (i = 0: S = Q K^T of block
             // 0 issued) and after iteration i - 1 (O += P V of block i - 1 and S = Q K^T of block i issued).
             // Once event i is complete, K's stage i % 2 (block i) and V's stage (i + 1) % 2 (block i - 1)
             // have been read, so K(i + 2) and V(i + 1) may overwrite them.
-            bool ok = true;
-            auto load_k = [&](int j) {
-                const int s = j % STAGES;
-                mbar_expect_tx(&bar->k_full[s], SM::K_BLOCK);
-                for (int kh = 0; kh < KH; ++kh)
-                    tma_load_3d(smem + SM::OFF_K + s * SM::K_BLOCK + kh * (BN * 128), &mapK, &bar->k_full[s], kh * 64, j * BN, prob);
-            };
-            auto load_v = [&](int j) {
-                const int s = j % STAGES;
-                mbar_expect_tx(&bar->v_full[s], SM::V_BLOCK);
-                for (int hh = 0; hh < 2; ++hh)
-                    tma_load_3d(smem + SM::OFF_V + s * SM::V_BLOCK + hh * (D * 128), &mapV, &bar->v_full[s], j * BN + hh * 64, 0, prob);
-            };
-            for (int j = 0; j < STAGES && j < nblk; ++j) { load_k(j); load_v(j); }
-            for (int i = 0; i + 2 < nblk && ok; ++i) {
+            for (int G = 0; G < STAGES && G < total; ++G) { load_k(G); load_v(G); k_loaded = G; }
+            feed_q();
+            for (int i = 0; i + 2 < total && ok; ++i) {
                 ok = mbar_wait(&bar->kv_free[i % STAGES], (uint32_t)(i / STAGES) & 1u);
                 if (!ok) break;
                 load_k(i + 2);
+                k_loaded = i + 2;
                 if (i >= 1) load_v(i + 1);
+                feed_q();
             }
-            // the last V block: freed by event nblk - 1
-            if (ok && nblk > STAGES) {
-                const int i = nblk - 2;
+            // the last V block: freed by event total - 1
+            if (ok && total > STAGES) {
+                const int i = total - 2;
                 ok = mbar_wait(&bar->kv_free[i % STAGES], (uint32_t)(i / STAGES) & 1u);
                 if (ok) load_v(i + 1);
             }
@@ -336,120 +367,150 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                 for (int hh = 0; hh < 2; ++hh)
 #pragma unroll
                     for (int ks = 0; ks < 4; ++ks)
-                        mma_ts(tmem + 256 + t * 128, tmem + t * 128 + hh * 64 + ks * 8,
+                        mma_ts(tmem + 256 + t * 128, tmem + t * 128 + (hh * 2 + (ks >> 1)) * 32 + (ks & 1) * 8,
                                b0 + (uint64_t)(hh * (D * 128 >> 4) + ks * 2), IDESC_PV, (acc || (hh | ks) != 0) ? 1u : 0u);
             };
             bool ok = mbar_wait(&bar->q_full, 0) && mbar_wait(&bar->k_full[0], 0);
             if (ok) {
                 tc_fence_after();
                 for (int t = 0; t < 2; ++t) { issue_qk(t, 0); tc_commit(&bar->s_full[t]); }
+                if (nblk == 1) tc_commit(&bar->q_free);                        // item 0 needs its queries no more
                 tc_commit(&bar->kv_free[0]);                                   // event 0
             }
-            for (int j = 0; j < nblk && ok; ++j) {
-                const int s = j % STAGES;
-                const bool more = j + 1 < nblk;
-                const int sn = (j + 1) % STAGES;
-                if (more) ok = mbar_wait(&bar->k_full[sn], (uint32_t)((j + 1) / STAGES) & 1u);
-                ok = ok && mbar_wait(&bar->v_full[s], (uint32_t)(j / STAGES) & 1u);
+            // Iteration G: O += P V of block G, then S = Q K^T of block G + 1 - which may be the first
+            // block of the next item: the tensor pipe runs on while the softmax warps finish an item.
+            int j = 0, k = 0;                                                  // block G = item k, block j
+            for (int G = 0; G < total && ok; ++G) {
+                const int s = G % STAGES;
+                const bool more = G + 1 < total;
+                const int sn = (G + 1) % STAGES;
+                const bool last = j == nblk - 1;                               // last block of item k
+                if (more) ok = mbar_wait(&bar->k_full[sn], (uint32_t)((G + 1) / STAGES) & 1u);
+                ok = ok && mbar_wait(&bar->v_full[s], (uint32_t)(G / STAGES) & 1u);
                 for (int t = 0; t < 2 && ok; ++t) {
-                    ok = mbar_wait(&bar->p_ready[t], (uint32_t)j & 1u);
+                    ok = mbar_wait(&bar->p_ready[t], (uint32_t)G & 1u);
+                    // a new item overwrites the accumulator: the epilogue of the previous one must have read it
+                    if (ok && j == 0 && k > 0) ok = mbar_wait(&bar->o_free[t], (uint32_t)(k - 1) & 1u);
                     if (!ok) break;
                     tc_fence_after();
                     issue_pv(t, s, j > 0);
                     // s_full also tells the softmax warps that O += P V of block j is complete (a commit
-                    // covers every earlier MMA); only the last block needs o_done for the epilogue
-                    if (more) { issue_qk(t, sn); tc_commit(&bar->s_full[t]); }
-                    else tc_commit(&bar->o_done[t]);
+                    // covers every earlier MMA); the last block of an item signals the epilogue
+                    if (last) tc_commit(&bar->o_done[t]);
+                    if (more) {
+                        // the next item's queries are needed only now, after this item's last O += P V went out
+                        if (last && t == 0) ok = mbar_wait(&bar->q_full, (uint32_t)(k + 1) & 1u);
+                        if (!ok) break;
+                        issue_qk(t, sn);
+                        tc_commit(&bar->s_full[t]);
+                    }
                 }
                 if (!ok) break;
-                tc_commit(&bar->kv_free[(j + 1) % STAGES]);                    // event j + 1
+                // the logits just issued belong to block j + 1 of item k, or to block 0 of item k + 1
+                const int jn = last ? 0 : j + 1;
+                if (more && jn == nblk - 1) tc_commit(&bar->q_free);
+                tc_commit(&bar->kv_free[(G + 1) % STAGES]);                    // event G + 1
+                j = jn;
+                if (last) ++k;
             }
             if (!ok) { atomicExch(status, 2); bar->abort_flag = 1; }
         }
     } else {
         // ------------------------------ softmax + epilogue ------------------------------
-        // 8 warps per query tile: warps with the same (warp % 4) share 32 rows (TMEM lanes) and split
-        // the block's 128 columns in two halves; the halves exchange their row maxima (and, at the
-        // end, their denominators) through shared memory.
-        const int t = warp >> 3;                                   // query tile
-        const int hh = (warp >> 2) & 1;                            // column half
+        // All 16 warps serve the query tile whose logits are ready, tile 0 and tile 1 in turn: while
+        // they work on one tile the tensor pipe works on the other.  Warps with the same (warp % 4)
+        // share 32 rows (TMEM lanes) and split the block's 128 columns in four quarters; the
+        // quarters exchange their row maxima (and, at the end, their denominators) through shared
+        // memory, in a buffer per tile so that a value is overwritten only two barriers later.
+        const int cq = warp >> 2;                                  // column quarter
         const int row = (warp & 3) * 32 + lane;                    // row in the tile = TMEM lane
         const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
-        const uint32_t tS = tmem + lane_addr + t * 128 + hh * 64;  // this thread's 64 logit columns
-        const uint32_t tP = tS;                                    // their bf16 probabilities overwrite the first 32 of them
-        const uint32_t tO = tmem + lane_addr + 256 + t * 128 + hh * (D / 2);   // its half of the accumulator
-        float *xmine = bar->xchg[t][hh], *xother = bar->xchg[t][hh ^ 1];
-        const bool use_bias = nonuniform[prob] != 0;
-        const float *bp = bias + (int64_t)prob * n_pad + hh * 64;
-        float m_ref = -INFINITY, l = 0.f;
         bool ok = true;
-        for (int j = 0; j < nblk; ++j) {
-            ok = mbar_wait(&bar->s_full[t], (uint32_t)j & 1u);
-            if (!ok) break;
-            tc_fence_after();
-            const int valid = n_core - j * BN - hh * 64;           // of this thread's 64 columns, how many exist
-            const bool special = use_bias || valid < 64;           // per-column bias and/or a ragged tail
-            const float *bcols = use_bias ? bp + j * BN : nullptr;
-            // ---- pass 1: row maximum over both halves ----
-            const float mh = special ? row_max<true, 2>(tS, scale_log2, bcols, valid)
-                                     : row_max<false, 2>(tS, scale_log2, bcols, valid);
-            xmine[row] = mh;
-            asm volatile("bar.sync %0, 256;" ::"r"(1 + t) : "memory");
-            const float mx = fmaxf(mh, xother[row]);
-            // lazy rescale: keep the old reference unless the maximum grew by more than 2^TAU
-            const bool grow = mx > m_ref + RESCALE_TAU;
-            if (__any_sync(0xffffffffu, grow)) {
-                if (j > 0) {
-                    // O += P V of block j-1 is complete: s_full of block j was committed after it
-                    const float alpha = grow ? fast_exp2(m_ref - mx) : 1.f;
+        int G = 0;
+        for (int k = 0; k < n_items && ok; ++k) {
+            const int bh = item_bh(k), q0 = item_q0(k), prob = prob_of(bh);
+            const bool use_bias = nonuniform[prob] != 0;
+            const float *bp = bias + (int64_t)prob * n_pad + cq * 32;
+            float m_ref[2] = {-INFINITY, -INFINITY}, l[2] = {0.f, 0.f};
+            for (int j = 0; j < nblk && ok; ++j, ++G) {
+                const int valid = n_core - j * BN - cq * 32;           // of this thread's 32 columns, how many exist
+                const bool special = use_bias || valid < 32;           // per-column bias and/or a ragged tail
+                const float *bcols = use_bias ? bp + j * BN : nullptr;
 #pragma unroll
-                    for (int q = 0; q < D / 64; ++q) {
-                        uint32_t o[32];
-                        tmem_ld32(tO + q * 32, o);
-                        tmem_wait_ld();
+                for (int t = 0; t < 2; ++t) {
+                    const uint32_t tS = tmem + lane_addr + t * 128 + cq * 32;   // this thread's 32 logit columns
+                    const uint32_t tP = tS;                 // their bf16 probabilities overwrite the first 16 of them
+                    const uint32_t tO = tmem + lane_addr + 256 + t * 128 + cq * (D / 4);   // its quarter of the accumulator
+                    ok = mbar_wait(&bar->s_full[t], (uint32_t)G & 1u);
+                    if (!ok) break;
+                    tc_fence_after();
+                    // ---- pass 1: row maximum over the four quarters ----
+                    const float mh = special ? row_max<true, 1>(tS, scale_log2, bcols, valid)
+                                             : row_max<false, 1>(tS, scale_log2, bcols, valid);
+                    bar->xchg[t][cq][row] = mh;
+                    asm volatile("bar.sync 1, 512;" ::: "memory");
+                    const float mx = fmaxf(fmaxf(bar->xchg[t][0][row], bar->xchg[t][1][row]),
+                                           fmaxf(bar->xchg[t][2][row], bar->xchg[t][3][row]));
+                    // lazy rescale: keep the old reference unless the maximum grew by more than 2^TAU
+                    const bool grow = mx > m_ref[t] + RESCALE_TAU;
+                    if (__any_sync(0xffffffffu, grow)) {
+                        if (j > 0) {
+                            // O += P V of block j-1 is complete: s_full of block j was committed after it
+                            const float alpha = grow ? fast_exp2(m_ref[t] - mx) : 1.f;
+                            uint32_t o[32];
+                            if (D == 128) tmem_ld32(tO, o);
+                            else tmem_ld16(tO, o);
+                            tmem_wait_ld();
 #pragma unroll
-                        for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
-                        tmem_st32(tO + q * 32, o);
+                            for (int c = 0; c < D / 4; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
+                            if (D == 128) tmem_st32(tO, o);
+                            else tmem_st16(tO, o);
+                            l[t] *= alpha;
+                        }
+                        if (grow) m_ref[t] = mx;
                     }
-                    l *= alpha;
+                    // ---- pass 2: probabilities and running denominator ----
+                    l[t] += special ? exp_pass<true, 1>(tS, tP, scale_log2, -m_ref[t], bcols, valid)
+                                    : exp_pass<false, 1>(tS, tP, scale_log2, -m_ref[t], bcols, valid);
+                    tmem_wait_st();
+                    tc_fence_before();
+                    mbar_arrive(&bar->p_ready[t]);
                 }
-                if (grow) m_ref = mx;
             }
-            // ---- pass 2: probabilities and running denominator ----
-            l += special ? exp_pass<true, 2>(tS, tP, scale_log2, -m_ref, bcols, valid)
-                         : exp_pass<false, 2>(tS, tP, scale_log2, -m_ref, bcols, valid);
-            tmem_wait_st();
-            tc_fence_before();
-            mbar_arrive(&bar->p_ready[t]);
-        }
-        if (ok) ok = mbar_wait(&bar->o_done[t], 0);
-        if (ok) {
-            tc_fence_after();
-            xmine[row] = l;
-            asm volatile("bar.sync %0, 256;" ::"r"(1 + t) : "memory");
-            const float inv = 1.f / (l + xother[row]);
-            const int64_t qrow = (int64_t)q0 + t * BM + row;
-            __nv_bfloat16 *dst = O + ((int64_t)bh * n_q + qrow) * D + hh * (D / 2);
+            if (!ok) break;
 #pragma unroll
-            for (int q = 0; q < D / 64; ++q) {
+            for (int t = 0; t < 2; ++t) {
+                const uint32_t tO = tmem + lane_addr + 256 + t * 128 + cq * (D / 4);
+                ok = mbar_wait(&bar->o_done[t], (uint32_t)k & 1u);
+                if (!ok) break;
+                tc_fence_after();
+                bar->xchg[t][cq][row] = l[t];
+                asm volatile("bar.sync 1, 512;" ::: "memory");
+                const float inv = 1.f / ((bar->xchg[t][0][row] + bar->xchg[t][1][row]) + (bar->xchg[t][2][row] + bar->xchg[t][3][row]));
+                const int64_t qrow = (int64_t)q0 + t * BM + row;
+                __nv_bfloat16 *dst = O + ((int64_t)bh * n_q + qrow) * D + cq * (D / 4);
                 uint32_t o[32];
-                tmem_ld32(tO + q * 32, o);
+                if (D == 128) tmem_ld32(tO, o);
+                else tmem_ld16(tO, o);
                 tmem_wait_ld();
+                // the accumulator is in registers: the next item may overwrite it
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&bar->o_free[t]);
                 if (qrow < n_q) {
 #pragma unroll
-                    for (int c = 0; c < 32; c += 8) {
+                    for (int c = 0; c < D / 4; c += 8) {
                         uint4 v;
                         v.x = pack_bf16x2(__uint_as_float(o[c]) * inv, __uint_as_float(o[c + 1]) * inv);
                         v.y = pack_bf16x2(__uint_as_float(o[c + 2]) * inv, __uint_as_float(o[c + 3]) * inv);
                         v.z = pack_bf16x2(__uint_as_float(o[c + 4]) * inv, __uint_as_float(o[c + 5]) * inv);
                         v.w = pack_bf16x2(__uint_as_float(o[c + 6]) * inv, __uint_as_float(o[c + 7]) * inv);
-                        *reinterpret_cast<uint4 *>(dst + q * 32 + c) = v;
+                        *reinterpret_cast<uint4 *>(dst + c) = v;
                     }
                 }
             }
-        } else if (lane == 0) {
-            atomicExch(status, 3);
         }
+        if (!ok && lane == 0) atomicExch(status, 3);
     }
     tc_fence_before();
     __syncthreads();
@@ -474,6 +535,17 @@ static bool make_map(CUtensorMap *map, const void *base, uint64_t d0, uint64_t d
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+static int sm_count()
+{
+    static int n = 0;
+    if (n == 0) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+            n = 148;
+    }
+    return n;
 }
 
 template <int D>
@@ -505,16 +577,19 @@ static int launch(const __nv_bfloat16 *Q, const __nv_bfloat16 *K, const __nv_bfl
     StageTimer t(timed ? ELM_STAGE_ATTEND : -1, st, 1);
     auto kern = attend_tc_kernel<D>;
     ELM_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<D>::TOTAL));
-    dim3 grid((unsigned)((p->n_q + 2 * BM - 1) / (2 * BM)), (unsigned)(p->batch * p->q_heads));
+    // one persistent CTA per SM, each taking every gridDim.x-th pair of query tiles
+    const int tiles_x = (p->n_q + 2 * BM - 1) / (2 * BM);
+    const int64_t items = (int64_t)tiles_x * p->batch * p->q_heads;
+    if (items > 0x7fffffff / 64) return ELM_ERR_SHAPE;
+    const int ctas = (int)(items < sm_count() ? items : sm_count());
     const float scale_log2 = (float)(1.4426950408889634 / sqrt((double)D));
-    kern<<<grid, NTHREADS, Smem<D>::TOTAL, st>>>(mQ, mK, mV, bias, flags, O, p->q_heads, p->kv_heads, p->n_q,
-                                                 n_core, n_pad, scale_log2, status);
+    kern<<<ctas, NTHREADS, Smem<D>::TOTAL, st>>>(mQ, mK, mV, bias, flags, O, p->q_heads, p->kv_heads, p->n_q,
+                                                 n_core, n_pad, scale_log2, tiles_x, (int)items, status);
     count_launches(1);
     return cuda_status(cudaGetLastError());
 }
 
 }  // namespace tc
-
 int attend_tc(const __nv_bfloat16 *Q, const __nv_bfloat16 *K, const __nv_bfloat16 *V, const int32_t *idx,
               const float *w, int n_core, const elm_params *p, __nv_bfloat16 *O, unsigned char *ws,
               cudaStream_t st, bool timed)
