@@ -149,8 +149,13 @@ int elm_attend_static(const void *Q, const void *K, const void *V, const int32_t
 
 /*
  * End-to-end convenience call on HOST buffers: copies Q, K, V to the device, runs elm_compress and
- * elm_attend, copies O (and, when non-NULL, idx and w) back, and synchronises `stream` before it
- * returns.  Host buffers may be pageable or pinned.  `device_scratch` is a DEVICE buffer of at
+ * elm_attend, copies O (and, when non-NULL, idx and w) back, and returns when everything has
+ * arrived.  The host link bounds this call, so uploads, kernels and downloads overlap: K and V go
+ * first on `stream` with the compression behind them; Q follows on a second, internal stream in
+ * chunks of one attention problem's query heads; each chunk is attended on `stream` as soon as it
+ * has landed and its part of O leaves on a third stream.  The internal streams and events are
+ * created and destroyed inside the call (no device memory is allocated).  Host buffers may be
+ * pageable or pinned; only pinned buffers overlap.  `device_scratch` is a DEVICE buffer of at
  * least elm_host_call_scratch_bytes(params) bytes, 256-byte aligned, owned by the caller.
  */
 int elm_host_call_scratch_bytes(const elm_params *params, size_t *bytes);

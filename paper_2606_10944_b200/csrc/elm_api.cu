@@ -5,6 +5,8 @@
 
 #include <atomic>
 
+#include <vector>
+
 #include "elm_attend.cuh"
 #include "elm_common.cuh"
 #include "elm_compress.cuh"
@@ -138,27 +140,88 @@ extern "C" int elm_compress_attend_host(const void *Q_host, const void *K_host, 
     cudaStream_t st = (cudaStream_t)stream;
     unsigned char *base = (unsigned char *)device_scratch;
     const size_t es = elt_bytes(params->dtype);
-    const size_t qo = (size_t)params->batch * params->q_heads * params->n_q * params->d * es;
     const size_t kv = (size_t)params->batch * params->kv_heads * params->n_kv * params->d * es;
     const size_t core = (size_t)params->batch * params->kv_heads * ((size_t)1 << params->log2_nout);
-    // K and V first: compression can start while Q is still in flight on a copy engine only if the
-    // caller splits streams; on one stream the order is simply K, V, Q.
-    ELM_CUDA_TRY(cudaMemcpyAsync(base + L.K, K_host, kv, cudaMemcpyHostToDevice, st));
-    ELM_CUDA_TRY(cudaMemcpyAsync(base + L.V, V_host, kv, cudaMemcpyHostToDevice, st));
-    ELM_CUDA_TRY(cudaMemcpyAsync(base + L.Q, Q_host, qo, cudaMemcpyHostToDevice, st));
-    rc = elm_compress(base + L.K, base + L.V, params, seed, (int32_t *)(base + L.idx), (float *)(base + L.w),
-                      base + L.ws_compress, compress_layout(params).total, stream);
-    if (rc != ELM_OK) return rc;
     const int32_t n_core = 1 << params->log2_nout;
-    rc = elm_attend(base + L.Q, base + L.K, base + L.V, (const int32_t *)(base + L.idx),
-                    (const float *)(base + L.w), n_core, params, base + L.O, base + L.ws_attend,
-                    attend_layout(params, n_core).total, stream);
+    // The link is the bottleneck of this call, so it is kept busy in both directions: K and V go
+    // first and the compression runs behind them; the queries follow on a second stream in chunks
+    // of one (batch entry, KV head) - the query heads that share a coreset are contiguous in Q - and
+    // each chunk is attended as soon as it has landed, while its output leaves on a third stream
+    // under the next chunk's upload.
+    const int chunks = params->batch * params->kv_heads;
+    const int rep = params->q_heads / params->kv_heads;
+    const size_t q_chunk = (size_t)rep * params->n_q * params->d * es;       // bytes of Q (and of O) per chunk
+    const size_t kv_chunk = (size_t)params->n_kv * params->d * es;
+    cudaStream_t cin = nullptr, cout = nullptr;
+    cudaEvent_t ev_kv = nullptr, ev_core = nullptr;
+    std::vector<cudaEvent_t> ev_q(chunks, nullptr), ev_o(chunks, nullptr);
+    auto cleanup = [&]() {
+        if (cin) cudaStreamDestroy(cin);
+        if (cout) cudaStreamDestroy(cout);
+        if (ev_kv) cudaEventDestroy(ev_kv);
+        if (ev_core) cudaEventDestroy(ev_core);
+        for (int c = 0; c < chunks; ++c) {
+            if (ev_q[c]) cudaEventDestroy(ev_q[c]);
+            if (ev_o[c]) cudaEventDestroy(ev_o[c]);
+        }
+    };
+#define ELM_HOST_TRY(expr)                                   \
+    do {                                                     \
+        if ((expr) != cudaSuccess) {                         \
+            cudaStreamSynchronize(st);                       \
+            if (cin) cudaStreamSynchronize(cin);             \
+            if (cout) cudaStreamSynchronize(cout);           \
+            cleanup();                                       \
+            return ELM_ERR_CUDA;                             \
+        }                                                    \
+    } while (0)
+    ELM_HOST_TRY(cudaStreamCreateWithFlags(&cin, cudaStreamNonBlocking));
+    ELM_HOST_TRY(cudaStreamCreateWithFlags(&cout, cudaStreamNonBlocking));
+    ELM_HOST_TRY(cudaEventCreateWithFlags(&ev_kv, cudaEventDisableTiming));
+    ELM_HOST_TRY(cudaEventCreateWithFlags(&ev_core, cudaEventDisableTiming));
+    for (int c = 0; c < chunks; ++c) {
+        ELM_HOST_TRY(cudaEventCreateWithFlags(&ev_q[c], cudaEventDisableTiming));
+        ELM_HOST_TRY(cudaEventCreateWithFlags(&ev_o[c], cudaEventDisableTiming));
+    }
+    ELM_HOST_TRY(cudaMemcpyAsync(base + L.K, K_host, kv, cudaMemcpyHostToDevice, st));
+    ELM_HOST_TRY(cudaMemcpyAsync(base + L.V, V_host, kv, cudaMemcpyHostToDevice, st));
+    ELM_HOST_TRY(cudaEventRecord(ev_kv, st));
+    ELM_HOST_TRY(cudaStreamWaitEvent(cin, ev_kv, 0));                        // K and V have the link first
+    for (int c = 0; c < chunks; ++c) {
+        ELM_HOST_TRY(cudaMemcpyAsync(base + L.Q + (size_t)c * q_chunk, (const unsigned char *)Q_host + (size_t)c * q_chunk,
+                                     q_chunk, cudaMemcpyHostToDevice, cin));
+        ELM_HOST_TRY(cudaEventRecord(ev_q[c], cin));
+    }
+    rc = compress_enqueue(base + L.K, base + L.V, params, seed, (int32_t *)(base + L.idx), (float *)(base + L.w),
+                          base + L.ws_compress, st, 0u);
+    if (rc == ELM_OK) {
+        ELM_HOST_TRY(cudaEventRecord(ev_core, st));
+        ELM_HOST_TRY(cudaStreamWaitEvent(cout, ev_core, 0));
+        if (idx_host) ELM_HOST_TRY(cudaMemcpyAsync(idx_host, base + L.idx, core * 4, cudaMemcpyDeviceToHost, cout));
+        if (w_host) ELM_HOST_TRY(cudaMemcpyAsync(w_host, base + L.w, core * 4, cudaMemcpyDeviceToHost, cout));
+    }
+    elm_params one = *params;                                                // one attention problem per chunk
+    one.batch = 1;
+    one.kv_heads = 1;
+    one.q_heads = rep;
+    for (int c = 0; c < chunks && rc == ELM_OK; ++c) {
+        ELM_HOST_TRY(cudaStreamWaitEvent(st, ev_q[c], 0));
+        rc = attend_enqueue(base + L.Q + (size_t)c * q_chunk, base + L.K + (size_t)c * kv_chunk,
+                            base + L.V + (size_t)c * kv_chunk, (const int32_t *)(base + L.idx) + (size_t)c * n_core,
+                            (const float *)(base + L.w) + (size_t)c * n_core, n_core, &one,
+                            base + L.O + (size_t)c * q_chunk, base + L.ws_attend, st);
+        if (rc != ELM_OK) break;
+        ELM_HOST_TRY(cudaEventRecord(ev_o[c], st));
+        ELM_HOST_TRY(cudaStreamWaitEvent(cout, ev_o[c], 0));
+        ELM_HOST_TRY(cudaMemcpyAsync((unsigned char *)O_host + (size_t)c * q_chunk, base + L.O + (size_t)c * q_chunk, q_chunk,
+                                     cudaMemcpyDeviceToHost, cout));
+    }
+    const bool sync_ok = cudaStreamSynchronize(st) == cudaSuccess && cudaStreamSynchronize(cin) == cudaSuccess &&
+                         cudaStreamSynchronize(cout) == cudaSuccess;
+    cleanup();
+#undef ELM_HOST_TRY
     if (rc != ELM_OK) return rc;
-    ELM_CUDA_TRY(cudaMemcpyAsync(O_host, base + L.O, qo, cudaMemcpyDeviceToHost, st));
-    if (idx_host) ELM_CUDA_TRY(cudaMemcpyAsync(idx_host, base + L.idx, core * 4, cudaMemcpyDeviceToHost, st));
-    if (w_host) ELM_CUDA_TRY(cudaMemcpyAsync(w_host, base + L.w, core * 4, cudaMemcpyDeviceToHost, st));
-    ELM_CUDA_TRY(cudaStreamSynchronize(st));
-    return ELM_OK;
+    return sync_ok ? ELM_OK : ELM_ERR_CUDA;
 }
 
 extern "C" int elm_compress_status(const void *workspace, const elm_params *params, int32_t *status_host, void *stream)
