@@ -148,6 +148,36 @@ int elm_attend_static(const void *Q, const void *K, const void *V, const int32_t
                       int32_t n_core, const elm_params *params, void *O, void *stream);
 
 /*
+ * Offline-Express (the recursive form of Algorithm 1, "Express", with Subsample - Algorithm 3 - and
+ * Compress2 - Algorithm 2 - inside and Halve = KH(delta) with the failure parameters of Corollary 2,
+ * i.e. KH-Express): the n_out points a streaming Express cache holds after n_kv = n_out 4^R key-value
+ * pairs, R >= 0, for every attention problem.  E starts as the first n_out points; round r = 0 .. R-1
+ * (thinning factor m = 2r) thins the next three segments of n_out 2^m points each - one stratified
+ * uniform draw per 2^(m - mbar) points when m > mbar, then Compress2 of depth min(m, mbar) - appends
+ * the three results to E and halves the 4 n_out points of E twice with KH(delta_m / 2), where
+ * delta_m = (delta/2)(1/log2(m/2 + 2) - 1/log2(m/2 + 3)); level i of a depth-q Compress2 uses
+ * KH(4^(i+1-q) delta_m / (3q)).
+ *   params     batch, kv_heads, n_kv, d, log2_nout (>= 1), dtype, precision and delta are used;
+ *              n_kv must equal 2^log2_nout * 4^R.  q_heads, n_q, m and delta_level are ignored.
+ *   mbar       inflation factor of Algorithm 1 (0 .. 30); the paper's experiments use log2_nout - 2
+ *              for prefill.
+ *   seed       uniforms as in elm_compress, with the counter's third word numbering the call's place
+ *              in the recursion: i + 64 (4r + j) for Halve_i of segment j in {1,2,3} of round r,
+ *              62 / 63 + 64 (4r) for the two halvings of E, 61 + 64 (4r + j) for the draws of
+ *              segment j (first word = stratum number, point = stratum start + floor(U 2^(m-mbar))).
+ *   idx_out    [batch][kv_heads][n_out] row numbers in [0, n_kv) in the order the last halving
+ *              appends them; w_out the same shape, every entry 1/n_out.
+ *   workspace  at least elm_express_workspace_bytes(params, mbar) bytes, 256-byte aligned.
+ * v_max of Eq. (katt) is taken over the whole sequence of the problem.  In fp64 mode a call of more
+ * than 2048 pairs (n_out > 1024 here) is not supported and returns ELM_ERR_SHAPE.
+ * This is the compression half of causal prefill with Thinformer Express (Algorithm 5); attention
+ * of every query over the cache as of its own position is not part of this library yet.
+ */
+int elm_express_workspace_bytes(const elm_params *params, int32_t mbar, size_t *bytes);
+int elm_express_compress(const void *K, const void *V, const elm_params *params, int32_t mbar, uint64_t seed,
+                         int32_t *idx_out, float *w_out, void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * End-to-end convenience call on HOST buffers: copies Q, K, V to the device, runs elm_compress and
  * elm_attend, copies O (and, when non-NULL, idx and w) back, and returns when everything has
  * arrived.  The host link bounds this call, so uploads, kernels and downloads overlap: K and V go

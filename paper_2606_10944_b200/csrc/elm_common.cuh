@@ -85,6 +85,21 @@ __device__ __forceinline__ uint32_t philox4x32_10_word0(uint32_t c0, uint32_t c1
 
 // The uniform of pair `pair` of Halve call `group` at `level` of attention problem `problem`:
 // top 24 bits of the first Philox word, so the value is exact in fp32 and fp64 alike.
+// Second and third counter words of Halve call g of a level.  `lvl` carries the level's third word in
+// its low half; a non-zero high half says that the level batches sibling segments of an Express round
+// with that many calls each: call g is then call g % calls of sibling g / calls, whose third word is
+// 64 further on per sibling.
+__device__ __forceinline__ void call_counter(int g, int64_t lvl, uint32_t &group, uint32_t &code)
+{
+    const uint32_t per = (uint32_t)(lvl >> 32);
+    code = (uint32_t)lvl;
+    group = (uint32_t)g;
+    if (per) {
+        group = (uint32_t)g % per;
+        code += 64u * ((uint32_t)g / per);
+    }
+}
+
 template <typename T>
 __device__ __forceinline__ T halving_uniform(uint64_t seed, uint32_t pair, uint32_t group,
                                              uint32_t level, uint32_t problem)

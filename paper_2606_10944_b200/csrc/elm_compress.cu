@@ -323,7 +323,7 @@ __global__ void __launch_bounds__(576) walk_cta_kernel(const T *__restrict__ F, 
                                                        const T *__restrict__ rdecay,
                                                        const int32_t *__restrict__ cur,
                                                        int32_t *__restrict__ out, int64_t out_stride,
-                                                       int64_t n, int P, int level, uint64_t seed,
+                                                       int64_t n, int P, int64_t lvl, uint64_t seed,
                                                        T logfac, uint32_t pbase)
 {
     constexpr int PW = 2048 / sizeof(T);                             // panel width in columns (64 KB / 2 buffers... per 32 rows)
@@ -367,12 +367,14 @@ __global__ void __launch_bounds__(576) walk_cta_kernel(const T *__restrict__ F, 
         else copy_tile(tiles, 0, 0);
         asm volatile("cp.async.commit_group;" ::: "memory");
     }
+    uint32_t cgroup, ccode;
+    call_counter(g, lvl, cgroup, ccode);
     for (int i = threadIdx.x; i < P; i += nthr) {
         alpha_s[i] = 0;
         const T d = Fg[(int64_t)i * P + i];
         b_s[i] = sqrt(d > 0 ? d : (T)0);
         r_s[i] = rdecay[(int64_t)p * (n / 2) + base + i];
-        U_s[i] = halving_uniform<T>(seed, (uint32_t)i, (uint32_t)g, (uint32_t)level, (uint32_t)p + pbase);
+        U_s[i] = halving_uniform<T>(seed, (uint32_t)i, cgroup, ccode, (uint32_t)p + pbase);
     }
     if (warp <= 1) asm volatile("cp.async.wait_group 0;" ::: "memory");
 
@@ -499,7 +501,7 @@ __global__ void __launch_bounds__(256) walk_warp_kernel(const T *__restrict__ F,
                                                         const T *__restrict__ rdecay,
                                                         const int32_t *__restrict__ cur,
                                                         int32_t *__restrict__ out, int64_t out_stride,
-                                                        int64_t n, int P, int groups, int level,
+                                                        int64_t n, int P, int groups, int64_t lvl,
                                                         uint64_t seed, T logfac, uint32_t pbase)
 {
     const int p = blockIdx.y;
@@ -511,7 +513,9 @@ __global__ void __launch_bounds__(256) walk_warp_kernel(const T *__restrict__ F,
     T bmax = 0;
     const bool live = lane < P;
     const T r = live ? rdecay[(int64_t)p * (n / 2) + base + lane] : (T)1;
-    const T U = halving_uniform<T>(seed, (uint32_t)lane, (uint32_t)g, (uint32_t)level, (uint32_t)p + pbase);
+    uint32_t cgroup, ccode;
+    call_counter(g, lvl, cgroup, ccode);
+    const T U = halving_uniform<T>(seed, (uint32_t)lane, cgroup, ccode, (uint32_t)p + pbase);
     uint32_t swaps = walk_block<T>(Fg, P, 0, P, (T)0, r, U, logfac, bmax, lane);
     if (live) {
         const uint32_t sw = (swaps >> lane) & 1u;
@@ -577,6 +581,101 @@ static int run_gram_simt(const Tin *K, const Tin *V, const elm_params *p, const 
     return cuda_status(cudaGetLastError());
 }
 
+// Everything one level needs besides its point lists.
+template <typename Tin, typename T> struct LevelCtx {
+    const Tin *K, *V;
+    const elm_params *p;
+    unsigned *vmax_bits;        // [BH] v_max bits, then the device status word
+    T *cnorm, *Mpair, *rdecay, *F;
+    int64_t F_stride;
+    uint64_t seed;
+    uint32_t pbase;
+    cudaStream_t st;
+};
+
+// One level: `groups` Halve calls KH(delta_call) of P pairs each per attention problem, on the point
+// lists `cur` ([BH][n_kv]-strided, the level's 2 P groups points at the front); survivors go to
+// `out` (stride out_stride) in call order.  `code` is the third word of the uniforms' counter; with
+// calls_per_sibling > 0 the level holds the calls of several sibling segments (see call_counter).
+template <typename Tin, typename T>
+static int run_halve_level(const LevelCtx<Tin, T> &c, const int32_t *cur, int32_t *out, int64_t out_stride, int groups,
+                           int P, int code, double delta_call, int calls_per_sibling = 0)
+{
+    const int64_t lvl = (int64_t)code | ((int64_t)calls_per_sibling << 32);
+    const elm_params *p = c.p;
+    const int BH = p->batch * p->kv_heads;
+    const int64_t n = p->n_kv;
+    const int64_t Ptotal = (int64_t)groups * P;
+    const T logfac = (T)(0.5 + log(2.0 * (double)(2 * P) / delta_call));
+    cudaStream_t st = c.st;
+    int *status = reinterpret_cast<int *>(c.vmax_bits + BH);
+    {
+        StageTimer t(ELM_STAGE_LEVEL_PREP, st, 1);
+        const int lp_threads = P >= 1024 ? 1024 : (P <= 32 ? 32 : (P + 31) / 32 * 32);
+        level_prep_kernel<T><<<dim3((unsigned)groups, (unsigned)BH), lp_threads, 0, st>>>(c.cnorm, cur, n, P, c.Mpair, c.rdecay);
+        count_launches(1);
+        ELM_CUDA_TRY(cudaGetLastError());
+    }
+    bool walked = false;                                       // the Gram kernel walked the level itself
+    {
+        StageTimer t(ELM_STAGE_GRAM, st, 1);
+        int rc;
+        if constexpr (std::is_same<Tin, __nv_bfloat16>::value && std::is_same<T, float>::value) {
+            // tensor cores once a Halve call fills at least a quarter of a 64-pair tile side; calls
+            // that fit a tile (<= 64 pairs) are also walked inside the Gram kernel
+            if (P >= 16) {
+                WalkArgs wk;
+                wk.fused = P <= 64;
+                wk.level = lvl;
+                wk.seed = c.seed;
+                wk.logfac = logfac;
+                wk.rdecay = c.rdecay;
+                wk.out = out;
+                wk.out_stride = out_stride;
+                wk.pbase = c.pbase;
+                walked = wk.fused;
+                rc = gram_tc(c.K, c.V, p, cur, c.Mpair, c.vmax_bits, P, Ptotal, groups, c.F, c.F_stride, status, wk, st);
+            } else {
+                rc = run_gram_simt<Tin, T>(c.K, c.V, p, cur, c.Mpair, c.vmax_bits, P, Ptotal, groups, c.F, c.F_stride, st);
+            }
+        } else {
+            rc = run_gram_simt<Tin, T>(c.K, c.V, p, cur, c.Mpair, c.vmax_bits, P, Ptotal, groups, c.F, c.F_stride, st);
+        }
+        if (rc != ELM_OK) return rc;
+    }
+    if (!walked) {
+        StageTimer t(ELM_STAGE_WALK, st, 1);
+        int chain_rc = 1;                                          // 1 = not taken
+        if (P >= walk_chain_min_pairs() && walk_chain_covers<T>(P)) {
+            chain_rc = walk_chain<T>(c.F, c.F_stride, c.rdecay, cur, out, out_stride, n, P, groups, (int)BH, lvl, c.seed,
+                                     logfac, c.pbase, status, st);
+            if (chain_rc < 0) return chain_rc;
+        }
+        if (chain_rc == ELM_OK) {
+            // launched by walk_chain
+        } else if (P >= 32) {
+            // walker warp + tile-copy warp + updaters (one per two pairs, at most 512 threads)
+            int upd = P / 2;
+            upd = upd < 32 ? 32 : (upd > 512 ? 512 : upd);
+            const int threads = P == 32 ? 32 : 64 + upd;
+            constexpr int PW = 2048 / sizeof(T);
+            const int pw_alloc = P - 64 < PW ? (P - 64 > 0 ? P - 64 : 32) : PW;
+            const size_t smem = (size_t)(4 * 1024 + 4 * P + 32 + 2 * 32 * pw_alloc) * sizeof(T) + (size_t)(P / 32) * 4;
+            if (smem > 227 * 1024) return ELM_ERR_SHAPE;               // a call this long needs the chain kernel
+            auto kern = walk_cta_kernel<T>;
+            ELM_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            kern<<<dim3((unsigned)groups, (unsigned)BH), threads, smem, st>>>(
+                c.F, c.F_stride, c.rdecay, cur, out, out_stride, n, P, lvl, c.seed, logfac, c.pbase);
+        } else {
+            walk_warp_kernel<T><<<dim3((unsigned)((groups + 7) / 8), (unsigned)BH), 256, 0, st>>>(
+                c.F, c.F_stride, c.rdecay, cur, out, out_stride, n, P, groups, lvl, c.seed, logfac, c.pbase);
+        }
+        count_launches(1);
+        ELM_CUDA_TRY(cudaGetLastError());
+    }
+    return ELM_OK;
+}
+
 template <typename Tin, typename T>
 static int compress_impl(const Tin *K, const Tin *V, const elm_params *p, uint64_t seed,
                          int32_t *idx_out, float *w_out, unsigned char *ws, cudaStream_t st, uint32_t pbase)
@@ -586,13 +685,17 @@ static int compress_impl(const Tin *K, const Tin *V, const elm_params *p, uint64
     const int64_t n = p->n_kv;
     const int64_t n_out = (int64_t)1 << p->log2_nout;
     const int m = p->m;
-    unsigned *vmax_bits = reinterpret_cast<unsigned *>(ws + L.vmax_bits);
-    T *cnorm = reinterpret_cast<T *>(ws + L.cnorm);
+    LevelCtx<Tin, T> c;
+    c.K = K; c.V = V; c.p = p;
+    c.vmax_bits = reinterpret_cast<unsigned *>(ws + L.vmax_bits);
+    c.cnorm = reinterpret_cast<T *>(ws + L.cnorm);
+    c.Mpair = reinterpret_cast<T *>(ws + L.Mpair);
+    c.rdecay = reinterpret_cast<T *>(ws + L.rdecay);
+    c.F = reinterpret_cast<T *>(ws + L.F);
+    c.F_stride = (int64_t)L.F_stride;
+    c.seed = seed; c.pbase = pbase; c.st = st;
     int32_t *cur = reinterpret_cast<int32_t *>(ws + L.cur);
     int32_t *nxt = reinterpret_cast<int32_t *>(ws + L.nxt);
-    T *Mpair = reinterpret_cast<T *>(ws + L.Mpair);
-    T *rdecay = reinterpret_cast<T *>(ws + L.rdecay);
-    T *F = reinterpret_cast<T *>(ws + L.F);
 
     double dl[32];
     if (p->delta_level) {
@@ -603,88 +706,198 @@ static int compress_impl(const Tin *K, const Tin *V, const elm_params *p, uint64
 
     if (m > 0) {
         StageTimer t(ELM_STAGE_PREPASS, st, 1);
-        ELM_CUDA_TRY(cudaMemsetAsync(vmax_bits, 0, (size_t)(BH + 1) * 4, st));
+        ELM_CUDA_TRY(cudaMemsetAsync(c.vmax_bits, 0, (size_t)(BH + 1) * 4, st));
         dim3 grid((unsigned)((n + 255) / 256), (unsigned)BH);
-        prepass_kernel<Tin, T><<<grid, 256, 0, st>>>(K, V, n, p->d, cnorm, vmax_bits, cur);
+        prepass_kernel<Tin, T><<<grid, 256, 0, st>>>(K, V, n, p->d, c.cnorm, c.vmax_bits, cur);
         count_launches(1);
         ELM_CUDA_TRY(cudaGetLastError());
     }
     for (int level = 0; level < m; ++level) {
         const int64_t len = n >> level;                            // points alive
         const int groups = 1 << (2 * (m - 1 - level));             // 4^(m-1-level) Halve calls
-        const int64_t s = len / groups;                            // points per call
-        const int P = (int)(s / 2);
-        const int64_t Ptotal = len / 2;
-        const T logfac = (T)(0.5 + log(2.0 * (double)s / dl[level]));
+        const int P = (int)(len / groups / 2);
         const bool last = level == m - 1;
-        int32_t *out = last ? idx_out : nxt;
-        const int64_t out_stride = last ? n_out : n;
-        {
-            StageTimer t(ELM_STAGE_LEVEL_PREP, st, 1);
-            const int lp_threads = P >= 1024 ? 1024 : (P <= 32 ? 32 : (P + 31) / 32 * 32);
-            level_prep_kernel<T><<<dim3((unsigned)groups, (unsigned)BH), lp_threads, 0, st>>>(cnorm, cur, n, P, Mpair, rdecay);
-            count_launches(1);
-            ELM_CUDA_TRY(cudaGetLastError());
-        }
-        bool walked = false;                                       // the Gram kernel walked the level itself
-        {
-            StageTimer t(ELM_STAGE_GRAM, st, 1);
-            int rc;
-            if constexpr (std::is_same<Tin, __nv_bfloat16>::value && std::is_same<T, float>::value) {
-                // tensor cores once a Halve call fills at least a quarter of a 64-pair tile side; calls
-                // that fit a tile (<= 64 pairs) are also walked inside the Gram kernel
-                if (P >= 16) {
-                    WalkArgs wk;
-                    wk.fused = P <= 64;
-                    wk.level = level;
-                    wk.seed = seed;
-                    wk.logfac = logfac;
-                    wk.rdecay = rdecay;
-                    wk.out = out;
-                    wk.out_stride = out_stride;
-                    wk.pbase = pbase;
-                    walked = wk.fused;
-                    rc = gram_tc(K, V, p, cur, Mpair, vmax_bits, P, Ptotal, groups, F, L.F_stride,
-                                 reinterpret_cast<int *>(vmax_bits + BH), wk, st);
-                } else {
-                    rc = run_gram_simt<Tin, T>(K, V, p, cur, Mpair, vmax_bits, P, Ptotal, groups, F, L.F_stride, st);
-                }
-            } else {
-                rc = run_gram_simt<Tin, T>(K, V, p, cur, Mpair, vmax_bits, P, Ptotal, groups, F, L.F_stride, st);
-            }
-            if (rc != ELM_OK) return rc;
-        }
-        if (!walked) {
-            StageTimer t(ELM_STAGE_WALK, st, 1);
-            if (P >= walk_chain_min_pairs() && walk_chain_covers<T>(P)) {
-                const int rc = walk_chain<T>(F, L.F_stride, rdecay, cur, out, out_stride, n, P, groups, (int)BH, level,
-                                             seed, logfac, pbase, reinterpret_cast<int *>(vmax_bits + BH), st);
-                if (rc != ELM_OK) return rc;
-            } else if (P >= 32) {
-                // walker warp + tile-copy warp + updaters (one per two pairs, at most 512 threads)
-                int upd = P / 2;
-                upd = upd < 32 ? 32 : (upd > 512 ? 512 : upd);
-                const int threads = P == 32 ? 32 : 64 + upd;
-                constexpr int PW = 2048 / sizeof(T);
-                const int pw_alloc = P - 64 < PW ? (P - 64 > 0 ? P - 64 : 32) : PW;
-                const size_t smem = (size_t)(4 * 1024 + 4 * P + 32 + 2 * 32 * pw_alloc) * sizeof(T) + (size_t)(P / 32) * 4;
-                auto kern = walk_cta_kernel<T>;
-                ELM_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-                kern<<<dim3((unsigned)groups, (unsigned)BH), threads, smem, st>>>(
-                    F, L.F_stride, rdecay, cur, out, out_stride, n, P, level, seed, logfac, pbase);
-            } else {
-                walk_warp_kernel<T><<<dim3((unsigned)((groups + 7) / 8), (unsigned)BH), 256, 0, st>>>(
-                    F, L.F_stride, rdecay, cur, out, out_stride, n, P, groups, level, seed, logfac, pbase);
-            }
-            count_launches(1);
-            ELM_CUDA_TRY(cudaGetLastError());
-        }
+        const int rc = run_halve_level<Tin, T>(c, cur, last ? idx_out : nxt, last ? n_out : n, groups, P, level, dl[level]);
+        if (rc != ELM_OK) return rc;
         int32_t *tmp = cur; cur = nxt; nxt = tmp;
     }
     {
         StageTimer t(ELM_STAGE_EMIT, st, 1);
         const int64_t total = (int64_t)BH * n_out;
         emit_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(w_out, idx_out, total, n_out, m == 0);
+        count_launches(1);
+        ELM_CUDA_TRY(cudaGetLastError());
+    }
+    return ELM_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Offline-Express: the cache a streaming Express run (Algorithm 1, with Subsample, Algorithm 3, and
+// Compress2, Algorithm 2, inside, Halve = KH with the failure parameters of Corollary 2) holds after
+// n = n_out 4^R points, computed by the equivalent recursion: E = first n_out points; round r
+// (thinning factor m = 2r) thins the next three segments of n_out 2^m points each - one stratified
+// draw per 2^(m - mbar) points when m > mbar, then Compress2 of depth min(m, mbar) - appends the three
+// results to E and halves E twice.  Every Halve call runs through the same level machinery as
+// elm_compress; the uniforms' counter words follow the call structure of the streaming run:
+//   third word = level i + 64 (4 r + j)    Halve_i inside sibling j in {1, 2, 3} of round r,
+//                62 / 63 + 64 (4 r)        the two halvings of E,
+//                61 + 64 (4 r + j)         the stratified draws of sibling j (first word = stratum).
+// v_max is taken over the whole sequence.
+// ---------------------------------------------------------------------------------------------
+struct ExpressLayout {
+    size_t vmax_bits, cnorm, listA, listB, E, T1, Mpair, rdecay, F, F_stride, total;
+};
+static ExpressLayout express_layout(const elm_params *p)
+{
+    ExpressLayout L;
+    const size_t ts = p->precision == ELM_PREC_FP64_DET ? 8 : 4;
+    const size_t BH = (size_t)p->batch * p->kv_heads;
+    const size_t n = (size_t)p->n_kv;
+    const size_t n_out = (size_t)1 << p->log2_nout;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+    L.vmax_bits = take((BH + 1) * 4);      // + one device status word
+    L.cnorm = take(BH * n * ts);
+    L.listA = take(BH * n * 4);
+    L.listB = take(BH * n * 4);
+    L.E = take(BH * n * 4);                // every point list is [BH][n]-strided, like the lists of elm_compress
+    L.T1 = take(BH * n * 4);
+    L.Mpair = take(BH * (n / 2 + 1) * ts);
+    L.rdecay = take(BH * (n / 2 + 1) * ts);
+    L.F_stride = 4 * n_out * n_out;        // the first halving of E is one call of 2 n_out pairs
+    L.F = take(BH * L.F_stride * ts);
+    L.total = off;
+    return L;
+}
+
+// n_kv = n_out 4^R ?  Returns R or -1.
+static int express_rounds(const elm_params *p)
+{
+    const int64_t n_out = (int64_t)1 << p->log2_nout;
+    int64_t v = n_out;
+    for (int R = 0; R <= 15; ++R, v *= 4)
+        if (v == (int64_t)p->n_kv) return R;
+    return -1;
+}
+static int validate_express(const elm_params *p, int32_t mbar)
+{
+    if (p->batch < 1 || p->kv_heads < 1) return ELM_ERR_SHAPE;
+    if (p->d != 64 && p->d != 128) return ELM_ERR_SHAPE;
+    if (p->log2_nout < 1 || p->log2_nout > 24 || mbar < 0 || mbar > 30) return ELM_ERR_SHAPE;
+    if (p->n_kv < 1 || express_rounds(p) < 0) return ELM_ERR_SHAPE;
+    if ((int64_t)p->batch * p->kv_heads > 65535) return ELM_ERR_SHAPE;
+    if (p->dtype != ELM_F32 && p->dtype != ELM_BF16) return ELM_ERR_DTYPE;
+    if (p->precision != ELM_PREC_FP64_DET && p->precision != ELM_PREC_FP32) return ELM_ERR_DTYPE;
+    if (!(p->delta > 0.0 && p->delta < 1.0)) return ELM_ERR_DELTA;
+    return ELM_OK;
+}
+
+// list[p][dst + i] = start + i
+__global__ void range_kernel(int32_t *__restrict__ list, int64_t stride, int64_t dst, int64_t start, int64_t count)
+{
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < count) list[(int64_t)blockIdx.y * stride + dst + i] = (int32_t)(start + i);
+}
+// dst[p][dst_off + i] = src[p][i]
+__global__ void copy_list_kernel(int32_t *__restrict__ dstl, int64_t dst_off, const int32_t *__restrict__ src, int64_t stride,
+                                 int64_t count)
+{
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < count) dstl[(int64_t)blockIdx.y * stride + dst_off + i] = src[(int64_t)blockIdx.y * stride + i];
+}
+// Subsample (Algorithm 3) of three consecutive sibling segments of `seg` points, the first starting at
+// `start`: stratum s of width 2^wlog of sibling j keeps point (segment start) + s 2^wlog + floor(U 2^wlog),
+// U the 24-bit uniform of counter (s, 0, code + 64 j, problem); `per` strata per sibling.
+__global__ void subsample_kernel(int32_t *__restrict__ list, int64_t stride, int64_t start, int64_t seg, int wlog,
+                                 int64_t per, uint64_t seed, uint32_t code, uint32_t pbase)
+{
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= 3 * per) return;
+    const int64_t j = t / per, s = t % per;
+    const double U = halving_uniform<double>(seed, (uint32_t)s, 0u, code + 64u * (uint32_t)j, (uint32_t)blockIdx.y + pbase);
+    list[(int64_t)blockIdx.y * stride + t] =
+        (int32_t)(start + j * seg + (s << wlog) + (int64_t)floor(U * (double)((int64_t)1 << wlog)));
+}
+
+static double kh_express_delta(double delta, int m)
+{
+    // Corollary 2: delta_m = (delta / 2) (1 / log2(m/2 + 2) - 1 / log2(m/2 + 3))
+    return 0.5 * delta * (1.0 / log2(0.5 * m + 2.0) - 1.0 / log2(0.5 * m + 3.0));
+}
+
+template <typename Tin, typename T>
+static int express_impl(const Tin *K, const Tin *V, const elm_params *p, int mbar, uint64_t seed, int32_t *idx_out,
+                        float *w_out, unsigned char *ws, cudaStream_t st, uint32_t pbase)
+{
+    const ExpressLayout L = express_layout(p);
+    const int BH = p->batch * p->kv_heads;
+    const int64_t n = p->n_kv;
+    const int64_t n_out = (int64_t)1 << p->log2_nout;
+    const int R = express_rounds(p);
+    LevelCtx<Tin, T> c;
+    c.K = K; c.V = V; c.p = p;
+    c.vmax_bits = reinterpret_cast<unsigned *>(ws + L.vmax_bits);
+    c.cnorm = reinterpret_cast<T *>(ws + L.cnorm);
+    c.Mpair = reinterpret_cast<T *>(ws + L.Mpair);
+    c.rdecay = reinterpret_cast<T *>(ws + L.rdecay);
+    c.F = reinterpret_cast<T *>(ws + L.F);
+    c.F_stride = (int64_t)L.F_stride;
+    c.seed = seed; c.pbase = pbase; c.st = st;
+    int32_t *listA = reinterpret_cast<int32_t *>(ws + L.listA);
+    int32_t *listB = reinterpret_cast<int32_t *>(ws + L.listB);
+    int32_t *E = reinterpret_cast<int32_t *>(ws + L.E);
+    int32_t *T1 = reinterpret_cast<int32_t *>(ws + L.T1);
+    auto blocks = [](int64_t count) { return (unsigned)((count + 255) / 256); };
+    {
+        StageTimer t(ELM_STAGE_PREPASS, st, 2);
+        ELM_CUDA_TRY(cudaMemsetAsync(c.vmax_bits, 0, (size_t)(BH + 1) * 4, st));
+        prepass_kernel<Tin, T><<<dim3(blocks(n), (unsigned)BH), 256, 0, st>>>(K, V, n, p->d, c.cnorm, c.vmax_bits, listA);
+        range_kernel<<<dim3(blocks(n_out), (unsigned)BH), 256, 0, st>>>(E, n, 0, 0, n_out);      // exact phase
+        count_launches(2);
+        ELM_CUDA_TRY(cudaGetLastError());
+    }
+    for (int r = 0; r < R; ++r) {
+        const int m = 2 * r, q = m < mbar ? m : mbar;
+        const int64_t seg = n_out << m, len0 = n_out << q;
+        const double dm = kh_express_delta(p->delta, m);
+        // The three sibling segments of the round are thinned together: their point lists are laid
+        // side by side, every level holds the calls of all three (call_counter keeps their uniforms
+        // apart), and the last level leaves their 3 n_out survivors behind the n_out points of E.
+        const int code1 = 64 * (4 * r + 1);                                   // sibling 1; siblings 2, 3 are 64 apart
+        if (m > mbar)
+            subsample_kernel<<<dim3(blocks(3 * len0), (unsigned)BH), 256, 0, st>>>(listA, n, seg, seg, m - mbar, len0, seed,
+                                                                                   (uint32_t)(61 + code1), pbase);
+        else
+            range_kernel<<<dim3(blocks(3 * seg), (unsigned)BH), 256, 0, st>>>(listA, n, 0, seg, 3 * seg);
+        count_launches(1);
+        ELM_CUDA_TRY(cudaGetLastError());
+        if (q == 0) {
+            copy_list_kernel<<<dim3(blocks(3 * n_out), (unsigned)BH), 256, 0, st>>>(E, n_out, listA, n, 3 * n_out);
+            count_launches(1);
+            ELM_CUDA_TRY(cudaGetLastError());
+        } else {
+            int32_t *cur = listA, *nxt = listB;
+            for (int i = 0; i < q; ++i) {
+                const int per = 1 << (2 * (q - 1 - i));                       // calls per sibling
+                const int P = (int)((len0 >> i) / per / 2);
+                const double dlt = ldexp(dm, 2 * (i + 1 - q)) / (3.0 * (double)q);
+                const int rc = run_halve_level<Tin, T>(c, cur, i == q - 1 ? E + n_out : nxt, n, 3 * per, P, i + code1, dlt, per);
+                if (rc != ELM_OK) return rc;
+                int32_t *tmp = cur; cur = nxt; nxt = tmp;
+            }
+        }
+        // halve phase: 4 n_out -> 2 n_out -> n_out
+        const bool last_round = r == R - 1;
+        int rc = run_halve_level<Tin, T>(c, E, T1, n, 1, (int)(2 * n_out), (int)(62 + 64 * 4 * r), 0.5 * dm);
+        if (rc != ELM_OK) return rc;
+        rc = run_halve_level<Tin, T>(c, T1, last_round ? idx_out : E, last_round ? n_out : n, 1, (int)n_out,
+                                     (int)(63 + 64 * 4 * r), 0.5 * dm);
+        if (rc != ELM_OK) return rc;
+    }
+    {
+        StageTimer t(ELM_STAGE_EMIT, st, 1);
+        const int64_t total = (int64_t)BH * n_out;
+        emit_kernel<<<blocks(total), 256, 0, st>>>(w_out, idx_out, total, n_out, R == 0);
         count_launches(1);
         ELM_CUDA_TRY(cudaGetLastError());
     }
@@ -723,4 +936,36 @@ extern "C" int elm_compress(const void *K, const void *V, const elm_params *para
     if ((uintptr_t)workspace & 255) return ELM_ERR_ALIGN;
     if (workspace_bytes < compress_layout(params).total) return ELM_ERR_WORKSPACE;
     return compress_enqueue(K, V, params, seed, idx_out, w_out, workspace, (cudaStream_t)stream, 0u);
+}
+
+extern "C" int elm_express_workspace_bytes(const elm_params *params, int32_t mbar, size_t *bytes)
+{
+    using namespace elm;
+    if (!params || !bytes) return ELM_ERR_NULL;
+    const int rc = validate_express(params, mbar);
+    if (rc != ELM_OK) return rc;
+    *bytes = express_layout(params).total;
+    return ELM_OK;
+}
+
+extern "C" int elm_express_compress(const void *K, const void *V, const elm_params *params, int32_t mbar, uint64_t seed,
+                                    int32_t *idx_out, float *w_out, void *workspace, size_t workspace_bytes, void *stream)
+{
+    using namespace elm;
+    if (!params) return ELM_ERR_NULL;
+    const int rc = validate_express(params, mbar);
+    if (rc != ELM_OK) return rc;
+    if (!K || !V || !idx_out || !w_out || !workspace) return ELM_ERR_NULL;
+    if (((uintptr_t)K | (uintptr_t)V | (uintptr_t)idx_out | (uintptr_t)w_out) & 15) return ELM_ERR_ALIGN;
+    if ((uintptr_t)workspace & 255) return ELM_ERR_ALIGN;
+    if (workspace_bytes < express_layout(params).total) return ELM_ERR_WORKSPACE;
+    unsigned char *ws = (unsigned char *)workspace;
+    cudaStream_t st = (cudaStream_t)stream;
+    const bool det = params->precision == ELM_PREC_FP64_DET;
+    if (params->dtype == ELM_F32) {
+        return det ? express_impl<float, double>((const float *)K, (const float *)V, params, mbar, seed, idx_out, w_out, ws, st, 0u)
+                   : express_impl<float, float>((const float *)K, (const float *)V, params, mbar, seed, idx_out, w_out, ws, st, 0u);
+    }
+    return det ? express_impl<__nv_bfloat16, double>((const __nv_bfloat16 *)K, (const __nv_bfloat16 *)V, params, mbar, seed, idx_out, w_out, ws, st, 0u)
+               : express_impl<__nv_bfloat16, float>((const __nv_bfloat16 *)K, (const __nv_bfloat16 *)V, params, mbar, seed, idx_out, w_out, ws, st, 0u);
 }

@@ -32,7 +32,7 @@ int compress_enqueue(const void *K, const void *V, const elm_params *params, uin
 // the survivors go straight to `out`.
 struct WalkArgs {
     int fused;
-    int level;
+    int64_t level;           // third counter word (+ calls per sibling in the high half, see call_counter)
     uint64_t seed;
     float logfac;
     const float *rdecay;     // [BH][n/2]
@@ -49,10 +49,12 @@ int gram_tc(const __nv_bfloat16 *K, const __nv_bfloat16 *V, const elm_params *p,
 
 // The halving walk of one level for calls of at least 32 pairs (one CTA or one cluster per call).
 // walk_chain_covers says whether a call size fits its shared-memory plan; `status` as above.
+// walk_chain returns ELM_OK, a negative elm_status, or 1 when the device cannot keep a cluster of the
+// needed size resident (nothing launched: use another kernel).
 template <typename T> bool walk_chain_covers(int P);
 template <typename T>
 int walk_chain(const T *F, int64_t F_stride, const T *rdecay, const int32_t *cur, int32_t *out, int64_t out_stride,
-               int64_t n, int P, int groups, int problems, int level, uint64_t seed, T logfac, uint32_t pbase,
+               int64_t n, int P, int groups, int problems, int64_t level, uint64_t seed, T logfac, uint32_t pbase,
                int *status, cudaStream_t st);
 
 }  // namespace elm

@@ -143,7 +143,9 @@ gram_tc_kernel(const __nv_bfloat16 *__restrict__ K, const __nv_bfloat16 *__restr
         if (wk.fused) {
             // everything the in-tile walk needs from global memory, fetched while the tile is built
             misc->rdec[tid] = jc < Ptotal ? wk.rdecay[(int64_t)p * (n / 2) + jc] : 1.f;
-            misc->unif[tid] = halving_uniform<float>(wk.seed, (uint32_t)(jc % P), (uint32_t)(jc / P), (uint32_t)wk.level, (uint32_t)p + wk.pbase);
+            uint32_t cgroup, ccode;
+            call_counter((int)(jc / P), wk.level, cgroup, ccode);
+            misc->unif[tid] = halving_uniform<float>(wk.seed, (uint32_t)(jc % P), cgroup, ccode, (uint32_t)p + wk.pbase);
         }
     }
     if (tid == 0) {

@@ -28,7 +28,7 @@
 namespace elm {
 namespace {
 
-constexpr int MAX_CLUSTER = 8;
+constexpr int MAX_CLUSTER = 16;          // above 8 the cluster size is "non-portable": opt-in, and checked for schedulability
 constexpr int UPD_THREADS_MAX = 256;
 constexpr uint32_t FULL = 0xffffffffu;
 
@@ -155,7 +155,7 @@ __global__ void __launch_bounds__(96 + UPD_THREADS_MAX)
 walk_chain_kernel(const __grid_constant__ CUtensorMap mapF, const T *__restrict__ F, int64_t F_stride,
                   const T *__restrict__ rdecay,
                   const int32_t *__restrict__ cur, int32_t *__restrict__ out, int64_t out_stride,
-                  int64_t n, int P, int level, uint64_t seed, T logfac, uint32_t pbase, int nb_cap, int *status)
+                  int64_t n, int P, int64_t lvl, uint64_t seed, T logfac, uint32_t pbase, int nb_cap, int *status)
 {
     using namespace sm100;
     constexpr bool EAGER = std::is_same<T, float>::value;            // the fp32 walker also scores the next block
@@ -245,9 +245,11 @@ walk_chain_kernel(const __grid_constant__ CUtensorMap mapF, const T *__restrict_
         }
     }
     for (int i = threadIdx.x; i < col0 + W; i += nthr) rall_s[i] = rdecay[(int64_t)p * (n / 2) + base + i];
+    uint32_t cgroup, ccode;
+    call_counter(g, lvl, cgroup, ccode);
     for (int i = threadIdx.x; i < W; i += nthr) {
         alpha_s[i] = 0;
-        U_s[i] = halving_uniform<T>(seed, (uint32_t)(col0 + i), (uint32_t)g, (uint32_t)level, (uint32_t)p + pbase);
+        U_s[i] = halving_uniform<T>(seed, (uint32_t)(col0 + i), cgroup, ccode, (uint32_t)p + pbase);
     }
     __syncthreads();
     if (C > 1) cluster_sync_all();                                   // every CTA's control words are initialised
@@ -388,7 +390,7 @@ template <typename T> bool walk_chain_covers(int P)
 
 template <typename T>
 int walk_chain(const T *F, int64_t F_stride, const T *rdecay, const int32_t *cur, int32_t *out, int64_t out_stride,
-               int64_t n, int P, int groups, int problems, int level, uint64_t seed, T logfac, uint32_t pbase,
+               int64_t n, int P, int groups, int problems, int64_t level, uint64_t seed, T logfac, uint32_t pbase,
                int *status, cudaStream_t st)
 {
     const int C = chain_cluster_size(P);
@@ -423,6 +425,16 @@ int walk_chain(const T *F, int64_t F_stride, const T *rdecay, const int32_t *cur
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
+    if (C > 8) {
+        // clusters of 16 CTAs need the opt-in and a GPC with 16 free SMs; if none can be resident
+        // the caller falls back to one CTA per call
+        ELM_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
+        int resident = 0;
+        if (cudaOccupancyMaxActiveClusters(&resident, kern, &cfg) != cudaSuccess || resident < 1) {
+            cudaGetLastError();
+            return 1;
+        }
+    }
     ELM_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, mapF, F, F_stride, rdecay, cur, out, out_stride, n, P, level, seed, logfac,
                                     pbase, nb_cap, status));
     return ELM_OK;
@@ -431,9 +443,9 @@ int walk_chain(const T *F, int64_t F_stride, const T *rdecay, const int32_t *cur
 template bool walk_chain_covers<float>(int);
 template bool walk_chain_covers<double>(int);
 template int walk_chain<float>(const float *, int64_t, const float *, const int32_t *, int32_t *, int64_t, int64_t, int,
-                               int, int, int, uint64_t, float, uint32_t, int *, cudaStream_t);
+                               int, int, int64_t, uint64_t, float, uint32_t, int *, cudaStream_t);
 template int walk_chain<double>(const double *, int64_t, const double *, const int32_t *, int32_t *, int64_t, int64_t,
-                                int, int, int, int, uint64_t, double, uint32_t, int *, cudaStream_t);
+                                int, int, int, int64_t, uint64_t, double, uint32_t, int *, cudaStream_t);
 
 }  // namespace elm
 
