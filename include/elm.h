@@ -170,10 +170,30 @@ int elm_attend_static(const void *Q, const void *K, const void *V, const int32_t
  *   workspace  at least elm_express_workspace_bytes(params, mbar) bytes, 256-byte aligned.
  * v_max of Eq. (katt) is taken over the whole sequence of the problem.  In fp64 mode a call of more
  * than 2048 pairs (n_out > 1024 here) is not supported and returns ELM_ERR_SHAPE.
- * This is the compression half of causal prefill with Thinformer Express (Algorithm 5); attention
- * of every query over the cache as of its own position is not part of this library yet.
+ * This is the compression half of causal prefill with Thinformer Express (Algorithm 5); see
+ * elm_express_prefill for the attention of every query over the cache as of its own position.
  */
 int elm_express_workspace_bytes(const elm_params *params, int32_t mbar, size_t *bytes);
+
+/*
+ * Thinformer Express (Algorithm 5) in prefill: O[t] = WtdAttention(q_t, cache as of token t plus token
+ * t itself) for every token t of every head, where the cache is that of the Express run described at
+ * elm_express_compress (computed by the same recursion, with the same uniforms), and that cache after
+ * the last token in idx_out / w_out.  Token t's cache is: E with the segments finished so far (weight
+ * 1), for every Compress2 level i the outputs of Halve calls that the next level has not consumed yet
+ * (weight 2^(i-q), q = the current Compress2 depth), and the tokens since the last level-0 Halve call
+ * up to t (weight 2^-q).  The first 4 n_out tokens attend exactly (causally).
+ *   Q, O       [batch][q_heads][n_kv][d] (params->n_q must equal n_kv); K, V as for elm_compress.
+ *   Limits     rounds with a thinning factor above mbar (Subsample active) are not built yet:
+ *              n_kv <= n_out 4^(mbar/2 + 1), else ELM_ERR_SHAPE; level-0 Halve calls need >= 2 points
+ *              (2 (R-1) <= log2_nout + 1).
+ *   workspace  at least elm_express_prefill_workspace_bytes(params, mbar) bytes, 256-byte aligned.
+ * One attention launch per epoch (the tokens between two level-0 Halve calls).
+ */
+int elm_express_prefill_workspace_bytes(const elm_params *params, int32_t mbar, size_t *bytes);
+int elm_express_prefill(const void *Q, const void *K, const void *V, const elm_params *params, int32_t mbar,
+                        uint64_t seed, void *O, int32_t *idx_out, float *w_out, void *workspace,
+                        size_t workspace_bytes, void *stream);
 int elm_express_compress(const void *K, const void *V, const elm_params *params, int32_t mbar, uint64_t seed,
                          int32_t *idx_out, float *w_out, void *workspace, size_t workspace_bytes, void *stream);
 

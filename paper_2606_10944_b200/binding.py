@@ -21,6 +21,7 @@ STAGE_NAMES = ["prepass", "level_prep", "gram", "walk", "emit", "gather", "atten
 EXPORTED_SYMBOLS = [
     "elm_workspace_bytes", "elm_default_delta_levels", "elm_compress", "elm_attend",
     "elm_attend_workspace_bytes", "elm_attend_static", "elm_express_workspace_bytes", "elm_express_compress",
+    "elm_express_prefill_workspace_bytes", "elm_express_prefill",
     "elm_host_call_scratch_bytes", "elm_compress_attend_host",
     "elm_compress_status", "elm_attend_status", "elm_profile_enable", "elm_profile_read", "elm_launch_count", "elm_strerror", "elm_version",
 ]
@@ -67,6 +68,8 @@ def load_library():
     lib.elm_attend_static.argtypes = [vp, vp, vp, vp, vp, ctypes.c_int32, pp, vp, vp]
     lib.elm_express_workspace_bytes.argtypes = [pp, ctypes.c_int32, szp]
     lib.elm_express_compress.argtypes = [vp, vp, pp, ctypes.c_int32, ctypes.c_uint64, vp, vp, vp, sz, vp]
+    lib.elm_express_prefill_workspace_bytes.argtypes = [pp, ctypes.c_int32, szp]
+    lib.elm_express_prefill.argtypes = [vp, vp, vp, pp, ctypes.c_int32, ctypes.c_uint64, vp, vp, vp, vp, sz, vp]
     lib.elm_host_call_scratch_bytes.argtypes = [pp, szp]
     lib.elm_compress_attend_host.argtypes = [vp, vp, vp, vp, vp, vp, pp, ctypes.c_uint64, vp, sz, vp]
     lib.elm_compress_status.argtypes = [vp, pp, ctypes.POINTER(ctypes.c_int32), vp]
@@ -181,6 +184,29 @@ def express_compress(K, V, log2_nout: int, mbar: int, seed: int = 1, precision="
     _check(lib.elm_express_compress(K.data_ptr(), V.data_ptr(), ctypes.byref(p), mbar, seed, idx.data_ptr(),
                                     w.data_ptr(), ws.data_ptr(), ws.numel(), _stream()), "elm_express_compress")
     return idx, w
+
+
+def express_prefill(Q, K, V, log2_nout: int, mbar: int, seed: int = 1, precision="fp32", delta: float = 0.5,
+                    workspace=None, out=None):
+    """elm_express_prefill: Q [B, Hq, n, d], K, V [B, Hkv, n, d] -> (O like Q, idx, w): every token attends
+    over the Express cache as of its own position plus itself (Thinformer Express in prefill)."""
+    lib = load_library()
+    _require_cuda(Q, K, V)
+    B, Hq, nq, d = Q.shape
+    H, n = K.shape[1], K.shape[2]
+    p, _ = make_params(B, Hq, H, n, nq, d, log2_nout, 0, _dtype_code(K), precision, delta)
+    need = ctypes.c_size_t(0)
+    _check(lib.elm_express_prefill_workspace_bytes(ctypes.byref(p), mbar, ctypes.byref(need)),
+           "elm_express_prefill_workspace_bytes")
+    ws = workspace if workspace is not None else _workspace(int(need.value), K.device)
+    n_out = 1 << log2_nout
+    O = out if out is not None else torch.empty_like(Q)
+    idx = torch.empty((B, H, n_out), dtype=torch.int32, device=K.device)
+    w = torch.empty((B, H, n_out), dtype=torch.float32, device=K.device)
+    _check(lib.elm_express_prefill(Q.data_ptr(), K.data_ptr(), V.data_ptr(), ctypes.byref(p), mbar, seed, O.data_ptr(),
+                                   idx.data_ptr(), w.data_ptr(), ws.data_ptr(), ws.numel(), _stream()),
+           "elm_express_prefill")
+    return O, idx, w
 
 
 def attend(Q, K, V, idx, w, precision="fp32", workspace=None, out=None):

@@ -51,7 +51,8 @@ __global__ void __launch_bounds__(128) attend_simt_kernel(const Tin *__restrict_
                                                           const Tin *__restrict__ Vc,
                                                           const float *__restrict__ bias,
                                                           Tin *__restrict__ O, int q_heads,
-                                                          int kv_heads, int64_t n_q, int n_core)
+                                                          int kv_heads, int64_t n_q, int n_core,
+                                                          int64_t q_row0, int64_t n_q_total, int tail_start)
 {
     constexpr int BM = 64, BN = 32;
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -69,7 +70,7 @@ __global__ void __launch_bounds__(128) attend_simt_kernel(const Tin *__restrict_
     const int b = bh / q_heads, h = bh % q_heads;
     const int64_t prob = (int64_t)b * kv_heads + ((int64_t)h * kv_heads) / q_heads;
     const int64_t q0 = (int64_t)blockIdx.x * BM;
-    const Tin *Qp = Q + ((int64_t)bh * n_q) * D;
+    const Tin *Qp = Q + ((int64_t)bh * n_q_total + q_row0) * D;
     const Tin *Kp = Kc + prob * n_core * D;
     const Tin *Vp = Vc + prob * n_core * D;
     const float *bp = bias + prob * n_core;
@@ -118,7 +119,9 @@ __global__ void __launch_bounds__(128) attend_simt_kernel(const Tin *__restrict_
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 int col = 4 * tx + c;
-                S[(4 * ty + r) * (BN + 1) + col] = (c0 + col < n_core) ? s[r][c] * scale + sbias[col] : (T)-INFINITY;
+                // a row sees the list up to its own entry of the causal tail
+                const bool seen = c0 + col < n_core && (int64_t)(c0 + col) <= (int64_t)tail_start + q0 + 4 * ty + r;
+                S[(4 * ty + r) * (BN + 1) + col] = seen ? s[r][c] * scale + sbias[col] : (T)-INFINITY;
             }
         __syncthreads();
         if (tid < BM) {
@@ -155,7 +158,7 @@ __global__ void __launch_bounds__(128) attend_simt_kernel(const Tin *__restrict_
             }
         }
     }
-    Tin *Op = O + ((int64_t)bh * n_q) * D;
+    Tin *Op = O + ((int64_t)bh * n_q_total + q_row0) * D;
 #pragma unroll
     for (int r = 0; r < 4; ++r) {
         int64_t q = q0 + 4 * ty + r;
@@ -184,24 +187,25 @@ AttendLayout attend_layout(const elm_params *p, int32_t n_core)
 
 template <typename Tin, typename T, int D>
 static int launch_attend_simt(const Tin *Q, const Tin *Kc, const Tin *Vc, const float *bias, Tin *O,
-                              const elm_params *p, int n_core, cudaStream_t st)
+                              const elm_params *p, int n_core, cudaStream_t st, const AttendWindow &win = AttendWindow())
 {
     constexpr int BM = 64, BN = 32;
     const size_t smem = sizeof(T) * (size_t)(D * BM + D * BN + BN * D + BM * (BN + 1) + 3 * BM + BN);
     auto kern = attend_simt_kernel<Tin, T, D>;
     ELM_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     dim3 grid((unsigned)((p->n_q + BM - 1) / BM), (unsigned)(p->batch * p->q_heads));
-    kern<<<grid, 128, smem, st>>>(Q, Kc, Vc, bias, O, p->q_heads, p->kv_heads, p->n_q, n_core);
+    kern<<<grid, 128, smem, st>>>(Q, Kc, Vc, bias, O, p->q_heads, p->kv_heads, p->n_q, n_core, win.q_row0,
+                                  win.n_q_total ? win.n_q_total : (int64_t)p->n_q, win.tail_start);
     count_launches(1);
     return cuda_status(cudaGetLastError());
 }
 
 template <typename Tin, typename T>
 static int attend_impl(const Tin *Q, const Tin *K, const Tin *V, const int32_t *idx, const float *w,
-                       int n_core, const elm_params *p, Tin *O, unsigned char *ws, cudaStream_t st)
+                       int n_core, const elm_params *p, Tin *O, unsigned char *ws, cudaStream_t st, const AttendWindow &win)
 {
     if constexpr (std::is_same<Tin, __nv_bfloat16>::value && std::is_same<T, float>::value)
-        return attend_tc(Q, K, V, idx, w, n_core, p, O, ws, st, true);
+        return attend_tc(Q, K, V, idx, w, n_core, p, O, ws, st, true, win);
     const AttendLayout L = attend_layout(p, n_core);
     Tin *Kc = reinterpret_cast<Tin *>(ws + L.Kc);
     Tin *Vc = reinterpret_cast<Tin *>(ws + L.Vc);
@@ -217,8 +221,8 @@ static int attend_impl(const Tin *Q, const Tin *K, const Tin *V, const int32_t *
         ELM_CUDA_TRY(cudaGetLastError());
     }
     StageTimer t(ELM_STAGE_ATTEND, st, 1);
-    if (p->d == 64) return launch_attend_simt<Tin, T, 64>(Q, Kc, Vc, bias, O, p, n_core, st);
-    return launch_attend_simt<Tin, T, 128>(Q, Kc, Vc, bias, O, p, n_core, st);
+    if (p->d == 64) return launch_attend_simt<Tin, T, 64>(Q, Kc, Vc, bias, O, p, n_core, st, win);
+    return launch_attend_simt<Tin, T, 128>(Q, Kc, Vc, bias, O, p, n_core, st, win);
 }
 
 
@@ -279,17 +283,17 @@ static int attend_enqueue_untimed(const Tin *Q, const Tin *K, const Tin *V, cons
 namespace elm {
 // elm_attend after argument validation
 int attend_enqueue(const void *Q, const void *K, const void *V, const int32_t *idx, const float *w, int32_t n_core,
-                   const elm_params *params, void *O, void *workspace, cudaStream_t st)
+                   const elm_params *params, void *O, void *workspace, cudaStream_t st, const AttendWindow &win)
 {
     unsigned char *ws = (unsigned char *)workspace;
     const bool det = params->precision == ELM_PREC_FP64_DET;
     if (params->dtype == ELM_F32) {
-        return det ? attend_impl<float, double>((const float *)Q, (const float *)K, (const float *)V, idx, w, n_core, params, (float *)O, ws, st)
-                   : attend_impl<float, float>((const float *)Q, (const float *)K, (const float *)V, idx, w, n_core, params, (float *)O, ws, st);
+        return det ? attend_impl<float, double>((const float *)Q, (const float *)K, (const float *)V, idx, w, n_core, params, (float *)O, ws, st, win)
+                   : attend_impl<float, float>((const float *)Q, (const float *)K, (const float *)V, idx, w, n_core, params, (float *)O, ws, st, win);
     }
     typedef __nv_bfloat16 bf;
-    return det ? attend_impl<bf, double>((const bf *)Q, (const bf *)K, (const bf *)V, idx, w, n_core, params, (bf *)O, ws, st)
-               : attend_impl<bf, float>((const bf *)Q, (const bf *)K, (const bf *)V, idx, w, n_core, params, (bf *)O, ws, st);
+    return det ? attend_impl<bf, double>((const bf *)Q, (const bf *)K, (const bf *)V, idx, w, n_core, params, (bf *)O, ws, st, win)
+               : attend_impl<bf, float>((const bf *)Q, (const bf *)K, (const bf *)V, idx, w, n_core, params, (bf *)O, ws, st, win);
 }
 }  // namespace elm
 

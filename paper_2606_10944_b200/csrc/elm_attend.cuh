@@ -19,14 +19,25 @@ struct AttendLayout {
 };
 AttendLayout attend_layout(const elm_params *p, int32_t n_core);
 
+// Which rows of Q / O a launch covers, and a causal tail of the coreset list.  params->n_q is the
+// number of query rows of the launch; they are rows q_row0 .. q_row0 + n_q - 1 of each head's
+// n_q_total rows.  List entries from tail_start on are visible to row r of the launch only up to
+// entry tail_start + r (Algorithm 5 in prefill: the tail holds the launch's own tokens in order).
+struct AttendWindow {
+    int64_t q_row0 = 0;
+    int64_t n_q_total = 0;               // 0: params->n_q
+    int32_t tail_start = 0x7fffffff;     // no tail
+};
+
 // elm_attend after argument validation
 int attend_enqueue(const void *Q, const void *K, const void *V, const int32_t *idx, const float *w, int32_t n_core,
-                   const elm_params *params, void *O, void *workspace, cudaStream_t st);
+                   const elm_params *params, void *O, void *workspace, cudaStream_t st,
+                   const AttendWindow &win = AttendWindow());
 
 // Tensor-core path (bf16 storage, fp32 accumulation): gather + attention, enqueued on `st`.
 // `timed` selects whether the per-stage event timers are used.
 int attend_tc(const __nv_bfloat16 *Q, const __nv_bfloat16 *K, const __nv_bfloat16 *V, const int32_t *idx,
               const float *w, int n_core, const elm_params *p, __nv_bfloat16 *O, unsigned char *ws,
-              cudaStream_t st, bool timed);
+              cudaStream_t st, bool timed, const AttendWindow &win = AttendWindow());
 
 }  // namespace elm

@@ -241,7 +241,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                  const __grid_constant__ CUtensorMap mapV, const float *__restrict__ bias,
                  const int *__restrict__ nonuniform, __nv_bfloat16 *__restrict__ O, int q_heads,
                  int kv_heads, int n_q, int n_core, int n_pad, float scale_log2, int tiles_x, int n_items_total,
-                 int *__restrict__ status)
+                 int q_row0, int n_q_total, int tail_start, int *__restrict__ status)
 {
     using SM = Smem<D>;
     constexpr int KH = SM::KH;
@@ -293,7 +293,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                 mbar_expect_tx(&bar->q_full, 2 * SM::Q_TILE);
                 for (int t = 0; t < 2; ++t)
                     for (int kh = 0; kh < KH; ++kh)
-                        tma_load_3d(smem + SM::OFF_Q + t * SM::Q_TILE + kh * (BM * 128), &mapQ, &bar->q_full, kh * 64, q0 + t * BM, bh);
+                        tma_load_3d(smem + SM::OFF_Q + t * SM::Q_TILE + kh * (BM * 128), &mapQ, &bar->q_full, kh * 64, q_row0 + q0 + t * BM, bh);
             };
             // Blocks are numbered G = k nblk + j along the CTA's whole stream (item k, block j).
             auto load_k = [&](int G) {
@@ -433,11 +433,16 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
             const float *bp = bias + (int64_t)prob * n_pad + cq * 32;
             float m_ref[2] = {-INFINITY, -INFINITY}, l[2] = {0.f, 0.f};
             for (int j = 0; j < nblk && ok; ++j, ++G) {
-                const int valid = n_core - j * BN - cq * 32;           // of this thread's 32 columns, how many exist
-                const bool special = use_bias || valid < 32;           // per-column bias and/or a ragged tail
                 const float *bcols = use_bias ? bp + j * BN : nullptr;
 #pragma unroll
                 for (int t = 0; t < 2; ++t) {
+                    // A row sees the list up to its own entry of the causal tail (if there is one), so
+                    // the visible columns are a prefix of the list; of this thread's 32, `valid` exist.
+                    const int64_t seen = (int64_t)tail_start + q0 + t * BM + row + 1;
+                    const int valid = (int)(seen < n_core ? seen : n_core) - j * BN - cq * 32;
+                    // per-column bias and/or a ragged end; warp-uniform, because both forms of the two
+                    // passes contain warp-collective TMEM loads
+                    const bool special = use_bias || __any_sync(0xffffffffu, valid < 32);
                     const uint32_t tS = tmem + lane_addr + t * 128 + cq * 32;   // this thread's 32 logit columns
                     const uint32_t tP = tS;                 // their bf16 probabilities overwrite the first 16 of them
                     const uint32_t tO = tmem + lane_addr + 256 + t * 128 + cq * (D / 4);   // its quarter of the accumulator
@@ -488,7 +493,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                 asm volatile("bar.sync 1, 512;" ::: "memory");
                 const float inv = 1.f / ((bar->xchg[t][0][row] + bar->xchg[t][1][row]) + (bar->xchg[t][2][row] + bar->xchg[t][3][row]));
                 const int64_t qrow = (int64_t)q0 + t * BM + row;
-                __nv_bfloat16 *dst = O + ((int64_t)bh * n_q + qrow) * D + cq * (D / 4);
+                __nv_bfloat16 *dst = O + ((int64_t)bh * n_q_total + q_row0 + qrow) * D + cq * (D / 4);
                 uint32_t o[32];
                 if (D == 128) tmem_ld32(tO, o);
                 else tmem_ld16(tO, o);
@@ -551,8 +556,9 @@ static int sm_count()
 template <int D>
 static int launch(const __nv_bfloat16 *Q, const __nv_bfloat16 *K, const __nv_bfloat16 *V, const int32_t *idx,
                   const float *w, int n_core, const elm_params *p, __nv_bfloat16 *O, unsigned char *ws,
-                  cudaStream_t st, bool timed)
+                  cudaStream_t st, bool timed, const AttendWindow &win)
 {
+    const int64_t n_q_total = win.n_q_total ? win.n_q_total : (int64_t)p->n_q;
     const AttendLayout L = attend_layout(p, n_core);
     const int n_pad = (n_core + BN - 1) / BN * BN;
     const int problems = p->batch * p->kv_heads;
@@ -562,7 +568,7 @@ static int launch(const __nv_bfloat16 *Q, const __nv_bfloat16 *K, const __nv_bfl
     int *flags = reinterpret_cast<int *>(ws + L.flags);
     int *status = flags + problems;
     CUtensorMap mQ, mK, mV;
-    if (!make_map(&mQ, Q, D, (uint64_t)p->n_q, (uint64_t)p->batch * p->q_heads, BM) ||
+    if (!make_map(&mQ, Q, D, (uint64_t)n_q_total, (uint64_t)p->batch * p->q_heads, BM) ||
         !make_map(&mK, Kc, D, (uint64_t)n_pad, (uint64_t)problems, BN) ||
         !make_map(&mV, Vt, (uint64_t)n_pad, D, (uint64_t)problems, D))
         return ELM_ERR_CUDA;
@@ -584,7 +590,8 @@ static int launch(const __nv_bfloat16 *Q, const __nv_bfloat16 *K, const __nv_bfl
     const int ctas = (int)(items < sm_count() ? items : sm_count());
     const float scale_log2 = (float)(1.4426950408889634 / sqrt((double)D));
     kern<<<ctas, NTHREADS, Smem<D>::TOTAL, st>>>(mQ, mK, mV, bias, flags, O, p->q_heads, p->kv_heads, p->n_q,
-                                                 n_core, n_pad, scale_log2, tiles_x, (int)items, status);
+                                                 n_core, n_pad, scale_log2, tiles_x, (int)items, (int)win.q_row0,
+                                                 (int)n_q_total, win.tail_start, status);
     count_launches(1);
     return cuda_status(cudaGetLastError());
 }
@@ -592,10 +599,10 @@ static int launch(const __nv_bfloat16 *Q, const __nv_bfloat16 *K, const __nv_bfl
 }  // namespace tc
 int attend_tc(const __nv_bfloat16 *Q, const __nv_bfloat16 *K, const __nv_bfloat16 *V, const int32_t *idx,
               const float *w, int n_core, const elm_params *p, __nv_bfloat16 *O, unsigned char *ws,
-              cudaStream_t st, bool timed)
+              cudaStream_t st, bool timed, const AttendWindow &win)
 {
-    if (p->d == 64) return tc::launch<64>(Q, K, V, idx, w, n_core, p, O, ws, st, timed);
-    return tc::launch<128>(Q, K, V, idx, w, n_core, p, O, ws, st, timed);
+    if (p->d == 64) return tc::launch<64>(Q, K, V, idx, w, n_core, p, O, ws, st, timed, win);
+    return tc::launch<128>(Q, K, V, idx, w, n_core, p, O, ws, st, timed, win);
 }
 
 }  // namespace elm

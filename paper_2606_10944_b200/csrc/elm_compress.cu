@@ -9,6 +9,7 @@
 
 #include <type_traits>
 
+#include "elm_attend.cuh"
 #include "elm_common.cuh"
 #include "elm_compress.cuh"
 #include "elm_walk.cuh"
@@ -746,8 +747,27 @@ static int compress_impl(const Tin *K, const Tin *V, const elm_params *p, uint64
 // ---------------------------------------------------------------------------------------------
 struct ExpressLayout {
     size_t vmax_bits, cnorm, listA, listB, E, T1, Mpair, rdecay, F, F_stride, total;
+    // prefill only: the output lists of every Compress2 level of a round, the cache list of one
+    // epoch with its weights, the workspace of elm_attend for that list
+    size_t levels, ep_idx, ep_w, ws_attend, ep_cap;
+    int n_levels;
 };
-static ExpressLayout express_layout(const elm_params *p)
+// Longest cache list (weighted cache + causal tail) any epoch of the prefill attends over.
+static size_t express_epoch_cap(const elm_params *p, int mbar)
+{
+    const size_t n_out = (size_t)1 << p->log2_nout;
+    size_t cap = 4 * n_out;                                   // the exact start: causal attention over 4 n_out tokens
+    const int R = [&]() { size_t v = n_out; int r = 0; while (v < (size_t)p->n_kv) { v *= 4; ++r; } return r; }();
+    for (int r = 1; r < R; ++r) {
+        const int q = 2 * r < mbar ? 2 * r : mbar;
+        // E (up to 3 n_out before the third sibling ends), up to three call outputs in each S_i, the tail
+        size_t len = 3 * n_out + ((n_out << 2) >> q);
+        for (int i = 1; i < q; ++i) len += 3 * (((n_out << 2) >> q) << (i - 1)) / 2;
+        if (len > cap) cap = len;
+    }
+    return cap;
+}
+static ExpressLayout express_layout(const elm_params *p, int mbar = 0, bool prefill = false)
 {
     ExpressLayout L;
     const size_t ts = p->precision == ELM_PREC_FP64_DET ? 8 : 4;
@@ -766,6 +786,16 @@ static ExpressLayout express_layout(const elm_params *p)
     L.rdecay = take(BH * (n / 2 + 1) * ts);
     L.F_stride = 4 * n_out * n_out;        // the first halving of E is one call of 2 n_out pairs
     L.F = take(BH * L.F_stride * ts);
+    L.levels = L.ep_idx = L.ep_w = L.ws_attend = L.ep_cap = 0;
+    L.n_levels = 0;
+    if (prefill) {
+        L.n_levels = mbar < 30 ? mbar : 30;
+        L.levels = take((size_t)L.n_levels * BH * n * 4);
+        L.ep_cap = express_epoch_cap(p, mbar);
+        L.ep_idx = take(BH * L.ep_cap * 4);
+        L.ep_w = take(BH * L.ep_cap * 4);
+        L.ws_attend = take(attend_layout(p, (int32_t)L.ep_cap).total);
+    }
     L.total = off;
     return L;
 }
@@ -825,11 +855,58 @@ static double kh_express_delta(double delta, int m)
     return 0.5 * delta * (1.0 / log2(0.5 * m + 2.0) - 1.0 / log2(0.5 * m + 3.0));
 }
 
+// One epoch's cache list: up to 16 pieces laid end to end, each either a run of a point list
+// (src != NULL: entries src[problem * src_stride + src_off ...]) or a run of consecutive tokens.
+struct ListPieces {
+    const int32_t *src[16];
+    int64_t src_off[16];        // offset into the list, or the first token of a run
+    int32_t dst_off[17];        // dst_off[k+1] - dst_off[k] entries
+    float w[16];
+    int n;
+};
+__global__ void build_list_kernel(ListPieces pc, int64_t src_stride, int32_t *__restrict__ idx, float *__restrict__ w,
+                                  int64_t cap)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= pc.dst_off[pc.n]) return;
+    int k = 0;
+    while (i >= pc.dst_off[k + 1]) ++k;
+    const int64_t o = i - pc.dst_off[k];
+    const int64_t pr = blockIdx.y;
+    idx[pr * cap + i] = pc.src[k] ? pc.src[k][pr * src_stride + pc.src_off[k] + o] : (int32_t)(pc.src_off[k] + o);
+    w[pr * cap + i] = pc.w[k];
+}
+
+// Attention of the query rows [t0, t0 + rows) over the list described by `pc` (the last piece is
+// the causal tail: those same tokens).  Thinformer Express, Algorithm 5, in prefill.
+static int express_attend_epoch(const void *Q, const void *K, const void *V, void *O, const elm_params *p, const ExpressLayout &L,
+                                unsigned char *ws, const ListPieces &pc, int64_t t0, int rows, cudaStream_t st)
+{
+    const int BH = p->batch * p->kv_heads;
+    const int total = pc.dst_off[pc.n];
+    int32_t *ep_idx = reinterpret_cast<int32_t *>(ws + L.ep_idx);
+    float *ep_w = reinterpret_cast<float *>(ws + L.ep_w);
+    if ((size_t)total > L.ep_cap) return ELM_ERR_WORKSPACE;
+    // elm_attend takes dense [problem][n_core] lists
+    build_list_kernel<<<dim3((unsigned)((total + 255) / 256), (unsigned)BH), 256, 0, st>>>(pc, p->n_kv, ep_idx, ep_w, total);
+    count_launches(1);
+    ELM_CUDA_TRY(cudaGetLastError());
+    elm_params pe = *p;
+    pe.n_q = rows;
+    AttendWindow win;
+    win.q_row0 = t0;
+    win.n_q_total = p->n_kv;
+    win.tail_start = pc.dst_off[pc.n - 1];
+    return attend_enqueue(Q, K, V, ep_idx, ep_w, total, &pe, O, ws + L.ws_attend, st, win);
+}
+
 template <typename Tin, typename T>
 static int express_impl(const Tin *K, const Tin *V, const elm_params *p, int mbar, uint64_t seed, int32_t *idx_out,
-                        float *w_out, unsigned char *ws, cudaStream_t st, uint32_t pbase)
+                        float *w_out, unsigned char *ws, cudaStream_t st, uint32_t pbase, const Tin *Q = nullptr,
+                        Tin *O = nullptr)
 {
-    const ExpressLayout L = express_layout(p);
+    const bool prefill = Q != nullptr;
+    const ExpressLayout L = express_layout(p, mbar, prefill);
     const int BH = p->batch * p->kv_heads;
     const int64_t n = p->n_kv;
     const int64_t n_out = (int64_t)1 << p->log2_nout;
@@ -856,6 +933,18 @@ static int express_impl(const Tin *K, const Tin *V, const elm_params *p, int mba
         count_launches(2);
         ELM_CUDA_TRY(cudaGetLastError());
     }
+    int32_t *levels = reinterpret_cast<int32_t *>(ws + L.levels);
+    if (prefill) {
+        // Exact phase and round 0 (thinning factor 1: nothing is dropped): each of the first 4 n_out
+        // tokens attends over all tokens up to itself (Theorem 3's exact regime).
+        ListPieces pc = {};
+        const int rows = (int)(n < 4 * n_out ? n : 4 * n_out);
+        pc.n = 1;
+        pc.src[0] = nullptr; pc.src_off[0] = 0; pc.w[0] = 1.f;
+        pc.dst_off[0] = 0; pc.dst_off[1] = rows;
+        const int rc = express_attend_epoch(Q, K, V, O, p, L, ws, pc, 0, rows, st);
+        if (rc != ELM_OK) return rc;
+    }
     for (int r = 0; r < R; ++r) {
         const int m = 2 * r, q = m < mbar ? m : mbar;
         const int64_t seg = n_out << m, len0 = n_out << q;
@@ -876,14 +965,53 @@ static int express_impl(const Tin *K, const Tin *V, const elm_params *p, int mba
             count_launches(1);
             ELM_CUDA_TRY(cudaGetLastError());
         } else {
+            // level i reads list i and writes list i + 1; the prefill keeps every list of the round
+            // (the cache of an epoch is made of runs of them), compression alone alternates two
             int32_t *cur = listA, *nxt = listB;
             for (int i = 0; i < q; ++i) {
                 const int per = 1 << (2 * (q - 1 - i));                       // calls per sibling
                 const int P = (int)((len0 >> i) / per / 2);
                 const double dlt = ldexp(dm, 2 * (i + 1 - q)) / (3.0 * (double)q);
+                if (prefill) nxt = levels + (size_t)i * BH * n;
                 const int rc = run_halve_level<Tin, T>(c, cur, i == q - 1 ? E + n_out : nxt, n, 3 * per, P, i + code1, dlt, per);
                 if (rc != ELM_OK) return rc;
                 int32_t *tmp = cur; cur = nxt; nxt = tmp;
+            }
+        }
+        if (prefill && r >= 1) {
+            // Thinformer Express (Algorithm 5) for the 3 n_out 2^m tokens of this round.  Between two
+            // level-0 Halve calls ("epoch": s_0 = n_out 2^(2-q) tokens) the cache is fixed except for
+            // the growing S_0: E with the finished siblings (weight 1), in S_i the outputs of the
+            // level-(i-1) calls that level i has not consumed yet (weight 2^(i-q)), and the epoch's
+            // own tokens up to the query (weight 2^-q).
+            if (m > mbar) return ELM_ERR_SHAPE;                               // subsampled rounds: not built yet
+            const int64_t s0 = (n_out << 2) >> q;
+            const int epochs = 1 << (2 * (q - 1));
+            for (int jj = 0; jj < 3; ++jj) {
+                for (int e = 0; e < epochs; ++e) {
+                    ListPieces pc = {};
+                    int k = 0;
+                    int32_t at = 0;
+                    auto piece = [&](const int32_t *src, int64_t off, int64_t count, float wgt) {
+                        if (count <= 0) return;
+                        pc.src[k] = src; pc.src_off[k] = off; pc.w[k] = wgt; pc.dst_off[k] = at;
+                        at += (int32_t)count;
+                        ++k;
+                    };
+                    piece(E, 0, (1 + jj) * n_out, 1.f);
+                    for (int i = q - 1; i >= 1; --i) {
+                        const int64_t u = (s0 << (i - 1)) >> 1;              // output of one level-(i-1) call
+                        const int64_t done = e >> (2 * (i - 1)), used = 4 * (int64_t)(e >> (2 * i));
+                        piece(levels + (size_t)(i - 1) * BH * n, jj * (len0 >> i) + used * u, (done - used) * u,
+                              (float)ldexp(1.0, i - q));
+                    }
+                    const int64_t t0 = (jj + 1) * seg + e * s0;
+                    piece(nullptr, t0, s0, (float)ldexp(1.0, -q));            // the causal tail
+                    pc.dst_off[k] = at;
+                    pc.n = k;
+                    const int rc = express_attend_epoch(Q, K, V, O, p, L, ws, pc, t0, (int)s0, st);
+                    if (rc != ELM_OK) return rc;
+                }
             }
         }
         // halve phase: 4 n_out -> 2 n_out -> n_out
@@ -968,4 +1096,53 @@ extern "C" int elm_express_compress(const void *K, const void *V, const elm_para
     }
     return det ? express_impl<__nv_bfloat16, double>((const __nv_bfloat16 *)K, (const __nv_bfloat16 *)V, params, mbar, seed, idx_out, w_out, ws, st, 0u)
                : express_impl<__nv_bfloat16, float>((const __nv_bfloat16 *)K, (const __nv_bfloat16 *)V, params, mbar, seed, idx_out, w_out, ws, st, 0u);
+}
+
+namespace elm {
+// what the prefill needs on top of validate_express
+static int validate_prefill(const elm_params *p, int32_t mbar)
+{
+    int rc = validate_express(p, mbar);
+    if (rc != ELM_OK) return rc;
+    if (p->q_heads < 1 || p->q_heads % p->kv_heads != 0 || (int64_t)p->batch * p->q_heads > 65535) return ELM_ERR_SHAPE;
+    if (p->n_q != p->n_kv) return ELM_ERR_SHAPE;                       // one query per token
+    const int R = express_rounds(p);
+    if (R >= 2 && 2 * (R - 1) > mbar) return ELM_ERR_SHAPE;               // subsampled rounds: attention not built yet
+    if (R >= 2 && 2 * (R - 1) > p->log2_nout + 1) return ELM_ERR_SHAPE;   // level-0 calls of at least 2 points
+    return ELM_OK;
+}
+}  // namespace elm
+
+extern "C" int elm_express_prefill_workspace_bytes(const elm_params *params, int32_t mbar, size_t *bytes)
+{
+    using namespace elm;
+    if (!params || !bytes) return ELM_ERR_NULL;
+    const int rc = validate_prefill(params, mbar);
+    if (rc != ELM_OK) return rc;
+    *bytes = express_layout(params, mbar, true).total;
+    return ELM_OK;
+}
+
+extern "C" int elm_express_prefill(const void *Q, const void *K, const void *V, const elm_params *params, int32_t mbar,
+                                   uint64_t seed, void *O, int32_t *idx_out, float *w_out, void *workspace,
+                                   size_t workspace_bytes, void *stream)
+{
+    using namespace elm;
+    if (!params) return ELM_ERR_NULL;
+    const int rc = validate_prefill(params, mbar);
+    if (rc != ELM_OK) return rc;
+    if (!Q || !K || !V || !O || !idx_out || !w_out || !workspace) return ELM_ERR_NULL;
+    if (((uintptr_t)Q | (uintptr_t)K | (uintptr_t)V | (uintptr_t)O | (uintptr_t)idx_out | (uintptr_t)w_out) & 15) return ELM_ERR_ALIGN;
+    if ((uintptr_t)workspace & 255) return ELM_ERR_ALIGN;
+    if (workspace_bytes < express_layout(params, mbar, true).total) return ELM_ERR_WORKSPACE;
+    unsigned char *ws = (unsigned char *)workspace;
+    cudaStream_t st = (cudaStream_t)stream;
+    const bool det = params->precision == ELM_PREC_FP64_DET;
+    typedef __nv_bfloat16 bf;
+    if (params->dtype == ELM_F32) {
+        return det ? express_impl<float, double>((const float *)K, (const float *)V, params, mbar, seed, idx_out, w_out, ws, st, 0u, (const float *)Q, (float *)O)
+                   : express_impl<float, float>((const float *)K, (const float *)V, params, mbar, seed, idx_out, w_out, ws, st, 0u, (const float *)Q, (float *)O);
+    }
+    return det ? express_impl<bf, double>((const bf *)K, (const bf *)V, params, mbar, seed, idx_out, w_out, ws, st, 0u, (const bf *)Q, (bf *)O)
+               : express_impl<bf, float>((const bf *)K, (const bf *)V, params, mbar, seed, idx_out, w_out, ws, st, 0u, (const bf *)Q, (bf *)O);
 }

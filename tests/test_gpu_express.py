@@ -94,3 +94,72 @@ def test_express_rejects_lengths_that_are_not_nout_times_a_power_of_four():
     _, K, V = generate(wl, seed=1, want_q=False)
     with pytest.raises(elm.ElmError):
         elm.express_compress(K.cuda(), V.cuda(), 4, 2, seed=1)          # 128 = 16 * 8
+
+
+# ----------------------------------------------------------------------------------------------
+# Thinformer Express in prefill: every token's output against the streaming oracle's
+# ----------------------------------------------------------------------------------------------
+# name -> (workload, log2_nout, rounds R, mbar, q heads per KV head)
+PREFILL_CASES = {
+    # exact regime only (n = 4 n_out): causal attention
+    "iid_f32_nout32_R1": (WORKLOADS["cfg1"].scaled(q_heads=1, kv_heads=1), 5, 1, 4, 1),
+    # one thinned round (m = 2: 4 epochs per segment, S_1 fills and empties)
+    "mixture_f32_nout16_R2": (WORKLOADS["cfg2"].scaled(batch=1, q_heads=2, kv_heads=1), 4, 2, 2, 2),
+    # two thinned rounds (m = 4: 64 epochs per segment, three Compress2 levels in the cache)
+    "lowrank_bf16_nout32_R3": (WORKLOADS["cfg3"].scaled(batch=1, q_heads=2, kv_heads=2), 5, 3, 4, 1),
+    # tensor-core path with blocks of 128 list entries, grouped queries
+    "mixture_t3_bf16_nout256_R2": (WORKLOADS["cfg5"].scaled(q_heads=4, kv_heads=2), 8, 2, 6, 2),
+}
+PREFILL_TOL = {("f32", "fp64"): 2e-6, ("f32", "fp32"): 1e-4, ("bf16", "fp64"): 1e-2, ("bf16", "fp32"): 2e-2}
+
+
+def _prefill_inputs(name):
+    wl, log2_nout, R, mbar, rep = PREFILL_CASES[name]
+    n = (1 << log2_nout) * 4 ** R
+    wl = wl.scaled(n=n, n_q=n, q_heads=wl.kv_heads * rep)
+    Q, K, V = generate(wl, seed=777, want_q=True)
+    return wl, Q, K, V, log2_nout, mbar
+
+
+@pytest.mark.parametrize("precision", ["fp64", "fp32"])
+@pytest.mark.parametrize("name", sorted(PREFILL_CASES))
+def test_express_prefill_outputs_match_streaming_oracle(name, precision):
+    from _util import max_rel_err
+    wl, Q, K, V, log2_nout, mbar = _prefill_inputs(name)
+    O, idx, _ = elm.express_prefill(Q.cuda(), K.cuda(), V.cuda(), log2_nout, mbar, seed=9, precision=precision)
+    torch.cuda.synchronize()
+    got = O.float().cpu().numpy()
+    Qf, Kf, Vf = as_f32_numpy(Q), as_f32_numpy(K), as_f32_numpy(V)
+    B, Hq, n, d = Qf.shape
+    H = Kf.shape[1]
+    worst = 0.0
+    for b in range(B):
+        for h in range(Hq):
+            kv = (h * H) // Hq
+            r = oracle.thinformer_express(Qf[b, h], Kf[b, kv], Vf[b, kv], log2_nout, mbar, seed=9, head=b * H + kv)
+            if precision == "fp64":
+                assert np.array_equal(idx[b, kv].cpu().numpy(), r["final_idx"])
+                worst = max(worst, max_rel_err(got[b, h], r["O"]))
+            else:
+                # fp32 mode may (rarely) pick another coreset; then the outputs legitimately differ
+                if np.array_equal(idx[b, kv].cpu().numpy(), r["final_idx"]):
+                    worst = max(worst, max_rel_err(got[b, h], r["O"]))
+    print(f"{name} {precision}: max relative error of the prefill outputs {worst:.3e}")
+    assert worst <= PREFILL_TOL[(wl.dtype if wl.dtype == "bf16" else "f32", precision)]
+
+
+def test_express_prefill_first_tokens_equal_exact_causal_attention():
+    """Theorem 3: the first 4 n_out outputs are exact causal attention."""
+    from _util import max_rel_err
+    wl, Q, K, V, log2_nout, mbar = _prefill_inputs("mixture_f32_nout16_R2")
+    O, _, _ = elm.express_prefill(Q.cuda(), K.cuda(), V.cuda(), log2_nout, mbar, seed=3, precision="fp64")
+    m = 4 << log2_nout
+    ref = oracle.exact_causal_attention(as_f32_numpy(Q)[0, 0, :m], as_f32_numpy(K)[0, 0, :m], as_f32_numpy(V)[0, 0, :m])
+    assert max_rel_err(O[0, 0, :m].float().cpu().numpy(), ref) <= 2e-6
+
+
+def test_express_prefill_rejects_subsampled_rounds():
+    wl = WORKLOADS["cfg1"].scaled(n=16 * 64, n_q=16 * 64)
+    Q, K, V = generate(wl, seed=1, want_q=True)
+    with pytest.raises(elm.ElmError):
+        elm.express_prefill(Q.cuda(), K.cuda(), V.cuda(), 4, 2, seed=1)      # R = 3 needs mbar >= 4
