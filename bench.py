@@ -200,9 +200,10 @@ def main():
     ap.add_argument("--ref-heads", type=int, default=None)
     ap.add_argument("--override", default="", help="comma list of Workload fields for small profiling "
                     "captures, e.g. q_heads=8,kv_heads=2,n=32768,n_q=32768 (the line then names the scaled case)")
-    ap.add_argument("--only", default="both", choices=["both", "compress", "attend", "express"],
-                    help="run one half of the step, or the Offline-Express compression of the same keys and "
-                         "values with mbar = log2(n_out) - 2 instead of the step (profiling captures only)")
+    ap.add_argument("--only", default="both", choices=["both", "compress", "attend", "express", "prefill"],
+                    help="run one half of the step; or, instead of the step, the Offline-Express compression "
+                         "(express) or the Thinformer Express prefill (prefill) of the same inputs with "
+                         "mbar = log2(n_out) - 2 (profiling captures only)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -249,6 +250,10 @@ def main():
     def step(seed):
         if flush is not None:
             flush.zero_()
+        if args.only == "prefill":
+            elm.express_prefill(Qd, Kd, Vd, wl.log2_nout, wl.log2_nout - 2, seed=seed, precision=args.precision,
+                                workspace=state.setdefault("ws_p", None), out=O)
+            return
         if args.only == "express":
             state["idx"], state["w"] = elm.express_compress(Kd, Vd, wl.log2_nout, wl.log2_nout - 2, seed=seed,
                                                             precision=args.precision, workspace=state.get("ws_x"))

@@ -745,11 +745,12 @@ static int compress_impl(const Tin *K, const Tin *V, const elm_params *p, uint64
 //                61 + 64 (4 r + j)         the stratified draws of sibling j (first word = stratum).
 // v_max is taken over the whole sequence.
 // ---------------------------------------------------------------------------------------------
+constexpr int EXPRESS_LANES = 6;       // side streams of the prefill: two per sibling segment
 struct ExpressLayout {
     size_t vmax_bits, cnorm, listA, listB, E, T1, Mpair, rdecay, F, F_stride, total;
     // prefill only: the output lists of every Compress2 level of a round, the cache list of one
     // epoch with its weights, the workspace of elm_attend for that list
-    size_t levels, ep_idx, ep_w, ws_attend, ep_cap;
+    size_t levels, ep_idx, ep_w, ws_attend, ep_cap, ep_stride, ws_attend_stride;
     int n_levels;
 };
 // Longest cache list (weighted cache + causal tail) any epoch of the prefill attends over.
@@ -786,15 +787,18 @@ static ExpressLayout express_layout(const elm_params *p, int mbar = 0, bool pref
     L.rdecay = take(BH * (n / 2 + 1) * ts);
     L.F_stride = 4 * n_out * n_out;        // the first halving of E is one call of 2 n_out pairs
     L.F = take(BH * L.F_stride * ts);
-    L.levels = L.ep_idx = L.ep_w = L.ws_attend = L.ep_cap = 0;
+    L.levels = L.ep_idx = L.ep_w = L.ws_attend = L.ep_cap = L.ep_stride = L.ws_attend_stride = 0;
     L.n_levels = 0;
     if (prefill) {
         L.n_levels = mbar < 30 ? mbar : 30;
         L.levels = take((size_t)L.n_levels * BH * n * 4);
         L.ep_cap = express_epoch_cap(p, mbar);
-        L.ep_idx = take(BH * L.ep_cap * 4);
-        L.ep_w = take(BH * L.ep_cap * 4);
-        L.ws_attend = take(attend_layout(p, (int32_t)L.ep_cap).total);
+        // one set per side stream: the epochs of a round are spread over EXPRESS_LANES streams
+        L.ep_stride = align_up(BH * L.ep_cap * 4, 256);
+        L.ep_idx = take(EXPRESS_LANES * L.ep_stride);
+        L.ep_w = take(EXPRESS_LANES * L.ep_stride);
+        L.ws_attend_stride = align_up(attend_layout(p, (int32_t)L.ep_cap).total, 256);
+        L.ws_attend = take(EXPRESS_LANES * L.ws_attend_stride);
     }
     L.total = off;
     return L;
@@ -880,12 +884,12 @@ __global__ void build_list_kernel(ListPieces pc, int64_t src_stride, int32_t *__
 // Attention of the query rows [t0, t0 + rows) over the list described by `pc` (the last piece is
 // the causal tail: those same tokens).  Thinformer Express, Algorithm 5, in prefill.
 static int express_attend_epoch(const void *Q, const void *K, const void *V, void *O, const elm_params *p, const ExpressLayout &L,
-                                unsigned char *ws, const ListPieces &pc, int64_t t0, int rows, cudaStream_t st)
+                                unsigned char *ws, const ListPieces &pc, int64_t t0, int rows, cudaStream_t st, int lane = 0)
 {
     const int BH = p->batch * p->kv_heads;
     const int total = pc.dst_off[pc.n];
-    int32_t *ep_idx = reinterpret_cast<int32_t *>(ws + L.ep_idx);
-    float *ep_w = reinterpret_cast<float *>(ws + L.ep_w);
+    int32_t *ep_idx = reinterpret_cast<int32_t *>(ws + L.ep_idx + lane * L.ep_stride);
+    float *ep_w = reinterpret_cast<float *>(ws + L.ep_w + lane * L.ep_stride);
     if ((size_t)total > L.ep_cap) return ELM_ERR_WORKSPACE;
     // elm_attend takes dense [problem][n_core] lists
     build_list_kernel<<<dim3((unsigned)((total + 255) / 256), (unsigned)BH), 256, 0, st>>>(pc, p->n_kv, ep_idx, ep_w, total);
@@ -897,7 +901,7 @@ static int express_attend_epoch(const void *Q, const void *K, const void *V, voi
     win.q_row0 = t0;
     win.n_q_total = p->n_kv;
     win.tail_start = pc.dst_off[pc.n - 1];
-    return attend_enqueue(Q, K, V, ep_idx, ep_w, total, &pe, O, ws + L.ws_attend, st, win);
+    return attend_enqueue(Q, K, V, ep_idx, ep_w, total, &pe, O, ws + L.ws_attend + lane * L.ws_attend_stride, st, win);
 }
 
 template <typename Tin, typename T>
@@ -934,6 +938,28 @@ static int express_impl(const Tin *K, const Tin *V, const elm_params *p, int mba
         ELM_CUDA_TRY(cudaGetLastError());
     }
     int32_t *levels = reinterpret_cast<int32_t *>(ws + L.levels);
+    struct SideStreams {                                             // released on every return path
+        cudaStream_t s[EXPRESS_LANES] = {};
+        cudaEvent_t fork = nullptr, join[EXPRESS_LANES] = {};
+        ~SideStreams()
+        {
+            for (int i = 0; i < EXPRESS_LANES; ++i) {
+                if (s[i]) cudaStreamDestroy(s[i]);                   // work already enqueued still completes
+                if (join[i]) cudaEventDestroy(join[i]);
+            }
+            if (fork) cudaEventDestroy(fork);
+        }
+    } sides;
+    cudaStream_t *side = sides.s;
+    cudaEvent_t &fork = sides.fork;
+    cudaEvent_t *join = sides.join;
+    if (prefill && R >= 2) {
+        ELM_CUDA_TRY(cudaEventCreateWithFlags(&fork, cudaEventDisableTiming));
+        for (int i = 0; i < EXPRESS_LANES; ++i) {
+            ELM_CUDA_TRY(cudaStreamCreateWithFlags(&side[i], cudaStreamNonBlocking));
+            ELM_CUDA_TRY(cudaEventCreateWithFlags(&join[i], cudaEventDisableTiming));
+        }
+    }
     if (prefill) {
         // Exact phase and round 0 (thinning factor 1: nothing is dropped): each of the first 4 n_out
         // tokens attends over all tokens up to itself (Theorem 3's exact regime).
@@ -987,8 +1013,15 @@ static int express_impl(const Tin *K, const Tin *V, const elm_params *p, int mba
             if (m > mbar) return ELM_ERR_SHAPE;                               // subsampled rounds: not built yet
             const int64_t s0 = (n_out << 2) >> q;
             const int epochs = 1 << (2 * (q - 1));
+            // An epoch's launch has one work item per 256 of its s_0 tokens and head - too few for the
+            // GPU when s_0 is small - and all epochs of a round are independent given the round's lists:
+            // they are dealt to EXPRESS_LANES streams (each with its own list buffers) between two events.
+            ELM_CUDA_TRY(cudaEventRecord(fork, st));
+            for (int i = 0; i < EXPRESS_LANES; ++i) ELM_CUDA_TRY(cudaStreamWaitEvent(side[i], fork, 0));
             for (int jj = 0; jj < 3; ++jj) {
                 for (int e = 0; e < epochs; ++e) {
+                    const int lane_id = (jj * epochs + e) % EXPRESS_LANES;
+                    cudaStream_t sj = side[lane_id];
                     ListPieces pc = {};
                     int k = 0;
                     int32_t at = 0;
@@ -1009,9 +1042,13 @@ static int express_impl(const Tin *K, const Tin *V, const elm_params *p, int mba
                     piece(nullptr, t0, s0, (float)ldexp(1.0, -q));            // the causal tail
                     pc.dst_off[k] = at;
                     pc.n = k;
-                    const int rc = express_attend_epoch(Q, K, V, O, p, L, ws, pc, t0, (int)s0, st);
+                    const int rc = express_attend_epoch(Q, K, V, O, p, L, ws, pc, t0, (int)s0, sj, lane_id);
                     if (rc != ELM_OK) return rc;
                 }
+            }
+            for (int i = 0; i < EXPRESS_LANES; ++i) {
+                ELM_CUDA_TRY(cudaEventRecord(join[i], side[i]));
+                ELM_CUDA_TRY(cudaStreamWaitEvent(st, join[i], 0));             // the halvings overwrite E
             }
         }
         // halve phase: 4 n_out -> 2 n_out -> n_out
