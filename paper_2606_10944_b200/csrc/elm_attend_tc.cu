@@ -423,6 +423,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
         // quarters exchange their row maxima (and, at the end, their denominators) through shared
         // memory, in a buffer per tile so that a value is overwritten only two barriers later.
         const int cq = warp >> 2;                                  // column quarter
+        const bool has_tail = tail_start != 0x7fffffff;
         const int row = (warp & 3) * 32 + lane;                    // row in the tile = TMEM lane
         const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
         bool ok = true;
@@ -438,11 +439,15 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                 for (int t = 0; t < 2; ++t) {
                     // A row sees the list up to its own entry of the causal tail (if there is one), so
                     // the visible columns are a prefix of the list; of this thread's 32, `valid` exist.
-                    const int64_t seen = (int64_t)tail_start + q0 + t * BM + row + 1;
-                    const int valid = (int)(seen < n_core ? seen : n_core) - j * BN - cq * 32;
-                    // per-column bias and/or a ragged end; warp-uniform, because both forms of the two
-                    // passes contain warp-collective TMEM loads
-                    const bool special = use_bias || __any_sync(0xffffffffu, valid < 32);
+                    int valid = n_core - j * BN - cq * 32;
+                    bool ragged = valid < 32;
+                    if (has_tail) {
+                        const int64_t seen = (int64_t)tail_start + q0 + t * BM + row + 1;
+                        if (seen < n_core) valid = (int)seen - j * BN - cq * 32;
+                        // warp-uniform, because both forms of the two passes contain warp-collective TMEM loads
+                        ragged = __any_sync(0xffffffffu, valid < 32);
+                    }
+                    const bool special = use_bias || ragged;           // per-column bias and/or a ragged end
                     const uint32_t tS = tmem + lane_addr + t * 128 + cq * 32;   // this thread's 32 logit columns
                     const uint32_t tP = tS;                 // their bf16 probabilities overwrite the first 16 of them
                     const uint32_t tO = tmem + lane_addr + 256 + t * 128 + cq * (D / 4);   // its quarter of the accumulator
