@@ -200,10 +200,11 @@ def main():
     ap.add_argument("--ref-heads", type=int, default=None)
     ap.add_argument("--override", default="", help="comma list of Workload fields for small profiling "
                     "captures, e.g. q_heads=8,kv_heads=2,n=32768,n_q=32768 (the line then names the scaled case)")
-    ap.add_argument("--only", default="both", choices=["both", "compress", "attend", "express", "prefill"],
+    ap.add_argument("--only", default="both", choices=["both", "compress", "attend", "express", "prefill", "decode"],
                     help="run one half of the step; or, instead of the step, the Offline-Express compression "
                          "(express) or the Thinformer Express prefill (prefill) of the same inputs with "
-                         "mbar = log2(n_out) - 2 (profiling captures only)")
+                         "mbar = log2(n_out) - 2; or (decode) one query per head over a cache of n_out and of "
+                         "6 n_out entries, printed as its own JSON line (profiling captures only)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -244,6 +245,44 @@ def main():
     O = torch.empty_like(Qd)
     small_inputs = not wl.name.startswith(("cfg4", "cfg5"))
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev) if small_inputs else None
+
+    if args.only == "decode":
+        # one new token per head over a weighted cache: HBM-bound; bytes = the cache rows of K and V once
+        peaks = load_peaks()
+        es = 2 if wl.dtype == "bf16" else 4
+        q1 = Qd[:, :, :1, :].contiguous()
+        out = []
+        for n_core in (wl.n_out, 6 * wl.n_out):
+            g = torch.Generator().manual_seed(7)
+            idx = torch.stack([torch.randperm(wl.n, generator=g)[:n_core] for _ in range(wl.batch * wl.kv_heads)])
+            idx = idx.reshape(wl.batch, wl.kv_heads, n_core).to(torch.int32).cuda()
+            w = (torch.rand(wl.batch, wl.kv_heads, n_core, generator=g) + 0.05).cuda()
+            p1, _ = elm.make_params(wl.batch, wl.q_heads, wl.kv_heads, wl.n, 1, wl.d, wl.log2_nout, wl.m,
+                                    1 if wl.dtype == "bf16" else 0, args.precision)
+            ws1 = torch.empty(elm.attend_workspace_bytes(p1, n_core), dtype=torch.uint8, device=dev)
+            o1 = torch.empty_like(q1)
+            for _ in range(warmup):
+                elm.attend(q1, Kd, Vd, idx, w, precision=args.precision, workspace=ws1, out=o1)
+            reps = max(args.steps, 20)
+            big = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+
+            # device time from the library's own stage events (recorded around the two launches of a
+            # call on its stream): the Python call itself takes longer than the kernels
+            elm.profile_enable(True)
+            for _ in range(reps):
+                big.zero_()                                      # the cache rows leave L2 between tokens
+                elm.attend(q1, Kd, Vd, idx, w, precision=args.precision, workspace=ws1, out=o1)
+            torch.cuda.synchronize()
+            total = elm.profile_read()["attend"][0]
+            elm.profile_enable(False)
+            us = total / reps * 1e3
+            nbytes = wl.batch * wl.kv_heads * n_core * (2 * wl.d * es + 8)
+            gbs = nbytes / (us * 1e-6) / 1e9
+            out.append({"n_core": n_core, "us_per_token": us, "algorithmic_bytes": nbytes, "achieved_GBps": gbs,
+                        "frac_of_measured_hbm": gbs / peaks["hbm_gbs"]})
+        if rank == 0:
+            print(json.dumps({"decode": out, "config": workload_config(wl, args), "l2": "256 MiB written between tokens"}))
+        return
 
     state = {}
 

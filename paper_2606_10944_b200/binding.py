@@ -209,6 +209,13 @@ def express_prefill(Q, K, V, log2_nout: int, mbar: int, seed: int = 1, precision
     return O, idx, w
 
 
+def attend_workspace_bytes(params: ElmParams, n_core: int) -> int:
+    need = ctypes.c_size_t(0)
+    _check(load_library().elm_attend_workspace_bytes(ctypes.byref(params), n_core, ctypes.byref(need)),
+           "elm_attend_workspace_bytes")
+    return int(need.value)
+
+
 def attend(Q, K, V, idx, w, precision="fp32", workspace=None, out=None):
     """elm_attend: Q [B, Hq, nq, d]; K, V [B, Hkv, n, d]; idx, w [B, Hkv, n_core] -> O like Q."""
     lib = load_library()

@@ -287,6 +287,8 @@ int attend_enqueue(const void *Q, const void *K, const void *V, const int32_t *i
 {
     unsigned char *ws = (unsigned char *)workspace;
     const bool det = params->precision == ELM_PREC_FP64_DET;
+    const bool whole = win.q_row0 == 0 && win.n_q_total == 0 && win.tail_start == 0x7fffffff;
+    if (whole && attend_decode_applies(params)) return attend_decode(Q, K, V, idx, w, n_core, params, O, ws, st, true);
     if (params->dtype == ELM_F32) {
         return det ? attend_impl<float, double>((const float *)Q, (const float *)K, (const float *)V, idx, w, n_core, params, (float *)O, ws, st, win)
                    : attend_impl<float, float>((const float *)Q, (const float *)K, (const float *)V, idx, w, n_core, params, (float *)O, ws, st, win);
@@ -343,6 +345,7 @@ extern "C" int elm_attend_static(const void *Q, const void *K, const void *V, co
     if (rc != ELM_OK) return rc;
     cudaStream_t st = (cudaStream_t)stream;
     const bool det = params->precision == ELM_PREC_FP64_DET;
+    if (attend_decode_applies(params)) return attend_decode(Q, K, V, idx, w, n_core, params, O, scratch, st, false);
     if (params->dtype == ELM_F32) {
         return det ? attend_enqueue_untimed<float, double>((const float *)Q, (const float *)K, (const float *)V, idx, w, n_core, params, (float *)O, scratch, st)
                    : attend_enqueue_untimed<float, float>((const float *)Q, (const float *)K, (const float *)V, idx, w, n_core, params, (float *)O, scratch, st);

@@ -188,6 +188,23 @@ def test_attend_arbitrary_weights_and_ragged_shapes(dtype, d, n_core, n_q, hq, h
         assert err <= tol, (precision, err)
 
 
+@pytest.mark.parametrize("dtype,d,n_core,n_q,hq,hkv", [
+    ("bf16", 128, 2048, 1, 8, 2),     # decode: one new token, 4 query heads per KV head
+    ("bf16", 128, 12288, 1, 4, 4),    # a full Express cache (6 n_out entries), no grouping
+    ("f32", 64, 301, 2, 4, 1),        # 8 query vectors per KV head, ragged list
+    ("bf16", 64, 1, 3, 2, 2),         # single entry
+    ("f32", 128, 70, 1, 1, 1),        # list shorter than one CTA's share
+    ("bf16", 128, 4096, 5, 8, 8),     # 5 rows per head (odd count, padded to 8 vectors)
+])
+def test_attend_few_queries_takes_the_decode_kernels(dtype, d, n_core, n_q, hq, hkv):
+    """(q_heads / kv_heads) * n_q <= 8 in fp32 mode: the HBM-bound decode kernels, same tolerances."""
+    wl = WORKLOADS["cfg2"].scaled(batch=2, q_heads=hq, kv_heads=hkv, n=16384, n_q=n_q, d=d, dtype=dtype)
+    before = elm.launch_count()
+    err, tol = _attend_case(wl, "fp32", weights="random", n_core=n_core)
+    assert elm.launch_count() - before == 2          # partial + merge: no gather launch
+    assert err <= tol, err
+
+
 def test_attend_weight_scale_invariance_and_single_point():
     wl = WORKLOADS["cfg2"].scaled(batch=1, q_heads=2, kv_heads=2, n=1024, n_q=100)
     Q, K, V = generate(wl, seed=5)
