@@ -198,6 +198,45 @@ int elm_express_compress(const void *K, const void *V, const elm_params *params,
                          int32_t *idx_out, float *w_out, void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * Streaming Thinformer Express (Algorithms 1, 2 and 5 with Halve = KH(delta) at the failure parameters
+ * of Corollary 2), one token per call: elm_stream_step first attends the new token's queries over the
+ * weighted cache plus the token itself, then feeds the token's key-value pair to the cache
+ * (Express.update: exact phase, Compress2 levels S_0..S_q with a Halve call whenever a level is full,
+ * hand-over to E at the end of a thin phase, two halvings of E at the end of a round).  The cache never
+ * exceeds 6 n_out points.  After n_out 4^R tokens it equals the result of elm_express_compress, and
+ * every output equals elm_express_prefill's.
+ *   elm_stream     plain HOST struct owned by the caller; elm_stream_init fills it, the library keeps no
+ *                  other state.  All arrays live in the caller's device workspace.
+ *   params         batch, q_heads, kv_heads, d, log2_nout, dtype, precision, delta as elsewhere; n_kv is
+ *                  the CAPACITY (rows of K and V per problem); n_q must be 1.
+ *   K, V           [batch][kv_heads][n_kv][d]; row t must be valid when step t is enqueued.
+ *   n_known        rows of K and V already valid at init: v_max of Eq. (katt) starts as the largest
+ *                  |v| over them and grows with the tokens seen later (with n_known = the whole
+ *                  sequence this is the v_max of elm_express_compress).
+ *   Q_t, O_t       [batch][q_heads][1][d]
+ *   Limits         thinning factors above mbar (Subsample active, more than n_out 4^(mbar/2+1) tokens)
+ *                  return ELM_ERR_SHAPE; mbar <= 12.
+ * Calls only enqueue work on `stream`; the host struct is updated immediately (the schedule of Halve
+ * calls depends on the token count alone).
+ */
+typedef struct elm_stream {
+    int64_t n, ell, n_E;          /* tokens seen, tokens of the current thin phase, points in E */
+    int32_t m, b, q, mbar;        /* thinning factor, finished segments of the round, Compress2 depth */
+    int64_t n_S[16], calls[16];   /* points in S_i; Halve calls made at level i of the current Compress2 */
+    int64_t n_known;
+    uint64_t seed;
+} elm_stream;
+int elm_stream_workspace_bytes(const elm_params *params, int32_t mbar, size_t *bytes);
+int elm_stream_init(elm_stream *s, const void *K, const void *V, int64_t n_known, const elm_params *params,
+                    int32_t mbar, uint64_t seed, void *workspace, size_t workspace_bytes, void *stream);
+int elm_stream_step(elm_stream *s, const void *Q_t, const void *K, const void *V, const elm_params *params,
+                    void *O_t, void *workspace, size_t workspace_bytes, void *stream);
+/* The current cache, wtd_cache() of Algorithm 1: at most 6 n_out entries per problem, [batch][kv_heads][count]
+ * row numbers and (unnormalised) weights 2^(i-q) / 1; *count_host receives the number of entries. */
+int elm_stream_cache(const elm_stream *s, const elm_params *params, int32_t *idx_out, float *w_out,
+                     int32_t *count_host, void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * End-to-end convenience call on HOST buffers: copies Q, K, V to the device, runs elm_compress and
  * elm_attend, copies O (and, when non-NULL, idx and w) back, and returns when everything has
  * arrived.  The host link bounds this call, so uploads, kernels and downloads overlap: K and V go

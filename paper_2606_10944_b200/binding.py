@@ -22,6 +22,7 @@ EXPORTED_SYMBOLS = [
     "elm_workspace_bytes", "elm_default_delta_levels", "elm_compress", "elm_attend",
     "elm_attend_workspace_bytes", "elm_attend_static", "elm_express_workspace_bytes", "elm_express_compress",
     "elm_express_prefill_workspace_bytes", "elm_express_prefill",
+    "elm_stream_workspace_bytes", "elm_stream_init", "elm_stream_step", "elm_stream_cache",
     "elm_host_call_scratch_bytes", "elm_compress_attend_host",
     "elm_compress_status", "elm_attend_status", "elm_profile_enable", "elm_profile_read", "elm_launch_count", "elm_strerror", "elm_version",
 ]
@@ -38,6 +39,15 @@ class ElmParams(ctypes.Structure):
         ("log2_nout", ctypes.c_int32), ("m", ctypes.c_int32),
         ("dtype", ctypes.c_int32), ("precision", ctypes.c_int32),
         ("delta", ctypes.c_double), ("delta_level", ctypes.POINTER(ctypes.c_double)),
+    ]
+
+
+class ElmStream(ctypes.Structure):
+    _fields_ = [
+        ("n", ctypes.c_int64), ("ell", ctypes.c_int64), ("n_E", ctypes.c_int64),
+        ("m", ctypes.c_int32), ("b", ctypes.c_int32), ("q", ctypes.c_int32), ("mbar", ctypes.c_int32),
+        ("n_S", ctypes.c_int64 * 16), ("calls", ctypes.c_int64 * 16),
+        ("n_known", ctypes.c_int64), ("seed", ctypes.c_uint64),
     ]
 
 
@@ -70,6 +80,11 @@ def load_library():
     lib.elm_express_compress.argtypes = [vp, vp, pp, ctypes.c_int32, ctypes.c_uint64, vp, vp, vp, sz, vp]
     lib.elm_express_prefill_workspace_bytes.argtypes = [pp, ctypes.c_int32, szp]
     lib.elm_express_prefill.argtypes = [vp, vp, vp, pp, ctypes.c_int32, ctypes.c_uint64, vp, vp, vp, vp, sz, vp]
+    sp = ctypes.POINTER(ElmStream)
+    lib.elm_stream_workspace_bytes.argtypes = [pp, ctypes.c_int32, szp]
+    lib.elm_stream_init.argtypes = [sp, vp, vp, ctypes.c_int64, pp, ctypes.c_int32, ctypes.c_uint64, vp, sz, vp]
+    lib.elm_stream_step.argtypes = [sp, vp, vp, vp, pp, vp, vp, sz, vp]
+    lib.elm_stream_cache.argtypes = [sp, pp, vp, vp, ctypes.POINTER(ctypes.c_int32), vp, sz, vp]
     lib.elm_host_call_scratch_bytes.argtypes = [pp, szp]
     lib.elm_compress_attend_host.argtypes = [vp, vp, vp, vp, vp, vp, pp, ctypes.c_uint64, vp, sz, vp]
     lib.elm_compress_status.argtypes = [vp, pp, ctypes.POINTER(ctypes.c_int32), vp]
@@ -207,6 +222,50 @@ def express_prefill(Q, K, V, log2_nout: int, mbar: int, seed: int = 1, precision
                                    idx.data_ptr(), w.data_ptr(), ws.data_ptr(), ws.numel(), _stream()),
            "elm_express_prefill")
     return O, idx, w
+
+
+class Stream:
+    """elm_stream_*: streaming Thinformer Express over K, V [B, Hkv, capacity, d] (one token per step)."""
+
+    def __init__(self, K, V, q_heads: int, log2_nout: int, mbar: int, seed: int = 1, precision="fp32",
+                 delta: float = 0.5, n_known=None):
+        lib = load_library()
+        _require_cuda(K, V)
+        B, H, n, d = K.shape
+        self.K, self.V = K, V
+        self.params, _ = make_params(B, q_heads, H, n, 1, d, log2_nout, 0, _dtype_code(K), precision, delta)
+        need = ctypes.c_size_t(0)
+        _check(lib.elm_stream_workspace_bytes(ctypes.byref(self.params), mbar, ctypes.byref(need)),
+               "elm_stream_workspace_bytes")
+        self.ws = _workspace(int(need.value), K.device)
+        self.state = ElmStream()
+        _check(lib.elm_stream_init(ctypes.byref(self.state), K.data_ptr(), V.data_ptr(), n if n_known is None else n_known,
+                                   ctypes.byref(self.params), mbar, seed, self.ws.data_ptr(), self.ws.numel(), _stream()),
+               "elm_stream_init")
+
+    def step(self, q_t, out=None):
+        """q_t [B, Hq, 1, d] -> O_t; the token is row state.n of K and V."""
+        O = out if out is not None else torch.empty_like(q_t)
+        _check(load_library().elm_stream_step(ctypes.byref(self.state), q_t.data_ptr(), self.K.data_ptr(), self.V.data_ptr(),
+                                              ctypes.byref(self.params), O.data_ptr(), self.ws.data_ptr(), self.ws.numel(),
+                                              _stream()), "elm_stream_step")
+        return O
+
+    def cache(self):
+        """(idx int32 [B, Hkv, count], w float32 [B, Hkv, count]) of wtd_cache()."""
+        p = self.params
+        cap = 6 * (1 << p.log2_nout) + 1
+        idx = torch.empty((p.batch, p.kv_heads, cap), dtype=torch.int32, device=self.K.device)
+        w = torch.empty((p.batch, p.kv_heads, cap), dtype=torch.float32, device=self.K.device)
+        count = ctypes.c_int32(0)
+        # the library writes dense [problem][count] arrays at the front of the buffers
+        _check(load_library().elm_stream_cache(ctypes.byref(self.state), ctypes.byref(p), idx.data_ptr(), w.data_ptr(),
+                                               ctypes.byref(count), self.ws.data_ptr(), self.ws.numel(), _stream()),
+               "elm_stream_cache")
+        c = int(count.value)
+        flat_i = idx.reshape(-1)[: p.batch * p.kv_heads * c].reshape(p.batch, p.kv_heads, c)
+        flat_w = w.reshape(-1)[: p.batch * p.kv_heads * c].reshape(p.batch, p.kv_heads, c)
+        return flat_i, flat_w
 
 
 def attend_workspace_bytes(params: ElmParams, n_core: int) -> int:

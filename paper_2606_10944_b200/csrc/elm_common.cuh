@@ -85,18 +85,27 @@ __device__ __forceinline__ uint32_t philox4x32_10_word0(uint32_t c0, uint32_t c1
 
 // The uniform of pair `pair` of Halve call `group` at `level` of attention problem `problem`:
 // top 24 bits of the first Philox word, so the value is exact in fp32 and fp64 alike.
-// Second and third counter words of Halve call g of a level.  `lvl` carries the level's third word in
-// its low half; a non-zero high half says that the level batches sibling segments of an Express round
-// with that many calls each: call g is then call g % calls of sibling g / calls, whose third word is
-// 64 further on per sibling.
+// Second and third counter words of Halve call g of a level.  `lvl` packs three fields:
+//   bits  0-15  the level's third counter word,
+//   bits 16-39  the number of the level's first call (a streaming run makes the calls of a level one
+//               launch at a time),
+//   bits 40-63  non-zero when the level batches sibling segments of an Express round with that many
+//               calls each: call g is then call g % calls of sibling g / calls, whose third word is
+//               64 further on per sibling.
+__host__ __device__ __forceinline__ int64_t pack_level(int code, int64_t first_call, int64_t calls_per_sibling)
+{
+    return (int64_t)code | (first_call << 16) | (calls_per_sibling << 40);
+}
 __device__ __forceinline__ void call_counter(int g, int64_t lvl, uint32_t &group, uint32_t &code)
 {
-    const uint32_t per = (uint32_t)(lvl >> 32);
-    code = (uint32_t)lvl;
-    group = (uint32_t)g;
+    const uint32_t per = (uint32_t)(lvl >> 40);
+    code = (uint32_t)lvl & 0xffffu;
+    group = (uint32_t)(lvl >> 16) & 0xffffffu;
     if (per) {
-        group = (uint32_t)g % per;
+        group += (uint32_t)g % per;
         code += 64u * ((uint32_t)g / per);
+    } else {
+        group += (uint32_t)g;
     }
 }
 

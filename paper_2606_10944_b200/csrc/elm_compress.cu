@@ -50,14 +50,16 @@ __global__ void __launch_bounds__(256) prepass_kernel(const Tin *__restrict__ K,
                                                       const Tin *__restrict__ V, int64_t n, int d,
                                                       T *__restrict__ cnorm,
                                                       unsigned *__restrict__ vmax_bits,
-                                                      int32_t *__restrict__ cur)
+                                                      int32_t *__restrict__ cur, int64_t first = 0,
+                                                      int64_t last = -1 /* rows [first, last); -1: n */)
 {
+    if (last < 0) last = n;
     constexpr int EPC = 16 / sizeof(Tin);                 // elements per 16-byte chunk
     const int p = blockIdx.y;
     const int lpr = d / EPC;                              // lanes per row: 8, 16 or 32
     const int rows_per_pass = 256 / lpr;
     const int sub = threadIdx.x % lpr, rloc = threadIdx.x / lpr;
-    const int64_t row0 = (int64_t)blockIdx.x * 256;       // 256 rows per CTA
+    const int64_t row0 = first + (int64_t)blockIdx.x * 256;   // 256 rows per CTA
     const Tin *Kp = K + (int64_t)p * n * d;
     const Tin *Vp = V + (int64_t)p * n * d;
     const T rsd = sqrt((T)d);
@@ -65,9 +67,9 @@ __global__ void __launch_bounds__(256) prepass_kernel(const Tin *__restrict__ K,
     for (int r = rloc; r < 256; r += rows_per_pass) {
         const int64_t t = row0 + r;
         T s = 0;
-        if (t < n) chunk_sq_absmax<T>(Kp + t * d + sub * EPC, Vp + t * d + sub * EPC, s, vm);
+        if (t < last) chunk_sq_absmax<T>(Kp + t * d + sub * EPC, Vp + t * d + sub * EPC, s, vm);
         for (int o = lpr >> 1; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-        if (sub == 0 && t < n) {
+        if (sub == 0 && t < last) {
             cnorm[(int64_t)p * n + t] = s / rsd;
             cur[(int64_t)p * n + t] = (int32_t)t;
         }
@@ -600,9 +602,9 @@ template <typename Tin, typename T> struct LevelCtx {
 // calls_per_sibling > 0 the level holds the calls of several sibling segments (see call_counter).
 template <typename Tin, typename T>
 static int run_halve_level(const LevelCtx<Tin, T> &c, const int32_t *cur, int32_t *out, int64_t out_stride, int groups,
-                           int P, int code, double delta_call, int calls_per_sibling = 0)
+                           int P, int code, double delta_call, int calls_per_sibling = 0, int64_t first_call = 0)
 {
-    const int64_t lvl = (int64_t)code | ((int64_t)calls_per_sibling << 32);
+    const int64_t lvl = pack_level(code, first_call, calls_per_sibling);
     const elm_params *p = c.p;
     const int BH = p->batch * p->kv_heads;
     const int64_t n = p->n_kv;
@@ -1182,4 +1184,278 @@ extern "C" int elm_express_prefill(const void *Q, const void *K, const void *V, 
     }
     return det ? express_impl<bf, double>((const bf *)K, (const bf *)V, params, mbar, seed, idx_out, w_out, ws, st, 0u, (const bf *)Q, (bf *)O)
                : express_impl<bf, float>((const bf *)K, (const bf *)V, params, mbar, seed, idx_out, w_out, ws, st, 0u, (const bf *)Q, (bf *)O);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Streaming Thinformer Express: the host struct elm_stream carries the counters of Algorithms 1-2
+// (they depend on the token count alone), the device workspace the point lists E, S_0..S_mbar.
+// ---------------------------------------------------------------------------------------------
+namespace elm {
+struct StreamLayout {
+    size_t vmax_bits, cnorm, E, T1, S, Mpair, rdecay, F, F_stride, ep_idx, ep_w, ws_attend, ep_cap, total;
+};
+static StreamLayout stream_layout(const elm_params *p, int mbar)
+{
+    StreamLayout L;
+    const size_t ts = p->precision == ELM_PREC_FP64_DET ? 8 : 4;
+    const size_t BH = (size_t)p->batch * p->kv_heads;
+    const size_t n = (size_t)p->n_kv;
+    const size_t n_out = (size_t)1 << p->log2_nout;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+    L.vmax_bits = take((BH + 1) * 4);
+    L.cnorm = take(BH * n * ts);
+    L.E = take(BH * n * 4);                    // every point list is [BH][n_kv]-strided, like the lists of elm_compress
+    L.T1 = take(BH * n * 4);
+    L.S = take((size_t)(mbar + 1) * BH * n * 4);
+    L.Mpair = take(BH * (n / 2 + 1) * ts);
+    L.rdecay = take(BH * (n / 2 + 1) * ts);
+    L.F_stride = 4 * n_out * n_out;
+    L.F = take(BH * L.F_stride * ts);
+    L.ep_cap = 6 * n_out + 1;                  // Theorem 1's cache bound, plus the token itself
+    L.ep_idx = take(BH * L.ep_cap * 4);
+    L.ep_w = take(BH * L.ep_cap * 4);
+    elm_params one = *p;
+    one.n_q = 1;
+    L.ws_attend = take(attend_layout(&one, (int32_t)L.ep_cap).total);
+    L.total = off;
+    return L;
+}
+static int validate_stream(const elm_params *p, int32_t mbar)
+{
+    if (p->batch < 1 || p->kv_heads < 1 || p->q_heads < 1 || p->q_heads % p->kv_heads != 0) return ELM_ERR_SHAPE;
+    if ((int64_t)p->batch * p->q_heads > 65535) return ELM_ERR_SHAPE;
+    if (p->d != 64 && p->d != 128) return ELM_ERR_SHAPE;
+    if (p->log2_nout < 1 || p->log2_nout > 24 || mbar < 0 || mbar > 12) return ELM_ERR_SHAPE;
+    if (p->n_kv < 2 || p->n_q != 1) return ELM_ERR_SHAPE;
+    if (p->dtype != ELM_F32 && p->dtype != ELM_BF16) return ELM_ERR_DTYPE;
+    if (p->precision != ELM_PREC_FP64_DET && p->precision != ELM_PREC_FP32) return ELM_ERR_DTYPE;
+    if (!(p->delta > 0.0 && p->delta < 1.0)) return ELM_ERR_DELTA;
+    return ELM_OK;
+}
+__global__ void append_kernel(int32_t *__restrict__ list, int64_t stride, int64_t pos, int32_t value, int problems)
+{
+    const int p = blockIdx.x * blockDim.x + threadIdx.x;
+    if (p < problems) list[(int64_t)p * stride + pos] = value;
+}
+
+// wtd_cache() of Algorithm 1 (+ the token t itself when t >= 0) as list pieces
+static void stream_pieces(const elm_stream *s, const StreamLayout &L, unsigned char *ws, const elm_params *p, int64_t t,
+                          ListPieces &pc)
+{
+    const size_t BH = (size_t)p->batch * p->kv_heads;
+    int32_t *S = reinterpret_cast<int32_t *>(ws + L.S);
+    int k = 0;
+    int32_t at = 0;
+    auto piece = [&](const int32_t *src, int64_t off, int64_t count, float wgt) {
+        if (count <= 0) return;
+        pc.src[k] = src; pc.src_off[k] = off; pc.w[k] = wgt; pc.dst_off[k] = at;
+        at += (int32_t)count;
+        ++k;
+    };
+    for (int i = 0; i <= s->q; ++i) piece(S + (size_t)i * BH * p->n_kv, 0, s->n_S[i], (float)ldexp(1.0, i - s->q));
+    piece(reinterpret_cast<int32_t *>(ws + L.E), 0, s->n_E, 1.f);
+    if (t >= 0) piece(nullptr, t, 1, (float)ldexp(1.0, -s->q));          // the token enters S_0
+    pc.dst_off[k] = at;
+    pc.n = k;
+}
+
+template <typename Tin, typename T>
+static int stream_step_impl(elm_stream *s, const Tin *Q, const Tin *K, const Tin *V, const elm_params *p, Tin *O,
+                            unsigned char *ws, cudaStream_t st)
+{
+    const StreamLayout L = stream_layout(p, s->mbar);
+    const int BH = p->batch * p->kv_heads;
+    const int64_t n = p->n_kv, n_out = (int64_t)1 << p->log2_nout;
+    const int64_t t = s->n;
+    if (t >= n) return ELM_ERR_SHAPE;                                      // capacity
+    if (s->m > s->mbar) return ELM_ERR_SHAPE;                              // Subsample: not built yet
+    if (s->q >= 1 && p->log2_nout + 2 - s->q < 1) return ELM_ERR_SHAPE;     // level-0 calls of at least 2 points
+    LevelCtx<Tin, T> c;
+    c.K = K; c.V = V; c.p = p;
+    c.vmax_bits = reinterpret_cast<unsigned *>(ws + L.vmax_bits);
+    c.cnorm = reinterpret_cast<T *>(ws + L.cnorm);
+    c.Mpair = reinterpret_cast<T *>(ws + L.Mpair);
+    c.rdecay = reinterpret_cast<T *>(ws + L.rdecay);
+    c.F = reinterpret_cast<T *>(ws + L.F);
+    c.F_stride = (int64_t)L.F_stride;
+    c.seed = s->seed; c.pbase = 0; c.st = st;
+    int32_t *E = reinterpret_cast<int32_t *>(ws + L.E);
+    int32_t *T1 = reinterpret_cast<int32_t *>(ws + L.T1);
+    int32_t *S = reinterpret_cast<int32_t *>(ws + L.S);
+    auto Slist = [&](int i) { return S + (size_t)i * BH * n; };
+    auto blocks = [](int64_t count) { return (unsigned)((count + 255) / 256); };
+    if (t >= s->n_known) {
+        // a token that was not there at init: its key norm, and v_max grows with it
+        prepass_kernel<Tin, T><<<dim3(1, (unsigned)BH), 256, 0, st>>>(K, V, n, p->d, c.cnorm, c.vmax_bits, T1, t, t + 1);
+        count_launches(1);
+        ELM_CUDA_TRY(cudaGetLastError());
+    }
+    // ---- Algorithm 5: attend over wtd_cache() plus the token ----
+    {
+        ListPieces pc = {};
+        stream_pieces(s, L, ws, p, t, pc);
+        const int total = pc.dst_off[pc.n];
+        int32_t *ep_idx = reinterpret_cast<int32_t *>(ws + L.ep_idx);
+        float *ep_w = reinterpret_cast<float *>(ws + L.ep_w);
+        build_list_kernel<<<dim3(blocks(total), (unsigned)BH), 256, 0, st>>>(pc, n, ep_idx, ep_w, total);
+        count_launches(1);
+        ELM_CUDA_TRY(cudaGetLastError());
+        const int rc = attend_enqueue(Q, K, V, ep_idx, ep_w, total, p, O, ws + L.ws_attend, st);
+        if (rc != ELM_OK) return rc;
+    }
+    // ---- Algorithm 1: Express.update ----
+    auto append = [&](int32_t *list, int64_t pos) {
+        append_kernel<<<(BH + 127) / 128, 128, 0, st>>>(list, n, pos, (int32_t)t, BH);
+        count_launches(1);
+        return cuda_status(cudaGetLastError());
+    };
+    s->n += 1;
+    if (s->n <= n_out) {                                                   // exact phase
+        const int rc = append(E, s->n_E);
+        s->n_E += 1;
+        return rc;
+    }
+    s->ell += 1;                                                           // thin phase: Compress2.update
+    {
+        const int q = s->q;
+        int rc = append(Slist(0), s->n_S[0]);
+        if (rc != ELM_OK) return rc;
+        s->n_S[0] += 1;
+        const double dm = kh_express_delta(p->delta, s->m);
+        for (int i = 0; i < q; ++i) {
+            const int64_t thresh = ((n_out << q) << i) >> (2 * (q - 1));  // n_in 2^i / 4^(q-1)
+            if (s->n_S[i] != thresh) continue;
+            const double dlt = ldexp(dm, 2 * (i + 1 - q)) / (3.0 * (double)q);
+            const int code = i + 64 * (4 * (s->m / 2) + s->b + 1);
+            rc = run_halve_level<Tin, T>(c, Slist(i), Slist(i + 1) + s->n_S[i + 1], n, 1, (int)(thresh / 2), code, dlt, 0,
+                                         s->calls[i]);
+            if (rc != ELM_OK) return rc;
+            s->calls[i] += 1;
+            s->n_S[i + 1] += thresh / 2;
+            s->n_S[i] = 0;
+        }
+    }
+    if (s->ell == (n_out << s->m)) {                                       // the segment is done: S_q joins E
+        copy_list_kernel<<<dim3(blocks(s->n_S[s->q]), (unsigned)BH), 256, 0, st>>>(E, s->n_E, Slist(s->q), n, s->n_S[s->q]);
+        count_launches(1);
+        ELM_CUDA_TRY(cudaGetLastError());
+        s->n_E += s->n_S[s->q];
+        s->n_S[s->q] = 0;
+        s->ell = 0;
+        s->b += 1;
+    }
+    if (s->n == 4 * (n_out << s->m)) {                                     // halve phase
+        const double dm = kh_express_delta(p->delta, s->m);
+        int rc = run_halve_level<Tin, T>(c, E, T1, n, 1, (int)(2 * n_out), 62 + 64 * 4 * (s->m / 2), 0.5 * dm);
+        if (rc != ELM_OK) return rc;
+        rc = run_halve_level<Tin, T>(c, T1, E, n, 1, (int)n_out, 63 + 64 * 4 * (s->m / 2), 0.5 * dm);
+        if (rc != ELM_OK) return rc;
+        s->n_E = n_out;
+        s->m += 2;
+        s->b = 0;
+    }
+    if (s->ell == 0) {                                                     // a new Compress2 instance
+        s->q = s->m < s->mbar ? s->m : s->mbar;
+        for (int i = 0; i < 16; ++i) { s->n_S[i] = 0; s->calls[i] = 0; }
+    }
+    return ELM_OK;
+}
+}  // namespace elm
+
+extern "C" int elm_stream_workspace_bytes(const elm_params *params, int32_t mbar, size_t *bytes)
+{
+    using namespace elm;
+    if (!params || !bytes) return ELM_ERR_NULL;
+    const int rc = validate_stream(params, mbar);
+    if (rc != ELM_OK) return rc;
+    *bytes = stream_layout(params, mbar).total;
+    return ELM_OK;
+}
+
+extern "C" int elm_stream_init(elm_stream *s, const void *K, const void *V, int64_t n_known, const elm_params *params,
+                               int32_t mbar, uint64_t seed, void *workspace, size_t workspace_bytes, void *stream)
+{
+    using namespace elm;
+    if (!s || !params || !workspace) return ELM_ERR_NULL;
+    const int rc = validate_stream(params, mbar);
+    if (rc != ELM_OK) return rc;
+    if (n_known < 0 || n_known > params->n_kv || (n_known > 0 && (!K || !V))) return ELM_ERR_SHAPE;
+    if ((uintptr_t)workspace & 255) return ELM_ERR_ALIGN;
+    const StreamLayout L = stream_layout(params, mbar);
+    if (workspace_bytes < L.total) return ELM_ERR_WORKSPACE;
+    unsigned char *ws = (unsigned char *)workspace;
+    cudaStream_t st = (cudaStream_t)stream;
+    const int BH = params->batch * params->kv_heads;
+    *s = elm_stream{};
+    s->mbar = mbar;
+    s->seed = seed;
+    s->n_known = n_known;
+    ELM_CUDA_TRY(cudaMemsetAsync(ws + L.vmax_bits, 0, (size_t)(BH + 1) * 4, st));
+    if (n_known > 0) {
+        const dim3 grid((unsigned)((n_known + 255) / 256), (unsigned)BH);
+        unsigned *vb = reinterpret_cast<unsigned *>(ws + L.vmax_bits);
+        int32_t *scratch = reinterpret_cast<int32_t *>(ws + L.T1);
+        const int64_t n = params->n_kv;
+        typedef __nv_bfloat16 bf;
+        if (params->dtype == ELM_F32) {
+            if (params->precision == ELM_PREC_FP64_DET)
+                prepass_kernel<float, double><<<grid, 256, 0, st>>>((const float *)K, (const float *)V, n, params->d, reinterpret_cast<double *>(ws + L.cnorm), vb, scratch, 0, n_known);
+            else
+                prepass_kernel<float, float><<<grid, 256, 0, st>>>((const float *)K, (const float *)V, n, params->d, reinterpret_cast<float *>(ws + L.cnorm), vb, scratch, 0, n_known);
+        } else {
+            if (params->precision == ELM_PREC_FP64_DET)
+                prepass_kernel<bf, double><<<grid, 256, 0, st>>>((const bf *)K, (const bf *)V, n, params->d, reinterpret_cast<double *>(ws + L.cnorm), vb, scratch, 0, n_known);
+            else
+                prepass_kernel<bf, float><<<grid, 256, 0, st>>>((const bf *)K, (const bf *)V, n, params->d, reinterpret_cast<float *>(ws + L.cnorm), vb, scratch, 0, n_known);
+        }
+        count_launches(1);
+        ELM_CUDA_TRY(cudaGetLastError());
+    }
+    return ELM_OK;
+}
+
+extern "C" int elm_stream_step(elm_stream *s, const void *Q_t, const void *K, const void *V, const elm_params *params,
+                               void *O_t, void *workspace, size_t workspace_bytes, void *stream)
+{
+    using namespace elm;
+    if (!s || !params) return ELM_ERR_NULL;
+    const int rc = validate_stream(params, s->mbar);
+    if (rc != ELM_OK) return rc;
+    if (!Q_t || !K || !V || !O_t || !workspace) return ELM_ERR_NULL;
+    if (((uintptr_t)Q_t | (uintptr_t)K | (uintptr_t)V | (uintptr_t)O_t) & 15) return ELM_ERR_ALIGN;
+    if ((uintptr_t)workspace & 255) return ELM_ERR_ALIGN;
+    if (workspace_bytes < stream_layout(params, s->mbar).total) return ELM_ERR_WORKSPACE;
+    unsigned char *ws = (unsigned char *)workspace;
+    cudaStream_t st = (cudaStream_t)stream;
+    const bool det = params->precision == ELM_PREC_FP64_DET;
+    typedef __nv_bfloat16 bf;
+    if (params->dtype == ELM_F32) {
+        return det ? stream_step_impl<float, double>(s, (const float *)Q_t, (const float *)K, (const float *)V, params, (float *)O_t, ws, st)
+                   : stream_step_impl<float, float>(s, (const float *)Q_t, (const float *)K, (const float *)V, params, (float *)O_t, ws, st);
+    }
+    return det ? stream_step_impl<bf, double>(s, (const bf *)Q_t, (const bf *)K, (const bf *)V, params, (bf *)O_t, ws, st)
+               : stream_step_impl<bf, float>(s, (const bf *)Q_t, (const bf *)K, (const bf *)V, params, (bf *)O_t, ws, st);
+}
+
+extern "C" int elm_stream_cache(const elm_stream *s, const elm_params *params, int32_t *idx_out, float *w_out,
+                                int32_t *count_host, void *workspace, size_t workspace_bytes, void *stream)
+{
+    using namespace elm;
+    if (!s || !params || !idx_out || !w_out || !count_host || !workspace) return ELM_ERR_NULL;
+    const int rc = validate_stream(params, s->mbar);
+    if (rc != ELM_OK) return rc;
+    const StreamLayout L = stream_layout(params, s->mbar);
+    if (workspace_bytes < L.total) return ELM_ERR_WORKSPACE;
+    ListPieces pc = {};
+    stream_pieces(s, L, (unsigned char *)workspace, params, -1, pc);
+    const int total = pc.dst_off[pc.n];
+    *count_host = total;
+    if (total > 0) {
+        build_list_kernel<<<dim3((unsigned)((total + 255) / 256), (unsigned)(params->batch * params->kv_heads)), 256, 0,
+                            (cudaStream_t)stream>>>(pc, params->n_kv, idx_out, w_out, total);
+        count_launches(1);
+        ELM_CUDA_TRY(cudaGetLastError());
+    }
+    return ELM_OK;
 }

@@ -32,7 +32,7 @@ int compress_enqueue(const void *K, const void *V, const elm_params *params, uin
 // the survivors go straight to `out`.
 struct WalkArgs {
     int fused;
-    int64_t level;           // third counter word (+ calls per sibling in the high half, see call_counter)
+    int64_t level;           // third counter word, first call and calls per sibling (pack_level in elm_common.cuh)
     uint64_t seed;
     float logfac;
     const float *rdecay;     // [BH][n/2]

@@ -163,3 +163,64 @@ def test_express_prefill_rejects_subsampled_rounds():
     Q, K, V = generate(wl, seed=1, want_q=True)
     with pytest.raises(elm.ElmError):
         elm.express_prefill(Q.cuda(), K.cuda(), V.cuda(), 4, 2, seed=1)      # R = 3 needs mbar >= 4
+
+
+# ----------------------------------------------------------------------------------------------
+# Streaming Thinformer Express: one token per call against the streaming oracle
+# ----------------------------------------------------------------------------------------------
+# name -> (workload, log2_nout, tokens, mbar, q heads per KV head): token counts that stop mid-round
+STREAM_CASES = {
+    # stops in the third segment of round 2 (m = 4): S_1 .. S_3 partly filled
+    "iid_f32_nout16_300": (WORKLOADS["cfg1"].scaled(q_heads=1, kv_heads=1), 4, 300, 4, 1),
+    # stops just before the end of round 2
+    "mixture_f32_nout8_500": (WORKLOADS["cfg2"].scaled(batch=1, q_heads=2, kv_heads=2), 3, 500, 4, 1),
+    # grouped queries, stops early in round 2
+    "lowrank_bf16_nout32_600_gqa": (WORKLOADS["cfg3"].scaled(batch=1, q_heads=2, kv_heads=1), 5, 600, 4, 2),
+}
+
+
+@pytest.mark.parametrize("precision", ["fp64", "fp32"])
+@pytest.mark.parametrize("name", sorted(STREAM_CASES))
+def test_stream_outputs_and_cache_match_streaming_oracle(name, precision):
+    from _util import max_rel_err
+    wl, log2_nout, n, mbar, rep = STREAM_CASES[name]
+    wl = wl.scaled(n=n, n_q=n, q_heads=wl.kv_heads * rep)
+    Q, K, V = generate(wl, seed=31, want_q=True)
+    Qd, Kd, Vd = Q.cuda(), K.cuda(), V.cuda()
+    st = elm.Stream(Kd, Vd, wl.q_heads, log2_nout, mbar, seed=11, precision=precision)
+    outs = [st.step(Qd[:, :, t:t + 1, :].contiguous()) for t in range(n)]
+    got = torch.cat(outs, dim=2).float().cpu().numpy()
+    cidx, cw = st.cache()
+    torch.cuda.synchronize()
+    Qf, Kf, Vf = as_f32_numpy(Q), as_f32_numpy(K), as_f32_numpy(V)
+    B, Hq = Qf.shape[:2]
+    H = Kf.shape[1]
+    worst = 0.0
+    for b in range(B):
+        for h in range(Hq):
+            kv = (h * H) // Hq
+            r = oracle.thinformer_express(Qf[b, h], Kf[b, kv], Vf[b, kv], log2_nout, mbar, seed=11, head=b * H + kv)
+            same = np.array_equal(cidx[b, kv].cpu().numpy(), r["final_idx"])
+            if precision == "fp64":
+                assert same
+                assert np.array_equal(cw[b, kv].cpu().numpy().astype(np.float64), r["final_w"])
+            if same:
+                worst = max(worst, max_rel_err(got[b, h], r["O"]))
+    print(f"{name} {precision}: max relative error of the streamed outputs {worst:.3e}")
+    assert worst <= PREFILL_TOL[(wl.dtype if wl.dtype == "bf16" else "f32", precision)]
+
+
+def test_stream_with_tokens_unknown_at_init_tracks_vmax():
+    """n_known = 0: every token's key norm and v_max are picked up as it arrives; with v_max growing the
+    kernel differs from the prefill reading, so only structure is checked: cache bound and exact start."""
+    from _util import max_rel_err
+    wl = WORKLOADS["cfg1"].scaled(n=200, n_q=200)
+    Q, K, V = generate(wl, seed=2, want_q=True)
+    Qd, Kd, Vd = Q.cuda(), K.cuda(), V.cuda()
+    st = elm.Stream(Kd, Vd, 1, 4, 2, seed=3, precision="fp64", n_known=0)
+    outs = [st.step(Qd[:, :, t:t + 1, :].contiguous()) for t in range(200)]
+    got = torch.cat(outs, dim=2).float().cpu().numpy()
+    ref = oracle.exact_causal_attention(as_f32_numpy(Q)[0, 0, :64], as_f32_numpy(K)[0, 0, :64], as_f32_numpy(V)[0, 0, :64])
+    assert max_rel_err(got[0, 0, :64], ref) <= 2e-6                       # the first 4 n_out tokens are exact
+    cidx, _ = st.cache()
+    assert cidx.shape[-1] < 6 * 16 and len(set(cidx[0, 0].cpu().tolist())) == cidx.shape[-1]
