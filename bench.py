@@ -200,7 +200,7 @@ def main():
     ap.add_argument("--ref-heads", type=int, default=None)
     ap.add_argument("--override", default="", help="comma list of Workload fields for small profiling "
                     "captures, e.g. q_heads=8,kv_heads=2,n=32768,n_q=32768 (the line then names the scaled case)")
-    ap.add_argument("--only", default="both", choices=["both", "compress", "attend", "express", "prefill", "decode"],
+    ap.add_argument("--only", default="both", choices=["both", "compress", "attend", "express", "prefill", "decode", "stream"],
                     help="run one half of the step; or, instead of the step, the Offline-Express compression "
                          "(express) or the Thinformer Express prefill (prefill) of the same inputs with "
                          "mbar = log2(n_out) - 2; or (decode) one query per head over a cache of n_out and of "
@@ -245,6 +245,33 @@ def main():
     O = torch.empty_like(Qd)
     small_inputs = not wl.name.startswith(("cfg4", "cfg5"))
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev) if small_inputs else None
+
+    if args.only == "stream":
+        # streaming Thinformer Express, one token per call, over the first tokens of the workload
+        T = min(wl.n, 10 * wl.n_out)
+        st = elm.Stream(Kd, Vd, wl.q_heads, wl.log2_nout, wl.log2_nout - 2, seed=args.seed, precision=args.precision)
+        o1 = torch.empty_like(Qd[:, :, :1, :])
+        qs = [Qd[:, :, t:t + 1, :].contiguous() for t in range(T)]
+        torch.cuda.synchronize()
+        import time
+        marks = {}
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        w0 = time.perf_counter()
+        e0.record()
+        for t in range(T):
+            st.step(qs[t], out=o1)
+            if t + 1 in (4 * wl.n_out, T):
+                torch.cuda.synchronize()
+                marks[t + 1] = time.perf_counter() - w0
+        e1.record()
+        torch.cuda.synchronize()
+        if rank == 0:
+            print(json.dumps({"stream": {"tokens": T, "ms_total": e0.elapsed_time(e1),
+                                         "us_per_token_first_4nout": marks[4 * wl.n_out] / (4 * wl.n_out) * 1e6,
+                                         "us_per_token_after": (marks[T] - marks[4 * wl.n_out]) / (T - 4 * wl.n_out) * 1e6,
+                                         "cache_entries_at_end": int(st.cache()[0].shape[-1])},
+                              "config": workload_config(wl, args)}))
+        return
 
     if args.only == "decode":
         # one new token per head over a weighted cache: HBM-bound; bytes = the cache rows of K and V once
