@@ -67,6 +67,11 @@ def _load():
                                              ctypes.c_double, _f64p, ctypes.c_uint64, _i32p,
                                              _f64p, _f64p]
     lib.oracle_compress2_batched.restype = ctypes.c_int
+    lib.oracle_compress2_stream.argtypes = [_f32p, _f32p, ctypes.c_int64, ctypes.c_int, ctypes.c_int,
+                                            ctypes.c_int, ctypes.c_double, _f64p, ctypes.c_uint64,
+                                            ctypes.c_uint32, ctypes.c_int32, ctypes.c_int32, _i32p, _f64p,
+                                            ctypes.c_int32, _i32p]
+    lib.oracle_compress2_stream.restype = ctypes.c_int
     lib.oracle_wtd_attention.argtypes = [_f32p, _f32p, _f32p, _i32p, _f64p, ctypes.c_int,
                                          ctypes.c_int64, ctypes.c_int, _f64p]
     lib.oracle_wtd_attention.restype = ctypes.c_int
@@ -209,6 +214,31 @@ def compress2_batched(K, V, log2_nout: int, m: int, delta: float = 0.5, delta_le
     if rc != 0:
         raise ValueError(f"oracle_compress2_batched failed with {rc}")
     return idx, w, mg
+
+
+def compress2_stream(K, V, log2_nout: int, m: int, n_sink: int = 0, n_window: int = 0, delta: float = 0.5,
+                     delta_level=None, seed: int = 1, head: int = 0):
+    """Algorithm 2 fed the middle rows one by one, sink / window rows kept; K, V are [n, d] with any n.
+
+    Returns (idx[count] int32, w[count] float64): sinks, S_0 .. S_m, window; weights sum to 1."""
+    K, kp = _f32(K)
+    V, vp = _f32(V)
+    n, d = K.shape
+    cap = n_sink + n_window + 5 * (1 << log2_nout) + 8 if m > 0 else n
+    idx = np.zeros(cap, dtype=np.int32)
+    w = np.zeros(cap, dtype=np.float64)
+    cnt = ctypes.c_int32(0)
+    dl = None
+    if delta_level is not None:
+        dl_arr, dl = _f64(delta_level)
+        assert dl_arr.shape[0] == m
+    rc = _load().oracle_compress2_stream(kp, vp, n, d, log2_nout, m, delta, dl, seed, head, n_sink, n_window,
+                                         idx.ctypes.data_as(_i32p), w.ctypes.data_as(_f64p), cap,
+                                         ctypes.byref(cnt))
+    if rc != 0:
+        raise ValueError(f"oracle_compress2_stream failed with {rc}")
+    c = int(cnt.value)
+    return idx[:c].copy(), w[:c].copy()
 
 
 def wtd_attention(Q, K, V, idx, w):

@@ -10,6 +10,7 @@
  *   oracle_katt               Eq. (katt): key-value attention kernel
  *   oracle_kh                 Algorithm A.1: KH(delta) kernel halving
  *   oracle_compress2          Algorithm "Offline-Compress2" (recursive form of Algorithm 2)
+ *   oracle_compress2_stream   Algorithm 2 itself, one update per point, any length, sink / window rows kept
  *   oracle_wtd_attention      Algorithm 5 / Eq. (def:att_approx): weighted attention
  *   oracle_exact_attention    Eq. (unmaskedatt): exact unmasked attention
  *   oracle_mmd2               squared kernel MMD between a point set and a weighted subset
@@ -297,6 +298,81 @@ int oracle_compress2_batched(const float *K, const float *V, int problems, int64
         }
     }
     return bad;
+}
+
+/* ------------------------------------------------------------------------------------ */
+/* Compress2 in its streaming form (Algorithm 2), for sequences of any length, with the  */
+/* first n_sink and last n_window rows kept exactly.                                     */
+/*                                                                                        */
+/*   Compress2(m, n_in = 2^m n_out, Halve): S_0 <- S_0 + {x}; for i = 0..m-1: when S_i    */
+/*   holds n_in 2^i / 4^(m-1) points, S_{i+1} <- S_{i+1} + Halve_i(S_i), S_i <- {}.        */
+/*   wtd_cache() = [(S_i, 2^(i-m))]_{i=0..m}.                                              */
+/*                                                                                        */
+/* The middle rows n_sink .. n - n_window - 1 are fed one by one (at most n_in of them);  */
+/* whatever has not been halved yet stays in its level with that level's weight.  The    */
+/* sink and window rows carry the weight of a raw point, 2^-m.  Readings:                */
+/*   R-norm    all weights are divided by their sum n 2^-m, so that they are positive and */
+/*             sum to 1 (Definition 1): a point of S_i gets 2^i / n, a sink 1 / n.        */
+/*   R-out     output order: sinks, S_0, S_1, ..., S_m (each in append order), window.    */
+/*   R-vmax    v_max over all n rows of the problem.                                      */
+/*   uniforms  as in oracle_compress2: counter (pair, number of the call at its level,    */
+/*             level, head); with n = n_in and no sinks the result equals Offline-Compress2. */
+/* ------------------------------------------------------------------------------------ */
+int oracle_compress2_stream(const float *K, const float *V, int64_t n, int d, int log2_nout, int m,
+                            double delta, const double *delta_level, uint64_t seed, uint32_t head,
+                            int32_t n_sink, int32_t n_window, int32_t *idx_out, double *w_out,
+                            int32_t capacity, int32_t *count)
+{
+    const int64_t n_out = (int64_t)1 << log2_nout;
+    const int64_t n_in = n_out << m;
+    const int64_t n_mid = n - n_sink - n_window;
+    if (m < 0 || m > 30 || n_sink < 0 || n_window < 0 || n_mid < 0 || n_mid > n_in) return -1;
+    if (m >= 1 && ((n_in >> (2 * (m - 1))) < 2)) return -1;            /* level-0 calls of at least one pair */
+    double dl[32];
+    if (delta_level) memcpy(dl, delta_level, sizeof(double) * (size_t)m);
+    else oracle_default_delta_levels(m, delta, dl);
+    const double vmax = oracle_vmax(V, n, d);
+    int32_t *S[32];
+    int64_t nS[32], calls[32], thresh[32];
+    int rc = 0;
+    for (int i = 0; i <= m; ++i) { S[i] = NULL; nS[i] = 0; calls[i] = 0; }
+    for (int i = 0; i <= m; ++i) {
+        thresh[i] = m >= 1 ? ((n_in << i) >> (2 * (m - 1))) : n_in + 1;
+        /* S_i never holds more than its threshold (S_m: n_out points, or everything when m = 0) */
+        const int64_t room = i < m ? thresh[i] : (m == 0 ? n_in : n_out);
+        S[i] = (int32_t *)malloc(sizeof(int32_t) * (size_t)(room > 0 ? room : 1));
+        if (!S[i]) rc = -2;
+    }
+    for (int64_t t = 0; t < n_mid && rc == 0; ++t) {
+        S[0][nS[0]++] = (int32_t)(n_sink + t);                          /* update(x) */
+        for (int i = 0; i < m && rc == 0; ++i) {
+            if (nS[i] != thresh[i]) continue;
+            const int64_t s = thresh[i];
+            double *U = (double *)malloc(sizeof(double) * (size_t)(s / 2));
+            if (!U) { rc = -2; break; }
+            for (int64_t a = 0; a < s / 2; ++a)
+                U[a] = oracle_uniform(seed, (uint32_t)a, (uint32_t)calls[i], (uint32_t)i, head);
+            rc = oracle_kh(K, V, d, vmax, S[i], (int)s, dl[i], 1, U, S[i + 1] + nS[i + 1], NULL, NULL);
+            free(U);
+            calls[i] += 1;
+            nS[i + 1] += s / 2;
+            nS[i] = 0;
+        }
+    }
+    if (rc == 0) {
+        int64_t c = 0, total = n_sink + n_window;
+        for (int i = 0; i <= m; ++i) total += nS[i];
+        if (count) *count = (int32_t)total;
+        if (total > capacity) rc = -3;
+        if (rc == 0) {
+            for (int32_t a = 0; a < n_sink; ++a) { idx_out[c] = a; w_out[c] = 1.0 / (double)n; ++c; }
+            for (int i = 0; i <= m; ++i)
+                for (int64_t a = 0; a < nS[i]; ++a) { idx_out[c] = S[i][a]; w_out[c] = ldexp(1.0, i) / (double)n; ++c; }
+            for (int32_t a = 0; a < n_window; ++a) { idx_out[c] = (int32_t)(n - n_window + a); w_out[c] = 1.0 / (double)n; ++c; }
+        }
+    }
+    for (int i = 0; i <= m; ++i) free(S[i]);
+    return rc;
 }
 
 /* ------------------------------------------------------------------------------------ */
