@@ -200,11 +200,13 @@ def main():
     ap.add_argument("--ref-heads", type=int, default=None)
     ap.add_argument("--override", default="", help="comma list of Workload fields for small profiling "
                     "captures, e.g. q_heads=8,kv_heads=2,n=32768,n_q=32768 (the line then names the scaled case)")
-    ap.add_argument("--only", default="both", choices=["both", "compress", "attend", "express", "prefill", "decode", "stream"],
+    ap.add_argument("--only", default="both", choices=["both", "compress", "attend", "express", "prefill", "decode", "stream", "ragged"],
                     help="run one half of the step; or, instead of the step, the Offline-Express compression "
                          "(express) or the Thinformer Express prefill (prefill) of the same inputs with "
                          "mbar = log2(n_out) - 2; or (decode) one query per head over a cache of n_out and of "
-                         "6 n_out entries, printed as its own JSON line (profiling captures only)")
+                         "6 n_out entries, printed as its own JSON line (profiling captures only); or (ragged) "
+                         "compress + attend on a sequence 7 %% shorter than the workload's, 32 sink and 32 "
+                         "window rows kept (elm_compress_ragged)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -270,6 +272,43 @@ def main():
                                          "us_per_token_first_4nout": marks[4 * wl.n_out] / (4 * wl.n_out) * 1e6,
                                          "us_per_token_after": (marks[T] - marks[4 * wl.n_out]) / (T - 4 * wl.n_out) * 1e6,
                                          "cache_entries_at_end": int(st.cache()[0].shape[-1])},
+                              "config": workload_config(wl, args)}))
+        return
+
+    if args.only == "ragged":
+        # a length that is not n_out 2^m: Algorithm 2 leaves points in every level; 32 + 32 rows kept exactly
+        n_r = wl.n - wl.n // 14 - 37
+        Kr, Vr = Kd[:, :, :n_r, :].contiguous(), Vd[:, :, :n_r, :].contiguous()
+        Qr = Qd[:, :, :min(n_r, wl.n_q), :].contiguous()
+        Or = torch.empty_like(Qr)
+        pr, _ = elm.make_params(wl.batch, wl.q_heads, wl.kv_heads, n_r, Qr.shape[2], wl.d, wl.log2_nout, wl.m,
+                                1 if wl.dtype == "bf16" else 0, args.precision)
+        count, need = elm.compress_ragged_count(pr, 32, 32)
+        ws_r = torch.empty(need, dtype=torch.uint8, device=dev)
+        ws_ar = torch.empty(elm.attend_workspace_bytes(pr, count), dtype=torch.uint8, device=dev)
+
+        def ragged_step(seed):
+            idx, w = elm.compress_ragged(Kr, Vr, wl.log2_nout, wl.m, 32, 32, seed=seed, precision=args.precision,
+                                         workspace=ws_r)
+            elm.attend(Qr, Kr, Vr, idx, w, precision=args.precision, workspace=ws_ar, out=Or)
+
+        for i in range(warmup):
+            ragged_step(args.seed + i)
+        torch.cuda.synchronize()
+        elm.profile_enable(True)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(args.steps):
+            ragged_step(args.seed + warmup + i)
+        e1.record()
+        torch.cuda.synchronize()
+        prof = elm.profile_read()
+        elm.profile_enable(False)
+        ms = e0.elapsed_time(e1) / args.steps
+        if rank == 0:
+            print(json.dumps({"ragged": {"n": n_r, "n_sink": 32, "n_window": 32, "cache_entries": count,
+                                         "ms_per_step": ms, "tokens_per_s": wl.batch * n_r / (ms * 1e-3),
+                                         "stage_ms": {k: v[0] / args.steps for k, v in prof.items()}},
                               "config": workload_config(wl, args)}))
         return
 

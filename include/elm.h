@@ -101,11 +101,37 @@ int elm_compress(const void *K, const void *V, const elm_params *params, uint64_
                  void *stream);
 
 /*
+ * Algorithm 2 (Compress2 in its streaming form) on a sequence of any length, the first n_sink and the
+ * last n_window rows kept exactly (the paper's experiments keep 32 and 32 and compress the rows in
+ * between).  The n_mid = n_kv - n_sink - n_window middle rows are what Compress2(m, n_in = 2^m n_out)
+ * holds after n_mid updates in row order: level i has made floor(a_i / t_i) Halve calls on consecutive
+ * stretches of t_i = n_in 2^i / 4^(m-1) points (a_0 = n_mid, a_(i+1) = half of what level i consumed);
+ * the a_i mod t_i points left over stay in S_i.  wtd_cache() gives a point of S_i the weight 2^(i-m);
+ * sink and window rows carry the weight of a raw point, 2^-m; all weights are then divided by their
+ * sum n_kv 2^-m (Definition 1: positive, summing to 1), i.e. 2^i / n_kv and 1 / n_kv.
+ *   params     n_kv: any length >= 1 with 0 <= n_mid <= 2^m n_out; m >= 1 needs log2_nout - m + 2 >= 1
+ *              as in elm_compress; q_heads and n_q are not used.
+ *   K, V       [batch][kv_heads][n_kv][d]; v_max and the uniforms as in elm_compress (call g of level l
+ *              is the g-th stretch of that level), so with n_kv = 2^m n_out and no sink or window rows
+ *              the result is that of elm_compress.
+ *   idx_out, w_out   [batch][kv_heads][count], count from elm_compress_ragged_count (it depends on the
+ *              sizes only): sink rows, S_0, S_1, ..., S_m (each in append order), window rows.
+ *   workspace  at least the bytes elm_compress_ragged_count reports, 256-byte aligned.
+ * The result feeds elm_attend (n_core = count) unchanged.
+ */
+int elm_compress_ragged_count(const elm_params *params, int32_t n_sink, int32_t n_window, int32_t *count,
+                              size_t *workspace_bytes);
+int elm_compress_ragged(const void *K, const void *V, const elm_params *params, int32_t n_sink, int32_t n_window,
+                        uint64_t seed, int32_t *idx_out, float *w_out, void *workspace, size_t workspace_bytes,
+                        void *stream);
+
+/*
  * Eq. (def:att_approx) with one coreset per attention problem (Algorithm 5's return line).
  *   Q          [batch][q_heads][n_q][d]
  *   K, V       the ORIGINAL [batch][kv_heads][n_kv][d] tensors; rows are gathered through idx.
  *   idx, w     [batch][kv_heads][n_core]; any positive finite weights (they need not sum to 1),
  *              1 <= n_core <= n_kv.
+ *   params     n_kv may be any length >= 1 here; log2_nout, m, delta are not used.
  *   O          [batch][q_heads][n_q][d], same dtype as Q.
  *   workspace  at least elm_attend_workspace_bytes(params, n_core), 256-byte aligned.
  * precision FP64_DET accumulates in fp64, FP32 in fp32 (bf16 inputs: tensor cores).
@@ -278,6 +304,8 @@ int elm_profile_read(float *ms_out, int64_t *launches_out, int32_t n_stages);
  * records a non-zero code in a status word inside the workspace and the launch winds down instead
  * of hanging, leaving its outputs undefined.  These calls copy that word to *status_host (0 = every
  * wait completed) after synchronising `stream`.  `params` / `n_core` must be those of the call.
+ * elm_compress_status reads batch and kv_heads only and serves the workspace of every compression
+ * call (elm_compress, elm_compress_ragged, elm_express_compress / _prefill, elm_stream_*).
  */
 int elm_compress_status(const void *workspace, const elm_params *params, int32_t *status_host, void *stream);
 int elm_attend_status(const void *workspace, const elm_params *params, int32_t n_core, int32_t *status_host,

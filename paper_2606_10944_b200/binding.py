@@ -20,7 +20,7 @@ STAGE_NAMES = ["prepass", "level_prep", "gram", "walk", "emit", "gather", "atten
 
 EXPORTED_SYMBOLS = [
     "elm_workspace_bytes", "elm_default_delta_levels", "elm_compress", "elm_attend",
-    "elm_attend_workspace_bytes", "elm_attend_static", "elm_express_workspace_bytes", "elm_express_compress",
+    "elm_attend_workspace_bytes", "elm_attend_static", "elm_compress_ragged_count", "elm_compress_ragged", "elm_express_workspace_bytes", "elm_express_compress",
     "elm_express_prefill_workspace_bytes", "elm_express_prefill",
     "elm_stream_workspace_bytes", "elm_stream_init", "elm_stream_step", "elm_stream_cache",
     "elm_host_call_scratch_bytes", "elm_compress_attend_host",
@@ -76,6 +76,8 @@ def load_library():
     lib.elm_attend.argtypes = [vp, vp, vp, vp, vp, ctypes.c_int32, pp, vp, vp, sz, vp]
     lib.elm_attend_workspace_bytes.argtypes = [pp, ctypes.c_int32, szp]
     lib.elm_attend_static.argtypes = [vp, vp, vp, vp, vp, ctypes.c_int32, pp, vp, vp]
+    lib.elm_compress_ragged_count.argtypes = [pp, ctypes.c_int32, ctypes.c_int32, ctypes.POINTER(ctypes.c_int32), szp]
+    lib.elm_compress_ragged.argtypes = [vp, vp, pp, ctypes.c_int32, ctypes.c_int32, ctypes.c_uint64, vp, vp, vp, sz, vp]
     lib.elm_express_workspace_bytes.argtypes = [pp, ctypes.c_int32, szp]
     lib.elm_express_compress.argtypes = [vp, vp, pp, ctypes.c_int32, ctypes.c_uint64, vp, vp, vp, sz, vp]
     lib.elm_express_prefill_workspace_bytes.argtypes = [pp, ctypes.c_int32, szp]
@@ -179,6 +181,31 @@ def compress(K, V, log2_nout: int, m: int, seed: int = 1, precision="fp32", delt
     w = torch.empty((B, H, n_out), dtype=torch.float32, device=K.device)
     _check(lib.elm_compress(K.data_ptr(), V.data_ptr(), ctypes.byref(p), seed, idx.data_ptr(),
                             w.data_ptr(), ws.data_ptr(), ws.numel(), _stream()), "elm_compress")
+    return idx, w
+
+
+def compress_ragged_count(params: ElmParams, n_sink: int = 0, n_window: int = 0):
+    """elm_compress_ragged_count -> (entries per attention problem, workspace bytes)."""
+    c, b = ctypes.c_int32(0), ctypes.c_size_t(0)
+    _check(load_library().elm_compress_ragged_count(ctypes.byref(params), n_sink, n_window, ctypes.byref(c),
+                                                    ctypes.byref(b)), "elm_compress_ragged_count")
+    return int(c.value), int(b.value)
+
+
+def compress_ragged(K, V, log2_nout: int, m: int, n_sink: int = 0, n_window: int = 0, seed: int = 1, precision="fp32",
+                    delta: float = 0.5, delta_level=None, workspace=None):
+    """elm_compress_ragged: K, V [B, Hkv, n, d] with any n -> (idx, w) [B, Hkv, count]: the sink rows,
+    Compress2's weighted cache after the middle rows, the window rows."""
+    lib = load_library()
+    _require_cuda(K, V)
+    B, H, n, d = K.shape
+    p, keep = make_params(B, H, H, n, 1, d, log2_nout, m, _dtype_code(K), precision, delta, delta_level)
+    count, need = compress_ragged_count(p, n_sink, n_window)
+    ws = workspace if workspace is not None else _workspace(need, K.device)
+    idx = torch.empty((B, H, max(count, 1)), dtype=torch.int32, device=K.device)[:, :, :count]
+    w = torch.empty((B, H, max(count, 1)), dtype=torch.float32, device=K.device)[:, :, :count]
+    _check(lib.elm_compress_ragged(K.data_ptr(), V.data_ptr(), ctypes.byref(p), n_sink, n_window, seed, idx.data_ptr(),
+                                   w.data_ptr(), ws.data_ptr(), ws.numel(), _stream()), "elm_compress_ragged")
     return idx, w
 
 

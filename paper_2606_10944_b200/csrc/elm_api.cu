@@ -65,6 +65,18 @@ int validate_params(const elm_params *p)
     return ELM_OK;
 }
 
+// The attention calls read K and V through an index list: any n_kv, and log2_nout / m are not used.
+int validate_attend_params(const elm_params *p)
+{
+    if (p->batch < 1 || p->kv_heads < 1 || p->q_heads < 1 || p->n_q < 1 || p->n_kv < 1) return ELM_ERR_SHAPE;
+    if (p->q_heads % p->kv_heads != 0) return ELM_ERR_SHAPE;
+    if (p->d != 64 && p->d != 128) return ELM_ERR_SHAPE;
+    if ((int64_t)p->batch * p->q_heads > 65535) return ELM_ERR_SHAPE;
+    if (p->dtype != ELM_F32 && p->dtype != ELM_BF16) return ELM_ERR_DTYPE;
+    if (p->precision != ELM_PREC_FP64_DET && p->precision != ELM_PREC_FP32) return ELM_ERR_DTYPE;
+    return ELM_OK;
+}
+
 }  // namespace elm
 
 using namespace elm;
@@ -227,11 +239,10 @@ extern "C" int elm_compress_attend_host(const void *Q_host, const void *K_host, 
 extern "C" int elm_compress_status(const void *workspace, const elm_params *params, int32_t *status_host, void *stream)
 {
     if (!workspace || !params || !status_host) return ELM_ERR_NULL;
-    int rc = validate_params(params);
-    if (rc != ELM_OK) return rc;
-    // the status word follows the per-problem v_max words at the head of the compress workspace
-    const unsigned char *word = (const unsigned char *)workspace + compress_layout(params).vmax_bits +
-                                4 * (size_t)params->batch * params->kv_heads;
+    if (params->batch < 1 || params->kv_heads < 1) return ELM_ERR_SHAPE;
+    // the status word follows the per-problem v_max words at the head of every compression workspace
+    // (elm_compress, elm_compress_ragged, elm_express_*, elm_stream_*)
+    const unsigned char *word = (const unsigned char *)workspace + 4 * (size_t)params->batch * params->kv_heads;
     ELM_CUDA_TRY(cudaMemcpyAsync(status_host, word, 4, cudaMemcpyDeviceToHost, (cudaStream_t)stream));
     ELM_CUDA_TRY(cudaStreamSynchronize((cudaStream_t)stream));
     return ELM_OK;
@@ -241,7 +252,7 @@ extern "C" int elm_attend_status(const void *workspace, const elm_params *params
                                  int32_t *status_host, void *stream)
 {
     if (!workspace || !params || !status_host) return ELM_ERR_NULL;
-    int rc = validate_params(params);
+    int rc = validate_attend_params(params);
     if (rc != ELM_OK) return rc;
     if (n_core < 1 || n_core > params->n_kv) return ELM_ERR_SHAPE;
     // the status word follows the per-problem "weights differ" flags

@@ -180,6 +180,7 @@ AttendLayout attend_layout(const elm_params *p, int32_t n_core)
     L.Kc = take(problems * n_pad * p->d * es);
     L.Vc = take(problems * n_pad * p->d * es);
     L.bias = take(problems * n_pad * 4);
+    L.bx = take(problems * n_pad * 32);
     L.flags = take((problems + 1) * 4);
     L.total = off;
     return L;
@@ -303,7 +304,7 @@ extern "C" int elm_attend_workspace_bytes(const elm_params *params, int32_t n_co
 {
     using namespace elm;
     if (!params || !bytes) return ELM_ERR_NULL;
-    int rc = validate_params(params);
+    int rc = validate_attend_params(params);
     if (rc != ELM_OK) return rc;
     if (n_core < 1 || n_core > params->n_kv) return ELM_ERR_SHAPE;
     *bytes = attend_layout(params, n_core).total;
@@ -316,7 +317,7 @@ extern "C" int elm_attend(const void *Q, const void *K, const void *V, const int
 {
     using namespace elm;
     if (!params) return ELM_ERR_NULL;
-    int rc = validate_params(params);
+    int rc = validate_attend_params(params);
     if (rc != ELM_OK) return rc;
     if (!Q || !K || !V || !idx || !w || !O || !workspace) return ELM_ERR_NULL;
     if (n_core < 1 || n_core > params->n_kv) return ELM_ERR_SHAPE;
@@ -333,7 +334,7 @@ extern "C" int elm_attend_static(const void *Q, const void *K, const void *V, co
 {
     using namespace elm;
     if (!params) return ELM_ERR_NULL;
-    int rc = validate_params(params);
+    int rc = validate_attend_params(params);
     if (rc != ELM_OK) return rc;
     if (!Q || !K || !V || !idx || !w || !O) return ELM_ERR_NULL;
     if (n_core < 1 || n_core > params->n_kv) return ELM_ERR_SHAPE;

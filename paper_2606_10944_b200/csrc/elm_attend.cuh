@@ -14,6 +14,7 @@ struct AttendLayout {
     size_t Kc;    // [problems][n_core][d] gathered keys, input dtype
     size_t Vc;    // [problems][n_core][d] gathered values, input dtype
     size_t bias;  // [problems][n_core] log2 of the weights, fp32
+    size_t bx;    // [problems][n_pad][16] bf16: the weights as an operand of the tensor-core path's bias MMA
     size_t flags; // [problems] "weights differ" flags + one device status word
     size_t total;
 };

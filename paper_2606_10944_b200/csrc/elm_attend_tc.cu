@@ -22,6 +22,12 @@
 // TMEM columns: [0,128) S of tile 0, [128,256) S of tile 1, [256,256+D) O of tile 0, [384,384+D) O of
 // tile 1.  The probabilities of the points of column quarter c are written over the first 16 columns
 // of that quarter's logits, so a thread only ever overwrites logits it has already read itself.
+// Weights: log2 w_c has to be added to column c of the logits.  When a problem's weights differ (or its
+// list does not fill the last block) the tensor pipe adds it: one more MMA per block with K = 16,
+// A = a constant tile of ones, B = per column (hi, mid, lo, 0, ...) with hi + mid + lo = log2 w_c /
+// (log2 e / sqrt(d)) split into three bf16 terms (columns beyond the list: -1e30, which the exponential
+// turns into 0).  The softmax warps then treat every block alike; only the rows of a causal tail,
+// whose visible columns end at different places, take the slower masked form of the two passes.
 // Every mbarrier wait is bounded; on expiry the CTA records a status word and leaves through the
 // common exit, which frees the TMEM it holds.
 #include <cuda.h>
@@ -65,14 +71,18 @@ template <int D> struct Smem {
     static constexpr int OFF_Q = 0;
     static constexpr int OFF_K = OFF_Q + 2 * Q_TILE;
     static constexpr int OFF_V = OFF_K + STAGES * K_BLOCK;
-    static constexpr int OFF_BAR = OFF_V + STAGES * V_BLOCK;
+    static constexpr int X_BLOCK = BN * 16 * 2;             // bias operand: 16 bf16 per column, 32-byte swizzle
+    static constexpr int OFF_X = OFF_V + STAGES * V_BLOCK;
+    static constexpr int OFF_ONES = OFF_X + STAGES * X_BLOCK;   // [BM][16] bf16: the constant A operand of the bias MMA
+    static constexpr int OFF_BAR = OFF_ONES + BM * 16 * 2;
     static constexpr int TOTAL = OFF_BAR + 5120 + 1024;     // barrier block + slack for 1024-byte alignment
 };
 
 // ---------------------------------------------------------------------------------------------
 // gather for the tensor-core path: Kc [p][n_pad][D] (zero rows beyond n_core), Vt [p][D][n_pad]
-// (transposed, zero columns beyond n_core), bias = log2 w, and a per-problem flag that says
-// whether all weights of the problem are equal (then the bias cancels in the ratio).
+// (transposed, zero columns beyond n_core), Bx [p][n_pad][16]: log2 w / scale_log2 as three bf16 terms
+// (then zeros), and a per-problem flag that says whether all weights of the problem are equal (then
+// the bias cancels in the ratio).
 // ---------------------------------------------------------------------------------------------
 template <int D>
 __global__ void __launch_bounds__(256) gather_tc_kernel(const __nv_bfloat16 *__restrict__ K,
@@ -81,7 +91,8 @@ __global__ void __launch_bounds__(256) gather_tc_kernel(const __nv_bfloat16 *__r
                                                         const float *__restrict__ w, int64_t n, int n_core,
                                                         int n_pad, __nv_bfloat16 *__restrict__ Kc,
                                                         __nv_bfloat16 *__restrict__ Vt,
-                                                        float *__restrict__ bias, int *__restrict__ nonuniform)
+                                                        __nv_bfloat16 *__restrict__ Bx, float inv_scale_log2,
+                                                        int *__restrict__ nonuniform)
 {
     __shared__ __nv_bfloat16 tile[32][D + 2];
     const int p = blockIdx.y;
@@ -100,10 +111,16 @@ __global__ void __launch_bounds__(256) gather_tc_kernel(const __nv_bfloat16 *__r
             kd[e] = ok ? ks[e] : __float2bfloat16(0.f);
             tile[r][e] = ok ? vs[e] : __float2bfloat16(0.f);
         }
-        if (lane == 0) {
-            float wc = ok ? w[(int64_t)p * n_core + c] : 0.f;
-            bias[(int64_t)p * n_pad + c] = ok ? log2f(wc) : -INFINITY;
-            if (ok && wc != w0) differs = true;
+        if (lane < 16) {
+            const float wc = ok ? w[(int64_t)p * n_core + c] : 0.f;
+            // in the logits' own units (they are multiplied by scale_log2 later); -1e30 hides a padded column
+            const float x = ok ? log2f(wc) * inv_scale_log2 : -1e30f;
+            const __nv_bfloat16 hi = __float2bfloat16(x);
+            const float r1 = ok ? x - __bfloat162float(hi) : 0.f;
+            const __nv_bfloat16 mid = __float2bfloat16(r1);
+            const __nv_bfloat16 lo = __float2bfloat16(r1 - __bfloat162float(mid));
+            Bx[((int64_t)p * n_pad + c) * 16 + lane] = lane == 0 ? hi : (lane == 1 ? mid : (lane == 2 ? lo : __float2bfloat16(0.f)));
+            if (lane == 0 && ok && wc != w0) differs = true;
         }
     }
     if (differs) atomicOr(nonuniform + p, 1);
@@ -118,9 +135,9 @@ __global__ void __launch_bounds__(256) gather_tc_kernel(const __nv_bfloat16 *__r
 // ---------------------------------------------------------------------------------------------
 // softmax helpers: a thread owns one row (TMEM lane) and NCH chunks of 32 logit columns
 // ---------------------------------------------------------------------------------------------
-// Row maximum in base-2 units (bias and tail mask applied when SPECIAL); the logits stay in TMEM.
+// Row maximum in base-2 units (SPECIAL: only the first `valid` columns count); the logits stay in TMEM.
 template <bool SPECIAL, int NCH>
-__device__ __forceinline__ float row_max(uint32_t tS, float scale_log2, const float *bias_cols, int valid)
+__device__ __forceinline__ float row_max(uint32_t tS, float scale_log2, int valid)
 {
     float m0 = -INFINITY, m1 = -INFINITY;
     uint32_t a[2][32];
@@ -139,7 +156,6 @@ __device__ __forceinline__ float row_max(uint32_t tS, float scale_log2, const fl
 #pragma unroll
             for (int c = 0; c < 32; ++c) {
                 float v = __uint_as_float(a[q & 1][c]) * scale_log2;
-                if (bias_cols) v += __ldg(bias_cols + q * 32 + c);
                 if (q * 32 + c >= valid) v = -INFINITY;
                 m0 = fmaxf(m0, v);
             }
@@ -152,8 +168,7 @@ __device__ __forceinline__ float row_max(uint32_t tS, float scale_log2, const fl
 // (16 columns per chunk) and returns their fp32 row sum.  Each chunk is staged (all scalings, then
 // all exponentials, ...) so that independent operations interleave.
 template <bool SPECIAL, int NCH>
-__device__ __forceinline__ float exp_pass(uint32_t tS, uint32_t tP, float scale_log2, float neg_m,
-                                          const float *bias_cols, int valid)
+__device__ __forceinline__ float exp_pass(uint32_t tS, uint32_t tP, float scale_log2, float neg_m, int valid)
 {
     const uint64_t scale2 = pack2(scale_log2, scale_log2), negm2 = pack2(neg_m, neg_m);
     uint64_t sum2 = pack2(0.f, 0.f), sum2b = pack2(0.f, 0.f);
@@ -212,8 +227,7 @@ __device__ __forceinline__ float exp_pass(uint32_t tS, uint32_t tP, float scale_
         } else {
 #pragma unroll
             for (int c = 0; c < 32; c += 2) {
-                float v0 = __uint_as_float(a[q & 1][c]) * scale_log2, v1 = __uint_as_float(a[q & 1][c + 1]) * scale_log2;
-                if (bias_cols) { v0 += __ldg(bias_cols + q * 32 + c); v1 += __ldg(bias_cols + q * 32 + c + 1); }
+                const float v0 = __uint_as_float(a[q & 1][c]) * scale_log2, v1 = __uint_as_float(a[q & 1][c + 1]) * scale_log2;
                 const float p0 = (q * 32 + c < valid) ? fast_exp2(v0 + neg_m) : 0.f;
                 const float p1 = (q * 32 + c + 1 < valid) ? fast_exp2(v1 + neg_m) : 0.f;
                 sum0 += p0 + p1;
@@ -238,7 +252,7 @@ __device__ __forceinline__ float exp_pass(uint32_t tS, uint32_t tP, float scale_
 template <int D>
 __global__ void __launch_bounds__(NTHREADS, 1)
 attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
-                 const __grid_constant__ CUtensorMap mapV, const float *__restrict__ bias,
+                 const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapX,
                  const int *__restrict__ nonuniform, __nv_bfloat16 *__restrict__ O, int q_heads,
                  int kv_heads, int n_q, int n_core, int n_pad, float scale_log2, int tiles_x, int n_items_total,
                  int q_row0, int n_q_total, int tail_start, int *__restrict__ status)
@@ -258,6 +272,9 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
     auto item_bh = [&](int k) { return ((int)blockIdx.x + k * (int)gridDim.x) / tiles_x; };
     auto item_q0 = [&](int k) { return (((int)blockIdx.x + k * (int)gridDim.x) % tiles_x) * (2 * BM); };
     auto prob_of = [&](int bh) { return (bh / q_heads) * kv_heads + (int)(((int64_t)(bh % q_heads) * kv_heads) / q_heads); };
+    // does item k take the bias MMA?  (weights differ, or the last block is only partly filled)
+    const bool ragged_end = n_core % BN != 0;
+    auto item_bias = [&](int k) { return ragged_end || __ldg(nonuniform + prob_of(item_bh(k))) != 0; };
 
     // a CTA that gave up on a wait poisons the launch: the remaining CTAs leave at once
     if (*reinterpret_cast<volatile int *>(status) != 0) return;
@@ -279,6 +296,11 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
         bar->abort_flag = 0;
         fence_barrier_init();
     }
+    // the constant A operand of the bias MMA: every row (1, 1, 1, 0, 0, 0, 0, 0) in both 16-byte halves,
+    // so that the 32-byte swizzle (which exchanges the halves of some rows) leaves it unchanged
+    for (int i = threadIdx.x; i < BM * 16 / 2; i += NTHREADS)
+        reinterpret_cast<uint32_t *>(smem + SM::OFF_ONES)[i] = (i & 3) == 0 ? 0x3F803F80u : ((i & 3) == 1 ? 0x00003F80u : 0u);
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     if (warp == MMA_WARP) tmem_alloc(&bar->tmem_base, TMEM_COLS);
     tc_fence_before();
     __syncthreads();
@@ -298,9 +320,11 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
             // Blocks are numbered G = k nblk + j along the CTA's whole stream (item k, block j).
             auto load_k = [&](int G) {
                 const int s = G % STAGES, prob = prob_of(item_bh(G / nblk));
-                mbar_expect_tx(&bar->k_full[s], SM::K_BLOCK);
+                const bool with_bias = item_bias(G / nblk);
+                mbar_expect_tx(&bar->k_full[s], SM::K_BLOCK + (with_bias ? SM::X_BLOCK : 0));
                 for (int kh = 0; kh < KH; ++kh)
                     tma_load_3d(smem + SM::OFF_K + s * SM::K_BLOCK + kh * (BN * 128), &mapK, &bar->k_full[s], kh * 64, (G % nblk) * BN, prob);
+                if (with_bias) tma_load_3d(smem + SM::OFF_X + s * SM::X_BLOCK, &mapX, &bar->k_full[s], 0, (G % nblk) * BN, prob);
             };
             auto load_v = [&](int G) {
                 const int s = G % STAGES, prob = prob_of(item_bh(G / nblk));
@@ -351,7 +375,9 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
             const uint64_t dQ = umma_desc_k128(smem_u32(smem + SM::OFF_Q));
             const uint64_t dK = umma_desc_k128(smem_u32(smem + SM::OFF_K));
             const uint64_t dV = umma_desc_k128(smem_u32(smem + SM::OFF_V));
-            auto issue_qk = [&](int t, int s) {
+            const uint64_t dX = umma_desc_k32(smem_u32(smem + SM::OFF_X));
+            const uint64_t dOnes = umma_desc_k32(smem_u32(smem + SM::OFF_ONES));
+            auto issue_qk = [&](int t, int s, bool with_bias) {
                 const uint64_t a0 = dQ + (uint64_t)(t * (SM::Q_TILE >> 4));
                 const uint64_t b0 = dK + (uint64_t)(s * (SM::K_BLOCK >> 4));
 #pragma unroll
@@ -360,6 +386,8 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                     for (int ks = 0; ks < 4; ++ks)
                         mma_ss(tmem + t * 128, a0 + (uint64_t)(kh * (BM * 128 >> 4) + ks * 2),
                                b0 + (uint64_t)(kh * (BN * 128 >> 4) + ks * 2), IDESC_QK, (kh | ks) != 0);
+                // S += ones x (log2 w / scale_log2 in three bf16 terms)^T
+                if (with_bias) mma_ss(tmem + t * 128, dOnes, dX + (uint64_t)(s * (SM::X_BLOCK >> 4)), IDESC_QK, 1u);
             };
             auto issue_pv = [&](int t, int s, bool acc) {
                 const uint64_t b0 = dV + (uint64_t)(s * (SM::V_BLOCK >> 4));
@@ -373,18 +401,21 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
             bool ok = mbar_wait(&bar->q_full, 0) && mbar_wait(&bar->k_full[0], 0);
             if (ok) {
                 tc_fence_after();
-                for (int t = 0; t < 2; ++t) { issue_qk(t, 0); tc_commit(&bar->s_full[t]); }
+                const bool b0 = item_bias(0);
+                for (int t = 0; t < 2; ++t) { issue_qk(t, 0, b0); tc_commit(&bar->s_full[t]); }
                 if (nblk == 1) tc_commit(&bar->q_free);                        // item 0 needs its queries no more
                 tc_commit(&bar->kv_free[0]);                                   // event 0
             }
             // Iteration G: O += P V of block G, then S = Q K^T of block G + 1 - which may be the first
             // block of the next item: the tensor pipe runs on while the softmax warps finish an item.
             int j = 0, k = 0;                                                  // block G = item k, block j
+            bool bias_next = n_items > 0 && item_bias(0);                      // of the item block G + 1 belongs to
             for (int G = 0; G < total && ok; ++G) {
                 const int s = G % STAGES;
                 const bool more = G + 1 < total;
                 const int sn = (G + 1) % STAGES;
                 const bool last = j == nblk - 1;                               // last block of item k
+                if (last && more) bias_next = item_bias(k + 1);
                 if (more) ok = mbar_wait(&bar->k_full[sn], (uint32_t)((G + 1) / STAGES) & 1u);
                 ok = ok && mbar_wait(&bar->v_full[s], (uint32_t)(G / STAGES) & 1u);
                 for (int t = 0; t < 2 && ok; ++t) {
@@ -401,7 +432,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                         // the next item's queries are needed only now, after this item's last O += P V went out
                         if (last && t == 0) ok = mbar_wait(&bar->q_full, (uint32_t)(k + 1) & 1u);
                         if (!ok) break;
-                        issue_qk(t, sn);
+                        issue_qk(t, sn, bias_next);
                         tc_commit(&bar->s_full[t]);
                     }
                 }
@@ -429,25 +460,23 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
         bool ok = true;
         int G = 0;
         for (int k = 0; k < n_items && ok; ++k) {
-            const int bh = item_bh(k), q0 = item_q0(k), prob = prob_of(bh);
-            const bool use_bias = nonuniform[prob] != 0;
-            const float *bp = bias + (int64_t)prob * n_pad + cq * 32;
+            const int bh = item_bh(k), q0 = item_q0(k);
             float m_ref[2] = {-INFINITY, -INFINITY}, l[2] = {0.f, 0.f};
             for (int j = 0; j < nblk && ok; ++j, ++G) {
-                const float *bcols = use_bias ? bp + j * BN : nullptr;
 #pragma unroll
                 for (int t = 0; t < 2; ++t) {
                     // A row sees the list up to its own entry of the causal tail (if there is one), so
                     // the visible columns are a prefix of the list; of this thread's 32, `valid` exist.
+                    // Without a tail every block takes the plain form: the bias MMA has added log2 w and
+                    // hidden the columns beyond the list.
                     int valid = n_core - j * BN - cq * 32;
-                    bool ragged = valid < 32;
+                    bool special = false;
                     if (has_tail) {
                         const int64_t seen = (int64_t)tail_start + q0 + t * BM + row + 1;
                         if (seen < n_core) valid = (int)seen - j * BN - cq * 32;
                         // warp-uniform, because both forms of the two passes contain warp-collective TMEM loads
-                        ragged = __any_sync(0xffffffffu, valid < 32);
+                        special = __any_sync(0xffffffffu, valid < 32);
                     }
-                    const bool special = use_bias || ragged;           // per-column bias and/or a ragged end
                     const uint32_t tS = tmem + lane_addr + t * 128 + cq * 32;   // this thread's 32 logit columns
                     const uint32_t tP = tS;                 // their bf16 probabilities overwrite the first 16 of them
                     const uint32_t tO = tmem + lane_addr + 256 + t * 128 + cq * (D / 4);   // its quarter of the accumulator
@@ -455,8 +484,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                     if (!ok) break;
                     tc_fence_after();
                     // ---- pass 1: row maximum over the four quarters ----
-                    const float mh = special ? row_max<true, 1>(tS, scale_log2, bcols, valid)
-                                             : row_max<false, 1>(tS, scale_log2, bcols, valid);
+                    const float mh = special ? row_max<true, 1>(tS, scale_log2, valid) : row_max<false, 1>(tS, scale_log2, valid);
                     bar->xchg[t][cq][row] = mh;
                     asm volatile("bar.sync 1, 512;" ::: "memory");
                     const float mx = fmaxf(fmaxf(bar->xchg[t][0][row], bar->xchg[t][1][row]),
@@ -480,8 +508,8 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                         if (grow) m_ref[t] = mx;
                     }
                     // ---- pass 2: probabilities and running denominator ----
-                    l[t] += special ? exp_pass<true, 1>(tS, tP, scale_log2, -m_ref[t], bcols, valid)
-                                    : exp_pass<false, 1>(tS, tP, scale_log2, -m_ref[t], bcols, valid);
+                    l[t] += special ? exp_pass<true, 1>(tS, tP, scale_log2, -m_ref[t], valid)
+                                    : exp_pass<false, 1>(tS, tP, scale_log2, -m_ref[t], valid);
                     tmem_wait_st();
                     tc_fence_before();
                     mbar_arrive(&bar->p_ready[t]);
@@ -533,18 +561,20 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
 // ---------------------------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------------------------
-// 3-D bf16 tensor [d2][d1][d0] (d0 contiguous), box {64, box_rows, 1}, 128-byte swizzle
-static bool make_map(CUtensorMap *map, const void *base, uint64_t d0, uint64_t d1, uint64_t d2, uint32_t box_rows)
+// 3-D bf16 tensor [d2][d1][d0] (d0 contiguous), box {64, box_rows, 1} with the 128-byte swizzle, or
+// (narrow) box {16, box_rows, 1} with the 32-byte swizzle
+static bool make_map(CUtensorMap *map, const void *base, uint64_t d0, uint64_t d1, uint64_t d2, uint32_t box_rows,
+                     bool narrow = false)
 {
     sm100::EncodeTiledFn fn = sm100::tensor_map_encoder();
     if (!fn) return false;
     cuuint64_t dims[3] = {d0, d1, d2};
     cuuint64_t strides[2] = {d0 * 2, d0 * d1 * 2};
-    cuuint32_t box[3] = {64, box_rows, 1};
+    cuuint32_t box[3] = {narrow ? 16u : 64u, box_rows, 1};
     cuuint32_t estr[3] = {1, 1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+              CU_TENSOR_MAP_INTERLEAVE_NONE, narrow ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_128B,
+              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 static int sm_count()
@@ -569,19 +599,21 @@ static int launch(const __nv_bfloat16 *Q, const __nv_bfloat16 *K, const __nv_bfl
     const int problems = p->batch * p->kv_heads;
     __nv_bfloat16 *Kc = reinterpret_cast<__nv_bfloat16 *>(ws + L.Kc);
     __nv_bfloat16 *Vt = reinterpret_cast<__nv_bfloat16 *>(ws + L.Vc);
-    float *bias = reinterpret_cast<float *>(ws + L.bias);
+    __nv_bfloat16 *Bx = reinterpret_cast<__nv_bfloat16 *>(ws + L.bx);
     int *flags = reinterpret_cast<int *>(ws + L.flags);
     int *status = flags + problems;
-    CUtensorMap mQ, mK, mV;
+    CUtensorMap mQ, mK, mV, mX;
     if (!make_map(&mQ, Q, D, (uint64_t)n_q_total, (uint64_t)p->batch * p->q_heads, BM) ||
         !make_map(&mK, Kc, D, (uint64_t)n_pad, (uint64_t)problems, BN) ||
-        !make_map(&mV, Vt, (uint64_t)n_pad, D, (uint64_t)problems, D))
+        !make_map(&mV, Vt, (uint64_t)n_pad, D, (uint64_t)problems, D) ||
+        !make_map(&mX, Bx, 16, (uint64_t)n_pad, (uint64_t)problems, BN, true))
         return ELM_ERR_CUDA;
+    const float scale_log2 = (float)(1.4426950408889634 / sqrt((double)D));
     {
         StageTimer t(timed ? ELM_STAGE_GATHER : -1, st, 1);
         ELM_CUDA_TRY(cudaMemsetAsync(flags, 0, sizeof(int) * (size_t)(problems + 1), st));
         gather_tc_kernel<D><<<dim3((unsigned)(n_pad / 32), (unsigned)problems), 256, 0, st>>>(
-            K, V, idx, w, p->n_kv, n_core, n_pad, Kc, Vt, bias, flags);
+            K, V, idx, w, p->n_kv, n_core, n_pad, Kc, Vt, Bx, 1.f / scale_log2, flags);
         count_launches(1);
         ELM_CUDA_TRY(cudaGetLastError());
     }
@@ -593,8 +625,7 @@ static int launch(const __nv_bfloat16 *Q, const __nv_bfloat16 *K, const __nv_bfl
     const int64_t items = (int64_t)tiles_x * p->batch * p->q_heads;
     if (items > 0x7fffffff / 64) return ELM_ERR_SHAPE;
     const int ctas = (int)(items < sm_count() ? items : sm_count());
-    const float scale_log2 = (float)(1.4426950408889634 / sqrt((double)D));
-    kern<<<ctas, NTHREADS, Smem<D>::TOTAL, st>>>(mQ, mK, mV, bias, flags, O, p->q_heads, p->kv_heads, p->n_q,
+    kern<<<ctas, NTHREADS, Smem<D>::TOTAL, st>>>(mQ, mK, mV, mX, flags, O, p->q_heads, p->kv_heads, p->n_q,
                                                  n_core, n_pad, scale_log2, tiles_x, (int)items, (int)win.q_row0,
                                                  (int)n_q_total, win.tail_start, status);
     count_launches(1);

@@ -45,6 +45,7 @@ inline int cuda_status(cudaError_t e) { return e == cudaSuccess ? ELM_OK : ELM_E
     } while (0)
 
 int validate_params(const elm_params *p);
+int validate_attend_params(const elm_params *p);
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 inline size_t elt_bytes(int dtype) { return dtype == ELM_BF16 ? 2 : 4; }
 

@@ -175,6 +175,17 @@ __device__ __forceinline__ uint64_t umma_desc_k128(uint32_t smem_addr)
     d |= (uint64_t)2 << 61;                            // SWIZZLE_128B
     return d;
 }
+// The same for a K-major tile of rows x 16 bf16 (32 B per row), 32-byte swizzle; 8-row groups 256 B apart.
+__device__ __forceinline__ uint64_t umma_desc_k32(uint32_t smem_addr)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3FFFF) >> 4);
+    d |= (uint64_t)1 << 16;
+    d |= (uint64_t)(256 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)6 << 61;                            // SWIZZLE_32B
+    return d;
+}
 // kind::f16 instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M x N tile
 __host__ __device__ constexpr uint32_t umma_idesc_bf16(int M, int N)
 {
