@@ -210,11 +210,12 @@ int elm_express_workspace_bytes(const elm_params *params, int32_t mbar, size_t *
  * (weight 2^(i-q), q = the current Compress2 depth), and the tokens since the last level-0 Halve call
  * up to t (weight 2^-q).  The first 4 n_out tokens attend exactly (causally).
  *   Q, O       [batch][q_heads][n_kv][d] (params->n_q must equal n_kv); K, V as for elm_compress.
- *   Limits     rounds with a thinning factor above mbar (Subsample active) are not built yet:
- *              n_kv <= n_out 4^(mbar/2 + 1), else ELM_ERR_SHAPE; level-0 Halve calls need >= 2 points
- *              (2 (R-1) <= log2_nout + 1).
+ *   Limits     level-0 Halve calls need >= 2 points: min(2 (R-1), mbar) <= log2_nout + 1, else ELM_ERR_SHAPE.
  *   workspace  at least elm_express_prefill_workspace_bytes(params, mbar) bytes, 256-byte aligned.
- * One attention launch per epoch (the tokens between two level-0 Halve calls).
+ * In a round whose thinning factor exceeds mbar (Subsample active) the kept points differ from problem to
+ * problem; a token that is not kept still attends to itself with the weight of a point of S_0.
+ * One attention launch per window of about 1024 tokens, over every cache entry that some token of the
+ * window sees; each entry carries the span of tokens that see it.
  */
 int elm_express_prefill_workspace_bytes(const elm_params *params, int32_t mbar, size_t *bytes);
 int elm_express_prefill(const void *Q, const void *K, const void *V, const elm_params *params, int32_t mbar,

@@ -52,7 +52,10 @@ __global__ void __launch_bounds__(128) attend_simt_kernel(const Tin *__restrict_
                                                           const float *__restrict__ bias,
                                                           Tin *__restrict__ O, int q_heads,
                                                           int kv_heads, int64_t n_q, int n_core,
-                                                          int64_t q_row0, int64_t n_q_total, int tail_start)
+                                                          int64_t q_row0, int64_t n_q_total, int tail_start,
+                                                          const int32_t *__restrict__ birth,
+                                                          const int32_t *__restrict__ death, int n_pad,
+                                                          float *__restrict__ lse)
 {
     constexpr int BM = 64, BN = 32;
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -64,6 +67,8 @@ __global__ void __launch_bounds__(128) attend_simt_kernel(const Tin *__restrict_
     T *rowsum = rowscale + BM;                      // [BM] running denominator
     T *rowmax = rowsum + BM;                        // [BM] running maximum
     T *sbias = rowmax + BM;                         // [BN]
+    int32_t *sbirth = reinterpret_cast<int32_t *>(sbias + BN);   // [BN] lifetimes of the chunk's entries
+    int32_t *sdeath = sbirth + BN;                               // [BN]
 
     const int tid = threadIdx.x;
     const int bh = blockIdx.y;                      // batch * q_heads + head
@@ -98,7 +103,13 @@ __global__ void __launch_bounds__(128) attend_simt_kernel(const Tin *__restrict_
             Kt[k * BN + c] = ok ? load_as<T>(Kp, (int64_t)(c0 + c) * D + k) : (T)0;
             Vs[c * D + k] = ok ? load_as<T>(Vp, (int64_t)(c0 + c) * D + k) : (T)0;
         }
-        if (tid < BN) sbias[tid] = (c0 + tid < n_core) ? (T)bp[c0 + tid] : (T)0;
+        if (tid < BN) {
+            sbias[tid] = (c0 + tid < n_core) ? (T)bp[c0 + tid] : (T)0;
+            if (birth) {
+                sbirth[tid] = (c0 + tid < n_core) ? birth[prob * n_pad + c0 + tid] : 0x7fffffff;
+                sdeath[tid] = (c0 + tid < n_core) ? death[prob * n_pad + c0 + tid] : 0x7fffffff;
+            }
+        }
         __syncthreads();
         T s[4][4];
 #pragma unroll
@@ -119,8 +130,12 @@ __global__ void __launch_bounds__(128) attend_simt_kernel(const Tin *__restrict_
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 int col = 4 * tx + c;
-                // a row sees the list up to its own entry of the causal tail
-                const bool seen = c0 + col < n_core && (int64_t)(c0 + col) <= (int64_t)tail_start + q0 + 4 * ty + r;
+                // a row sees the entries alive at its own position, or (tail rule) the list up to its own
+                // entry of the causal tail
+                const int64_t trow = q_row0 + q0 + 4 * ty + r;
+                const bool seen = c0 + col < n_core &&
+                                  (birth ? (sbirth[col] <= trow && trow < sdeath[col])
+                                         : (int64_t)(c0 + col) <= (int64_t)tail_start + q0 + 4 * ty + r);
                 S[(4 * ty + r) * (BN + 1) + col] = seen ? s[r][c] * scale + sbias[col] : (T)-INFINITY;
             }
         __syncthreads();
@@ -166,6 +181,7 @@ __global__ void __launch_bounds__(128) attend_simt_kernel(const Tin *__restrict_
         T inv = (T)1 / rowsum[4 * ty + r];
 #pragma unroll
         for (int o = 0; o < OC; ++o) store_from(Op, q * D + tx + 8 * o, acc[r][o] * inv);
+        if (lse && tx == 0) lse[(int64_t)bh * n_q_total + q_row0 + q] = (float)(rowmax[4 * ty + r] + log2(rowsum[4 * ty + r]));
     }
 }
 
@@ -191,12 +207,13 @@ static int launch_attend_simt(const Tin *Q, const Tin *Kc, const Tin *Vc, const 
                               const elm_params *p, int n_core, cudaStream_t st, const AttendWindow &win = AttendWindow())
 {
     constexpr int BM = 64, BN = 32;
-    const size_t smem = sizeof(T) * (size_t)(D * BM + D * BN + BN * D + BM * (BN + 1) + 3 * BM + BN);
+    const size_t smem = sizeof(T) * (size_t)(D * BM + D * BN + BN * D + BM * (BN + 1) + 3 * BM + BN) + 2 * BN * sizeof(int32_t);
     auto kern = attend_simt_kernel<Tin, T, D>;
     ELM_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     dim3 grid((unsigned)((p->n_q + BM - 1) / BM), (unsigned)(p->batch * p->q_heads));
     kern<<<grid, 128, smem, st>>>(Q, Kc, Vc, bias, O, p->q_heads, p->kv_heads, p->n_q, n_core, win.q_row0,
-                                  win.n_q_total ? win.n_q_total : (int64_t)p->n_q, win.tail_start);
+                                  win.n_q_total ? win.n_q_total : (int64_t)p->n_q, win.tail_start, win.birth, win.death,
+                                  (n_core + 127) / 128 * 128, win.lse);
     count_launches(1);
     return cuda_status(cudaGetLastError());
 }
@@ -288,7 +305,7 @@ int attend_enqueue(const void *Q, const void *K, const void *V, const int32_t *i
 {
     unsigned char *ws = (unsigned char *)workspace;
     const bool det = params->precision == ELM_PREC_FP64_DET;
-    const bool whole = win.q_row0 == 0 && win.n_q_total == 0 && win.tail_start == 0x7fffffff;
+    const bool whole = win.q_row0 == 0 && win.n_q_total == 0 && win.tail_start == 0x7fffffff && !win.birth && !win.lse;
     if (whole && attend_decode_applies(params)) return attend_decode(Q, K, V, idx, w, n_core, params, O, ws, st, true);
     if (params->dtype == ELM_F32) {
         return det ? attend_impl<float, double>((const float *)Q, (const float *)K, (const float *)V, idx, w, n_core, params, (float *)O, ws, st, win)

@@ -24,10 +24,21 @@ AttendLayout attend_layout(const elm_params *p, int32_t n_core);
 // number of query rows of the launch; they are rows q_row0 .. q_row0 + n_q - 1 of each head's
 // n_q_total rows.  List entries from tail_start on are visible to row r of the launch only up to
 // entry tail_start + r (Algorithm 5 in prefill: the tail holds the launch's own tokens in order).
+//
+// Lifetimes (Thinformer Express in prefill, where the cache changes from token to token): when `birth` is
+// set, entry c of problem p is visible to the query row whose index within its head is t iff
+// birth[p][c] <= t < death[p][c], and the tail rule is not used.  Both arrays are [problems][n_pad],
+// n_pad = n_core rounded up to 128; blk_birth / blk_death [problems][n_pad / 128] hold the largest birth and
+// the smallest death of each block of 128 entries (a block that every row of a tile sees whole takes the
+// unmasked path).  `lse`, if set, receives log2 of each row's softmax denominator (logits in base 2,
+// weights included) at [batch * q_heads][n_q_total].
 struct AttendWindow {
     int64_t q_row0 = 0;
     int64_t n_q_total = 0;               // 0: params->n_q
     int32_t tail_start = 0x7fffffff;     // no tail
+    const int32_t *birth = nullptr, *death = nullptr;
+    const int32_t *blk_birth = nullptr, *blk_death = nullptr;
+    float *lse = nullptr;
 };
 
 // elm_attend after argument validation

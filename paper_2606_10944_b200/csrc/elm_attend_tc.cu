@@ -135,9 +135,10 @@ __global__ void __launch_bounds__(256) gather_tc_kernel(const __nv_bfloat16 *__r
 // ---------------------------------------------------------------------------------------------
 // softmax helpers: a thread owns one row (TMEM lane) and NCH chunks of 32 logit columns
 // ---------------------------------------------------------------------------------------------
-// Row maximum in base-2 units (SPECIAL: only the first `valid` columns count); the logits stay in TMEM.
+// Row maximum in base-2 units (SPECIAL: only the columns whose bit is set in `vmask` count); the logits
+// stay in TMEM.
 template <bool SPECIAL, int NCH>
-__device__ __forceinline__ float row_max(uint32_t tS, float scale_log2, int valid)
+__device__ __forceinline__ float row_max(uint32_t tS, float scale_log2, uint32_t vmask)
 {
     float m0 = -INFINITY, m1 = -INFINITY;
     uint32_t a[2][32];
@@ -156,7 +157,7 @@ __device__ __forceinline__ float row_max(uint32_t tS, float scale_log2, int vali
 #pragma unroll
             for (int c = 0; c < 32; ++c) {
                 float v = __uint_as_float(a[q & 1][c]) * scale_log2;
-                if (q * 32 + c >= valid) v = -INFINITY;
+                if (!((vmask >> c) & 1u)) v = -INFINITY;
                 m0 = fmaxf(m0, v);
             }
         }
@@ -168,7 +169,7 @@ __device__ __forceinline__ float row_max(uint32_t tS, float scale_log2, int vali
 // (16 columns per chunk) and returns their fp32 row sum.  Each chunk is staged (all scalings, then
 // all exponentials, ...) so that independent operations interleave.
 template <bool SPECIAL, int NCH>
-__device__ __forceinline__ float exp_pass(uint32_t tS, uint32_t tP, float scale_log2, float neg_m, int valid)
+__device__ __forceinline__ float exp_pass(uint32_t tS, uint32_t tP, float scale_log2, float neg_m, uint32_t vmask)
 {
     const uint64_t scale2 = pack2(scale_log2, scale_log2), negm2 = pack2(neg_m, neg_m);
     uint64_t sum2 = pack2(0.f, 0.f), sum2b = pack2(0.f, 0.f);
@@ -228,8 +229,8 @@ __device__ __forceinline__ float exp_pass(uint32_t tS, uint32_t tP, float scale_
 #pragma unroll
             for (int c = 0; c < 32; c += 2) {
                 const float v0 = __uint_as_float(a[q & 1][c]) * scale_log2, v1 = __uint_as_float(a[q & 1][c + 1]) * scale_log2;
-                const float p0 = (q * 32 + c < valid) ? fast_exp2(v0 + neg_m) : 0.f;
-                const float p1 = (q * 32 + c + 1 < valid) ? fast_exp2(v1 + neg_m) : 0.f;
+                const float p0 = ((vmask >> c) & 1u) ? fast_exp2(v0 + neg_m) : 0.f;
+                const float p1 = ((vmask >> (c + 1)) & 1u) ? fast_exp2(v1 + neg_m) : 0.f;
                 sum0 += p0 + p1;
                 pk[c >> 1] = __byte_perm(__float_as_uint(p0) + 0x8000u, __float_as_uint(p1) + 0x8000u, 0x7632);
             }
@@ -255,7 +256,9 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                  const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapX,
                  const int *__restrict__ nonuniform, __nv_bfloat16 *__restrict__ O, int q_heads,
                  int kv_heads, int n_q, int n_core, int n_pad, float scale_log2, int tiles_x, int n_items_total,
-                 int q_row0, int n_q_total, int tail_start, int *__restrict__ status)
+                 int q_row0, int n_q_total, int tail_start, const int32_t *__restrict__ birth,
+                 const int32_t *__restrict__ death, const int32_t *__restrict__ blk_birth,
+                 const int32_t *__restrict__ blk_death, float *__restrict__ lse, int *__restrict__ status)
 {
     using SM = Smem<D>;
     constexpr int KH = SM::KH;
@@ -461,6 +464,8 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
         int G = 0;
         for (int k = 0; k < n_items && ok; ++k) {
             const int bh = item_bh(k), q0 = item_q0(k);
+            const int64_t life0 = (int64_t)prob_of(bh) * n_pad + cq * 32;     // this thread's first entry of the lifetime arrays
+            const int64_t blk0 = (int64_t)prob_of(bh) * nblk;
             float m_ref[2] = {-INFINITY, -INFINITY}, l[2] = {0.f, 0.f};
             for (int j = 0; j < nblk && ok; ++j, ++G) {
 #pragma unroll
@@ -469,13 +474,28 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                     // the visible columns are a prefix of the list; of this thread's 32, `valid` exist.
                     // Without a tail every block takes the plain form: the bias MMA has added log2 w and
                     // hidden the columns beyond the list.
-                    int valid = n_core - j * BN - cq * 32;
+                    // `special` must be warp-uniform: both forms of the two passes contain warp-collective TMEM loads.
+                    uint32_t vmask = 0xffffffffu;
                     bool special = false;
-                    if (has_tail) {
+                    if (birth) {
+                        // lifetimes: the block is seen whole by this warp's 32 rows unless an entry is born
+                        // after the first or dies before the last of them
+                        const int t_first = q_row0 + q0 + t * BM + (warp & 3) * 32;
+                        special = !(__ldg(blk_birth + blk0 + j) <= t_first && __ldg(blk_death + blk0 + j) > t_first + 31);
+                        if (special) {
+                            const int t_row = t_first + lane;
+                            const int32_t *bp = birth + life0 + j * BN, *dp = death + life0 + j * BN;
+                            vmask = 0u;
+#pragma unroll 8
+                            for (int c = 0; c < 32; ++c)
+                                vmask |= (uint32_t)(__ldg(bp + c) <= t_row && t_row < __ldg(dp + c)) << c;
+                        }
+                    } else if (has_tail) {
+                        int valid = n_core - j * BN - cq * 32;
                         const int64_t seen = (int64_t)tail_start + q0 + t * BM + row + 1;
                         if (seen < n_core) valid = (int)seen - j * BN - cq * 32;
-                        // warp-uniform, because both forms of the two passes contain warp-collective TMEM loads
                         special = __any_sync(0xffffffffu, valid < 32);
+                        vmask = valid >= 32 ? 0xffffffffu : (valid <= 0 ? 0u : (1u << valid) - 1u);
                     }
                     const uint32_t tS = tmem + lane_addr + t * 128 + cq * 32;   // this thread's 32 logit columns
                     const uint32_t tP = tS;                 // their bf16 probabilities overwrite the first 16 of them
@@ -484,7 +504,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                     if (!ok) break;
                     tc_fence_after();
                     // ---- pass 1: row maximum over the four quarters ----
-                    const float mh = special ? row_max<true, 1>(tS, scale_log2, valid) : row_max<false, 1>(tS, scale_log2, valid);
+                    const float mh = special ? row_max<true, 1>(tS, scale_log2, vmask) : row_max<false, 1>(tS, scale_log2, vmask);
                     bar->xchg[t][cq][row] = mh;
                     asm volatile("bar.sync 1, 512;" ::: "memory");
                     const float mx = fmaxf(fmaxf(bar->xchg[t][0][row], bar->xchg[t][1][row]),
@@ -508,8 +528,8 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                         if (grow) m_ref[t] = mx;
                     }
                     // ---- pass 2: probabilities and running denominator ----
-                    l[t] += special ? exp_pass<true, 1>(tS, tP, scale_log2, -m_ref[t], valid)
-                                    : exp_pass<false, 1>(tS, tP, scale_log2, -m_ref[t], valid);
+                    l[t] += special ? exp_pass<true, 1>(tS, tP, scale_log2, -m_ref[t], vmask)
+                                    : exp_pass<false, 1>(tS, tP, scale_log2, -m_ref[t], vmask);
                     tmem_wait_st();
                     tc_fence_before();
                     mbar_arrive(&bar->p_ready[t]);
@@ -524,8 +544,10 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                 tc_fence_after();
                 bar->xchg[t][cq][row] = l[t];
                 asm volatile("bar.sync 1, 512;" ::: "memory");
-                const float inv = 1.f / ((bar->xchg[t][0][row] + bar->xchg[t][1][row]) + (bar->xchg[t][2][row] + bar->xchg[t][3][row]));
+                const float l_all = (bar->xchg[t][0][row] + bar->xchg[t][1][row]) + (bar->xchg[t][2][row] + bar->xchg[t][3][row]);
+                const float inv = 1.f / l_all;
                 const int64_t qrow = (int64_t)q0 + t * BM + row;
+                if (lse && cq == 0 && qrow < n_q) lse[(int64_t)bh * n_q_total + q_row0 + qrow] = m_ref[t] + log2f(l_all);
                 __nv_bfloat16 *dst = O + ((int64_t)bh * n_q_total + q_row0 + qrow) * D + cq * (D / 4);
                 uint32_t o[32];
                 if (D == 128) tmem_ld32(tO, o);
@@ -627,7 +649,8 @@ static int launch(const __nv_bfloat16 *Q, const __nv_bfloat16 *K, const __nv_bfl
     const int ctas = (int)(items < sm_count() ? items : sm_count());
     kern<<<ctas, NTHREADS, Smem<D>::TOTAL, st>>>(mQ, mK, mV, mX, flags, O, p->q_heads, p->kv_heads, p->n_q,
                                                  n_core, n_pad, scale_log2, tiles_x, (int)items, (int)win.q_row0,
-                                                 (int)n_q_total, win.tail_start, status);
+                                                 (int)n_q_total, win.tail_start, win.birth, win.death, win.blk_birth,
+                                                 win.blk_death, win.lse, status);
     count_launches(1);
     return cuda_status(cudaGetLastError());
 }

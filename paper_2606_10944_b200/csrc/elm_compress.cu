@@ -750,23 +750,111 @@ static int compress_impl(const Tin *K, const Tin *V, const elm_params *p, uint64
 constexpr int EXPRESS_LANES = 6;       // side streams of the prefill: two per sibling segment
 struct ExpressLayout {
     size_t vmax_bits, cnorm, listA, listB, E, T1, Mpair, rdecay, F, F_stride, total;
-    // prefill only: the output lists of every Compress2 level of a round, the cache list of one
-    // epoch with its weights, the workspace of elm_attend for that list
-    size_t levels, ep_idx, ep_w, ws_attend, ep_cap, ep_stride, ws_attend_stride;
+    // prefill only: the output lists of every Compress2 level of a round; per side stream the cache list
+    // of one launch with its weights and lifetimes and the workspace of elm_attend for that list; log2 of
+    // the softmax denominators (rounds with Subsample: the tokens that were not kept are merged in afterwards)
+    size_t levels, ep_idx, ep_w, ep_birth, ep_death, ep_blk, ws_attend, ep_cap, ep_pad, ep_stride, ws_attend_stride, lse;
     int n_levels;
 };
-// Longest cache list (weighted cache + causal tail) any epoch of the prefill attends over.
-static size_t express_epoch_cap(const elm_params *p, int mbar)
+// Geometry of round r of an Express run (thinning factor m = 2r): Compress2 depth q = min(m, mbar), one
+// point kept per 2^wlog tokens (Subsample, when m > mbar), `seg` tokens and len0 kept points per sibling
+// segment, s0 kept points per level-0 Halve call.
+struct RoundGeom {
+    int m, q, wlog;
+    bool sub;
+    int64_t seg, len0, s0;
+};
+static RoundGeom round_geom(const elm_params *p, int mbar, int r)
 {
-    const size_t n_out = (size_t)1 << p->log2_nout;
-    size_t cap = 4 * n_out;                                   // the exact start: causal attention over 4 n_out tokens
-    const int R = [&]() { size_t v = n_out; int r = 0; while (v < (size_t)p->n_kv) { v *= 4; ++r; } return r; }();
+    RoundGeom g;
+    const int64_t n_out = (int64_t)1 << p->log2_nout;
+    g.m = 2 * r;
+    g.q = g.m < mbar ? g.m : mbar;
+    g.sub = g.m > mbar;
+    g.wlog = g.m - g.q;
+    g.seg = n_out << g.m;
+    g.len0 = n_out << g.q;
+    g.s0 = g.q >= 1 ? (n_out << 2) >> g.q : g.len0;        // q = 0: no Halve call, S_0 only grows
+    return g;
+}
+// Tokens per attention launch of the prefill: windows of about 1024 tokens (whole strata, at most a segment).
+static int64_t prefill_window(const RoundGeom &g)
+{
+    int64_t W = (int64_t)1 << g.wlog;
+    if (W < 1024) W = 1024;
+    return W < g.seg ? W : g.seg;
+}
+
+// The cache entries some token of a window can see, as runs of the round's point lists, each entry with
+// the span of tokens that see it.  In terms of G = the number of kept points of the sibling segment
+// that have arrived (a window covers G in [G0, G1)):
+//   kind 0   E and the finished siblings: always
+//   kind 1   S_i, 1 <= i < q: the output of call c of level i - 1 (u entries) exists from G = (c + 1) A,
+//            A = s0 4^(i-1), until the level-i call that consumes it completes at G = (c / 4 + 1) 4 A
+//   kind 2   S_0: kept point g exists from its own token (which sees itself) until G = (g / s0 + 1) s0
+//   kind 3   S_q: the output of the segment's last call, from G = len0 on
+// G = X is reached right after the X-th kept point: at token kept[X - 1] + 1.
+struct WindowPieces {
+    const int32_t *src[16];
+    int64_t src_off[16];
+    int64_t first[16];          // kind 1: index of the run's first entry within the sibling's part of the list; kind 2: its g
+    int64_t per_call[16];       // kind 1: A
+    int32_t dst_off[17];
+    int32_t unit[16];           // kind 1: u; kind 2: s0
+    float w[16];
+    int8_t kind[16];
+    int n;
+    const int32_t *kept;        // kept points of the round's three siblings (the level-0 input list)
+    int64_t kept_off, len0;
+    int32_t q;
+};
+static int32_t window_pieces(const RoundGeom &g, int64_t n_out, int jj, int64_t G0, int64_t G1, const int32_t *E,
+                             const int32_t *levels, size_t level_stride, const int32_t *kept, WindowPieces &pc)
+{
+    int k = 0;
+    int32_t at = 0;
+    auto piece = [&](const int32_t *src, int64_t off, int64_t count, double wgt, int kind, int64_t first, int64_t unit,
+                     int64_t per_call) {
+        if (count <= 0) return;
+        pc.src[k] = src; pc.src_off[k] = off; pc.w[k] = (float)wgt; pc.dst_off[k] = at;
+        pc.kind[k] = (int8_t)kind; pc.first[k] = first; pc.unit[k] = (int32_t)unit; pc.per_call[k] = per_call;
+        at += (int32_t)count;
+        ++k;
+    };
+    const int q = g.q;
+    piece(E, 0, (1 + jj) * n_out, 1.0, 0, 0, 1, 1);
+    for (int i = q - 1; i >= 1; --i) {
+        const int64_t A = g.s0 << (2 * (i - 1)), u = (g.s0 << (i - 1)) >> 1;
+        const int64_t c_lo = 4 * (G0 / (4 * A)), c_end = G1 / A;
+        piece(levels ? levels + (size_t)(i - 1) * level_stride : nullptr, jj * (g.len0 >> i) + c_lo * u, (c_end - c_lo) * u,
+              ldexp(1.0, i - q), 1, c_lo * u, u, A);
+    }
+    if (q >= 1 && g.sub && G1 >= g.len0) piece(E, (1 + jj) * n_out, n_out, 1.0, 3, 0, 1, 1);
+    const int64_t g_lo = q >= 1 ? (G0 / g.s0) * g.s0 : 0;
+    piece(kept, jj * g.len0 + g_lo, G1 - g_lo, ldexp(1.0, -q), 2, g_lo, g.s0, 1);
+    pc.dst_off[k] = at;
+    pc.n = k;
+    pc.kept = kept;
+    pc.kept_off = jj * g.len0;
+    pc.len0 = g.len0;
+    pc.q = q;
+    return at;
+}
+// Longest cache list any launch of the prefill attends over.
+static size_t express_list_cap(const elm_params *p, int mbar)
+{
+    const int64_t n_out = (int64_t)1 << p->log2_nout;
+    size_t cap = (size_t)(4 * n_out);                         // the exact start: causal attention over 4 n_out tokens
+    const int R = [&]() { int64_t v = n_out; int r = 0; while (v < (int64_t)p->n_kv) { v *= 4; ++r; } return r; }();
     for (int r = 1; r < R; ++r) {
-        const int q = 2 * r < mbar ? 2 * r : mbar;
-        // E (up to 3 n_out before the third sibling ends), up to three call outputs in each S_i, the tail
-        size_t len = 3 * n_out + ((n_out << 2) >> q);
-        for (int i = 1; i < q; ++i) len += 3 * (((n_out << 2) >> q) << (i - 1)) / 2;
-        if (len > cap) cap = len;
+        const RoundGeom g = round_geom(p, mbar, r);
+        const int64_t Wg = prefill_window(g) >> g.wlog;
+        for (int jj = 0; jj < 3; ++jj)
+            for (int64_t G0 = 0; G0 < g.len0; G0 += Wg) {
+                WindowPieces pc;
+                const size_t len = (size_t)window_pieces(g, n_out, jj, G0, G0 + Wg, nullptr, nullptr, 0, nullptr, pc);
+                if (len > cap) cap = len;
+            }
     }
     return cap;
 }
@@ -789,16 +877,22 @@ static ExpressLayout express_layout(const elm_params *p, int mbar = 0, bool pref
     L.rdecay = take(BH * (n / 2 + 1) * ts);
     L.F_stride = 4 * n_out * n_out;        // the first halving of E is one call of 2 n_out pairs
     L.F = take(BH * L.F_stride * ts);
-    L.levels = L.ep_idx = L.ep_w = L.ws_attend = L.ep_cap = L.ep_stride = L.ws_attend_stride = 0;
+    L.levels = L.ep_idx = L.ep_w = L.ep_birth = L.ep_death = L.ep_blk = L.ws_attend = L.ep_cap = L.ep_pad = L.ep_stride = 0;
+    L.ws_attend_stride = L.lse = 0;
     L.n_levels = 0;
     if (prefill) {
         L.n_levels = mbar < 30 ? mbar : 30;
         L.levels = take((size_t)L.n_levels * BH * n * 4);
-        L.ep_cap = express_epoch_cap(p, mbar);
-        // one set per side stream: the epochs of a round are spread over EXPRESS_LANES streams
-        L.ep_stride = align_up(BH * L.ep_cap * 4, 256);
+        L.ep_cap = express_list_cap(p, mbar);
+        L.ep_pad = (L.ep_cap + 127) / 128 * 128;
+        // one set per side stream: the launches of a round are spread over EXPRESS_LANES streams
+        L.ep_stride = align_up(BH * L.ep_pad * 4, 256);
         L.ep_idx = take(EXPRESS_LANES * L.ep_stride);
         L.ep_w = take(EXPRESS_LANES * L.ep_stride);
+        L.ep_birth = take(EXPRESS_LANES * L.ep_stride);
+        L.ep_death = take(EXPRESS_LANES * L.ep_stride);
+        L.ep_blk = take(EXPRESS_LANES * L.ep_stride);          // two arrays of [BH][ep_pad / 128]
+        L.lse = take((size_t)p->batch * p->q_heads * n * 4);
         L.ws_attend_stride = align_up(attend_layout(p, (int32_t)L.ep_cap).total, 256);
         L.ws_attend = take(EXPRESS_LANES * L.ws_attend_stride);
     }
@@ -883,18 +977,146 @@ __global__ void build_list_kernel(ListPieces pc, int64_t src_stride, int32_t *__
     w[pr * cap + i] = pc.w[k];
 }
 
-// Attention of the query rows [t0, t0 + rows) over the list described by `pc` (the last piece is
-// the causal tail: those same tokens).  Thinformer Express, Algorithm 5, in prefill.
-static int express_attend_epoch(const void *Q, const void *K, const void *V, void *O, const elm_params *p, const ExpressLayout &L,
-                                unsigned char *ws, const ListPieces &pc, int64_t t0, int rows, cudaStream_t st, int lane = 0)
+// The list of one prefill window (see WindowPieces): indices, weights, and for every entry the first
+// token that sees it (birth) and the first that does not any more (death); per block of 128 entries the
+// largest birth and the smallest death.  Entries beyond the list (up to n_pad) are given the lifetime
+// "always": the attention kernel hides them by other means.
+__global__ void __launch_bounds__(256) build_window_kernel(WindowPieces pc, int64_t src_stride, int32_t *__restrict__ idx,
+                                                           float *__restrict__ w, int n_core, int n_pad,
+                                                           int32_t *__restrict__ birth, int32_t *__restrict__ death,
+                                                           int32_t *__restrict__ blk_birth, int32_t *__restrict__ blk_death)
+{
+    __shared__ int32_t sb[8], sd[8];
+    const int i = blockIdx.x * 256 + threadIdx.x;
+    const int64_t pr = blockIdx.y;
+    int32_t bt = 0, dt = 0x7fffffff;
+    if (i < n_core) {
+        int k = 0;
+        while (i >= pc.dst_off[k + 1]) ++k;
+        const int64_t o = i - pc.dst_off[k];
+        const int32_t *kept = pc.kept + pr * src_stride + pc.kept_off;
+        auto token_after = [&](int64_t X) { return X > pc.len0 ? 0x7fffffff : kept[X - 1] + 1; };   // G = X is reached
+        idx[pr * n_core + i] = pc.src[k][pr * src_stride + pc.src_off[k] + o];
+        w[pr * n_core + i] = pc.w[k];
+        if (pc.kind[k] == 1) {
+            const int64_t c = (pc.first[k] + o) / pc.unit[k];
+            bt = token_after((c + 1) * pc.per_call[k]);
+            dt = token_after((c / 4 + 1) * 4 * pc.per_call[k]);
+        } else if (pc.kind[k] == 2) {
+            const int64_t g = pc.first[k] + o;
+            bt = kept[g];
+            if (pc.q >= 1) dt = token_after((g / pc.unit[k] + 1) * pc.unit[k]);
+        } else if (pc.kind[k] == 3) {
+            bt = token_after(pc.len0);
+        }
+    }
+    if (i < n_pad) {
+        birth[pr * n_pad + i] = bt;
+        death[pr * n_pad + i] = dt;
+    }
+    int32_t bm = bt, dm = dt;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        bm = max(bm, __shfl_xor_sync(0xffffffffu, bm, o));
+        dm = min(dm, __shfl_xor_sync(0xffffffffu, dm, o));
+    }
+    if ((threadIdx.x & 31) == 0) { sb[threadIdx.x >> 5] = bm; sd[threadIdx.x >> 5] = dm; }
+    __syncthreads();
+    if (threadIdx.x < 2) {
+        const int blk = blockIdx.x * 2 + threadIdx.x, h = threadIdx.x * 4;
+        if (blk < n_pad / 128) {
+            blk_birth[pr * (n_pad / 128) + blk] = max(max(sb[h], sb[h + 1]), max(sb[h + 2], sb[h + 3]));
+            blk_death[pr * (n_pad / 128) + blk] = min(min(sd[h], sd[h + 1]), min(sd[h + 2], sd[h + 3]));
+        }
+    }
+}
+
+// Rounds with Subsample: a token that was not kept is in no list, but Algorithm 5 still lets it attend to
+// itself with the weight of a point of S_0.  One warp per (head, token): merges that single term into the
+// output row, given log2 of the row's denominator over the cache.
+template <typename Tin, typename T>
+__global__ void __launch_bounds__(256) self_merge_kernel(const Tin *__restrict__ Q, const Tin *__restrict__ K,
+                                                         const Tin *__restrict__ V, Tin *__restrict__ O,
+                                                         const float *__restrict__ lse, const int32_t *__restrict__ kept,
+                                                         int q_heads, int kv_heads, int64_t n, int d, int64_t seg,
+                                                         int64_t len0, int wlog, T log2w)
+{
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int64_t rel = (int64_t)blockIdx.x * 8 + warp;                   // token within the round's 3 segments
+    if (rel >= 3 * seg) return;
+    const int bh = blockIdx.y;
+    const int64_t prob = (int64_t)(bh / q_heads) * kv_heads + ((int64_t)(bh % q_heads) * kv_heads) / q_heads;
+    const int64_t t = seg + rel, jj = rel / seg, stratum = (rel % seg) >> wlog;
+    if (kept[prob * n + jj * len0 + stratum] == (int32_t)t) return;        // a kept token is an entry of S_0
+    const Tin *q = Q + ((int64_t)bh * n + t) * d, *k = K + (prob * n + t) * d, *v = V + (prob * n + t) * d;
+    Tin *o = O + ((int64_t)bh * n + t) * d;
+    T dot = 0;
+    for (int e = lane; e < d; e += 32) dot += load_as<T>(q, e) * load_as<T>(k, e);
+#pragma unroll
+    for (int s = 16; s > 0; s >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, s);
+    const T sc = dot * (T)(1.4426950408889634 / sqrt((double)d)) + log2w;
+    const T L = (T)lse[(int64_t)bh * n + t];
+    const T M = sc > L ? sc : L;
+    const T a = (T)exp2((T)(L - M)), b = (T)exp2((T)(sc - M));
+    const T inv = (T)1 / (a + b);
+    for (int e = lane; e < d; e += 32) store_from(o, e, (a * load_as<T>(o, e) + b * load_as<T>(v, e)) * inv);
+}
+
+// Launch-side state of one side stream of the prefill.
+struct PrefillLane {
+    int32_t *idx, *birth, *death, *blk_birth, *blk_death;
+    float *w;
+    unsigned char *ws_attend;
+};
+static PrefillLane prefill_lane(const ExpressLayout &L, unsigned char *ws, int BH, int lane)
+{
+    PrefillLane pl;
+    pl.idx = reinterpret_cast<int32_t *>(ws + L.ep_idx + lane * L.ep_stride);
+    pl.w = reinterpret_cast<float *>(ws + L.ep_w + lane * L.ep_stride);
+    pl.birth = reinterpret_cast<int32_t *>(ws + L.ep_birth + lane * L.ep_stride);
+    pl.death = reinterpret_cast<int32_t *>(ws + L.ep_death + lane * L.ep_stride);
+    pl.blk_birth = reinterpret_cast<int32_t *>(ws + L.ep_blk + lane * L.ep_stride);
+    pl.blk_death = pl.blk_birth + (size_t)BH * (L.ep_pad / 128);
+    pl.ws_attend = ws + L.ws_attend + lane * L.ws_attend_stride;
+    return pl;
+}
+
+// The exact start of Thinformer Express (Algorithm 5) in prefill: token t < rows attends over the tokens 0 .. t.
+static int express_attend_start(const void *Q, const void *K, const void *V, void *O, const elm_params *p, const ExpressLayout &L,
+                                unsigned char *ws, int rows, cudaStream_t st)
+{
+    const int BH = p->batch * p->kv_heads;
+    const PrefillLane pl = prefill_lane(L, ws, BH, 0);
+    if ((size_t)rows > L.ep_cap) return ELM_ERR_WORKSPACE;
+    ListPieces pc = {};
+    pc.n = 1;
+    pc.src[0] = nullptr; pc.src_off[0] = 0; pc.w[0] = 1.f;
+    pc.dst_off[0] = 0; pc.dst_off[1] = rows;
+    build_list_kernel<<<dim3((unsigned)((rows + 255) / 256), (unsigned)BH), 256, 0, st>>>(pc, p->n_kv, pl.idx, pl.w, rows);
+    count_launches(1);
+    ELM_CUDA_TRY(cudaGetLastError());
+    elm_params pe = *p;
+    pe.n_q = rows;
+    AttendWindow win;
+    win.q_row0 = 0;
+    win.n_q_total = p->n_kv;
+    win.tail_start = 0;                  // the whole list is the causal tail
+    return attend_enqueue(Q, K, V, pl.idx, pl.w, rows, &pe, O, pl.ws_attend, st, win);
+}
+
+// Attention of the tokens [t0, t0 + rows) over the entries of `pc`, each seen by the tokens of its lifetime.
+static int express_attend_window(const void *Q, const void *K, const void *V, void *O, const elm_params *p,
+                                 const ExpressLayout &L, unsigned char *ws, const WindowPieces &pc, int64_t t0, int rows,
+                                 float *lse, cudaStream_t st, int lane)
 {
     const int BH = p->batch * p->kv_heads;
     const int total = pc.dst_off[pc.n];
-    int32_t *ep_idx = reinterpret_cast<int32_t *>(ws + L.ep_idx + lane * L.ep_stride);
-    float *ep_w = reinterpret_cast<float *>(ws + L.ep_w + lane * L.ep_stride);
+    const int n_pad = (total + 127) / 128 * 128;
     if ((size_t)total > L.ep_cap) return ELM_ERR_WORKSPACE;
-    // elm_attend takes dense [problem][n_core] lists
-    build_list_kernel<<<dim3((unsigned)((total + 255) / 256), (unsigned)BH), 256, 0, st>>>(pc, p->n_kv, ep_idx, ep_w, total);
+    const PrefillLane pl = prefill_lane(L, ws, BH, lane);
+    int32_t *blk_death = pl.blk_birth + (size_t)BH * (n_pad / 128);
+    build_window_kernel<<<dim3((unsigned)((n_pad + 255) / 256), (unsigned)BH), 256, 0, st>>>(
+        pc, p->n_kv, pl.idx, pl.w, total, n_pad, pl.birth, pl.death, pl.blk_birth, blk_death);
     count_launches(1);
     ELM_CUDA_TRY(cudaGetLastError());
     elm_params pe = *p;
@@ -902,8 +1124,12 @@ static int express_attend_epoch(const void *Q, const void *K, const void *V, voi
     AttendWindow win;
     win.q_row0 = t0;
     win.n_q_total = p->n_kv;
-    win.tail_start = pc.dst_off[pc.n - 1];
-    return attend_enqueue(Q, K, V, ep_idx, ep_w, total, &pe, O, ws + L.ws_attend + lane * L.ws_attend_stride, st, win);
+    win.birth = pl.birth;
+    win.death = pl.death;
+    win.blk_birth = pl.blk_birth;
+    win.blk_death = blk_death;
+    win.lse = lse;
+    return attend_enqueue(Q, K, V, pl.idx, pl.w, total, &pe, O, pl.ws_attend, st, win);
 }
 
 template <typename Tin, typename T>
@@ -965,12 +1191,7 @@ static int express_impl(const Tin *K, const Tin *V, const elm_params *p, int mba
     if (prefill) {
         // Exact phase and round 0 (thinning factor 1: nothing is dropped): each of the first 4 n_out
         // tokens attends over all tokens up to itself (Theorem 3's exact regime).
-        ListPieces pc = {};
-        const int rows = (int)(n < 4 * n_out ? n : 4 * n_out);
-        pc.n = 1;
-        pc.src[0] = nullptr; pc.src_off[0] = 0; pc.w[0] = 1.f;
-        pc.dst_off[0] = 0; pc.dst_off[1] = rows;
-        const int rc = express_attend_epoch(Q, K, V, O, p, L, ws, pc, 0, rows, st);
+        const int rc = express_attend_start(Q, K, V, O, p, L, ws, (int)(n < 4 * n_out ? n : 4 * n_out), st);
         if (rc != ELM_OK) return rc;
     }
     for (int r = 0; r < R; ++r) {
@@ -1007,50 +1228,41 @@ static int express_impl(const Tin *K, const Tin *V, const elm_params *p, int mba
             }
         }
         if (prefill && r >= 1) {
-            // Thinformer Express (Algorithm 5) for the 3 n_out 2^m tokens of this round.  Between two
-            // level-0 Halve calls ("epoch": s_0 = n_out 2^(2-q) tokens) the cache is fixed except for
-            // the growing S_0: E with the finished siblings (weight 1), in S_i the outputs of the
-            // level-(i-1) calls that level i has not consumed yet (weight 2^(i-q)), and the epoch's
-            // own tokens up to the query (weight 2^-q).
-            if (m > mbar) return ELM_ERR_SHAPE;                               // subsampled rounds: not built yet
-            const int64_t s0 = (n_out << 2) >> q;
-            const int epochs = 1 << (2 * (q - 1));
-            // An epoch's launch has one work item per 256 of its s_0 tokens and head - too few for the
-            // GPU when s_0 is small - and all epochs of a round are independent given the round's lists:
-            // they are dealt to EXPRESS_LANES streams (each with its own list buffers) between two events.
+            // Thinformer Express (Algorithm 5) for the 3 n_out 2^m tokens of this round.  The cache a token
+            // sees is E with the finished siblings (weight 1), in every S_i the outputs of level-(i-1)
+            // Halve calls that level i has not consumed yet (weight 2^(i-q)), and in S_0 the kept points
+            // since the last level-0 call, itself included (weight 2^-q).  It changes with every level-0
+            // call, so the tokens are taken in windows: one attention launch per window over every entry
+            // that some token of the window sees, each entry carrying the span of tokens that see it.
+            // The launches are independent given the round's lists; they are dealt to EXPRESS_LANES
+            // streams (each with its own list buffers) between two events.
+            const RoundGeom g = round_geom(p, mbar, r);
+            const int64_t W = prefill_window(g), Wg = W >> g.wlog;
+            float *lse = g.sub ? reinterpret_cast<float *>(ws + L.lse) : nullptr;
             ELM_CUDA_TRY(cudaEventRecord(fork, st));
             for (int i = 0; i < EXPRESS_LANES; ++i) ELM_CUDA_TRY(cudaStreamWaitEvent(side[i], fork, 0));
+            int launch = 0;
             for (int jj = 0; jj < 3; ++jj) {
-                for (int e = 0; e < epochs; ++e) {
-                    const int lane_id = (jj * epochs + e) % EXPRESS_LANES;
-                    cudaStream_t sj = side[lane_id];
-                    ListPieces pc = {};
-                    int k = 0;
-                    int32_t at = 0;
-                    auto piece = [&](const int32_t *src, int64_t off, int64_t count, float wgt) {
-                        if (count <= 0) return;
-                        pc.src[k] = src; pc.src_off[k] = off; pc.w[k] = wgt; pc.dst_off[k] = at;
-                        at += (int32_t)count;
-                        ++k;
-                    };
-                    piece(E, 0, (1 + jj) * n_out, 1.f);
-                    for (int i = q - 1; i >= 1; --i) {
-                        const int64_t u = (s0 << (i - 1)) >> 1;              // output of one level-(i-1) call
-                        const int64_t done = e >> (2 * (i - 1)), used = 4 * (int64_t)(e >> (2 * i));
-                        piece(levels + (size_t)(i - 1) * BH * n, jj * (len0 >> i) + used * u, (done - used) * u,
-                              (float)ldexp(1.0, i - q));
-                    }
-                    const int64_t t0 = (jj + 1) * seg + e * s0;
-                    piece(nullptr, t0, s0, (float)ldexp(1.0, -q));            // the causal tail
-                    pc.dst_off[k] = at;
-                    pc.n = k;
-                    const int rc = express_attend_epoch(Q, K, V, O, p, L, ws, pc, t0, (int)s0, sj, lane_id);
+                for (int64_t G0 = 0; G0 < g.len0; G0 += Wg, ++launch) {
+                    const int lane_id = launch % EXPRESS_LANES;
+                    WindowPieces pc;
+                    window_pieces(g, n_out, jj, G0, G0 + Wg, E, levels, (size_t)BH * n, listA, pc);
+                    const int64_t t0 = (jj + 1) * seg + (G0 << g.wlog);
+                    const int rc = express_attend_window(Q, K, V, O, p, L, ws, pc, t0, (int)W, lse, side[lane_id], lane_id);
                     if (rc != ELM_OK) return rc;
                 }
             }
             for (int i = 0; i < EXPRESS_LANES; ++i) {
                 ELM_CUDA_TRY(cudaEventRecord(join[i], side[i]));
                 ELM_CUDA_TRY(cudaStreamWaitEvent(st, join[i], 0));             // the halvings overwrite E
+            }
+            if (g.sub) {
+                // the tokens Subsample dropped still attend to themselves
+                const dim3 grid((unsigned)((3 * seg + 7) / 8), (unsigned)(p->batch * p->q_heads));
+                self_merge_kernel<Tin, T><<<grid, 256, 0, st>>>(Q, K, V, O, lse, listA, p->q_heads, p->kv_heads, n, p->d, seg,
+                                                                g.len0, g.wlog, (T)(-g.q));
+                count_launches(1);
+                ELM_CUDA_TRY(cudaGetLastError());
             }
         }
         // halve phase: 4 n_out -> 2 n_out -> n_out
@@ -1146,8 +1358,8 @@ static int validate_prefill(const elm_params *p, int32_t mbar)
     if (p->q_heads < 1 || p->q_heads % p->kv_heads != 0 || (int64_t)p->batch * p->q_heads > 65535) return ELM_ERR_SHAPE;
     if (p->n_q != p->n_kv) return ELM_ERR_SHAPE;                       // one query per token
     const int R = express_rounds(p);
-    if (R >= 2 && 2 * (R - 1) > mbar) return ELM_ERR_SHAPE;               // subsampled rounds: attention not built yet
-    if (R >= 2 && 2 * (R - 1) > p->log2_nout + 1) return ELM_ERR_SHAPE;   // level-0 calls of at least 2 points
+    const int qmax = 2 * (R - 1) < mbar ? 2 * (R - 1) : mbar;            // deepest Compress2 of the run
+    if (R >= 2 && qmax > p->log2_nout + 1) return ELM_ERR_SHAPE;          // level-0 calls of at least 2 points
     return ELM_OK;
 }
 }  // namespace elm

@@ -109,6 +109,12 @@ PREFILL_CASES = {
     "lowrank_bf16_nout32_R3": (WORKLOADS["cfg3"].scaled(batch=1, q_heads=2, kv_heads=2), 5, 3, 4, 1),
     # tensor-core path with blocks of 128 list entries, grouped queries
     "mixture_t3_bf16_nout256_R2": (WORKLOADS["cfg5"].scaled(q_heads=4, kv_heads=2), 8, 2, 6, 2),
+    # Subsample active in round 2 (m = 4 > mbar = 2: one token kept per 4, a different one in every head)
+    "iid_f32_nout16_R3_subsample": (WORKLOADS["cfg1"].scaled(q_heads=2, kv_heads=2), 4, 3, 2, 1),
+    # mbar = 0: no Halve call inside a segment, strata of 4 and of 16 tokens
+    "mixture_f32_nout8_R3_mbar0": (WORKLOADS["cfg2"].scaled(batch=1, q_heads=2, kv_heads=1), 3, 3, 0, 2),
+    # tensor-core path, odd mbar: round 2 keeps one token of every 2 and runs Compress2 of depth 3
+    "mixture_t3_bf16_nout128_R3_subsample": (WORKLOADS["cfg5"].scaled(q_heads=4, kv_heads=2), 7, 3, 3, 2),
 }
 PREFILL_TOL = {("f32", "fp64"): 2e-6, ("f32", "fp32"): 1e-4, ("bf16", "fp64"): 1e-2, ("bf16", "fp32"): 2e-2}
 
@@ -158,11 +164,11 @@ def test_express_prefill_first_tokens_equal_exact_causal_attention():
     assert max_rel_err(O[0, 0, :m].float().cpu().numpy(), ref) <= 2e-6
 
 
-def test_express_prefill_rejects_subsampled_rounds():
-    wl = WORKLOADS["cfg1"].scaled(n=16 * 64, n_q=16 * 64)
+def test_express_prefill_rejects_level0_calls_below_one_pair():
+    wl = WORKLOADS["cfg1"].scaled(n=2 * 4 ** 4, n_q=2 * 4 ** 4)
     Q, K, V = generate(wl, seed=1, want_q=True)
     with pytest.raises(elm.ElmError):
-        elm.express_prefill(Q.cuda(), K.cuda(), V.cuda(), 4, 2, seed=1)      # R = 3 needs mbar >= 4
+        elm.express_prefill(Q.cuda(), K.cuda(), V.cuda(), 1, 6, seed=1)      # depth 6 Compress2 of 2^7 points
 
 
 # ----------------------------------------------------------------------------------------------
