@@ -214,7 +214,7 @@ int elm_express_workspace_bytes(const elm_params *params, int32_t mbar, size_t *
  *   workspace  at least elm_express_prefill_workspace_bytes(params, mbar) bytes, 256-byte aligned.
  * In a round whose thinning factor exceeds mbar (Subsample active) the kept points differ from problem to
  * problem; a token that is not kept still attends to itself with the weight of a point of S_0.
- * One attention launch per window of about 1024 tokens, over every cache entry that some token of the
+ * One attention launch per window of about 512 tokens, over every cache entry that some token of the
  * window sees; each entry carries the span of tokens that see it.
  */
 int elm_express_prefill_workspace_bytes(const elm_params *params, int32_t mbar, size_t *bytes);

@@ -777,11 +777,16 @@ static RoundGeom round_geom(const elm_params *p, int mbar, int r)
     g.s0 = g.q >= 1 ? (n_out << 2) >> g.q : g.len0;        // q = 0: no Halve call, S_0 only grows
     return g;
 }
-// Tokens per attention launch of the prefill: windows of about 1024 tokens (whole strata, at most a segment).
+// Tokens per attention launch of the prefill: windows of about 512 tokens (whole strata, at most a segment).
 static int64_t prefill_window(const RoundGeom &g)
 {
+    static const int64_t target = []() {
+        const char *e = getenv("ELM_PREFILL_WINDOW");           // tuning aid: a power of two
+        const long v = e ? atol(e) : 0;
+        return (int64_t)(v >= 64 && (v & (v - 1)) == 0 ? v : 512);
+    }();
     int64_t W = (int64_t)1 << g.wlog;
-    if (W < 1024) W = 1024;
+    if (W < target) W = target;
     return W < g.seg ? W : g.seg;
 }
 
