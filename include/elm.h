@@ -241,10 +241,15 @@ int elm_express_compress(const void *K, const void *V, const elm_params *params,
  *                  |v| over them and grows with the tokens seen later (with n_known = the whole
  *                  sequence this is the v_max of elm_express_compress).
  *   Q_t, O_t       [batch][q_heads][1][d]
- *   Limits         thinning factors above mbar (Subsample active, more than n_out 4^(mbar/2+1) tokens)
- *                  return ELM_ERR_SHAPE; mbar <= 12.
+ *   Limits         mbar <= 12; level-0 Halve calls need >= 2 points.
+ * Thinning factors above mbar (Subsample, Algorithm 3): problem p keeps one token of every stratum of
+ * 2^(m - mbar), chosen by the uniform of counter (stratum, 0, 61 + 64 (4 r + j), p), so inside a stratum
+ * the problems take their Compress2.update - and the Halve calls it triggers, one problem at a time - at
+ * different tokens; the counters in elm_stream describe the state at the stratum's start and move on at
+ * its end.  Where the problems' lists then differ in length, a shorter one repeats its last entry with
+ * that entry's weight split over the copies (every weighted sum over the list is unchanged).
  * Calls only enqueue work on `stream`; the host struct is updated immediately (the schedule of Halve
- * calls depends on the token count alone).
+ * calls depends on the token count and the draws alone).
  */
 typedef struct elm_stream {
     int64_t n, ell, n_E;          /* tokens seen, tokens of the current thin phase, points in E */
@@ -259,7 +264,8 @@ int elm_stream_init(elm_stream *s, const void *K, const void *V, int64_t n_known
 int elm_stream_step(elm_stream *s, const void *Q_t, const void *K, const void *V, const elm_params *params,
                     void *O_t, void *workspace, size_t workspace_bytes, void *stream);
 /* The current cache, wtd_cache() of Algorithm 1: at most 6 n_out entries per problem, [batch][kv_heads][count]
- * row numbers and (unnormalised) weights 2^(i-q) / 1; *count_host receives the number of entries. */
+ * row numbers and (unnormalised) weights 2^(i-q) / 1; *count_host receives the number of entries (inside a
+ * stratum of a subsampled phase: of the longest list; see above for the padding of the others). */
 int elm_stream_cache(const elm_stream *s, const elm_params *params, int32_t *idx_out, float *w_out,
                      int32_t *count_host, void *workspace, size_t workspace_bytes, void *stream);
 

@@ -69,13 +69,14 @@ __device__ __forceinline__ void store_from(__nv_bfloat16 *p, int64_t i, float v)
 }
 
 // Philox4x32-10 (Salmon et al., SC'11), first output word only.
-__device__ __forceinline__ uint32_t philox4x32_10_word0(uint32_t c0, uint32_t c1, uint32_t c2,
-                                                        uint32_t c3, uint32_t k0, uint32_t k1)
+__host__ __device__ __forceinline__ uint32_t philox4x32_10_word0(uint32_t c0, uint32_t c1, uint32_t c2,
+                                                                 uint32_t c3, uint32_t k0, uint32_t k1)
 {
 #pragma unroll
     for (int r = 0; r < 10; ++r) {
-        uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
-        uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+        const uint64_t p0 = (uint64_t)0xD2511F53u * c0, p1 = (uint64_t)0xCD9E8D57u * c2;
+        uint32_t hi0 = (uint32_t)(p0 >> 32), lo0 = (uint32_t)p0;
+        uint32_t hi1 = (uint32_t)(p1 >> 32), lo1 = (uint32_t)p1;
         uint32_t n0 = hi1 ^ c1 ^ k0, n2 = hi0 ^ c3 ^ k1;
         c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
         k0 += 0x9E3779B9u;
@@ -111,8 +112,8 @@ __device__ __forceinline__ void call_counter(int g, int64_t lvl, uint32_t &group
 }
 
 template <typename T>
-__device__ __forceinline__ T halving_uniform(uint64_t seed, uint32_t pair, uint32_t group,
-                                             uint32_t level, uint32_t problem)
+__host__ __device__ __forceinline__ T halving_uniform(uint64_t seed, uint32_t pair, uint32_t group,
+                                                      uint32_t level, uint32_t problem)
 {
     uint32_t w = philox4x32_10_word0(pair, group, level, problem, (uint32_t)seed, (uint32_t)(seed >> 32));
     return (T)(w >> 8) * (T)(1.0 / 16777216.0);

@@ -588,7 +588,8 @@ static int run_gram_simt(const Tin *K, const Tin *V, const elm_params *p, const 
 template <typename Tin, typename T> struct LevelCtx {
     const Tin *K, *V;
     const elm_params *p;
-    unsigned *vmax_bits;        // [BH] v_max bits, then the device status word
+    unsigned *vmax_bits;        // [BH] v_max bits (the workspace keeps the device status word behind them)
+    int *status;                // that status word
     T *cnorm, *Mpair, *rdecay, *F;
     int64_t F_stride;
     uint64_t seed;
@@ -611,7 +612,7 @@ static int run_halve_level(const LevelCtx<Tin, T> &c, const int32_t *cur, int32_
     const int64_t Ptotal = (int64_t)groups * P;
     const T logfac = (T)(0.5 + log(2.0 * (double)(2 * P) / delta_call));
     cudaStream_t st = c.st;
-    int *status = reinterpret_cast<int *>(c.vmax_bits + BH);
+    int *status = c.status;
     {
         StageTimer t(ELM_STAGE_LEVEL_PREP, st, 1);
         const int lp_threads = P >= 1024 ? 1024 : (P <= 32 ? 32 : (P + 31) / 32 * 32);
@@ -691,6 +692,7 @@ static int compress_impl(const Tin *K, const Tin *V, const elm_params *p, uint64
     LevelCtx<Tin, T> c;
     c.K = K; c.V = V; c.p = p;
     c.vmax_bits = reinterpret_cast<unsigned *>(ws + L.vmax_bits);
+    c.status = reinterpret_cast<int *>(c.vmax_bits + BH);
     c.cnorm = reinterpret_cast<T *>(ws + L.cnorm);
     c.Mpair = reinterpret_cast<T *>(ws + L.Mpair);
     c.rdecay = reinterpret_cast<T *>(ws + L.rdecay);
@@ -1151,6 +1153,7 @@ static int express_impl(const Tin *K, const Tin *V, const elm_params *p, int mba
     LevelCtx<Tin, T> c;
     c.K = K; c.V = V; c.p = p;
     c.vmax_bits = reinterpret_cast<unsigned *>(ws + L.vmax_bits);
+    c.status = reinterpret_cast<int *>(c.vmax_bits + BH);
     c.cnorm = reinterpret_cast<T *>(ws + L.cnorm);
     c.Mpair = reinterpret_cast<T *>(ws + L.Mpair);
     c.rdecay = reinterpret_cast<T *>(ws + L.rdecay);
@@ -1458,6 +1461,7 @@ static int ragged_impl(const Tin *K, const Tin *V, const elm_params *p, const Ra
     LevelCtx<Tin, T> c;
     c.K = K; c.V = V; c.p = p;
     c.vmax_bits = reinterpret_cast<unsigned *>(ws + L.vmax_bits);
+    c.status = reinterpret_cast<int *>(c.vmax_bits + BH);
     c.cnorm = reinterpret_cast<T *>(ws + L.cnorm);
     c.Mpair = reinterpret_cast<T *>(ws + L.Mpair);
     c.rdecay = reinterpret_cast<T *>(ws + L.rdecay);
@@ -1612,8 +1616,8 @@ __global__ void append_kernel(int32_t *__restrict__ list, int64_t stride, int64_
 }
 
 // wtd_cache() of Algorithm 1 (+ the token t itself when t >= 0) as list pieces
-static void stream_pieces(const elm_stream *s, const StreamLayout &L, unsigned char *ws, const elm_params *p, int64_t t,
-                          ListPieces &pc)
+static void stream_pieces(const elm_stream *s, const int64_t *n_S, const StreamLayout &L, unsigned char *ws,
+                          const elm_params *p, int64_t t, ListPieces &pc)
 {
     const size_t BH = (size_t)p->batch * p->kv_heads;
     int32_t *S = reinterpret_cast<int32_t *>(ws + L.S);
@@ -1625,11 +1629,75 @@ static void stream_pieces(const elm_stream *s, const StreamLayout &L, unsigned c
         at += (int32_t)count;
         ++k;
     };
-    for (int i = 0; i <= s->q; ++i) piece(S + (size_t)i * BH * p->n_kv, 0, s->n_S[i], (float)ldexp(1.0, i - s->q));
+    for (int i = 0; i <= s->q; ++i) piece(S + (size_t)i * BH * p->n_kv, 0, n_S[i], (float)ldexp(1.0, i - s->q));
     piece(reinterpret_cast<int32_t *>(ws + L.E), 0, s->n_E, 1.f);
     if (t >= 0) piece(nullptr, t, 1, (float)ldexp(1.0, -s->q));          // the token enters S_0
     pc.dst_off[k] = at;
     pc.n = k;
+}
+
+// Subsample (Algorithm 3) in a streaming run.  Inside a stratum of 2^wlog tokens problem p keeps the token
+// at offset floor(U 2^wlog), U the uniform of counter (stratum, 0, code, p): the problems take their
+// Compress2.update at different tokens of the stratum, so at the token with offset o a problem is either
+// still in the state the stratum began with (`a`) or already in the state it ends with (`b`: kept offset
+// < o).  The two states differ only in how many entries of the same lists count.
+struct StratumDraw {
+    uint64_t seed;
+    uint32_t stratum, code;
+    int32_t wlog;
+    int64_t o;
+};
+__host__ __device__ __forceinline__ int64_t kept_offset(const StratumDraw &d, uint32_t problem)
+{
+    return (int64_t)floor(halving_uniform<double>(d.seed, d.stratum, 0u, d.code, problem) * (double)((int64_t)1 << d.wlog));
+}
+// Like build_list_kernel with the list chosen per problem.  The two lists may differ in length; a list
+// shorter than `total` repeats its last entry over the remaining slots with that entry's weight divided
+// among the copies, which leaves every weighted sum over the list unchanged.
+__global__ void build_list_choice_kernel(ListPieces a, ListPieces b, StratumDraw dr, int64_t src_stride,
+                                         int32_t *__restrict__ idx, float *__restrict__ w, int total)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= total) return;
+    const int64_t pr = blockIdx.y;
+    const ListPieces &pc = kept_offset(dr, (uint32_t)pr) < dr.o ? b : a;
+    const int len = pc.dst_off[pc.n];
+    const int ii = i < len ? i : len - 1;
+    int k = 0;
+    while (ii >= pc.dst_off[k + 1]) ++k;
+    const int64_t o = ii - pc.dst_off[k];
+    idx[pr * total + i] = pc.src[k] ? pc.src[k][pr * src_stride + pc.src_off[k] + o] : (int32_t)(pc.src_off[k] + o);
+    w[pr * total + i] = ii == len - 1 ? pc.w[k] / (float)(total - len + 1) : pc.w[k];
+}
+// S_0 of every problem that keeps the token gets it at position `pos`.
+__global__ void append_kept_kernel(int32_t *__restrict__ list, int64_t stride, int64_t pos, int32_t value, int problems,
+                                   StratumDraw dr)
+{
+    const int p = blockIdx.x * blockDim.x + threadIdx.x;
+    if (p < problems && kept_offset(dr, (uint32_t)p) == dr.o) list[(int64_t)p * stride + pos] = value;
+}
+
+// The stratum the next token of a subsampled thin phase falls in, and the level counters a problem has after
+// it took the stratum's update (n_S plus one point in S_0, then the Halve calls that come due).
+// Returns false when Subsample is not active.
+static bool stratum_state(const elm_stream *s, int64_t n_out, StratumDraw &dr, int64_t nS_after[16], bool call_due[16])
+{
+    for (int i = 0; i < 16; ++i) { nS_after[i] = s->n_S[i]; call_due[i] = false; }
+    if (!(s->m > s->mbar && s->n >= n_out)) return false;                  // thin phase with thinning factor above mbar
+    dr.seed = s->seed;
+    dr.wlog = s->m - s->mbar;
+    dr.stratum = (uint32_t)(s->ell >> dr.wlog);
+    dr.o = s->ell & (((int64_t)1 << dr.wlog) - 1);
+    dr.code = (uint32_t)(61 + 64 * (4 * (s->m / 2) + s->b + 1));
+    nS_after[0] += 1;
+    for (int i = 0; i < s->q; ++i) {
+        const int64_t thresh = ((n_out << s->q) << i) >> (2 * (s->q - 1));
+        if (nS_after[i] != thresh) continue;
+        call_due[i] = true;
+        nS_after[i + 1] += thresh / 2;
+        nS_after[i] = 0;
+    }
+    return true;
 }
 
 template <typename Tin, typename T>
@@ -1641,11 +1709,11 @@ static int stream_step_impl(elm_stream *s, const Tin *Q, const Tin *K, const Tin
     const int64_t n = p->n_kv, n_out = (int64_t)1 << p->log2_nout;
     const int64_t t = s->n;
     if (t >= n) return ELM_ERR_SHAPE;                                      // capacity
-    if (s->m > s->mbar) return ELM_ERR_SHAPE;                              // Subsample: not built yet
     if (s->q >= 1 && p->log2_nout + 2 - s->q < 1) return ELM_ERR_SHAPE;     // level-0 calls of at least 2 points
     LevelCtx<Tin, T> c;
     c.K = K; c.V = V; c.p = p;
     c.vmax_bits = reinterpret_cast<unsigned *>(ws + L.vmax_bits);
+    c.status = reinterpret_cast<int *>(c.vmax_bits + BH);
     c.cnorm = reinterpret_cast<T *>(ws + L.cnorm);
     c.Mpair = reinterpret_cast<T *>(ws + L.Mpair);
     c.rdecay = reinterpret_cast<T *>(ws + L.rdecay);
@@ -1663,14 +1731,28 @@ static int stream_step_impl(elm_stream *s, const Tin *Q, const Tin *K, const Tin
         count_launches(1);
         ELM_CUDA_TRY(cudaGetLastError());
     }
+    // ---- Subsample bookkeeping: the stratum of this token and the state a problem is in after its update ----
+    StratumDraw dr = {};
+    int64_t nS_after[16];
+    bool call_due[16];
+    const bool sub = stratum_state(s, n_out, dr, nS_after, call_due);
     // ---- Algorithm 5: attend over wtd_cache() plus the token ----
     {
         ListPieces pc = {};
-        stream_pieces(s, L, ws, p, t, pc);
-        const int total = pc.dst_off[pc.n];
+        stream_pieces(s, s->n_S, L, ws, p, t, pc);
+        int total = pc.dst_off[pc.n];
         int32_t *ep_idx = reinterpret_cast<int32_t *>(ws + L.ep_idx);
         float *ep_w = reinterpret_cast<float *>(ws + L.ep_w);
-        build_list_kernel<<<dim3(blocks(total), (unsigned)BH), 256, 0, st>>>(pc, n, ep_idx, ep_w, total);
+        if (sub && dr.o > 0) {
+            // some problems have taken this stratum's update already
+            ListPieces pb = {};
+            stream_pieces(s, nS_after, L, ws, p, t, pb);
+            if (pb.dst_off[pb.n] > total) total = pb.dst_off[pb.n];
+            if ((size_t)total > L.ep_cap) return ELM_ERR_WORKSPACE;
+            build_list_choice_kernel<<<dim3(blocks(total), (unsigned)BH), 256, 0, st>>>(pc, pb, dr, n, ep_idx, ep_w, total);
+        } else {
+            build_list_kernel<<<dim3(blocks(total), (unsigned)BH), 256, 0, st>>>(pc, n, ep_idx, ep_w, total);
+        }
         count_launches(1);
         ELM_CUDA_TRY(cudaGetLastError());
         const int rc = attend_enqueue(Q, K, V, ep_idx, ep_w, total, p, O, ws + L.ws_attend, st);
@@ -1689,7 +1771,48 @@ static int stream_step_impl(elm_stream *s, const Tin *Q, const Tin *K, const Tin
         return rc;
     }
     s->ell += 1;                                                           // thin phase: Compress2.update
-    {
+    if (sub) {
+        // Subsample: only the problems whose draw is this token take the update now; the counters in *s
+        // move on when the stratum ends
+        append_kept_kernel<<<(BH + 127) / 128, 128, 0, st>>>(Slist(0), n, s->n_S[0], (int32_t)t, BH, dr);
+        count_launches(1);
+        ELM_CUDA_TRY(cudaGetLastError());
+        if (call_due[0]) {
+            const double dm = kh_express_delta(p->delta, s->m);
+            const int q = s->q;
+            for (int pi = 0; pi < BH; ++pi) {
+                if (kept_offset(dr, (uint32_t)pi) != dr.o) continue;
+                // the Halve calls of this one problem: the level machinery on its slice of every array
+                elm_params p1 = *p;
+                p1.batch = 1; p1.kv_heads = 1; p1.q_heads = 1;
+                LevelCtx<Tin, T> c1 = c;
+                c1.p = &p1;
+                c1.K = K + (int64_t)pi * n * p->d;
+                c1.V = V + (int64_t)pi * n * p->d;
+                c1.vmax_bits = c.vmax_bits + pi;
+                c1.cnorm = c.cnorm + (int64_t)pi * n;
+                c1.Mpair = c.Mpair + (int64_t)pi * (n / 2);
+                c1.rdecay = c.rdecay + (int64_t)pi * (n / 2);
+                c1.F = c.F + (int64_t)pi * c.F_stride;
+                c1.pbase = (uint32_t)pi;
+                for (int i = 0; i < q && call_due[i]; ++i) {
+                    const int64_t thresh = ((n_out << q) << i) >> (2 * (q - 1));
+                    const double dlt = ldexp(dm, 2 * (i + 1 - q)) / (3.0 * (double)q);
+                    const int code = i + 64 * (4 * (s->m / 2) + s->b + 1);
+                    const int rc = run_halve_level<Tin, T>(c1, Slist(i) + (int64_t)pi * n,
+                                                           Slist(i + 1) + (int64_t)pi * n + s->n_S[i + 1], n, 1,
+                                                           (int)(thresh / 2), code, dlt, 0, s->calls[i]);
+                    if (rc != ELM_OK) return rc;
+                }
+            }
+        }
+        if (dr.o == ((int64_t)1 << dr.wlog) - 1) {                         // the stratum ends: every problem has updated
+            for (int i = 0; i < 16; ++i) {
+                s->n_S[i] = nS_after[i];
+                if (call_due[i]) s->calls[i] += 1;
+            }
+        }
+    } else {
         const int q = s->q;
         int rc = append(Slist(0), s->n_S[0]);
         if (rc != ELM_OK) return rc;
@@ -1820,12 +1943,26 @@ extern "C" int elm_stream_cache(const elm_stream *s, const elm_params *params, i
     const StreamLayout L = stream_layout(params, s->mbar);
     if (workspace_bytes < L.total) return ELM_ERR_WORKSPACE;
     ListPieces pc = {};
-    stream_pieces(s, L, (unsigned char *)workspace, params, -1, pc);
-    const int total = pc.dst_off[pc.n];
+    stream_pieces(s, s->n_S, L, (unsigned char *)workspace, params, -1, pc);
+    int total = pc.dst_off[pc.n];
+    // Inside a stratum of a subsampled phase the problems that have kept their point hold one update more
+    // than the others; a shorter list is padded by repeating its last entry with the weight split.
+    StratumDraw dr = {};
+    int64_t nS_after[16];
+    bool call_due[16];
+    const bool mixed = stratum_state(s, (int64_t)1 << params->log2_nout, dr, nS_after, call_due) && dr.o > 0;
+    ListPieces pb = {};
+    if (mixed) {
+        stream_pieces(s, nS_after, L, (unsigned char *)workspace, params, -1, pb);
+        if (pb.dst_off[pb.n] > total) total = pb.dst_off[pb.n];
+    }
     *count_host = total;
     if (total > 0) {
-        build_list_kernel<<<dim3((unsigned)((total + 255) / 256), (unsigned)(params->batch * params->kv_heads)), 256, 0,
-                            (cudaStream_t)stream>>>(pc, params->n_kv, idx_out, w_out, total);
+        const dim3 grid((unsigned)((total + 255) / 256), (unsigned)(params->batch * params->kv_heads));
+        if (mixed)
+            build_list_choice_kernel<<<grid, 256, 0, (cudaStream_t)stream>>>(pc, pb, dr, params->n_kv, idx_out, w_out, total);
+        else
+            build_list_kernel<<<grid, 256, 0, (cudaStream_t)stream>>>(pc, params->n_kv, idx_out, w_out, total);
         count_launches(1);
         ELM_CUDA_TRY(cudaGetLastError());
     }
