@@ -250,7 +250,9 @@ __device__ __forceinline__ float exp_pass(uint32_t tS, uint32_t tP, float scale_
 // ---------------------------------------------------------------------------------------------
 // the attention kernel
 // ---------------------------------------------------------------------------------------------
-template <int D>
+// MASKED = false: every row sees the whole list (no causal tail, no lifetimes); the masked form of the
+// softmax passes is then not compiled in, which keeps the plain form's register allocation to itself.
+template <int D, bool MASKED>
 __global__ void __launch_bounds__(NTHREADS, 1)
 attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
                  const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapX,
@@ -321,9 +323,17 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                         tma_load_3d(smem + SM::OFF_Q + t * SM::Q_TILE + kh * (BM * 128), &mapQ, &bar->q_full, kh * 64, q_row0 + q0 + t * BM, bh);
             };
             // Blocks are numbered G = k nblk + j along the CTA's whole stream (item k, block j).
+            int flag_item = -1;
+            bool flag_now = false, flag_next = n_items > 0 && item_bias(0);
             auto load_k = [&](int G) {
                 const int s = G % STAGES, prob = prob_of(item_bh(G / nblk));
-                const bool with_bias = item_bias(G / nblk);
+                // the flag of an item is fetched while the item before it streams, off the critical path
+                if (G / nblk != flag_item) {
+                    flag_item = G / nblk;
+                    flag_now = flag_next;
+                    flag_next = flag_item + 1 < n_items && item_bias(flag_item + 1);
+                }
+                const bool with_bias = flag_now;
                 mbar_expect_tx(&bar->k_full[s], SM::K_BLOCK + (with_bias ? SM::X_BLOCK : 0));
                 for (int kh = 0; kh < KH; ++kh)
                     tma_load_3d(smem + SM::OFF_K + s * SM::K_BLOCK + kh * (BN * 128), &mapK, &bar->k_full[s], kh * 64, (G % nblk) * BN, prob);
@@ -413,12 +423,14 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
             // block of the next item: the tensor pipe runs on while the softmax warps finish an item.
             int j = 0, k = 0;                                                  // block G = item k, block j
             bool bias_next = n_items > 0 && item_bias(0);                      // of the item block G + 1 belongs to
+            bool bias_after = false;
             for (int G = 0; G < total && ok; ++G) {
                 const int s = G % STAGES;
                 const bool more = G + 1 < total;
                 const int sn = (G + 1) % STAGES;
                 const bool last = j == nblk - 1;                               // last block of item k
-                if (last && more) bias_next = item_bias(k + 1);
+                if (j == 0) bias_after = k + 1 < n_items && item_bias(k + 1);   // fetched early, used at the item's last block
+                if (last) bias_next = bias_after;
                 if (more) ok = mbar_wait(&bar->k_full[sn], (uint32_t)((G + 1) / STAGES) & 1u);
                 ok = ok && mbar_wait(&bar->v_full[s], (uint32_t)(G / STAGES) & 1u);
                 for (int t = 0; t < 2 && ok; ++t) {
@@ -477,25 +489,27 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                     // `special` must be warp-uniform: both forms of the two passes contain warp-collective TMEM loads.
                     uint32_t vmask = 0xffffffffu;
                     bool special = false;
-                    if (birth) {
-                        // lifetimes: the block is seen whole by this warp's 32 rows unless an entry is born
-                        // after the first or dies before the last of them
-                        const int t_first = q_row0 + q0 + t * BM + (warp & 3) * 32;
-                        special = !(__ldg(blk_birth + blk0 + j) <= t_first && __ldg(blk_death + blk0 + j) > t_first + 31);
-                        if (special) {
-                            const int t_row = t_first + lane;
-                            const int32_t *bp = birth + life0 + j * BN, *dp = death + life0 + j * BN;
-                            vmask = 0u;
+                    if constexpr (MASKED) {
+                        if (birth) {
+                            // lifetimes: the block is seen whole by this warp's 32 rows unless an entry is born
+                            // after the first or dies before the last of them
+                            const int t_first = q_row0 + q0 + t * BM + (warp & 3) * 32;
+                            special = !(__ldg(blk_birth + blk0 + j) <= t_first && __ldg(blk_death + blk0 + j) > t_first + 31);
+                            if (special) {
+                                const int t_row = t_first + lane;
+                                const int32_t *bp = birth + life0 + j * BN, *dp = death + life0 + j * BN;
+                                vmask = 0u;
 #pragma unroll 8
-                            for (int c = 0; c < 32; ++c)
-                                vmask |= (uint32_t)(__ldg(bp + c) <= t_row && t_row < __ldg(dp + c)) << c;
+                                for (int c = 0; c < 32; ++c)
+                                    vmask |= (uint32_t)(__ldg(bp + c) <= t_row && t_row < __ldg(dp + c)) << c;
+                            }
+                        } else if (has_tail) {
+                            int valid = n_core - j * BN - cq * 32;
+                            const int64_t seen = (int64_t)tail_start + q0 + t * BM + row + 1;
+                            if (seen < n_core) valid = (int)seen - j * BN - cq * 32;
+                            special = __any_sync(0xffffffffu, valid < 32);
+                            vmask = valid >= 32 ? 0xffffffffu : (valid <= 0 ? 0u : (1u << valid) - 1u);
                         }
-                    } else if (has_tail) {
-                        int valid = n_core - j * BN - cq * 32;
-                        const int64_t seen = (int64_t)tail_start + q0 + t * BM + row + 1;
-                        if (seen < n_core) valid = (int)seen - j * BN - cq * 32;
-                        special = __any_sync(0xffffffffu, valid < 32);
-                        vmask = valid >= 32 ? 0xffffffffu : (valid <= 0 ? 0u : (1u << valid) - 1u);
                     }
                     const uint32_t tS = tmem + lane_addr + t * 128 + cq * 32;   // this thread's 32 logit columns
                     const uint32_t tP = tS;                 // their bf16 probabilities overwrite the first 16 of them
@@ -504,7 +518,9 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                     if (!ok) break;
                     tc_fence_after();
                     // ---- pass 1: row maximum over the four quarters ----
-                    const float mh = special ? row_max<true, 1>(tS, scale_log2, vmask) : row_max<false, 1>(tS, scale_log2, vmask);
+                    float mh;
+                    if constexpr (MASKED) mh = special ? row_max<true, 1>(tS, scale_log2, vmask) : row_max<false, 1>(tS, scale_log2, vmask);
+                    else mh = row_max<false, 1>(tS, scale_log2, vmask);
                     bar->xchg[t][cq][row] = mh;
                     asm volatile("bar.sync 1, 512;" ::: "memory");
                     const float mx = fmaxf(fmaxf(bar->xchg[t][0][row], bar->xchg[t][1][row]),
@@ -528,8 +544,11 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                         if (grow) m_ref[t] = mx;
                     }
                     // ---- pass 2: probabilities and running denominator ----
-                    l[t] += special ? exp_pass<true, 1>(tS, tP, scale_log2, -m_ref[t], vmask)
-                                    : exp_pass<false, 1>(tS, tP, scale_log2, -m_ref[t], vmask);
+                    if constexpr (MASKED)
+                        l[t] += special ? exp_pass<true, 1>(tS, tP, scale_log2, -m_ref[t], vmask)
+                                        : exp_pass<false, 1>(tS, tP, scale_log2, -m_ref[t], vmask);
+                    else
+                        l[t] += exp_pass<false, 1>(tS, tP, scale_log2, -m_ref[t], vmask);
                     tmem_wait_st();
                     tc_fence_before();
                     mbar_arrive(&bar->p_ready[t]);
@@ -640,7 +659,8 @@ static int launch(const __nv_bfloat16 *Q, const __nv_bfloat16 *K, const __nv_bfl
         ELM_CUDA_TRY(cudaGetLastError());
     }
     StageTimer t(timed ? ELM_STAGE_ATTEND : -1, st, 1);
-    auto kern = attend_tc_kernel<D>;
+    const bool masked = win.birth != nullptr || win.tail_start != 0x7fffffff;
+    auto kern = masked ? attend_tc_kernel<D, true> : attend_tc_kernel<D, false>;
     ELM_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<D>::TOTAL));
     // one persistent CTA per SM, each taking every gridDim.x-th pair of query tiles
     const int tiles_x = (p->n_q + 2 * BM - 1) / (2 * BM);
