@@ -407,7 +407,7 @@ def main():
 
     # end to end through the host-buffer entry point (pinned inputs, copies inside the timed region)
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and args.only not in ("prefill", "express"):
         Qp, Kp, Vp = Q.pin_memory(), K.pin_memory(), V.pin_memory()
         Oh = torch.empty_like(Q).pin_memory()
         scratch = torch.empty(elm.host_call_scratch_bytes(wl.batch, wl.q_heads, wl.kv_heads, wl.n, wl.n_q, wl.d,
@@ -430,6 +430,18 @@ def main():
         del scratch
 
     if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    if args.only in ("prefill", "express"):
+        # not the step of the headline metric: its own line (profiling captures only)
+        what = "Thinformer Express prefill" if args.only == "prefill" else "Offline-Express compression"
+        print(json.dumps({args.only: {"what": what, "mbar": wl.log2_nout - 2, "ms_per_call": ms_step,
+                                      "tokens_per_s": value, "launches_per_call": launches // args.steps,
+                                      "stage_ms": {k: v[0] / args.steps for k, v in stage.items()}},
+                          "n_gpus": world, "steps": args.steps, "warmup": warmup,
+                          "config": workload_config(wl, args)}))
         if dist is not None:
             dist.destroy_process_group()
         return
