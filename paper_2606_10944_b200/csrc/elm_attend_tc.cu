@@ -48,9 +48,13 @@ constexpr int TMA_WARP = 16, MMA_WARP = 17;
 constexpr uint32_t TMEM_COLS = 512;
 constexpr float RESCALE_TAU = 8.0f;      // rescale the accumulator only if the max grew by > 2^8
 #ifndef ELM_EMU_PAIRS
-#define ELM_EMU_PAIRS 4
+#define ELM_EMU_PAIRS 0
 #endif
-constexpr int EMU_PAIRS = ELM_EMU_PAIRS;  // of every 16 column pairs, how many take exp2 from the FMA pipe
+// Of every 16 column pairs, how many take exp2 from the FMA pipe instead of the special-function unit.
+// Measured on cfg5 (same box, alternating): 0: 4.04 ms, 1: 4.06, 2: 4.08, 3: 4.15 ... 4.25, 4: 4.25, 6: 4.26 ... 4.37,
+// 8: 4.35 ... 4.43 - since the kernel became persistent the softmax warps are short of issue slots and
+// latency, not of exp2 throughput, so the default is none.
+constexpr int EMU_PAIRS = ELM_EMU_PAIRS;
 
 using namespace sm100;
 
@@ -187,8 +191,8 @@ __device__ __forceinline__ float exp_pass(uint32_t tS, uint32_t tP, float scale_
             for (int i = 0; i < 16; ++i)
                 x2[i] = fma2(pack2(__uint_as_float(a[q & 1][2 * i]), __uint_as_float(a[q & 1][2 * i + 1])), scale2, negm2);
             float pe[32];
-            // The special-function unit (16 exp2 per clock per SM) is the scarcest pipe of this loop, so
-            // EMU_PAIRS of the 16 pairs take 2^x from the FMA pipe instead: x = n + f with n = round(x)
+            // EMU_PAIRS of the 16 pairs can take 2^x from the FMA pipe instead of the special-function unit
+            // (16 exp2 per clock per SM): x = n + f with n = round(x)
             // (magic-number add), 2^f by a cubic on [-1/2, 1/2] (relative error 1e-4, below the bf16
             // rounding of the probabilities), n added to the exponent field.
 #pragma unroll
@@ -221,10 +225,10 @@ __device__ __forceinline__ float exp_pass(uint32_t tS, uint32_t tP, float scale_
                 sum2 = add2(sum2, pack2(pe[2 * i], pe[2 * i + 1]));
                 sum2b = add2(sum2b, pack2(pe[2 * i + 2], pe[2 * i + 3]));
             }
-            // round to bf16 on the integer pipe: add half an ulp, keep the upper halves
+            // one conversion per pair (rounding by two integer adds and a byte permute was 2 % slower: 4.05
+            // against 3.98 ms)
 #pragma unroll
-            for (int i = 0; i < 16; ++i)
-                pk[i] = __byte_perm(__float_as_uint(pe[2 * i]) + 0x8000u, __float_as_uint(pe[2 * i + 1]) + 0x8000u, 0x7632);
+            for (int i = 0; i < 16; ++i) pk[i] = pack_bf16x2(pe[2 * i], pe[2 * i + 1]);
         } else {
 #pragma unroll
             for (int c = 0; c < 32; c += 2) {
@@ -232,7 +236,7 @@ __device__ __forceinline__ float exp_pass(uint32_t tS, uint32_t tP, float scale_
                 const float p0 = ((vmask >> c) & 1u) ? fast_exp2(v0 + neg_m) : 0.f;
                 const float p1 = ((vmask >> (c + 1)) & 1u) ? fast_exp2(v1 + neg_m) : 0.f;
                 sum0 += p0 + p1;
-                pk[c >> 1] = __byte_perm(__float_as_uint(p0) + 0x8000u, __float_as_uint(p1) + 0x8000u, 0x7632);
+                pk[c >> 1] = pack_bf16x2(p0, p1);
             }
         }
         asm volatile(
