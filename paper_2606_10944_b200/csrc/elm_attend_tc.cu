@@ -526,7 +526,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                     if constexpr (MASKED) mh = special ? row_max<true, 1>(tS, scale_log2, vmask) : row_max<false, 1>(tS, scale_log2, vmask);
                     else mh = row_max<false, 1>(tS, scale_log2, vmask);
                     bar->xchg[t][cq][row] = mh;
-                    asm volatile("bar.sync 1, 512;" ::: "memory");
+                    asm volatile("bar.sync %0, 128;" ::"r"(1 + (warp & 3)) : "memory");
                     const float mx = fmaxf(fmaxf(bar->xchg[t][0][row], bar->xchg[t][1][row]),
                                            fmaxf(bar->xchg[t][2][row], bar->xchg[t][3][row]));
                     // lazy rescale: keep the old reference unless the maximum grew by more than 2^TAU
@@ -566,7 +566,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                 if (!ok) break;
                 tc_fence_after();
                 bar->xchg[t][cq][row] = l[t];
-                asm volatile("bar.sync 1, 512;" ::: "memory");
+                asm volatile("bar.sync %0, 128;" ::"r"(1 + (warp & 3)) : "memory");
                 const float l_all = (bar->xchg[t][0][row] + bar->xchg[t][1][row]) + (bar->xchg[t][2][row] + bar->xchg[t][3][row]);
                 const float inv = 1.f / l_all;
                 const int64_t qrow = (int64_t)q0 + t * BM + row;
