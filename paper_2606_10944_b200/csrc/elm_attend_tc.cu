@@ -251,6 +251,47 @@ __device__ __forceinline__ float exp_pass(uint32_t tS, uint32_t tP, float scale_
     return sum0 + s_lo + s_hi;
 }
 
+// The plain form for one chunk with the 32 logits kept in registers between the two passes (one TMEM load
+// per block instead of two).
+__device__ __forceinline__ float row_max_keep(uint32_t tS, float scale_log2, uint32_t (&a)[32])
+{
+    float m0 = -INFINITY, m1 = -INFINITY;
+    tmem_ld32(tS, a);
+    tmem_wait_ld();
+#pragma unroll
+    for (int c = 0; c < 32; c += 4) {
+        m0 = max3(m0, __uint_as_float(a[c]), __uint_as_float(a[c + 1]));
+        m1 = max3(m1, __uint_as_float(a[c + 2]), __uint_as_float(a[c + 3]));
+    }
+    return fmaxf(m0, m1) * scale_log2;
+}
+__device__ __forceinline__ float exp_pass_keep(uint32_t tP, float scale_log2, float neg_m, const uint32_t (&a)[32])
+{
+    const uint64_t scale2 = pack2(scale_log2, scale_log2), negm2 = pack2(neg_m, neg_m);
+    uint64_t sum2 = pack2(0.f, 0.f), sum2b = pack2(0.f, 0.f);
+    uint32_t pk[16];
+#pragma unroll
+    for (int i = 0; i < 16; i += 2) {
+        float x0, x1, x2, x3;
+        unpack2(fma2(pack2(__uint_as_float(a[2 * i]), __uint_as_float(a[2 * i + 1])), scale2, negm2), x0, x1);
+        unpack2(fma2(pack2(__uint_as_float(a[2 * i + 2]), __uint_as_float(a[2 * i + 3])), scale2, negm2), x2, x3);
+        const float p0 = fast_exp2(x0), p1 = fast_exp2(x1), p2 = fast_exp2(x2), p3 = fast_exp2(x3);
+        sum2 = add2(sum2, pack2(p0, p1));
+        sum2b = add2(sum2b, pack2(p2, p3));
+        pk[i] = pack_bf16x2(p0, p1);
+        pk[i + 1] = pack_bf16x2(p2, p3);
+    }
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%16], {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15};"
+        ::"r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3]), "r"(pk[4]), "r"(pk[5]), "r"(pk[6]), "r"(pk[7]),
+          "r"(pk[8]), "r"(pk[9]), "r"(pk[10]), "r"(pk[11]), "r"(pk[12]), "r"(pk[13]), "r"(pk[14]), "r"(pk[15]),
+          "r"(tP)
+        : "memory");
+    float s_lo, s_hi;
+    unpack2(add2(sum2, sum2b), s_lo, s_hi);
+    return s_lo + s_hi;
+}
+
 // ---------------------------------------------------------------------------------------------
 // the attention kernel
 // ---------------------------------------------------------------------------------------------
@@ -523,8 +564,9 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                     tc_fence_after();
                     // ---- pass 1: row maximum over the four quarters ----
                     float mh;
+                    uint32_t kept[32];                               // plain form: the logits between the two passes
                     if constexpr (MASKED) mh = special ? row_max<true, 1>(tS, scale_log2, vmask) : row_max<false, 1>(tS, scale_log2, vmask);
-                    else mh = row_max<false, 1>(tS, scale_log2, vmask);
+                    else mh = row_max_keep(tS, scale_log2, kept);
                     bar->xchg[t][cq][row] = mh;
                     asm volatile("bar.sync %0, 128;" ::"r"(1 + (warp & 3)) : "memory");
                     const float mx = fmaxf(fmaxf(bar->xchg[t][0][row], bar->xchg[t][1][row]),
@@ -552,7 +594,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                         l[t] += special ? exp_pass<true, 1>(tS, tP, scale_log2, -m_ref[t], vmask)
                                         : exp_pass<false, 1>(tS, tP, scale_log2, -m_ref[t], vmask);
                     else
-                        l[t] += exp_pass<false, 1>(tS, tP, scale_log2, -m_ref[t], vmask);
+                        l[t] += exp_pass_keep(tP, scale_log2, -m_ref[t], kept);
                     tmem_wait_st();
                     tc_fence_before();
                     mbar_arrive(&bar->p_ready[t]);
