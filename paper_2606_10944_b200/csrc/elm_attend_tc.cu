@@ -4,7 +4,7 @@
 //
 // One persistent CTA per SM takes every gridDim.x-th pair of 128-query tiles (numbered with the head
 // slowest, so that the CTAs running at one time share one head's coreset in L2) and streams the
-// head's coreset in blocks of 128 points for each pair.  Roles (576 threads):
+// head's coreset in blocks of 128 points for each pair.  Roles (608 threads):
 //   warps 0-15       softmax: all 16 warps serve the tile whose logits are ready, tile 0 and tile 1
 //                    in turn, while the tensor pipe works on the other tile.  A thread owns one row
 //                    and a quarter of the block's columns; two passes over the logits in TMEM (row
@@ -14,7 +14,7 @@
 //                    Same warps: epilogue of each pair of tiles.
 //   warp 16          TMA producer: the queries of each pair, K / V^T blocks through a 2-stage ring
 //                    that runs on across pairs
-//   warp 17          tcgen05.mma issuer: S = Q K^T (operands in shared memory), O += P V (P read
+//   warps 17, 18     tcgen05.mma issuers, one per query tile: S = Q K^T (operands in shared memory), O += P V (P read
 //                    from TMEM, V^T from shared memory); owns the TMEM allocation.  The logits of the
 //                    next pair's first block are issued right behind the last O += P V of the
 //                    current pair, so the tensor pipe does not drain while a pair is normalised and
@@ -43,7 +43,7 @@ namespace tc {
 constexpr int BM = 128;          // query rows per tile (= TMEM lanes)
 constexpr int BN = 128;          // coreset points per block
 constexpr int STAGES = 2;
-constexpr int NTHREADS = 576;          // 16 softmax warps + TMA producer + MMA issuer
+constexpr int NTHREADS = 608;          // 16 softmax warps + TMA producer + two MMA issuers (one per query tile)
 constexpr int TMA_WARP = 16, MMA_WARP = 17;
 constexpr uint32_t TMEM_COLS = 512;
 constexpr float RESCALE_TAU = 8.0f;      // rescale the accumulator only if the max grew by > 2^8
@@ -331,11 +331,11 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
 
     if (threadIdx.x == 0) {
         mbar_init(&bar->q_full, 1);
-        mbar_init(&bar->q_free, 1);
+        mbar_init(&bar->q_free, 2);
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(&bar->k_full[s], 1);
             mbar_init(&bar->v_full[s], 1);
-            mbar_init(&bar->kv_free[s], 1);
+            mbar_init(&bar->kv_free[s], 2);
         }
         for (int t = 0; t < 2; ++t) {
             mbar_init(&bar->s_full[t], 1);
@@ -424,9 +424,14 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
             }
             if (!ok) { atomicExch(status, 1); bar->abort_flag = 1; }
         }
-    } else if (warp == MMA_WARP) {
-        // ------------------------------ MMA issuer ------------------------------
+    } else if (warp == MMA_WARP || warp == MMA_WARP + 1) {
+        // ------------------------------ MMA issuers ------------------------------
+        // One issuing thread per query tile.  A tcgen05.mma holds its issuing thread until the tensor pipe
+        // takes it, and the waits and commits around a block cost that thread several hundred cycles in
+        // which it feeds nothing: with one thread for both tiles the pipe idled a quarter of the time.
+        // Each thread commits its own MMAs, so the barriers that release shared memory count two arrivals.
         if (lane == 0) {
+            const int t = warp - MMA_WARP;
             constexpr uint32_t IDESC_QK = umma_idesc_bf16(BM, BN);
             constexpr uint32_t IDESC_PV = umma_idesc_bf16(BM, D);
             // descriptors differ only in the 14-bit start-address field (address / 16)
@@ -460,7 +465,8 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
             if (ok) {
                 tc_fence_after();
                 const bool b0 = item_bias(0);
-                for (int t = 0; t < 2; ++t) { issue_qk(t, 0, b0); tc_commit(&bar->s_full[t]); }
+                issue_qk(t, 0, b0);
+                tc_commit(&bar->s_full[t]);
                 if (nblk == 1) tc_commit(&bar->q_free);                        // item 0 needs its queries no more
                 tc_commit(&bar->kv_free[0]);                                   // event 0
             }
@@ -478,23 +484,21 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                 if (last) bias_next = bias_after;
                 if (more) ok = mbar_wait(&bar->k_full[sn], (uint32_t)((G + 1) / STAGES) & 1u);
                 ok = ok && mbar_wait(&bar->v_full[s], (uint32_t)(G / STAGES) & 1u);
-                for (int t = 0; t < 2 && ok; ++t) {
-                    ok = mbar_wait(&bar->p_ready[t], (uint32_t)G & 1u);
-                    // a new item overwrites the accumulator: the epilogue of the previous one must have read it
-                    if (ok && j == 0 && k > 0) ok = mbar_wait(&bar->o_free[t], (uint32_t)(k - 1) & 1u);
+                ok = ok && mbar_wait(&bar->p_ready[t], (uint32_t)G & 1u);
+                // a new item overwrites the accumulator: the epilogue of the previous one must have read it
+                if (ok && j == 0 && k > 0) ok = mbar_wait(&bar->o_free[t], (uint32_t)(k - 1) & 1u);
+                if (!ok) break;
+                tc_fence_after();
+                issue_pv(t, s, j > 0);
+                // s_full also tells the softmax warps that O += P V of block j is complete (a commit
+                // covers every earlier MMA of this thread); the last block of an item signals the epilogue
+                if (last) tc_commit(&bar->o_done[t]);
+                if (more) {
+                    // the next item's queries are needed only now, after this item's last O += P V went out
+                    if (last) ok = mbar_wait(&bar->q_full, (uint32_t)(k + 1) & 1u);
                     if (!ok) break;
-                    tc_fence_after();
-                    issue_pv(t, s, j > 0);
-                    // s_full also tells the softmax warps that O += P V of block j is complete (a commit
-                    // covers every earlier MMA); the last block of an item signals the epilogue
-                    if (last) tc_commit(&bar->o_done[t]);
-                    if (more) {
-                        // the next item's queries are needed only now, after this item's last O += P V went out
-                        if (last && t == 0) ok = mbar_wait(&bar->q_full, (uint32_t)(k + 1) & 1u);
-                        if (!ok) break;
-                        issue_qk(t, sn, bias_next);
-                        tc_commit(&bar->s_full[t]);
-                    }
+                    issue_qk(t, sn, bias_next);
+                    tc_commit(&bar->s_full[t]);
                 }
                 if (!ok) break;
                 // the logits just issued belong to block j + 1 of item k, or to block 0 of item k + 1
