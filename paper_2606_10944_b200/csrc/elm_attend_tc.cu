@@ -5,17 +5,20 @@
 // One persistent CTA per SM takes every gridDim.x-th pair of 128-query tiles (numbered with the head
 // slowest, so that the CTAs running at one time share one head's coreset in L2) and streams the
 // head's coreset in blocks of 128 points for each pair.  Roles (608 threads):
-//   warps 0-15       softmax: all 16 warps serve the tile whose logits are ready, tile 0 and tile 1
-//                    in turn, while the tensor pipe works on the other tile.  A thread owns one row
-//                    and a quarter of the block's columns; two passes over the logits in TMEM (row
-//                    maximum, then probabilities); the quarters exchange row maxima through shared
-//                    memory.  Probabilities go back to TMEM as packed bf16 (over the logits); the
-//                    output accumulator is rescaled only when the maximum grew by more than 2^8.
-//                    Same warps: epilogue of each pair of tiles.
+//   warps 0-15       softmax, two passes over the logits in TMEM (row maximum, then probabilities).
+//                    Launches without a mask: warps 0-7 own tile 0, warps 8-15 tile 1, a thread owns one
+//                    row and half of the block's columns (kept in registers between the passes); the
+//                    two groups run out of phase.  Launches with a mask (causal tail, lifetimes): all
+//                    16 warps serve the tile whose logits are ready, tile 0 and tile 1 in turn, a thread
+//                    owns one row and a quarter of the columns.  Threads that share a row exchange row
+//                    maxima through shared memory behind a barrier of their own.  Probabilities go back
+//                    to TMEM as packed bf16 (over the logits); the output accumulator is rescaled only
+//                    when the maximum grew by more than 2^8.  Same warps: epilogue of each pair of tiles.
 //   warp 16          TMA producer: the queries of each pair, K / V^T blocks through a 2-stage ring
 //                    that runs on across pairs
-//   warps 17, 18     tcgen05.mma issuers, one per query tile: S = Q K^T (operands in shared memory), O += P V (P read
-//                    from TMEM, V^T from shared memory); owns the TMEM allocation.  The logits of the
+//   warps 17, 18     tcgen05.mma issuers, one per query tile: S = Q K^T (operands in shared memory),
+//                    O += P V (P read from TMEM, V^T from shared memory); warp 17 owns the TMEM
+//                    allocation.  The logits of the
 //                    next pair's first block are issued right behind the last O += P V of the
 //                    current pair, so the tensor pipe does not drain while a pair is normalised and
 //                    stored.
@@ -339,9 +342,9 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
         }
         for (int t = 0; t < 2; ++t) {
             mbar_init(&bar->s_full[t], 1);
-                        mbar_init(&bar->p_ready[t], 512);
+                        mbar_init(&bar->p_ready[t], MASKED ? 512 : 256);
             mbar_init(&bar->o_done[t], 1);
-            mbar_init(&bar->o_free[t], 16);
+            mbar_init(&bar->o_free[t], MASKED ? 16 : 8);
         }
         bar->abort_flag = 0;
         fence_barrier_init();
@@ -512,6 +515,137 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
         }
     } else {
         // ------------------------------ softmax + epilogue ------------------------------
+        if constexpr (!MASKED) {
+        // No mask: warps 0-7 own query tile 0, warps 8-15 tile 1, so the two tiles' passes run out of
+        // phase - while one group waits for the tensor pipe, or is between its passes, the other keeps
+        // the special-function unit busy (the exponentials of a block are what a pass mostly waits for).
+        // Warps with the same (warp % 4) share 32 rows; a thread owns one row and half of the block's
+        // columns (two quarters, the logits kept in registers between the passes); the two halves
+        // exchange their row maxima through shared memory behind a 64-thread barrier of their own.
+        const int t = warp >> 3, ch = (warp >> 2) & 1;
+        const int row = (warp & 3) * 32 + lane;                    // row in the tile = TMEM lane
+        const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t tS = tmem + lane_addr + t * 128 + ch * 64;  // this thread's 64 logit columns
+        const uint32_t tO = tmem + lane_addr + 256 + t * 128 + ch * (D / 2);   // its half of the accumulator
+        const int bar_id = 1 + t * 4 + (warp & 3);
+        const uint64_t scale2 = pack2(scale_log2, scale_log2);
+        bool ok = true;
+        int G = 0, xc = 0;                                         // xc: exchanges so far (buffers alternate)
+        for (int k = 0; k < n_items && ok; ++k) {
+            const int bh = item_bh(k), q0 = item_q0(k);
+            float m_ref = -INFINITY, l = 0.f;
+            for (int j = 0; j < nblk && ok; ++j, ++G, ++xc) {
+                ok = mbar_wait(&bar->s_full[t], (uint32_t)G & 1u);
+                if (!ok) break;
+                tc_fence_after();
+                // ---- pass 1: row maximum over the two halves ----
+                uint32_t a0[32], a1[32];
+                tmem_ld32(tS, a0);
+                tmem_ld32(tS + 32, a1);
+                tmem_wait_ld();
+                float m0 = -INFINITY, m1 = -INFINITY;
+#pragma unroll
+                for (int c = 0; c < 32; c += 2) {
+                    m0 = max3(m0, __uint_as_float(a0[c]), __uint_as_float(a0[c + 1]));
+                    m1 = max3(m1, __uint_as_float(a1[c]), __uint_as_float(a1[c + 1]));
+                }
+                bar->xchg[xc & 1][t * 2 + ch][row] = fmaxf(m0, m1) * scale_log2;
+                asm volatile("bar.sync %0, 64;" ::"r"(bar_id) : "memory");
+                const float mx = fmaxf(bar->xchg[xc & 1][t * 2][row], bar->xchg[xc & 1][t * 2 + 1][row]);
+                // lazy rescale: keep the old reference unless the maximum grew by more than 2^TAU
+                const bool grow = mx > m_ref + RESCALE_TAU;
+                if (__any_sync(0xffffffffu, grow)) {
+                    if (j > 0) {
+                        // O += P V of block j-1 is complete: s_full of block j was committed after it
+                        const float alpha = grow ? fast_exp2(m_ref - mx) : 1.f;
+#pragma unroll 1
+                        for (int c0 = 0; c0 < D / 2; c0 += 32) {
+                            uint32_t o[32];
+                            tmem_ld32(tO + c0, o);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
+                            tmem_st32(tO + c0, o);
+                        }
+                        l *= alpha;
+                        // the logits are fetched again rather than kept alive across this (rare) path
+                        tmem_ld32(tS, a0);
+                        tmem_ld32(tS + 32, a1);
+                        tmem_wait_ld();
+                    }
+                    if (grow) m_ref = mx;
+                }
+                // ---- pass 2: probabilities (bf16, over the first 16 columns of each quarter) and denominator ----
+                const uint64_t negm2 = pack2(-m_ref, -m_ref);
+                uint64_t sum2 = pack2(0.f, 0.f), sum2b = pack2(0.f, 0.f);
+                auto chunk = [&](const uint32_t (&a)[32], uint32_t tP) {
+                    uint32_t pk[16];
+#pragma unroll
+                    for (int i = 0; i < 16; i += 2) {
+                        const int c = 2 * i;
+                        float x0, x1, x2, x3;
+                        unpack2(fma2(pack2(__uint_as_float(a[c]), __uint_as_float(a[c + 1])), scale2, negm2), x0, x1);
+                        unpack2(fma2(pack2(__uint_as_float(a[c + 2]), __uint_as_float(a[c + 3])), scale2, negm2), x2, x3);
+                        const float p0 = fast_exp2(x0), p1 = fast_exp2(x1), p2 = fast_exp2(x2), p3 = fast_exp2(x3);
+                        sum2 = add2(sum2, pack2(p0, p1));
+                        sum2b = add2(sum2b, pack2(p2, p3));
+                        pk[i] = pack_bf16x2(p0, p1);
+                        pk[i + 1] = pack_bf16x2(p2, p3);
+                    }
+                    asm volatile(
+                        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%16], {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15};"
+                        ::"r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3]), "r"(pk[4]), "r"(pk[5]), "r"(pk[6]), "r"(pk[7]),
+                          "r"(pk[8]), "r"(pk[9]), "r"(pk[10]), "r"(pk[11]), "r"(pk[12]), "r"(pk[13]), "r"(pk[14]), "r"(pk[15]),
+                          "r"(tP)
+                        : "memory");
+                };
+                chunk(a0, tS);
+                chunk(a1, tS + 32);
+                float s_lo, s_hi;
+                unpack2(add2(sum2, sum2b), s_lo, s_hi);
+                l += s_lo + s_hi;
+                tmem_wait_st();
+                tc_fence_before();
+                mbar_arrive(&bar->p_ready[t]);
+            }
+            if (!ok) break;
+            ok = mbar_wait(&bar->o_done[t], (uint32_t)k & 1u);
+            if (!ok) break;
+            tc_fence_after();
+            bar->xchg[xc & 1][t * 2 + ch][row] = l;
+            asm volatile("bar.sync %0, 64;" ::"r"(bar_id) : "memory");
+            const float l_all = bar->xchg[xc & 1][t * 2][row] + bar->xchg[xc & 1][t * 2 + 1][row];
+            ++xc;
+            const float inv = 1.f / l_all;
+            const int64_t qrow = (int64_t)q0 + t * BM + row;
+            if (lse && ch == 0 && qrow < n_q) lse[(int64_t)bh * n_q_total + q_row0 + qrow] = m_ref + log2f(l_all);
+            __nv_bfloat16 *dst = O + ((int64_t)bh * n_q_total + q_row0 + qrow) * D + ch * (D / 2);
+#pragma unroll 1
+            for (int c0 = 0; c0 < D / 2; c0 += 32) {
+                uint32_t o[32];
+                tmem_ld32(tO + c0, o);
+                tmem_wait_ld();
+                if (c0 + 32 >= D / 2) {
+                    // the accumulator is in registers: the next item may overwrite it
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&bar->o_free[t]);
+                }
+                if (qrow < n_q) {
+#pragma unroll
+                    for (int c = 0; c < 32; c += 8) {
+                        uint4 v;
+                        v.x = pack_bf16x2(__uint_as_float(o[c]) * inv, __uint_as_float(o[c + 1]) * inv);
+                        v.y = pack_bf16x2(__uint_as_float(o[c + 2]) * inv, __uint_as_float(o[c + 3]) * inv);
+                        v.z = pack_bf16x2(__uint_as_float(o[c + 4]) * inv, __uint_as_float(o[c + 5]) * inv);
+                        v.w = pack_bf16x2(__uint_as_float(o[c + 6]) * inv, __uint_as_float(o[c + 7]) * inv);
+                        *reinterpret_cast<uint4 *>(dst + c0 + c) = v;
+                    }
+                }
+            }
+        }
+        if (!ok && lane == 0) atomicExch(status, 3);
+        } else {
         // All 16 warps serve the query tile whose logits are ready, tile 0 and tile 1 in turn: while
         // they work on one tile the tensor pipe works on the other.  Warps with the same (warp % 4)
         // share 32 rows (TMEM lanes) and split the block's 128 columns in four quarters; the
@@ -640,6 +774,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
             }
         }
         if (!ok && lane == 0) atomicExch(status, 3);
+        }
     }
     tc_fence_before();
     __syncthreads();
