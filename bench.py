@@ -23,7 +23,7 @@ if ROOT not in sys.path:
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one attend launch, from the ncu capture summarised
 # in profiles/attend_tc_cfg5_dram_traffic.md (read 1 084 004 352 + write 1 027 012 096 bytes)
-NCU_DRAM_BYTES_PER_ATTEND_LAUNCH = {"cfg5": 2111372800}
+NCU_DRAM_BYTES_PER_ATTEND_LAUNCH = {"cfg5": 2108260096}
 
 METRIC = "compress+attend tokens/sec per B200"
 UNIT = "tokens/s"
