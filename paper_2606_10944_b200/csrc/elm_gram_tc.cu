@@ -290,6 +290,7 @@ gram_tc_kernel(const __nv_bfloat16 *__restrict__ K, const __nv_bfloat16 *__restr
 // ---------------------------------------------------------------------------------------------
 constexpr int PNS = 3;                       // operand ring depth (jobs)
 constexpr int PTHREADS = 13 * 32;
+constexpr int PTAB = 256;                    // items of a CTA whose tiles are decoded up front
 
 struct PBarriers {
     uint64_t full[PNS], empty[PNS], accfull[2], accempty[2];
@@ -331,6 +332,28 @@ gram_tc_persistent_kernel(const __nv_bfloat16 *__restrict__ K, const __nv_bfloat
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
     if (*reinterpret_cast<volatile int *>(status) != 0) return;
+    // Which tile is item k of this CTA?  Decoding a tile number (two divisions, a square root) costs a lone
+    // thread about 900 cycles - a quarter of a tile's time on the MMA issuer - so all threads decode the CTA's
+    // items once, in parallel, into a table.
+    __shared__ int tab_p[PTAB], tab_jr[PTAB], tab_jc[PTAB];
+    for (int i = tid; i < PTAB; i += PTHREADS) {
+        const int it = blockIdx.x + i * gridDim.x;
+        if (it < total_items) {
+            int64_t jr, jc;
+            decode_tile(it % tiles_per_problem, P, jr, jc);
+            tab_p[i] = it / tiles_per_problem;
+            tab_jr[i] = (int)jr;
+            tab_jc[i] = (int)jc;
+        }
+    }
+    auto item = [&](int k, int it, int &p, int64_t &JR, int64_t &JC) {
+        if (k < PTAB) {
+            p = tab_p[k]; JR = tab_jr[k]; JC = tab_jc[k];
+        } else {
+            p = it / tiles_per_problem;
+            decode_tile(it % tiles_per_problem, P, JR, JC);
+        }
+    };
     if (tid == 0) {
         for (int b = 0; b < PNS; ++b) { mbar_init(&bar->full[b], 128); mbar_init(&bar->empty[b], 1); }
         for (int s = 0; s < 2; ++s) { mbar_init(&bar->accfull[s], 1); mbar_init(&bar->accempty[s], 256); }
@@ -345,11 +368,11 @@ gram_tc_persistent_kernel(const __nv_bfloat16 *__restrict__ K, const __nv_bfloat
 
     if (warp < 4) {
         // ------------------------------ loaders ------------------------------
-        int job = 0;
-        for (int it = blockIdx.x; it < total_items && ok; it += gridDim.x) {
-            const int p = it / tiles_per_problem, tile = it % tiles_per_problem;
+        int job = 0, lk = 0;
+        for (int it = blockIdx.x; it < total_items && ok; it += gridDim.x, ++lk) {
+            int p;
             int64_t JR, JC;
-            decode_tile(tile, P, JR, JC);
+            item(lk, it, p, JR, JC);
             const bool diagonal = JR == JC;
             const int32_t *curp = cur + (int64_t)p * n;
             // chunk q = tid + 128 i of a 128-row tile lies in row tid / CHUNKS + (128 / CHUNKS) i
@@ -388,9 +411,9 @@ gram_tc_persistent_kernel(const __nv_bfloat16 *__restrict__ K, const __nv_bfloat
             constexpr uint32_t IDESC = umma_idesc_bf16(TR, TR);
             int job = 0, k = 0;
             for (int it = blockIdx.x; it < total_items && ok; it += gridDim.x, ++k) {
-                const int tile = it % tiles_per_problem;
+                int p;
                 int64_t JR, JC;
-                decode_tile(tile, P, JR, JC);
+                item(k, it, p, JR, JC);
                 const bool diagonal = JR == JC;
                 const int slot = k & 1;
                 ok = mbar_wait(&bar->accempty[slot], ((uint32_t)(k >> 1) & 1u) ^ 1u);
@@ -425,9 +448,9 @@ gram_tc_persistent_kernel(const __nv_bfloat16 *__restrict__ K, const __nv_bfloat
         const float qscale = LOG2E / sqrtf((float)D);
         int k = 0;
         for (int it = blockIdx.x; it < total_items && ok; it += gridDim.x, ++k) {
-            const int p = it / tiles_per_problem, tile = it % tiles_per_problem;
+            int p;
             int64_t JR, JC;
-            decode_tile(tile, P, JR, JC);
+            item(k, it, p, JR, JC);
             const int slot = k & 1;
             const float vm = __uint_as_float(vmax_bits[p]);
             const float vm2 = vm * vm;
