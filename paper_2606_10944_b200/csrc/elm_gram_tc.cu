@@ -289,7 +289,8 @@ gram_tc_kernel(const __nv_bfloat16 *__restrict__ K, const __nv_bfloat16 *__restr
 //               next tile is gathered and multiplied
 // ---------------------------------------------------------------------------------------------
 constexpr int PNS = 3;                       // operand ring depth (jobs)
-constexpr int PTHREADS = 13 * 32;
+constexpr int PLOAD = 4;                      // loader warps (8 were slower: 0.76 against 0.71 ms per cfg5 step)
+constexpr int PTHREADS = (PLOAD + 1 + 8) * 32;   // loaders, the MMA issuer, 8 epilogue warps
 constexpr int PTAB = 256;                    // items of a CTA whose tiles are decoded up front
 
 struct PBarriers {
@@ -355,18 +356,18 @@ gram_tc_persistent_kernel(const __nv_bfloat16 *__restrict__ K, const __nv_bfloat
         }
     };
     if (tid == 0) {
-        for (int b = 0; b < PNS; ++b) { mbar_init(&bar->full[b], 128); mbar_init(&bar->empty[b], 1); }
+        for (int b = 0; b < PNS; ++b) { mbar_init(&bar->full[b], PLOAD * 32); mbar_init(&bar->empty[b], 1); }
         for (int s = 0; s < 2; ++s) { mbar_init(&bar->accfull[s], 1); mbar_init(&bar->accempty[s], 256); }
         fence_barrier_init();
     }
-    if (warp == 4) tmem_alloc(&bar->tmem_base, 512);
+    if (warp == PLOAD) tmem_alloc(&bar->tmem_base, 512);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = bar->tmem_base;
     bool ok = true;
 
-    if (warp < 4) {
+    if (warp < PLOAD) {
         // ------------------------------ loaders ------------------------------
         int job = 0, lk = 0;
         for (int it = blockIdx.x; it < total_items && ok; it += gridDim.x, ++lk) {
@@ -375,12 +376,13 @@ gram_tc_persistent_kernel(const __nv_bfloat16 *__restrict__ K, const __nv_bfloat
             item(lk, it, p, JR, JC);
             const bool diagonal = JR == JC;
             const int32_t *curp = cur + (int64_t)p * n;
-            // chunk q = tid + 128 i of a 128-row tile lies in row tid / CHUNKS + (128 / CHUNKS) i
-            constexpr int RPT = TR * CHUNKS / 128;            // chunks (= distinct rows) per thread and tile
+            // chunk q = tid + NL i of a 128-row tile lies in row tid / CHUNKS + (NL / CHUNKS) i, NL loader threads
+            constexpr int NL = PLOAD * 32;
+            constexpr int RPT = TR * CHUNKS / NL;            // chunks (= distinct rows) per thread and tile
             int32_t ra[RPT], rb[RPT];
 #pragma unroll
             for (int i = 0; i < RPT; ++i) {
-                const int r = tid / CHUNKS + (128 / CHUNKS) * i;
+                const int r = tid / CHUNKS + (NL / CHUNKS) * i;
                 ra[i] = __ldg(curp + 2 * JR + r);
                 rb[i] = diagonal ? 0 : __ldg(curp + 2 * JC + r);
             }
@@ -393,7 +395,7 @@ gram_tc_persistent_kernel(const __nv_bfloat16 *__restrict__ K, const __nv_bfloat
                 const uint32_t dstA = smem_u32(smem + b * SM::JOB), dstB = dstA + TR * D * 2;
 #pragma unroll
                 for (int i = 0; i < RPT; ++i) {
-                    const int r = tid / CHUNKS + (128 / CHUNKS) * i;
+                    const int r = tid / CHUNKS + (NL / CHUNKS) * i;
                     const uint32_t off = kh * (TR * 128) + (r >> 3) * 1024 + (r & 7) * 128 + ((c ^ (r & 7)) << 4);
                     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dstA + off), "l"(X + (int64_t)ra[i] * D + ch * 8) : "memory");
                     if (!diagonal)
@@ -405,7 +407,7 @@ gram_tc_persistent_kernel(const __nv_bfloat16 *__restrict__ K, const __nv_bfloat
         }
         asm volatile("cp.async.wait_all;" ::: "memory");
         if (!ok && lane == 0) atomicExch(status, 5);
-    } else if (warp == 4) {
+    } else if (warp == PLOAD) {
         // ------------------------------ MMA issuer ------------------------------
         if (lane == 0) {
             constexpr uint32_t IDESC = umma_idesc_bf16(TR, TR);
@@ -440,7 +442,7 @@ gram_tc_persistent_kernel(const __nv_bfloat16 *__restrict__ K, const __nv_bfloat
         }
     } else {
         // ------------------------------ epilogue ------------------------------
-        const int e = warp - 5;                               // 0..7
+        const int e = warp - (PLOAD + 1);                     // 0..7
         const int q4 = warp & 3;                              // TMEM lane quarter this warp may access
         const int ch = e >> 2;                                // column half
         const int r = q4 * 32 + lane;                         // point row in the tile
@@ -509,7 +511,7 @@ gram_tc_persistent_kernel(const __nv_bfloat16 *__restrict__ K, const __nv_bfloat
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 4) {
+    if (warp == PLOAD) {
         tc_fence_after();
         tmem_dealloc(tmem, 512);
     }
