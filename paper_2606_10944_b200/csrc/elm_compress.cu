@@ -626,10 +626,13 @@ static int run_halve_level(const LevelCtx<Tin, T> &c, const int32_t *cur, int32_
         int rc;
         if constexpr (std::is_same<Tin, __nv_bfloat16>::value && std::is_same<T, float>::value) {
             // tensor cores once a Halve call fills at least a quarter of a 64-pair tile side; calls
-            // that fit a tile (<= 64 pairs) are also walked inside the Gram kernel
+            // that share a tile (< 64 pairs) are also walked inside the Gram kernel.  Calls of exactly 64
+            // pairs - level 0 of the large workloads, one tile per call - go through the persistent
+            // kernel and a walk launch of their own: 0.61 + 0.32 ms of Gram + walk per cfg5 step against
+            // 0.70 + 0.27 with the walk inside the (one CTA per tile) Gram kernel
             if (P >= 16) {
                 WalkArgs wk;
-                wk.fused = P <= 64;
+                wk.fused = P < 64;
                 wk.level = lvl;
                 wk.seed = c.seed;
                 wk.logfac = logfac;

@@ -530,7 +530,7 @@ static int launch(const __nv_bfloat16 *K, const __nv_bfloat16 *V, const elm_para
     } else {
         tiles = (Ptotal + TP - 1) / TP;
     }
-    if (P > TP) {
+    if (P > TP || (P == TP && !wk.fused)) {
         // calls that span several tiles: persistent, pipelined kernel, one CTA per SM
         static int sm_count = 0;
         if (sm_count == 0) {
