@@ -458,8 +458,15 @@ gram_tc_persistent_kernel(const __nv_bfloat16 *__restrict__ K, const __nv_bfloat
             const float vm2 = vm * vm;
             // running shifts of this thread's 32 pair columns (in log2 units), fetched while the MMAs run
             float sh[32];
+            {
+                // 32 consecutive floats, 128-byte aligned (n / 2 and JC are multiples of 32)
+                const float4 *mp = reinterpret_cast<const float4 *>(Mpair + (int64_t)p * (n / 2) + JC + ch * 32);
 #pragma unroll
-            for (int i = 0; i < 32; ++i) sh[i] = __ldg(Mpair + (int64_t)p * (n / 2) + JC + ch * 32 + i) * LOG2E;
+                for (int i = 0; i < 8; ++i) {
+                    const float4 v = __ldg(mp + i);
+                    sh[4 * i] = v.x * LOG2E; sh[4 * i + 1] = v.y * LOG2E; sh[4 * i + 2] = v.z * LOG2E; sh[4 * i + 3] = v.w * LOG2E;
+                }
+            }
             ok = mbar_wait(&bar->accfull[slot], (uint32_t)(k >> 1) & 1u);
             if (!ok) break;
             tc_fence_after();
@@ -496,16 +503,12 @@ gram_tc_persistent_kernel(const __nv_bfloat16 *__restrict__ K, const __nv_bfloat
             const int64_t jc0 = JC + ch * 32 + (odd ? 16 : 0);
             const int64_t gr = jr / P;
             float *Fp = F + (int64_t)p * F_stride + jr * P - gr * P;
-            if (JR < JC) {
-                // a tile above the diagonal of its call: every entry is wanted, 64 contiguous bytes per thread
+            // 64 contiguous bytes per thread.  On a diagonal tile half of them lie below the diagonal of the
+            // call's P x P block, which nothing reads: written all the same, four vector stores being
+            // cheaper than sixteen predicated ones.
 #pragma unroll
-                for (int i = 0; i < 16; i += 4)
-                    *reinterpret_cast<float4 *>(Fp + jc0 + i) = make_float4(f[i], f[i + 1], f[i + 2], f[i + 3]);
-            } else {
-#pragma unroll
-                for (int i = 0; i < 16; ++i)
-                    if (jr <= jc0 + i) Fp[jc0 + i] = f[i];
-            }
+            for (int i = 0; i < 16; i += 4)
+                *reinterpret_cast<float4 *>(Fp + jc0 + i) = make_float4(f[i], f[i + 1], f[i + 2], f[i + 3]);
         }
         if (!ok && lane == 0) atomicExch(status, 7);
     }
