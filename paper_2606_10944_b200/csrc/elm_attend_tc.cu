@@ -91,6 +91,7 @@ template <int D> struct Smem {
 // (then zeros), and a per-problem flag that says whether all weights of the problem are equal (then
 // the bias cancels in the ratio).
 // ---------------------------------------------------------------------------------------------
+constexpr int GATHER_COLS = 64;          // list entries per CTA of the gather
 template <int D>
 __global__ void __launch_bounds__(256) gather_tc_kernel(const __nv_bfloat16 *__restrict__ K,
                                                         const __nv_bfloat16 *__restrict__ V,
@@ -101,22 +102,29 @@ __global__ void __launch_bounds__(256) gather_tc_kernel(const __nv_bfloat16 *__r
                                                         __nv_bfloat16 *__restrict__ Bx, float inv_scale_log2,
                                                         int *__restrict__ nonuniform)
 {
-    __shared__ __nv_bfloat16 tile[32][D + 2];
+    constexpr int CH = D / 8;                                  // 16-byte chunks per row
+    __shared__ __align__(16) __nv_bfloat16 tile[GATHER_COLS][D + 8];      // rows 16-byte aligned
     const int p = blockIdx.y;
-    const int c0 = blockIdx.x * 32;
+    const int c0 = blockIdx.x * GATHER_COLS;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const float w0 = w[(int64_t)p * n_core];
     bool differs = false;
-    for (int r = warp; r < 32; r += 8) {
+    // rows move in 16-byte chunks: lanes 0 .. CH-1 the key row (straight to Kc), lanes 16 .. 16+CH-1 the
+    // value row (to shared memory, to be written transposed)
+    for (int r = warp; r < GATHER_COLS; r += 8) {
         const int c = c0 + r;
         const bool ok = c < n_core;
         const int64_t row = ok ? idx[(int64_t)p * n_core + c] : 0;
-        const __nv_bfloat16 *ks = K + ((int64_t)p * n + row) * D;
-        const __nv_bfloat16 *vs = V + ((int64_t)p * n + row) * D;
-        __nv_bfloat16 *kd = Kc + ((int64_t)p * n_pad + c) * D;
-        for (int e = lane; e < D; e += 32) {
-            kd[e] = ok ? ks[e] : __float2bfloat16(0.f);
-            tile[r][e] = ok ? vs[e] : __float2bfloat16(0.f);
+        const int chunk = lane & 15;
+        if (chunk < CH) {
+            const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+            if (lane < 16) {
+                const uint4 v = ok ? __ldg(reinterpret_cast<const uint4 *>(K + ((int64_t)p * n + row) * D) + chunk) : zero;
+                reinterpret_cast<uint4 *>(Kc + ((int64_t)p * n_pad + c) * D)[chunk] = v;
+            } else {
+                const uint4 v = ok ? __ldg(reinterpret_cast<const uint4 *>(V + ((int64_t)p * n + row) * D) + chunk) : zero;
+                *reinterpret_cast<uint4 *>(&tile[r][chunk * 8]) = v;
+            }
         }
         if (lane < 16) {
             const float wc = ok ? w[(int64_t)p * n_core + c] : 0.f;
@@ -132,10 +140,10 @@ __global__ void __launch_bounds__(256) gather_tc_kernel(const __nv_bfloat16 *__r
     }
     if (differs) atomicOr(nonuniform + p, 1);
     __syncthreads();
-    // transposed write: thread -> (dimension e, point r) with r fastest
-    for (int i = threadIdx.x; i < 32 * D; i += 256) {
-        const int e = i >> 5, r = i & 31;
-        Vt[((int64_t)p * D + e) * n_pad + c0 + r] = tile[r][e];
+    // transposed write: a warp writes the 64 entries of one dimension e, 128 contiguous bytes
+    for (int e = warp; e < D; e += 8) {
+        const uint32_t lo = __bfloat16_as_ushort(tile[2 * lane][e]), hi = __bfloat16_as_ushort(tile[2 * lane + 1][e]);
+        *reinterpret_cast<uint32_t *>(Vt + ((int64_t)p * D + e) * n_pad + c0 + 2 * lane) = lo | (hi << 16);
     }
 }
 
@@ -838,7 +846,7 @@ static int launch(const __nv_bfloat16 *Q, const __nv_bfloat16 *K, const __nv_bfl
     {
         StageTimer t(timed ? ELM_STAGE_GATHER : -1, st, 1);
         ELM_CUDA_TRY(cudaMemsetAsync(flags, 0, sizeof(int) * (size_t)(problems + 1), st));
-        gather_tc_kernel<D><<<dim3((unsigned)(n_pad / 32), (unsigned)problems), 256, 0, st>>>(
+        gather_tc_kernel<D><<<dim3((unsigned)(n_pad / GATHER_COLS), (unsigned)problems), 256, 0, st>>>(
             K, V, idx, w, p->n_kv, n_core, n_pad, Kc, Vt, Bx, 1.f / scale_log2, flags);
         count_launches(1);
         ELM_CUDA_TRY(cudaGetLastError());
