@@ -88,3 +88,77 @@ def test_compute_call_without_a_device_fails_loudly():
     K = torch.zeros(1, 1, 64, 64)
     with pytest.raises(binding.ElmError):
         binding.compress(K, K, 4, 2)
+
+
+# ----------------------------------------------------------------------------------------------
+# host logic of the ragged-length, Express and streaming entry points (no device needed)
+# ----------------------------------------------------------------------------------------------
+def _level_sizes(n_mid, n_out, m):
+    sizes, a = [], n_mid
+    for i in range(m):
+        thresh = (n_out << (m + i)) >> (2 * (m - 1))
+        calls = a // thresh
+        sizes.append(a - calls * thresh)
+        a = calls * (thresh // 2)
+    return sizes + [a]
+
+
+@pytest.mark.parametrize("n,log2_nout,m,n_sink,n_window", [
+    (500, 4, 5, 0, 0), (500, 4, 5, 32, 32), (120, 3, 4, 5, 0), (63, 3, 3, 0, 9), (14, 3, 0, 4, 4), (9, 3, 3, 4, 5),
+    (121673, 11, 6, 32, 32), (131072, 11, 6, 0, 0)])
+def test_ragged_count_is_the_closed_form_of_algorithm_2(n, log2_nout, m, n_sink, n_window):
+    """elm_compress_ragged_count = sinks + window + the points Algorithm 2 leaves in S_0..S_m after the middle
+    rows: level i makes floor(a_i / t_i) calls, t_i = n_in 2^i / 4^(m-1)."""
+    p = _params(n_kv=n, log2_nout=log2_nout, m=m, q_heads=2)
+    count, ws = binding.compress_ragged_count(p, n_sink, n_window)
+    assert count == n_sink + n_window + sum(_level_sizes(n - n_sink - n_window, 1 << log2_nout, m))
+    assert ws > 0
+    if n == 131072:
+        assert count == 1 << log2_nout                      # the full length: elm_compress's coreset size
+
+
+@pytest.mark.parametrize("kw,sink,window,code", [
+    (dict(n_kv=50, log2_nout=3, m=2), 0, 0, -2),             # 50 middle rows > n_in = 32
+    (dict(n_kv=50, log2_nout=3, m=3), 30, 30, -2),           # sinks + window exceed the sequence
+    (dict(n_kv=50, log2_nout=1, m=6), 0, 0, -2),             # level-0 stretches below one pair
+    (dict(n_kv=50, log2_nout=3, m=3), -1, 0, -2),
+    (dict(n_kv=50, log2_nout=3, m=3, delta=1.5), 0, 0, -6),
+])
+def test_ragged_rejects_bad_sizes_on_the_host(kw, sink, window, code):
+    lib = binding.load_library()
+    p = _params(**kw)
+    assert lib.elm_compress_ragged_count(ctypes.byref(p), sink, window, None, None) == code
+    assert lib.elm_compress_ragged(256, 256, ctypes.byref(p), sink, window, 1, 256, 256, 256, 1 << 40, None) == code
+
+
+def test_attend_takes_any_sequence_length():
+    """The attention calls read K and V through the index list: n_kv need not be n_out 2^m."""
+    p = _params(n_kv=1000, log2_nout=0, m=0)
+    assert binding.attend_workspace_bytes(p, 300) > 0
+    lib = binding.load_library()
+    need = ctypes.c_size_t(0)
+    assert lib.elm_attend_workspace_bytes(ctypes.byref(p), 1001, ctypes.byref(need)) == -2     # n_core > n_kv
+    assert lib.elm_attend_workspace_bytes(ctypes.byref(_params(n_kv=1000, d=96)), 10, ctypes.byref(need)) == -2
+
+
+def test_express_and_stream_argument_checks():
+    lib = binding.load_library()
+    need = ctypes.c_size_t(0)
+    ok = _params(n_kv=16 * 64, n_q=16 * 64, log2_nout=4, m=0)
+    assert lib.elm_express_workspace_bytes(ctypes.byref(ok), 2, ctypes.byref(need)) == 0 and need.value > 0
+    small = need.value
+    # the prefill also holds the round's level lists, the window lists with their lifetimes and log-denominators
+    assert lib.elm_express_prefill_workspace_bytes(ctypes.byref(ok), 2, ctypes.byref(need)) == 0 and need.value > small
+    # a length that is not n_out 4^R
+    bad = _params(n_kv=16 * 8, n_q=16 * 8, log2_nout=4, m=0)
+    assert lib.elm_express_workspace_bytes(ctypes.byref(bad), 2, ctypes.byref(need)) == -2
+    # level-0 Halve calls of a single point: Compress2 of depth 6 on 2^7 points
+    deep = _params(n_kv=2 * 4 ** 4, n_q=2 * 4 ** 4, log2_nout=1, m=0)
+    assert lib.elm_express_prefill_workspace_bytes(ctypes.byref(deep), 6, ctypes.byref(need)) == -2
+    # one query per token in the prefill; one query per step in the stream
+    assert lib.elm_express_prefill_workspace_bytes(ctypes.byref(_params(n_kv=1024, n_q=100, log2_nout=4, m=0)), 2,
+                                                   ctypes.byref(need)) == -2
+    assert lib.elm_stream_workspace_bytes(ctypes.byref(_params(n_kv=1024, n_q=2, log2_nout=4, m=0)), 2,
+                                          ctypes.byref(need)) == -2
+    assert lib.elm_stream_workspace_bytes(ctypes.byref(_params(n_kv=1024, n_q=1, log2_nout=4, m=0)), 2,
+                                          ctypes.byref(need)) == 0 and need.value > 0
