@@ -690,9 +690,16 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                                 const int t_row = t_first + lane;
                                 const int32_t *bp = birth + life0 + j * BN, *dp = death + life0 + j * BN;
                                 vmask = 0u;
-#pragma unroll 8
-                                for (int c = 0; c < 32; ++c)
-                                    vmask |= (uint32_t)(__ldg(bp + c) <= t_row && t_row < __ldg(dp + c)) << c;
+                                // 32 consecutive entries of each array, 128-byte aligned: vector loads
+#pragma unroll
+                                for (int c = 0; c < 32; c += 4) {
+                                    const int4 b4 = __ldg(reinterpret_cast<const int4 *>(bp + c));
+                                    const int4 d4 = __ldg(reinterpret_cast<const int4 *>(dp + c));
+                                    vmask |= (uint32_t)(b4.x <= t_row && t_row < d4.x) << c;
+                                    vmask |= (uint32_t)(b4.y <= t_row && t_row < d4.y) << (c + 1);
+                                    vmask |= (uint32_t)(b4.z <= t_row && t_row < d4.z) << (c + 2);
+                                    vmask |= (uint32_t)(b4.w <= t_row && t_row < d4.w) << (c + 3);
+                                }
                             }
                         } else if (has_tail) {
                             int valid = n_core - j * BN - cq * 32;
