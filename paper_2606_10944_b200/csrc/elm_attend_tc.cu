@@ -169,15 +169,19 @@ __device__ __forceinline__ float row_max(uint32_t tS, float scale_log2, uint32_t
                 m1 = max3(m1, __uint_as_float(a[q & 1][c + 2]), __uint_as_float(a[q & 1][c + 3]));
             }
         } else {
+            // the same in the logits' own units (scale_log2 > 0), a masked column counting as -inf
 #pragma unroll
-            for (int c = 0; c < 32; ++c) {
-                float v = __uint_as_float(a[q & 1][c]) * scale_log2;
-                if (!((vmask >> c) & 1u)) v = -INFINITY;
-                m0 = fmaxf(m0, v);
+            for (int c = 0; c < 32; c += 4) {
+                const float v0 = ((vmask >> c) & 1u) ? __uint_as_float(a[q & 1][c]) : -INFINITY;
+                const float v1 = ((vmask >> (c + 1)) & 1u) ? __uint_as_float(a[q & 1][c + 1]) : -INFINITY;
+                const float v2 = ((vmask >> (c + 2)) & 1u) ? __uint_as_float(a[q & 1][c + 2]) : -INFINITY;
+                const float v3 = ((vmask >> (c + 3)) & 1u) ? __uint_as_float(a[q & 1][c + 3]) : -INFINITY;
+                m0 = max3(m0, v0, v1);
+                m1 = max3(m1, v2, v3);
             }
         }
     }
-    return SPECIAL ? m0 : fmaxf(m0, m1) * scale_log2;
+    return fmaxf(m0, m1) * scale_log2;
 }
 
 // p = 2^(logit - reference): reads the logits, writes the probabilities as packed bf16 to tP
@@ -241,13 +245,19 @@ __device__ __forceinline__ float exp_pass(uint32_t tS, uint32_t tP, float scale_
 #pragma unroll
             for (int i = 0; i < 16; ++i) pk[i] = pack_bf16x2(pe[2 * i], pe[2 * i + 1]);
         } else {
+            // the packed arithmetic of the plain form, a masked column's probability replaced by 0
 #pragma unroll
-            for (int c = 0; c < 32; c += 2) {
-                const float v0 = __uint_as_float(a[q & 1][c]) * scale_log2, v1 = __uint_as_float(a[q & 1][c + 1]) * scale_log2;
-                const float p0 = ((vmask >> c) & 1u) ? fast_exp2(v0 + neg_m) : 0.f;
-                const float p1 = ((vmask >> (c + 1)) & 1u) ? fast_exp2(v1 + neg_m) : 0.f;
-                sum0 += p0 + p1;
-                pk[c >> 1] = pack_bf16x2(p0, p1);
+            for (int i = 0; i < 16; i += 2) {
+                const int c = 2 * i;
+                float x0, x1, x2, x3;
+                unpack2(fma2(pack2(__uint_as_float(a[q & 1][c]), __uint_as_float(a[q & 1][c + 1])), scale2, negm2), x0, x1);
+                unpack2(fma2(pack2(__uint_as_float(a[q & 1][c + 2]), __uint_as_float(a[q & 1][c + 3])), scale2, negm2), x2, x3);
+                const float p0 = ((vmask >> c) & 1u) ? fast_exp2(x0) : 0.f, p1 = ((vmask >> (c + 1)) & 1u) ? fast_exp2(x1) : 0.f;
+                const float p2 = ((vmask >> (c + 2)) & 1u) ? fast_exp2(x2) : 0.f, p3 = ((vmask >> (c + 3)) & 1u) ? fast_exp2(x3) : 0.f;
+                sum2 = add2(sum2, pack2(p0, p1));
+                sum2b = add2(sum2b, pack2(p2, p3));
+                pk[i] = pack_bf16x2(p0, p1);
+                pk[i + 1] = pack_bf16x2(p2, p3);
             }
         }
         asm volatile(
