@@ -130,7 +130,9 @@ int elm_compress_ragged(const void *K, const void *V, const elm_params *params, 
  *   Q          [batch][q_heads][n_q][d]
  *   K, V       the ORIGINAL [batch][kv_heads][n_kv][d] tensors; rows are gathered through idx.
  *   idx, w     [batch][kv_heads][n_core]; any positive finite weights (they need not sum to 1),
- *              1 <= n_core <= n_kv.
+ *              1 <= n_core <= n_kv.  Every entry of idx must lie in [0, n_kv): the rows are read
+ *              through it unchecked (the caller's obligation; a build with -DELM_BOUNDS_CHECK
+ *              skips such an entry and reports it through the status word instead).
  *   params     n_kv may be any length >= 1 here; log2_nout, m, delta are not used.
  *   O          [batch][q_heads][n_q][d], same dtype as Q.
  *   workspace  at least elm_attend_workspace_bytes(params, n_core), 256-byte aligned.
@@ -168,10 +170,15 @@ int elm_attend_workspace_bytes(const elm_params *params, int32_t n_core, size_t 
  *     kernels can overlap on the GPU (different streams, no ordering between them) race on it:
  *     order them, or use elm_attend with separate workspaces.
  *   - Per-stage timing (elm_profile_enable) does not cover this entry point.
+ *   - The bounded waits of the tensor-core kernels report through a status word that lives in the
+ *     same array; elm_attend_static_status copies it to *status_host (0 = every wait completed) after
+ *     synchronising `stream`, for the (params, n_core) of the last call on this device.  It allocates
+ *     nothing either.  A non-zero word means O of that call is undefined.
  */
 #define ELM_ATTEND_STATIC_SCRATCH_BYTES (16u << 20)
 int elm_attend_static(const void *Q, const void *K, const void *V, const int32_t *idx, const float *w,
                       int32_t n_core, const elm_params *params, void *O, void *stream);
+int elm_attend_static_status(const elm_params *params, int32_t n_core, int32_t *status_host, void *stream);
 
 /*
  * Offline-Express (the recursive form of Algorithm 1, "Express", with Subsample - Algorithm 3 - and

@@ -62,6 +62,9 @@ def _load():
                                      ctypes.c_int, ctypes.c_double, _f64p, ctypes.c_uint64,
                                      ctypes.c_uint32, _i32p, _f64p, _f64p]
     lib.oracle_compress2.restype = ctypes.c_int
+    lib.oracle_compress2_calls.argtypes = lib.oracle_compress2.argtypes + [_f64p, ctypes.c_int64,
+                                                                           ctypes.POINTER(ctypes.c_int64)]
+    lib.oracle_compress2_calls.restype = ctypes.c_int
     lib.oracle_compress2_batched.argtypes = [_f32p, _f32p, ctypes.c_int, ctypes.c_int64,
                                              ctypes.c_int, ctypes.c_int, ctypes.c_int,
                                              ctypes.c_double, _f64p, ctypes.c_uint64, _i32p,
@@ -94,6 +97,8 @@ def _load():
                                               ctypes.c_int, ctypes.c_double, ctypes.c_uint64, ctypes.c_uint32,
                                               _f64p, _i32p, _i32p, _f64p, _i32p, _i64p]
     lib.oracle_thinformer_express.restype = ctypes.c_int
+    lib.oracle_thinformer_express_log.argtypes = lib.oracle_thinformer_express.argtypes + [_f64p, ctypes.c_int64]
+    lib.oracle_thinformer_express_log.restype = ctypes.c_int
     lib.oracle_exact_causal_attention.argtypes = [_f32p, _f32p, _f32p, ctypes.c_int64, ctypes.c_int, _f64p]
     lib.oracle_exact_causal_attention.restype = ctypes.c_int
     lib.oracle_num_threads.argtypes = []
@@ -192,6 +197,34 @@ def compress2(K, V, log2_nout: int, m: int, delta: float = 0.5, delta_level=None
     if rc != 0:
         raise ValueError(f"oracle_compress2 failed with {rc}")
     return idx, w, float(mg.value)
+
+
+def compress2_calls(K, V, log2_nout: int, m: int, delta: float = 0.5, delta_level=None, seed: int = 1,
+                    head: int = 0):
+    """Offline-Compress2 as ``compress2``, also returning the record of its Halve calls.
+
+    Returns (idx, w, calls[n_calls, 4]): per call, in the order made, level, number of the call at
+    its level, points in, delta used."""
+    K, kp = _f32(K)
+    V, vp = _f32(V)
+    n, d = K.shape
+    n_out = 1 << log2_nout
+    idx = np.zeros(n_out, dtype=np.int32)
+    w = np.zeros(n_out, dtype=np.float64)
+    cap = sum(4 ** i for i in range(max(m, 1)))
+    log = np.zeros((cap, 4), dtype=np.float64)
+    cnt = ctypes.c_int64(0)
+    dl = None
+    if delta_level is not None:
+        dl_arr, dl = _f64(delta_level)
+        assert dl_arr.shape[0] == m
+    rc = _load().oracle_compress2_calls(kp, vp, n, d, log2_nout, m, delta, dl, seed, head,
+                                        idx.ctypes.data_as(_i32p), w.ctypes.data_as(_f64p), None,
+                                        log.ctypes.data_as(_f64p), cap, ctypes.byref(cnt))
+    if rc != 0:
+        raise ValueError(f"oracle_compress2_calls failed with {rc}")
+    assert cnt.value <= cap
+    return idx, w, log[:cnt.value].copy()
 
 
 def compress2_batched(K, V, log2_nout: int, m: int, delta: float = 0.5, delta_level=None,
@@ -314,7 +347,9 @@ def thinformer_express(Q, K, V, log2_nout: int, mbar: int, delta: float = 0.5, s
     """Algorithms 1-5 streaming over one attention problem (Q, K, V are [n, d]).
 
     Returns a dict: O [n, d] (or None), cache_size [n] (points in wtd_cache() when token t arrives),
-    final_idx / final_w (wtd_cache() after the last update), halve_calls."""
+    final_idx / final_w (wtd_cache() after the last update), halve_calls, halve_log [halve_calls, 5]
+    (per KH call in the order made: thinning factor m, level i or -1 / -2 for the two halvings of E,
+    points in, delta used, sibling 1..3 or 0 for E)."""
     Q, qp = _f32(Q)
     K, kp = _f32(K)
     V, vp = _f32(V)
@@ -326,15 +361,20 @@ def thinformer_express(Q, K, V, log2_nout: int, mbar: int, delta: float = 0.5, s
     fw = np.zeros(6 * n_out + 1, dtype=np.float64)
     fc = ctypes.c_int32(0)
     hc = ctypes.c_int64(0)
-    rc = _load().oracle_thinformer_express(qp, kp, vp, n, d, log2_nout, mbar, delta, seed, head,
-                                           O.ctypes.data_as(_f64p) if want_outputs else None,
-                                           cache.ctypes.data_as(_i32p), fidx.ctypes.data_as(_i32p),
-                                           fw.ctypes.data_as(_f64p), ctypes.byref(fc), ctypes.byref(hc))
+    # a KH call consumes at least two points of its level and levels shrink by half: fewer than n calls
+    log_cap = n + 8
+    hlog = np.zeros((log_cap, 5), dtype=np.float64)
+    rc = _load().oracle_thinformer_express_log(qp, kp, vp, n, d, log2_nout, mbar, delta, seed, head,
+                                               O.ctypes.data_as(_f64p) if want_outputs else None,
+                                               cache.ctypes.data_as(_i32p), fidx.ctypes.data_as(_i32p),
+                                               fw.ctypes.data_as(_f64p), ctypes.byref(fc), ctypes.byref(hc),
+                                               hlog.ctypes.data_as(_f64p), log_cap)
     if rc != 0:
         raise ValueError(f"oracle_thinformer_express failed with {rc}")
     c = int(fc.value)
+    assert hc.value <= log_cap
     return {"O": O, "cache_size": cache, "final_idx": fidx[:c].copy(), "final_w": fw[:c].copy(),
-            "halve_calls": int(hc.value)}
+            "halve_calls": int(hc.value), "halve_log": hlog[:int(hc.value)].copy()}
 
 
 def exact_causal_attention(Q, K, V):

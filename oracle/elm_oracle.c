@@ -216,6 +216,8 @@ typedef struct {
     uint64_t seed;
     uint32_t head;
     double min_margin;     /* min_i |U_i - p_i| over all calls */
+    double *call_log;      /* optional [cap][4]: level, call number, points in, delta used */
+    int64_t call_log_cap, call_log_n;
 } compress2_ctx;
 
 /* One recursion of Offline-Compress2: `x` holds n_in = 2^m * n_out points; `level` counts
@@ -236,6 +238,11 @@ static int compress2_rec(compress2_ctx *c, int m, int level, int32_t *x, int64_t
             U[i] = oracle_uniform(c->seed, (uint32_t)i, (uint32_t)g, (uint32_t)level, c->head);
         rc = oracle_kh(c->K, c->V, c->d, c->vmax, x + g * gs, (int)gs, c->delta_level[level],
                        1, U, next + g * (gs / 2), NULL, diag);
+        if (c->call_log && c->call_log_n < c->call_log_cap) {
+            double *r = c->call_log + 4 * c->call_log_n;
+            r[0] = (double)level; r[1] = (double)g; r[2] = (double)gs; r[3] = c->delta_level[level];
+        }
+        c->call_log_n += 1;
         for (int64_t i = 0; i < gs / 2; ++i) {
             double mg = fabs(U[i] - diag[4 * i + 2]);
             if (mg < c->min_margin) c->min_margin = mg;
@@ -254,10 +261,14 @@ static int compress2_rec(compress2_ctx *c, int m, int level, int32_t *x, int64_t
  * idx_out[n_out] receives the coreset rows (R-order), w_out[n_out] the weights 1/n_out
  * (positive, summing to 1).  delta_level[m] may be NULL (R-delta with `delta`).
  * min_margin (optional) receives min |U - p| over every decision taken.
+ * call_log (optional, [call_log_cap][4]) receives one row per Halve call in the order the calls are
+ * made: level, number of the call at its level, points in, delta used; call_log_count the number
+ * of calls made (rows beyond the capacity are counted, not written).
  */
-int oracle_compress2(const float *K, const float *V, int64_t n, int d, int log2_nout, int m,
-                     double delta, const double *delta_level, uint64_t seed, uint32_t head,
-                     int32_t *idx_out, double *w_out, double *min_margin)
+int oracle_compress2_calls(const float *K, const float *V, int64_t n, int d, int log2_nout, int m,
+                           double delta, const double *delta_level, uint64_t seed, uint32_t head,
+                           int32_t *idx_out, double *w_out, double *min_margin,
+                           double *call_log, int64_t call_log_cap, int64_t *call_log_count)
 {
     int64_t n_out = (int64_t)1 << log2_nout;
     if (m < 0 || n != (n_out << m)) return -1;
@@ -267,14 +278,23 @@ int oracle_compress2(const float *K, const float *V, int64_t n, int d, int log2_
     if (delta_level) memcpy(dl, delta_level, sizeof(double) * (size_t)m);
     else oracle_default_delta_levels(m, delta, dl);
     for (int64_t i = 0; i < n; ++i) x[i] = (int32_t)i;
-    compress2_ctx c = { K, V, d, oracle_vmax(V, n, d), dl, seed, head, 2.0 };
+    compress2_ctx c = { K, V, d, oracle_vmax(V, n, d), dl, seed, head, 2.0, call_log, call_log_cap, 0 };
     int rc = compress2_rec(&c, m, 0, x, n);
     if (rc == 0) {
         for (int64_t i = 0; i < n_out; ++i) { idx_out[i] = x[i]; w_out[i] = 1.0 / (double)n_out; }
         if (min_margin) *min_margin = c.min_margin;
+        if (call_log_count) *call_log_count = c.call_log_n;
     }
     free(dl); free(x);
     return rc;
+}
+
+int oracle_compress2(const float *K, const float *V, int64_t n, int d, int log2_nout, int m,
+                     double delta, const double *delta_level, uint64_t seed, uint32_t head,
+                     int32_t *idx_out, double *w_out, double *min_margin)
+{
+    return oracle_compress2_calls(K, V, n, d, log2_nout, m, delta, delta_level, seed, head, idx_out, w_out,
+                                  min_margin, NULL, 0, NULL);
 }
 
 /* The same for `problems` independent attention problems laid out back to back
@@ -552,6 +572,9 @@ typedef struct {
     int64_t nS[40];
     int64_t calls[40];
     int64_t halve_calls;   /* total KH calls made (cost accounting) */
+    double *halve_log;     /* optional [cap][5]: thinning factor m, level i (-1, -2: first, second halving
+                              of E), points in, delta used, sibling j (0 for E) */
+    int64_t halve_log_cap;
 } express_state;
 
 static double kh_express_delta_m(double delta, int m)
@@ -568,8 +591,13 @@ static void express_reset_thin(express_state *st)
 }
 
 static int express_halve(express_state *st, int32_t *x, int64_t s, double dlt, uint32_t code, uint32_t call,
-                         int32_t *out)
+                         int32_t *out, int level)
 {
+    if (st->halve_log && st->halve_calls < st->halve_log_cap) {
+        double *r = st->halve_log + 5 * st->halve_calls;
+        r[0] = (double)st->m; r[1] = (double)level; r[2] = (double)s; r[3] = dlt;
+        r[4] = level >= 0 ? (double)(st->b + 1) : 0.0;
+    }
     double *U = (double *)malloc(sizeof(double) * (size_t)(s / 2));
     if (!U) return -2;
     for (int64_t i = 0; i < s / 2; ++i) U[i] = oracle_uniform(st->seed, (uint32_t)i, call, code, st->head);
@@ -591,7 +619,7 @@ static int express_compress2_update(express_state *st, int32_t x)
             const double dm = kh_express_delta_m(st->delta, st->m);
             const double dlt = pow(4.0, (double)(i + 1 - q)) * dm / (3.0 * (double)q);
             const uint32_t code = (uint32_t)i + 64u * (uint32_t)(4 * (st->m / 2) + st->b + 1);
-            int rc = express_halve(st, st->S[i], thresh, dlt, code, (uint32_t)st->calls[i], st->S[i + 1] + st->nS[i + 1]);
+            int rc = express_halve(st, st->S[i], thresh, dlt, code, (uint32_t)st->calls[i], st->S[i + 1] + st->nS[i + 1], i);
             if (rc != 0) return rc;
             st->calls[i] += 1;
             st->nS[i + 1] += thresh / 2;
@@ -635,8 +663,8 @@ static int express_update(express_state *st, int32_t x)
         const double dm = kh_express_delta_m(st->delta, st->m);
         int32_t *tmp = (int32_t *)malloc(sizeof(int32_t) * (size_t)(2 * st->n_out));
         if (!tmp) return -2;
-        int rc = express_halve(st, st->E, 4 * st->n_out, 0.5 * dm, 62u + 64u * (uint32_t)(4 * (st->m / 2)), 0u, tmp);
-        if (rc == 0) rc = express_halve(st, tmp, 2 * st->n_out, 0.5 * dm, 63u + 64u * (uint32_t)(4 * (st->m / 2)), 0u, st->E);
+        int rc = express_halve(st, st->E, 4 * st->n_out, 0.5 * dm, 62u + 64u * (uint32_t)(4 * (st->m / 2)), 0u, tmp, -1);
+        if (rc == 0) rc = express_halve(st, tmp, 2 * st->n_out, 0.5 * dm, 63u + 64u * (uint32_t)(4 * (st->m / 2)), 0u, st->E, -2);
         free(tmp);
         if (rc != 0) return rc;
         st->nE = st->n_out;
@@ -655,11 +683,14 @@ static int express_update(express_state *st, int32_t x)
  *   cache_size[n]    points in wtd_cache() when token t arrives (the input token not counted)
  *   final_idx/final_w/final_count  wtd_cache() after the last update (capacity 6 n_out)
  *   halve_calls      number of KH calls made
+ *   halve_log        [halve_log_cap][5], one row per KH call in the order made: thinning factor m of
+ *                    the round, level i of the Compress2 call (-1 / -2 for the first / second halving
+ *                    of the Express coreset), points in, delta used, sibling (1..3; 0 for E)
  */
-int oracle_thinformer_express(const float *Q, const float *K, const float *V, int64_t n, int d, int log2_nout,
-                              int mbar, double delta, uint64_t seed, uint32_t head, double *O,
-                              int32_t *cache_size, int32_t *final_idx, double *final_w, int32_t *final_count,
-                              int64_t *halve_calls)
+int oracle_thinformer_express_log(const float *Q, const float *K, const float *V, int64_t n, int d, int log2_nout,
+                                  int mbar, double delta, uint64_t seed, uint32_t head, double *O,
+                                  int32_t *cache_size, int32_t *final_idx, double *final_w, int32_t *final_count,
+                                  int64_t *halve_calls, double *halve_log, int64_t halve_log_cap)
 {
     if (log2_nout < 0 || mbar < 0 || !(delta > 0.0 && delta < 1.0)) return -1;
     express_state st;
@@ -667,6 +698,7 @@ int oracle_thinformer_express(const float *Q, const float *K, const float *V, in
     st.K = K; st.V = V; st.d = d; st.delta = delta; st.seed = seed; st.head = head;
     st.n_out = (int64_t)1 << log2_nout;
     st.mbar = mbar;
+    st.halve_log = halve_log; st.halve_log_cap = halve_log_cap;
     st.vmax = oracle_vmax(V, n, d);                                       /* R-vmax-causal */
     st.E = (int32_t *)malloc(sizeof(int32_t) * (size_t)(4 * st.n_out));
     int rc = st.E ? 0 : -2;
@@ -716,6 +748,15 @@ int oracle_thinformer_express(const float *Q, const float *K, const float *V, in
     for (int i = 0; i <= mbar; ++i) free(st.S[i]);
     free(cidx); free(cw); free(qrow);
     return rc;
+}
+
+int oracle_thinformer_express(const float *Q, const float *K, const float *V, int64_t n, int d, int log2_nout,
+                              int mbar, double delta, uint64_t seed, uint32_t head, double *O,
+                              int32_t *cache_size, int32_t *final_idx, double *final_w, int32_t *final_count,
+                              int64_t *halve_calls)
+{
+    return oracle_thinformer_express_log(Q, K, V, n, d, log2_nout, mbar, delta, seed, head, O, cache_size,
+                                         final_idx, final_w, final_count, halve_calls, NULL, 0);
 }
 
 /* Exact causal attention, Eq. (def:att): query t over the pairs 1..t. */

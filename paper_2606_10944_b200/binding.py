@@ -20,7 +20,7 @@ STAGE_NAMES = ["prepass", "level_prep", "gram", "walk", "emit", "gather", "atten
 
 EXPORTED_SYMBOLS = [
     "elm_workspace_bytes", "elm_default_delta_levels", "elm_compress", "elm_attend",
-    "elm_attend_workspace_bytes", "elm_attend_static", "elm_compress_ragged_count", "elm_compress_ragged", "elm_express_workspace_bytes", "elm_express_compress",
+    "elm_attend_workspace_bytes", "elm_attend_static", "elm_attend_static_status", "elm_compress_ragged_count", "elm_compress_ragged", "elm_express_workspace_bytes", "elm_express_compress",
     "elm_express_prefill_workspace_bytes", "elm_express_prefill",
     "elm_stream_workspace_bytes", "elm_stream_init", "elm_stream_step", "elm_stream_cache",
     "elm_host_call_scratch_bytes", "elm_compress_attend_host",
@@ -76,6 +76,7 @@ def load_library():
     lib.elm_attend.argtypes = [vp, vp, vp, vp, vp, ctypes.c_int32, pp, vp, vp, sz, vp]
     lib.elm_attend_workspace_bytes.argtypes = [pp, ctypes.c_int32, szp]
     lib.elm_attend_static.argtypes = [vp, vp, vp, vp, vp, ctypes.c_int32, pp, vp, vp]
+    lib.elm_attend_static_status.argtypes = [pp, ctypes.c_int32, ctypes.POINTER(ctypes.c_int32), vp]
     lib.elm_compress_ragged_count.argtypes = [pp, ctypes.c_int32, ctypes.c_int32, ctypes.POINTER(ctypes.c_int32), szp]
     lib.elm_compress_ragged.argtypes = [vp, vp, pp, ctypes.c_int32, ctypes.c_int32, ctypes.c_uint64, vp, vp, vp, sz, vp]
     lib.elm_express_workspace_bytes.argtypes = [pp, ctypes.c_int32, szp]
@@ -347,6 +348,18 @@ def attend_static(Q, K, V, idx, w, precision="fp32", out=None):
                                  idx.shape[-1], ctypes.byref(p), O.data_ptr(), _stream()),
            "elm_attend_static")
     return O
+
+
+def attend_static_status(Q, K, n_core: int, precision="fp32") -> int:
+    """elm_attend_static_status after an attend_static call with these tensors' shapes: 0 unless a bounded
+    device wait expired during it."""
+    B, Hq, nq, d = Q.shape
+    Hkv, n = K.shape[1], K.shape[2]
+    p, _ = make_params(B, Hq, Hkv, n, nq, d, n.bit_length() - 1, 0, _dtype_code(Q), precision)
+    out = ctypes.c_int32(-1)
+    _check(load_library().elm_attend_static_status(ctypes.byref(p), n_core, ctypes.byref(out), _stream()),
+           "elm_attend_static_status")
+    return int(out.value)
 
 
 def compress_attend_host(Q, K, V, log2_nout: int, m: int, seed: int = 1, precision="fp32",

@@ -288,6 +288,8 @@ static int attend_enqueue_untimed(const Tin *Q, const Tin *K, const Tin *V, cons
     Tin *Vc = reinterpret_cast<Tin *>(scratch + L.Vc);
     float *bias = reinterpret_cast<float *>(scratch + L.bias);
     const int problems = p->batch * p->kv_heads;
+    // this path has no bounded waits: its status word reads 0
+    ELM_CUDA_TRY(cudaMemsetAsync(scratch + L.flags, 0, sizeof(int) * (size_t)(problems + 1), st));
     gather_kernel<Tin><<<dim3((unsigned)((n_core + 7) / 8), (unsigned)problems), 256, 0, st>>>(
         K, V, idx, w, p->n_kv, p->d, n_core, Kc, Vc, bias);
     count_launches(1);
@@ -371,4 +373,23 @@ extern "C" int elm_attend_static(const void *Q, const void *K, const void *V, co
     typedef __nv_bfloat16 bf;
     return det ? attend_enqueue_untimed<bf, double>((const bf *)Q, (const bf *)K, (const bf *)V, idx, w, n_core, params, (bf *)O, scratch, st)
                : attend_enqueue_untimed<bf, float>((const bf *)Q, (const bf *)K, (const bf *)V, idx, w, n_core, params, (bf *)O, scratch, st);
+}
+
+extern "C" int elm_attend_static_status(const elm_params *params, int32_t n_core, int32_t *status_host, void *stream)
+{
+    using namespace elm;
+    if (!params || !status_host) return ELM_ERR_NULL;
+    int rc = validate_attend_params(params);
+    if (rc != ELM_OK) return rc;
+    if (n_core < 1 || n_core > params->n_kv) return ELM_ERR_SHAPE;
+    const AttendLayout L = attend_layout(params, n_core);
+    if (L.total > (size_t)ELM_ATTEND_STATIC_SCRATCH_BYTES) return ELM_ERR_STATIC_LIMIT;
+    unsigned char *scratch = nullptr;
+    rc = static_scratch_address(&scratch);
+    if (rc != ELM_OK) return rc;
+    // the status word follows the per-problem "weights differ" flags, as in a caller's workspace
+    const unsigned char *word = scratch + L.flags + 4 * (size_t)params->batch * params->kv_heads;
+    ELM_CUDA_TRY(cudaMemcpyAsync(status_host, word, 4, cudaMemcpyDeviceToHost, (cudaStream_t)stream));
+    ELM_CUDA_TRY(cudaStreamSynchronize((cudaStream_t)stream));
+    return ELM_OK;
 }

@@ -138,19 +138,23 @@ def test_express_prefill_outputs_match_streaming_oracle(name, precision):
     Qf, Kf, Vf = as_f32_numpy(Q), as_f32_numpy(K), as_f32_numpy(V)
     B, Hq, n, d = Qf.shape
     H = Kf.shape[1]
-    worst = 0.0
+    worst, compared = 0.0, 0
     for b in range(B):
         for h in range(Hq):
             kv = (h * H) // Hq
             r = oracle.thinformer_express(Qf[b, h], Kf[b, kv], Vf[b, kv], log2_nout, mbar, seed=9, head=b * H + kv)
             if precision == "fp64":
                 assert np.array_equal(idx[b, kv].cpu().numpy(), r["final_idx"])
+            # fp32 mode may (rarely) pick another coreset; then the outputs legitimately differ
+            if np.array_equal(idx[b, kv].cpu().numpy(), r["final_idx"]):
                 worst = max(worst, max_rel_err(got[b, h], r["O"]))
-            else:
-                # fp32 mode may (rarely) pick another coreset; then the outputs legitimately differ
-                if np.array_equal(idx[b, kv].cpu().numpy(), r["final_idx"]):
-                    worst = max(worst, max_rel_err(got[b, h], r["O"]))
-    print(f"{name} {precision}: max relative error of the prefill outputs {worst:.3e}")
+                compared += 1
+            # whatever the cache, the first 4 n_out outputs are exact causal attention and do not depend on it
+            m4 = 4 << log2_nout
+            worst = max(worst, max_rel_err(got[b, h, :m4], r["O"][:m4]))
+    print(f"{name} {precision}: max relative error of the prefill outputs {worst:.3e} ({compared} of {B * Hq} heads whole)")
+    # every head in fp64 mode; in fp32 mode at least half of them (no mismatch has been seen on these cases)
+    assert compared >= (B * Hq if precision == "fp64" else max(1, B * Hq // 2))
     assert worst <= PREFILL_TOL[(wl.dtype if wl.dtype == "bf16" else "f32", precision)]
 
 
@@ -219,7 +223,7 @@ def test_stream_outputs_and_cache_match_streaming_oracle(name, precision):
     Qf, Kf, Vf = as_f32_numpy(Q), as_f32_numpy(K), as_f32_numpy(V)
     B, Hq = Qf.shape[:2]
     H = Kf.shape[1]
-    worst = 0.0
+    worst, compared = 0.0, 0
     for b in range(B):
         for h in range(Hq):
             kv = (h * H) // Hq
@@ -228,10 +232,14 @@ def test_stream_outputs_and_cache_match_streaming_oracle(name, precision):
             same = np.array_equal(gi, r["final_idx"])
             if precision == "fp64":
                 assert same
-                assert np.allclose(gw, r["final_w"], rtol=1e-6, atol=0)
             if same:
+                assert np.allclose(gw, r["final_w"], rtol=1e-6, atol=0)
                 worst = max(worst, max_rel_err(got[b, h], r["O"]))
-    print(f"{name} {precision}: max relative error of the streamed outputs {worst:.3e}")
+                compared += 1
+            m4 = 4 << log2_nout                       # the exact regime does not depend on any decision
+            worst = max(worst, max_rel_err(got[b, h, :m4], r["O"][:m4]))
+    print(f"{name} {precision}: max relative error of the streamed outputs {worst:.3e} ({compared} of {B * Hq} heads whole)")
+    assert compared >= (B * Hq if precision == "fp64" else max(1, B * Hq // 2))
     assert worst <= PREFILL_TOL[(wl.dtype if wl.dtype == "bf16" else "f32", precision)]
 
 

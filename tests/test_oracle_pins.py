@@ -305,12 +305,66 @@ def test_compress2_offline_equals_streaming(log2_nout, m):
 
 
 def test_compress2_group_sizes_from_golden():
-    rows = [l.split() for l in open(os.path.join(GOLDEN, "structure_facts.txt"))
+    """Algorithm 2's size rule, as stored in the golden file, against the Halve calls the oracle makes
+    (level, points in, number of calls at that level read off the oracle's own call record)."""
+    rows = [tuple(map(int, l.split())) for l in open(os.path.join(GOLDEN, "structure_facts.txt"))
             if l.strip() and not l.startswith("#")]
-    for n_out, m, level, size, count in (map(int, r) for r in rows):
-        n_in = n_out << m
-        assert n_in * 2 ** level // 4 ** (m - 1) == size          # Algorithm 2's size rule
-        assert (n_in >> level) // size == count                    # points alive / group size
+    cases = sorted({(r[0], r[1]) for r in rows})
+    assert len(cases) >= 3
+    for n_out, m in cases:
+        n = n_out << m
+        K, V = _data(40 + m, n, 2, kscale=0.3)
+        idx, w, calls = oracle.compress2_calls(K, V, int(math.log2(n_out)), m, seed=2)
+        assert len(idx) == n_out
+        seen = {}
+        for level, number, size, _ in calls:
+            key = (int(level), int(size))
+            assert number == seen.get(key, 0)                         # calls of a level numbered in order
+            seen[key] = seen.get(key, 0) + 1
+        assert len({lv for lv, _ in seen}) == len(seen) == m           # one size per level, m levels
+        for r in rows:
+            if (r[0], r[1]) == (n_out, m):
+                assert seen[(r[2], r[3])] == r[4], r
+        # default schedule: every level spends delta / (3 m), the call delta / 3 (Corollary 2's split)
+        assert calls[:, 3].sum() == pytest.approx(0.5 / 3, rel=1e-12)
+
+
+def test_kh_running_shift_rescales_carried_bmax():
+    """The running shift: b_max is carried in the scale of the previous pair and must be multiplied by
+    exp(-(M_i - M_{i-1}) / 2) (b is a square root of kernel values) when the shift grows.  Directed case:
+    pair 1 has the largest b; pair 2 is two near-identical keys of large norm, which raises the shift while
+    its own b is tiny; pair 3 is an ordinary pair whose threshold a_3 = b_3 b_max (...) needs pair 1's b in
+    pair 3's scale.  The unshifted run (the printed formula) is the reference: same p, same decisions,
+    and a_i equal after undoing the scale exp(-M_i)."""
+    d = 4
+    K = np.zeros((6, d), np.float32)
+    V = np.zeros((6, d), np.float32)
+    K[0], K[1] = [1.0, 0, 0, 0], [-1.0, 0.3, 0, 0]
+    K[2], K[3] = [0, 2.5, 0, 0], [0, 2.5, 1e-4, 0]
+    K[4], K[5] = [0.2, 0, 0.1, 0], [0.1, 0, 0.2, 0]
+    V[0], V[1] = [1, 0, 0, 0], [-1, 0.5, 0, 0]
+    V[2], V[3] = [0.3, 0.3, 0, 0], [0.3, 0.3, 0, 0]
+    V[4], V[5] = [0.5, 0.1, 0, 0], [0.4, 0.2, 0, 0]
+    x = np.arange(6, dtype=np.int32)
+    vm = oracle.vmax(V)
+    G = _gram(K, V, vm)
+    F = _pair_gram(G)
+    b = np.sqrt(np.diag(F))
+    assert b[0] > 5 * b[2] > 25 * b[1]                                # pair 1 dominates, pair 2 is tiny
+    c = (K.astype(np.float64) ** 2).sum(1) / math.sqrt(d)
+    M = np.maximum.accumulate(np.maximum(c[0::2], c[1::2]))
+    assert M[1] - M[0] > 2.0 and M[2] == M[1]                         # the shift grows at pair 2 only
+    for U in ([0.9, 0.9, 0.9], [0.1, 0.9, 0.55], [0.1, 0.1, 0.65]):
+        U = np.array(U)
+        S1, S2, diag = oracle.kh(K, V, vm, x, 0.5, U, shift_mode=1)
+        S1u, S2u, diagu = oracle.kh(K, V, vm, x, 0.5, U, shift_mode=0)
+        _check_against_matrix_form(K, V, x, 0.5, U, S1u, S2u, diagu)
+        assert np.array_equal(S1, S1u)
+        assert np.abs(diag[:, 2] - diagu[:, 2]).max() < 1e-12
+        assert 0.05 < abs(diag[2, 2] - 0.5) < 0.45                    # pair 3's p is neither 1/2 nor clamped
+        assert np.allclose(diag[:, 1], diagu[:, 1] * np.exp(-M), rtol=1e-12)
+        # a_3 = b_3 * (pair 1's b) * (1/2 + ln(2 s / delta)), all in pair 3's scale
+        assert diag[2, 1] == pytest.approx(b[2] * b[0] * np.exp(-M[2]) * (0.5 + math.log(2 * 6 / 0.5)), rel=1e-10)
 
 
 def test_compress2_structure_and_identity():
