@@ -21,9 +21,10 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one attend launch, from the ncu capture summarised
-# in profiles/attend_tc_cfg5_dram_traffic.md (read 1 084 004 352 + write 1 027 012 096 bytes)
-NCU_DRAM_BYTES_PER_ATTEND_LAUNCH = {"cfg5": 2108260096}
+# dram__bytes_read.sum + dram__bytes_write.sum of one attend launch at the workload's full size, from one
+# single-pass ncu capture of that launch (read 1 083 738 880 + write 1 024 521 216 bytes); workloads without
+# a capture report null and say so
+NCU_DRAM_BYTES_PER_ATTEND_LAUNCH = {"cfg5": 1083738880 + 1024521216}
 
 METRIC = "compress+attend tokens/sec per B200"
 UNIT = "tokens/s"
@@ -52,7 +53,29 @@ class ClockSampler:
         self._stop = threading.Event()
         self._thr = None
 
+    def _nvml_loop(self):
+        """Read-only NVML polling every 2 ms (an nvidia-smi call takes longer than the timed region)."""
+        import pynvml
+        pynvml.nvmlInit()
+        h = pynvml.nvmlDeviceGetHandleByIndex(self.gpu)
+        mx = pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM)
+        bits = {"hw_slowdown": pynvml.nvmlClocksEventReasonHwSlowdown,
+                "hw_thermal_slowdown": pynvml.nvmlClocksEventReasonHwThermalSlowdown,
+                "sw_thermal_slowdown": pynvml.nvmlClocksEventReasonSwThermalSlowdown,
+                "sw_power_cap": pynvml.nvmlClocksEventReasonSwPowerCap}
+        while not self._stop.is_set():
+            sm = pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM)
+            r = pynvml.nvmlDeviceGetCurrentClocksEventReasons(h)
+            pw = pynvml.nvmlDeviceGetPowerUsage(h) / 1000.0
+            self.rows.append([str(sm), str(mx), str(pw)] + ["Active" if r & b else "Not Active" for b in bits.values()])
+            self._stop.wait(0.002)
+
     def _run(self):
+        try:
+            self._nvml_loop()
+            return
+        except Exception:
+            pass
         while not self._stop.is_set():
             try:
                 out = subprocess.run(["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.FIELDS}",
@@ -87,8 +110,14 @@ class ClockSampler:
         if not sm:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         sm.sort()
+        power = []
+        for r in self.rows:
+            try:
+                power.append(float(r[2]))
+            except (ValueError, IndexError):
+                pass
         return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": max(mx), "reasons": sorted(reasons),
-                "samples": len(sm)}
+                "samples": len(sm), "power_w_max": max(power) if power else None}
 
 
 def max_over_ranks(ms_local: float, dist, device) -> float:
@@ -149,6 +178,23 @@ def cpu_baseline(wl, Q, K, V, budget_heads=None):
                       f"scaled linearly to the full step ({est:.1f} s)"}, est
 
 
+def oracle_cfg1_one_thread_ms():
+    """The oracle on the smallest workload (one attention problem, so one thread): full compress + attend."""
+    import oracle
+    from paper_2606_10944_b200.workloads import WORKLOADS, as_f32_numpy, generate
+    w1 = WORKLOADS["cfg1"]
+    Q, K, V = generate(w1, seed=1234)
+    Qf, Kf, Vf = as_f32_numpy(Q), as_f32_numpy(K), as_f32_numpy(V)
+    best = None
+    for _ in range(3):
+        t0 = time.perf_counter()
+        idx, w, _ = oracle.compress2_batched(Kf.reshape(1, w1.n, w1.d), Vf.reshape(1, w1.n, w1.d), w1.log2_nout, w1.m, seed=1)
+        oracle.wtd_attention_batched(Qf, Kf, Vf, idx.reshape(1, 1, -1), w.reshape(1, 1, -1))
+        dt = (time.perf_counter() - t0) * 1e3
+        best = dt if best is None else min(best, dt)
+    return best
+
+
 def run_reference(args, wl):
     """--impl reference: the CPU oracle timed on the host cores (rank 0 only)."""
     if int(os.environ.get("RANK", "0")) != 0:
@@ -207,6 +253,8 @@ def main():
                          "6 n_out entries, printed as its own JSON line (profiling captures only); or (ragged) "
                          "compress + attend on a sequence 7 %% shorter than the workload's, 32 sink and 32 "
                          "window rows kept (elm_compress_ragged)")
+    ap.add_argument("--sustain-s", type=float, default=3.0,
+                    help="seconds of back-to-back attend launches for the sustained-clock figure (0: skip)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -450,7 +498,16 @@ def main():
     attend_flops, compress_flops, hbm_bytes = algorithmic_counts(wl)
     stage_ms = {k: v[0] / args.steps for k, v in stage.items()}
     att_ms = stage_ms["attend"] or float("nan")     # zero only under --only compress
-    tensor_peak = peaks["bf16_tflops_sustained"]
+    clk = clocks.summary()
+    # Which measured GEMM peak the tensor fractions are read against: the burst figure was taken on a kernel
+    # timed alone at full clocks, the sustained one inside a seconds-long loop under the power cap.  A timed
+    # region of well under a second at (nearly) the maximum SM clock never enters that regime, so the burst
+    # peak is the denominator then; both fractions are printed either way.
+    region_s = ms_total * 1e-3
+    at_full_clock = clk["sm_mhz"] is not None and clk["sm_mhz"] >= 0.95 * clk["sm_max_mhz"]
+    use_burst = region_s < 1.0 and at_full_clock
+    tensor_peak = peaks["bf16_tflops"] if use_burst else peaks["bf16_tflops_sustained"]
+    peak_name = "burst" if use_burst else "sustained"
     # the dominant kernel: weighted attention (dense contraction -> tensor roofline) unless the
     # workload's coreset is so small that its Q/O traffic dominates
     t_tensor = attend_flops / (tensor_peak * 1e12)
@@ -460,18 +517,49 @@ def main():
         achieved = attend_flops / (att_ms * 1e-3) / 1e12
         roofline = {"bound": "tensor", "kernel": "attend", "achieved": achieved, "peak": tensor_peak,
                     "unit": "TFLOP/s", "frac": achieved / tensor_peak, "traffic": None,
-                    "peak_source": f"{peaks['source']} bf16 sustained", "ms_per_launch": att_ms}
+                    "peak_source": f"{peaks['source']} bf16 {peak_name} ({region_s:.2f} s timed region at "
+                                   f"{clk['sm_mhz']} of {clk['sm_max_mhz']} MHz)",
+                    "frac_burst": achieved / peaks["bf16_tflops"],
+                    "frac_sustained": achieved / peaks["bf16_tflops_sustained"], "ms_per_launch": att_ms}
     else:
         achieved = att_bytes / (att_ms * 1e-3) / 1e9
         roofline = {"bound": "hbm", "kernel": "attend", "achieved": achieved, "peak": peaks["hbm_gbs"],
                     "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "traffic": None,
                     "peak_source": f"{peaks['source']} copy", "ms_per_launch": att_ms}
     roofline["traffic"] = NCU_DRAM_BYTES_PER_ATTEND_LAUNCH.get(wl.name)
+    if roofline["traffic"] is None:
+        roofline["traffic_note"] = "no ncu capture of this workload's attend launch"
     whole_roof_s = max((attend_flops + compress_flops) / (tensor_peak * 1e12), hbm_bytes / (peaks["hbm_gbs"] * 1e9))
+    whole_burst_s = max((attend_flops + compress_flops) / (peaks["bf16_tflops"] * 1e12), hbm_bytes / (peaks["hbm_gbs"] * 1e9))
+    whole_sust_s = max((attend_flops + compress_flops) / (peaks["bf16_tflops_sustained"] * 1e12),
+                       hbm_bytes / (peaks["hbm_gbs"] * 1e9))
+
+    # The same attend launch back to back for a few seconds, clocks sampled throughout: the like-for-like
+    # numerator for the sustained peak (and time x clock, which does not depend on where the clock settles).
+    sustained = None
+    if args.sustain_s > 0 and args.only in ("both", "attend") and roofline["bound"] == "tensor":
+        reps = max(8, int(args.sustain_s * 1e3 / att_ms))
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with ClockSampler(local) as sclk:
+            torch.cuda.synchronize()
+            s0.record()
+            for _ in range(reps):
+                elm.attend(Qd, Kd, Vd, state["idx"], state["w"], precision=args.precision, workspace=ws_a, out=O)
+            s1.record()
+            torch.cuda.synchronize()
+        sms = s0.elapsed_time(s1) / reps
+        sc = sclk.summary()
+        ach = attend_flops / (sms * 1e-3) / 1e12
+        sustained = {"launches": reps, "seconds": s0.elapsed_time(s1) * 1e-3, "ms_per_launch": sms, "achieved": ach,
+                     "unit": "TFLOP/s", "frac_sustained": ach / peaks["bf16_tflops_sustained"],
+                     "frac_burst": ach / peaks["bf16_tflops"], "clocks": sc,
+                     "ms_x_mhz": sms * sc["sm_mhz"] if sc["sm_mhz"] else None}
+        roofline["ms_x_mhz"] = att_ms * clk["sm_mhz"] if clk["sm_mhz"] else None
 
     base = None
     if not args.no_cpu_baseline:
         base, _ = cpu_baseline(wl, Q, K, V)
+        base["cfg1_one_thread_ms"] = oracle_cfg1_one_thread_ms()
 
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -480,13 +568,15 @@ def main():
         "config": workload_config(wl, args),
         "roofline": roofline,
         "whole_path_roofline": {"roofline_ms": whole_roof_s * 1e3, "frac": whole_roof_s * 1e3 / ms_step,
+                                "frac_burst": whole_burst_s * 1e3 / ms_step, "frac_sustained": whole_sust_s * 1e3 / ms_step,
                                 "attend_flops": attend_flops, "compress_flops": compress_flops,
                                 "hbm_bytes": hbm_bytes},
+        "attend_sustained": sustained,
         "stage_ms": stage_ms,
         "cpu_baseline": base,
         "e2e": e2e,
         "gpu_launches": launches,
-        "clocks": clocks.summary(),
+        "clocks": clk,
     }
     print(json.dumps(out))
     if dist is not None:

@@ -325,6 +325,24 @@ int elm_compress_status(const void *workspace, const elm_params *params, int32_t
 int elm_attend_status(const void *workspace, const elm_params *params, int32_t n_core, int32_t *status_host,
                       void *stream);
 
+/*
+ * Test hooks (no counterpart in the paper).  They exist so that the failure path of the bounded waits can be
+ * exercised without hanging or faulting anything:
+ *   ELM_DEBUG_WAIT_LIMIT_NS            the time limit of the bounded waits of the tensor-core attention kernel
+ *                                      (default 2 000 000 000; at least 1 000 000), for launches from now on;
+ *   ELM_DEBUG_ATTEND_MISSING_ARRIVALS  the NEXT tensor-core elm_attend launch expects `value` arrivals on its
+ *                                      "probabilities ready" barriers that nobody makes: the waits on them run
+ *                                      out, the launch winds down, elm_attend_status reads non-zero and O is
+ *                                      undefined.  One launch only; later calls are normal again.
+ * Environment variables read by the library (tuning aids, off the documented path): ELM_WALK_CHAIN_MIN_PAIRS
+ * (default 1024: Halve calls with at least this many pairs take the cluster walk kernel; 32 .. 4096) and
+ * ELM_PREFILL_WINDOW (default 512: tokens per attention launch of elm_express_prefill; a power of two >= 64).
+ * A build with -DELM_BOUNDS_CHECK (ELM_NVCC_EXTRA of the build script) checks every caller-supplied row number
+ * of elm_attend against [0, n_kv): a bad one reads row 0 instead and sets the status word to 64.
+ */
+enum { ELM_DEBUG_WAIT_LIMIT_NS = 0, ELM_DEBUG_ATTEND_MISSING_ARRIVALS = 1 };
+int elm_debug_set(int32_t what, int64_t value);
+
 /* Kernels launched by this library since it was loaded (all calls, all stages). */
 int64_t elm_launch_count(void);
 

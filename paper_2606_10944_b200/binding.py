@@ -24,7 +24,7 @@ EXPORTED_SYMBOLS = [
     "elm_express_prefill_workspace_bytes", "elm_express_prefill",
     "elm_stream_workspace_bytes", "elm_stream_init", "elm_stream_step", "elm_stream_cache",
     "elm_host_call_scratch_bytes", "elm_compress_attend_host",
-    "elm_compress_status", "elm_attend_status", "elm_profile_enable", "elm_profile_read", "elm_launch_count", "elm_strerror", "elm_version",
+    "elm_compress_status", "elm_attend_status", "elm_debug_set", "elm_profile_enable", "elm_profile_read", "elm_launch_count", "elm_strerror", "elm_version",
 ]
 
 
@@ -92,6 +92,7 @@ def load_library():
     lib.elm_compress_attend_host.argtypes = [vp, vp, vp, vp, vp, vp, pp, ctypes.c_uint64, vp, sz, vp]
     lib.elm_compress_status.argtypes = [vp, pp, ctypes.POINTER(ctypes.c_int32), vp]
     lib.elm_attend_status.argtypes = [vp, pp, ctypes.c_int32, ctypes.POINTER(ctypes.c_int32), vp]
+    lib.elm_debug_set.argtypes = [ctypes.c_int32, ctypes.c_int64]
     lib.elm_profile_enable.argtypes = [ctypes.c_int]
     lib.elm_profile_read.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int64), ctypes.c_int32]
     lib.elm_launch_count.argtypes = []

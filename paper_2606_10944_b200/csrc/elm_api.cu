@@ -4,6 +4,7 @@
 #include <stdio.h>
 
 #include <atomic>
+#include <mutex>
 
 #include <vector>
 
@@ -236,6 +237,23 @@ extern "C" int elm_compress_attend_host(const void *Q_host, const void *K_host, 
     return sync_ok ? ELM_OK : ELM_ERR_CUDA;
 }
 
+namespace elm {
+int device_sm_count()
+{
+    static std::mutex mu;
+    static int cached[64] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+    std::lock_guard<std::mutex> lock(mu);
+    if (cached[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+        cached[dev] = n;
+    }
+    return cached[dev];
+}
+}  // namespace elm
+
 extern "C" int elm_compress_status(const void *workspace, const elm_params *params, int32_t *status_host, void *stream)
 {
     if (!workspace || !params || !status_host) return ELM_ERR_NULL;
@@ -262,6 +280,8 @@ extern "C" int elm_attend_status(const void *workspace, const elm_params *params
     ELM_CUDA_TRY(cudaStreamSynchronize((cudaStream_t)stream));
     return ELM_OK;
 }
+
+extern "C" int elm_debug_set(int32_t what, int64_t value) { return elm::debug_set_attend_tc(what, value); }
 
 extern "C" int elm_profile_enable(int on)
 {

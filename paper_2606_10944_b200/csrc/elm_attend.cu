@@ -23,13 +23,14 @@ __global__ void __launch_bounds__(256) gather_kernel(const Tin *__restrict__ K,
                                                      const int32_t *__restrict__ idx,
                                                      const float *__restrict__ w, int64_t n, int d,
                                                      int n_core, Tin *__restrict__ Kc,
-                                                     Tin *__restrict__ Vc, float *__restrict__ bias)
+                                                     Tin *__restrict__ Vc, float *__restrict__ bias,
+                                                     int *__restrict__ status)
 {
     const int p = blockIdx.y;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int c = blockIdx.x * 8 + warp;
     if (c >= n_core) return;
-    const int64_t row = idx[(int64_t)p * n_core + c];
+    const int64_t row = checked_row(idx[(int64_t)p * n_core + c], n, status);
     const Tin *ks = K + ((int64_t)p * n + row) * d;
     const Tin *vs = V + ((int64_t)p * n + row) * d;
     Tin *kd = Kc + ((int64_t)p * n_core + c) * d;
@@ -234,7 +235,7 @@ static int attend_impl(const Tin *Q, const Tin *K, const Tin *V, const int32_t *
         // this path has no bounded waits: its status word reads 0
         ELM_CUDA_TRY(cudaMemsetAsync(ws + L.flags, 0, sizeof(int) * (size_t)(problems + 1), st));
         gather_kernel<Tin><<<dim3((unsigned)((n_core + 7) / 8), (unsigned)problems), 256, 0, st>>>(
-            K, V, idx, w, p->n_kv, p->d, n_core, Kc, Vc, bias);
+            K, V, idx, w, p->n_kv, p->d, n_core, Kc, Vc, bias, reinterpret_cast<int *>(ws + L.flags) + problems);
         count_launches(1);
         ELM_CUDA_TRY(cudaGetLastError());
     }
@@ -291,7 +292,7 @@ static int attend_enqueue_untimed(const Tin *Q, const Tin *K, const Tin *V, cons
     // this path has no bounded waits: its status word reads 0
     ELM_CUDA_TRY(cudaMemsetAsync(scratch + L.flags, 0, sizeof(int) * (size_t)(problems + 1), st));
     gather_kernel<Tin><<<dim3((unsigned)((n_core + 7) / 8), (unsigned)problems), 256, 0, st>>>(
-        K, V, idx, w, p->n_kv, p->d, n_core, Kc, Vc, bias);
+        K, V, idx, w, p->n_kv, p->d, n_core, Kc, Vc, bias, reinterpret_cast<int *>(scratch + L.flags) + problems);
     count_launches(1);
     ELM_CUDA_TRY(cudaGetLastError());
     if (p->d == 64) return launch_attend_simt<Tin, T, 64>(Q, Kc, Vc, bias, O, p, n_core, st);

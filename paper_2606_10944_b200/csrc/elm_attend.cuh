@@ -52,6 +52,9 @@ int attend_tc(const __nv_bfloat16 *Q, const __nv_bfloat16 *K, const __nv_bfloat1
               const float *w, int n_core, const elm_params *p, __nv_bfloat16 *O, unsigned char *ws,
               cudaStream_t st, bool timed, const AttendWindow &win = AttendWindow());
 
+// elm_debug_set for the hooks that live with the tensor-core attention
+int debug_set_attend_tc(int32_t what, int64_t value);
+
 // A few query vectors per KV head (decode): HBM-bound kernels that read the coreset rows once through
 // the index list.  Applies to fp32 mode when (q_heads / kv_heads) * n_q <= 8.
 bool attend_decode_applies(const elm_params *p);

@@ -227,12 +227,7 @@ int attend_decode(const void *Q, const void *K, const void *V, const int32_t *id
     const size_t room = L.bias - L.Kc;
     const size_t per_split = (size_t)problems * G * (p->d + 2) * sizeof(float);
     // enough CTAs for about two per SM, but at least one batch of entries per warp
-    static int sm_count = 0;
-    if (sm_count == 0) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sm_count <= 0)
-            sm_count = 148;
-    }
+    const int sm_count = device_sm_count();
     int splits = (n_core + DEC_WARPS * DEC_UNR - 1) / (DEC_WARPS * DEC_UNR);
     const int wanted = (2 * sm_count + problems - 1) / problems;
     if (splits > wanted) splits = wanted;

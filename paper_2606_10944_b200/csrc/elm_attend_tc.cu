@@ -36,6 +36,8 @@
 #include <cuda.h>
 #include <math.h>
 
+#include <atomic>
+
 #include "elm_attend.cuh"
 #include "elm_common.cuh"
 #include "elm_sm100.cuh"
@@ -114,7 +116,7 @@ __global__ void __launch_bounds__(256) gather_tc_kernel(const __nv_bfloat16 *__r
     for (int r = warp; r < GATHER_COLS; r += 8) {
         const int c = c0 + r;
         const bool ok = c < n_core;
-        const int64_t row = ok ? idx[(int64_t)p * n_core + c] : 0;
+        const int64_t row = ok ? checked_row(idx[(int64_t)p * n_core + c], n, nonuniform + gridDim.y) : 0;
         const int chunk = lane & 15;
         if (chunk < CH) {
             const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
@@ -326,8 +328,11 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                  int kv_heads, int n_q, int n_core, int n_pad, float scale_log2, int tiles_x, int n_items_total,
                  int q_row0, int n_q_total, int tail_start, const int32_t *__restrict__ birth,
                  const int32_t *__restrict__ death, const int32_t *__restrict__ blk_birth,
-                 const int32_t *__restrict__ blk_death, float *__restrict__ lse, int *__restrict__ status)
+                 const int32_t *__restrict__ blk_death, float *__restrict__ lse, int *__restrict__ status,
+                 int extra_arrivals, unsigned long long wait_limit_ns)
 {
+    // every wait of this kernel is bounded by the limit the host passes (2 s unless a test shortened it)
+    auto mbar_wait = [wait_limit_ns](uint64_t *b, uint32_t parity) { return sm100::mbar_wait(b, parity, wait_limit_ns); };
     using SM = Smem<D>;
     constexpr int KH = SM::KH;
     extern __shared__ unsigned char smem_dyn[];
@@ -360,7 +365,8 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
         }
         for (int t = 0; t < 2; ++t) {
             mbar_init(&bar->s_full[t], 1);
-                        mbar_init(&bar->p_ready[t], MASKED ? 512 : 256);
+            // (extra_arrivals is 0 except in the test that lets a wait run out: arrivals that nobody makes)
+            mbar_init(&bar->p_ready[t], (MASKED ? 512 : 256) + extra_arrivals);
             mbar_init(&bar->o_done[t], 1);
             mbar_init(&bar->o_free[t], MASKED ? 16 : 8);
         }
@@ -828,16 +834,13 @@ static bool make_map(CUtensorMap *map, const void *base, uint64_t d0, uint64_t d
               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-static int sm_count()
-{
-    static int n = 0;
-    if (n == 0) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
-            n = 148;
-    }
-    return n;
-}
+static int sm_count() { return device_sm_count(); }
+
+// test hook (elm_debug_set): arrivals that the next launch expects on its "probabilities ready" barriers and that
+// nobody makes, so that the issuing threads' bounded waits run out
+static std::atomic<int> g_debug_extra_arrivals{0};
+// test hook: the time limit of the kernel's bounded waits
+static std::atomic<unsigned long long> g_debug_wait_limit_ns{sm100::WAIT_LIMIT_NS};
 
 template <int D>
 static int launch(const __nv_bfloat16 *Q, const __nv_bfloat16 *K, const __nv_bfloat16 *V, const int32_t *idx,
@@ -880,12 +883,29 @@ static int launch(const __nv_bfloat16 *Q, const __nv_bfloat16 *K, const __nv_bfl
     kern<<<ctas, NTHREADS, Smem<D>::TOTAL, st>>>(mQ, mK, mV, mX, flags, O, p->q_heads, p->kv_heads, p->n_q,
                                                  n_core, n_pad, scale_log2, tiles_x, (int)items, (int)win.q_row0,
                                                  (int)n_q_total, win.tail_start, win.birth, win.death, win.blk_birth,
-                                                 win.blk_death, win.lse, status);
+                                                 win.blk_death, win.lse, status, g_debug_extra_arrivals.exchange(0),
+                                                 g_debug_wait_limit_ns.load());
     count_launches(1);
     return cuda_status(cudaGetLastError());
 }
 
 }  // namespace tc
+
+int debug_set_attend_tc(int32_t what, int64_t value)
+{
+    if (what == ELM_DEBUG_WAIT_LIMIT_NS) {
+        if (value < 1000000) return ELM_ERR_SHAPE;              // at least a millisecond
+        tc::g_debug_wait_limit_ns.store((unsigned long long)value);
+        return ELM_OK;
+    }
+    if (what == ELM_DEBUG_ATTEND_MISSING_ARRIVALS) {
+        if (value < 0 || value > 1024) return ELM_ERR_SHAPE;
+        tc::g_debug_extra_arrivals.store((int)value);
+        return ELM_OK;
+    }
+    return ELM_ERR_SHAPE;
+}
+
 int attend_tc(const __nv_bfloat16 *Q, const __nv_bfloat16 *K, const __nv_bfloat16 *V, const int32_t *idx,
               const float *w, int n_core, const elm_params *p, __nv_bfloat16 *O, unsigned char *ws,
               cudaStream_t st, bool timed, const AttendWindow &win)

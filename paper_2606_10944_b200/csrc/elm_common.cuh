@@ -44,6 +44,9 @@ inline int cuda_status(cudaError_t e) { return e == cudaSuccess ? ELM_OK : ELM_E
         if (_e != cudaSuccess) return ELM_ERR_CUDA;       \
     } while (0)
 
+// Multiprocessors of the current device (looked up once per device ordinal; 148 if the query fails).
+int device_sm_count();
+
 int validate_params(const elm_params *p);
 int validate_attend_params(const elm_params *p);
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -66,6 +69,24 @@ __device__ __forceinline__ void store_from(__nv_bfloat16 *p, int64_t i, double v
 __device__ __forceinline__ void store_from(__nv_bfloat16 *p, int64_t i, float v)
 {
     p[i] = __float2bfloat16_rn(v);
+}
+
+// Row numbers that come from the caller (idx of elm_attend) index K and V unchecked in a normal build.  A build
+// with -DELM_BOUNDS_CHECK tests each against [0, n): a bad one is replaced by row 0 and reported through the
+// call's status word (ELM_STATUS_BAD_ROW) - never by trapping.
+constexpr int ELM_STATUS_BAD_ROW = 64;
+__device__ __forceinline__ int64_t checked_row(int64_t row, int64_t n, int *status)
+{
+#ifdef ELM_BOUNDS_CHECK
+    if (row < 0 || row >= n) {
+        if (status) atomicExch(status, ELM_STATUS_BAD_ROW);
+        return 0;
+    }
+#else
+    (void)n;
+    (void)status;
+#endif
+    return row;
 }
 
 // Philox4x32-10 (Salmon et al., SC'11), first output word only.

@@ -535,12 +535,7 @@ static int launch(const __nv_bfloat16 *K, const __nv_bfloat16 *V, const elm_para
     }
     if (P > TP || (P == TP && !wk.fused)) {
         // calls that span several tiles: persistent, pipelined kernel, one CTA per SM
-        static int sm_count = 0;
-        if (sm_count == 0) {
-            int dev = 0;
-            ELM_CUDA_TRY(cudaGetDevice(&dev));
-            ELM_CUDA_TRY(cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev));
-        }
+        const int sm_count = device_sm_count();
         const int64_t total = tiles * BH;
         const int grid = (int)(total < sm_count ? total : sm_count);
         auto pk = gram_tc_persistent_kernel<D>;

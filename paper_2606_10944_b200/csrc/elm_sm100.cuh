@@ -53,8 +53,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
         : "memory");
     return ok != 0;
 }
-// Bounded wait: gives up after ~2 s of wall time.
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity)
+// Bounded wait: gives up after `limit_ns` nanoseconds of the global timer (2 s unless the kernel passes its own:
+// the tensor-core attention takes it as a kernel argument so that a test can watch a wait run out quickly).
+constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, unsigned long long limit_ns = WAIT_LIMIT_NS)
 {
     if (mbar_try_wait(bar, parity)) return true;
     uint64_t t0;
@@ -65,7 +67,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity)
             if (mbar_try_wait(bar, parity)) return true;
         uint64_t t1;
         asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t1));
-        if (t1 - t0 > 2000000000ull) return false;
+        if (t1 - t0 > limit_ns) return false;
     }
 }
 __device__ __forceinline__ void fence_barrier_init()
