@@ -136,10 +136,11 @@ def whole_job_tokens_per_s(tokens_per_rank_step: int, world: int, ms_per_step: f
 
 def algorithmic_counts(wl):
     """Flops and bytes the method itself needs per step (not what exact attention would need)."""
-    es = 2 if wl.dtype == "bf16" else 4
+    es = {"bf16": 2, "e4m3": 1}.get(wl.dtype, 4)
+    eo = 2 if wl.dtype == "e4m3" else es                      # O is bf16 for 8-bit inputs
     attend_flops = wl.batch * wl.q_heads * wl.n_q * wl.n_out * 4 * wl.d
     compress_flops = wl.batch * wl.kv_heads * wl.m * 8 * wl.d * wl.n_out ** 2
-    hbm_bytes = 2 * wl.batch * wl.q_heads * wl.n_q * wl.d * es + 2 * wl.batch * wl.kv_heads * wl.n * wl.d * es
+    hbm_bytes = wl.batch * wl.q_heads * wl.n_q * wl.d * (es + eo) + 2 * wl.batch * wl.kv_heads * wl.n * wl.d * es
     return attend_flops, compress_flops, hbm_bytes
 
 
@@ -240,6 +241,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg5")
     ap.add_argument("--precision", default="fp32", choices=["fp32", "fp64"])
+    ap.add_argument("--storage", default=None, choices=["f32", "bf16", "e4m3"],
+                    help="storage type of Q, K, V instead of the workload's own (e4m3: 8-bit inputs, d = 128, O in bf16; "
+                         "S = Q K^T then runs on 8-bit tensor-core operands)")
     ap.add_argument("--data-seed", type=int, default=1234)
     ap.add_argument("--seed", type=int, default=1)
     ap.add_argument("--e2e-steps", type=int, default=3)
@@ -264,6 +268,8 @@ def main():
     if args.override:
         kv = dict(item.split("=") for item in args.override.split(","))
         wl = wl.scaled(name=f"{wl.name}[{args.override}]", **{k: int(v) for k, v in kv.items()})
+    if args.storage and args.storage != wl.dtype:
+        wl = wl.scaled(name=f"{wl.name}[storage={args.storage}]", dtype=args.storage)
     if args.impl == "reference":
         run_reference(args, wl)
         return
@@ -287,12 +293,14 @@ def main():
     Q, K, V = generate(wl, seed=args.data_seed + rank)      # each replica has its own batch
     Qd, Kd, Vd = Q.cuda(), K.cuda(), V.cuda()
     dev = Qd.device
-    p, _ = elm.make_params(wl.batch, wl.q_heads, wl.kv_heads, wl.n, wl.n_q, wl.d, wl.log2_nout, wl.m,
-                           1 if wl.dtype == "bf16" else 0, args.precision)
+    dcode = {"f32": 0, "bf16": 1, "e4m3": 2}[wl.dtype]
+    p, _ = elm.make_params(wl.batch, wl.q_heads, wl.kv_heads, wl.n, wl.n_q, wl.d, wl.log2_nout, wl.m, dcode, args.precision)
     cb, ab = elm.workspace_bytes(p)
     ws_c = torch.empty(cb, dtype=torch.uint8, device=dev)
     ws_a = torch.empty(ab, dtype=torch.uint8, device=dev)
-    O = torch.empty_like(Qd)
+    O = torch.empty(Qd.shape, dtype=torch.bfloat16 if wl.dtype == "e4m3" else Qd.dtype, device=dev)
+    if wl.dtype == "e4m3":
+        args.no_e2e = True          # the host-buffer entry point takes f32 and bf16 only
     small_inputs = not wl.name.startswith(("cfg4", "cfg5"))
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev) if small_inputs else None
 
@@ -508,19 +516,26 @@ def main():
     use_burst = region_s < 1.0 and at_full_clock
     tensor_peak = peaks["bf16_tflops"] if use_burst else peaks["bf16_tflops_sustained"]
     peak_name = "burst" if use_burst else "sustained"
+    # 8-bit inputs: half of attend's flops (S = Q K^T) run at the 8-bit rate, nominally twice the bf16 rate, the
+    # other half (P V) at the bf16 rate: the blended peak for the whole contraction is 4/3 of the bf16 figure
+    fp8 = wl.dtype == "e4m3"
+    blend = 4.0 / 3.0 if fp8 else 1.0
+    tensor_peak *= blend
     # the dominant kernel: weighted attention (dense contraction -> tensor roofline) unless the
     # workload's coreset is so small that its Q/O traffic dominates
     t_tensor = attend_flops / (tensor_peak * 1e12)
-    att_bytes = 2 * wl.batch * wl.q_heads * wl.n_q * wl.d * (2 if wl.dtype == "bf16" else 4)
+    att_bytes = wl.batch * wl.q_heads * wl.n_q * wl.d * ({"bf16": 4, "e4m3": 3}.get(wl.dtype, 8))
     t_hbm = att_bytes / (peaks["hbm_gbs"] * 1e9)
-    if wl.dtype == "bf16" and t_tensor >= t_hbm:
+    if wl.dtype in ("bf16", "e4m3") and t_tensor >= t_hbm:
         achieved = attend_flops / (att_ms * 1e-3) / 1e12
         roofline = {"bound": "tensor", "kernel": "attend", "achieved": achieved, "peak": tensor_peak,
                     "unit": "TFLOP/s", "frac": achieved / tensor_peak, "traffic": None,
                     "peak_source": f"{peaks['source']} bf16 {peak_name} ({region_s:.2f} s timed region at "
                                    f"{clk['sm_mhz']} of {clk['sm_max_mhz']} MHz)",
-                    "frac_burst": achieved / peaks["bf16_tflops"],
-                    "frac_sustained": achieved / peaks["bf16_tflops_sustained"], "ms_per_launch": att_ms}
+                    "frac_burst": achieved / (peaks["bf16_tflops"] * blend),
+                    "frac_sustained": achieved / (peaks["bf16_tflops_sustained"] * blend), "ms_per_launch": att_ms}
+        if fp8:
+            roofline["peak_source"] += "; x 4/3: S = Q K^T at the nominal 2x rate of 8-bit operands, P V at the bf16 rate"
     else:
         achieved = att_bytes / (att_ms * 1e-3) / 1e9
         roofline = {"bound": "hbm", "kernel": "attend", "achieved": achieved, "peak": peaks["hbm_gbs"],
@@ -529,10 +544,10 @@ def main():
     roofline["traffic"] = NCU_DRAM_BYTES_PER_ATTEND_LAUNCH.get(wl.name)
     if roofline["traffic"] is None:
         roofline["traffic_note"] = "no ncu capture of this workload's attend launch"
-    whole_roof_s = max((attend_flops + compress_flops) / (tensor_peak * 1e12), hbm_bytes / (peaks["hbm_gbs"] * 1e9))
-    whole_burst_s = max((attend_flops + compress_flops) / (peaks["bf16_tflops"] * 1e12), hbm_bytes / (peaks["hbm_gbs"] * 1e9))
-    whole_sust_s = max((attend_flops + compress_flops) / (peaks["bf16_tflops_sustained"] * 1e12),
+    whole_burst_s = max((attend_flops / blend + compress_flops) / (peaks["bf16_tflops"] * 1e12), hbm_bytes / (peaks["hbm_gbs"] * 1e9))
+    whole_sust_s = max((attend_flops / blend + compress_flops) / (peaks["bf16_tflops_sustained"] * 1e12),
                        hbm_bytes / (peaks["hbm_gbs"] * 1e9))
+    whole_roof_s = whole_burst_s if use_burst else whole_sust_s
 
     # The same attend launch back to back for a few seconds, clocks sampled throughout: the like-for-like
     # numerator for the sustained peak (and time x clock, which does not depend on where the clock settles).
@@ -551,8 +566,8 @@ def main():
         sc = sclk.summary()
         ach = attend_flops / (sms * 1e-3) / 1e12
         sustained = {"launches": reps, "seconds": s0.elapsed_time(s1) * 1e-3, "ms_per_launch": sms, "achieved": ach,
-                     "unit": "TFLOP/s", "frac_sustained": ach / peaks["bf16_tflops_sustained"],
-                     "frac_burst": ach / peaks["bf16_tflops"], "clocks": sc,
+                     "unit": "TFLOP/s", "frac_sustained": ach / (peaks["bf16_tflops_sustained"] * blend),
+                     "frac_burst": ach / (peaks["bf16_tflops"] * blend), "clocks": sc,
                      "ms_x_mhz": sms * sc["sm_mhz"] if sc["sm_mhz"] else None}
         roofline["ms_x_mhz"] = att_ms * clk["sm_mhz"] if clk["sm_mhz"] else None
 
@@ -564,7 +579,7 @@ def main():
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "bf16" if wl.dtype == "bf16" else "f32", "data": "synthetic",
+        "vs_baseline": None, "dtype": {"bf16": "bf16", "e4m3": "e4m3 (Q K^T) / bf16 (P V)"}.get(wl.dtype, "f32"), "data": "synthetic",
         "config": workload_config(wl, args),
         "roofline": roofline,
         "whole_path_roofline": {"roofline_ms": whole_roof_s * 1e3, "frac": whole_roof_s * 1e3 / ms_step,

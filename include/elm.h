@@ -35,7 +35,14 @@
 extern "C" {
 #endif
 
-typedef enum { ELM_F32 = 0, ELM_BF16 = 1 } elm_dtype;
+/* ELM_E4M3: 8-bit floats (OCP E4M3, the finite-only variant: 4 exponent bits, 3 mantissa bits, no infinities) for
+ * Q, K and V, taken as the numbers they encode - no scale factors.  The paper's Conclusion names FP8 as future
+ * work; this library accepts it in elm_workspace_bytes, elm_compress, elm_attend (and their helper calls) with
+ * d = 128.  O is then bf16.  Every E4M3 value is also a bf16 value, so the compression and the fp64-mode
+ * attention run on an exact widened copy (in the workspace) and give what they would give on bf16 inputs holding
+ * the same numbers; the fp32-mode attention computes S = Q K^T with 8-bit tensor-core operands and fp32
+ * accumulation (products of E4M3 numbers are exact in fp32), the probabilities and P V in bf16 as for bf16 inputs. */
+typedef enum { ELM_F32 = 0, ELM_BF16 = 1, ELM_E4M3 = 2 } elm_dtype;
 
 typedef enum {
     ELM_PREC_FP64_DET = 0, /* all kernel-halving arithmetic in fp64: decisions reproduce an fp64
@@ -67,7 +74,7 @@ typedef struct elm_params {
     int32_t log2_nout;   /* coreset size n_out = 2^log2_nout (Algorithm 4's h) */
     int32_t m;           /* Compress2 depth (Algorithm 2); 0 returns every point; the level-0
                             groups hold n_kv / 4^(m-1) points and must hold at least 2 */
-    int32_t dtype;       /* elm_dtype of Q, K, V, O */
+    int32_t dtype;       /* elm_dtype of Q, K, V and O (ELM_E4M3: of Q, K, V; O is bf16) */
     int32_t precision;   /* elm_precision */
     double delta;        /* failure budget delta in (0,1); the paper's experiments use 1/2 */
     const double *delta_level; /* optional HOST array[m]: KH failure parameter of level i.  NULL

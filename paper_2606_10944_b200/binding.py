@@ -12,7 +12,7 @@ from pathlib import Path
 
 import torch
 
-ELM_F32, ELM_BF16 = 0, 1
+ELM_F32, ELM_BF16, ELM_E4M3 = 0, 1, 2
 PREC_FP64_DET, PREC_FP32 = 0, 1
 _PRECISIONS = {"fp64": PREC_FP64_DET, "fp64_det": PREC_FP64_DET, "fp32": PREC_FP32,
                PREC_FP64_DET: PREC_FP64_DET, PREC_FP32: PREC_FP32}
@@ -125,6 +125,8 @@ def _dtype_code(t: torch.Tensor) -> int:
         return ELM_F32
     if t.dtype == torch.bfloat16:
         return ELM_BF16
+    if t.dtype == torch.float8_e4m3fn:
+        return ELM_E4M3
     raise ElmError(f"unsupported dtype {t.dtype}")
 
 
@@ -319,7 +321,9 @@ def attend(Q, K, V, idx, w, precision="fp32", workspace=None, out=None):
     _check(lib.elm_attend_workspace_bytes(ctypes.byref(p), n_core, ctypes.byref(need)),
            "elm_attend_workspace_bytes")
     ws = workspace if workspace is not None else _workspace(int(need.value), Q.device)
-    O = out if out is not None else torch.empty_like(Q)
+    # 8-bit inputs: the output is bf16
+    O = out if out is not None else torch.empty(Q.shape, dtype=torch.bfloat16 if Q.dtype == torch.float8_e4m3fn else Q.dtype,
+                                                device=Q.device)
     _check(lib.elm_attend(Q.data_ptr(), K.data_ptr(), V.data_ptr(), idx.data_ptr(), w.data_ptr(),
                           n_core, ctypes.byref(p), O.data_ptr(), ws.data_ptr(), ws.numel(), _stream()),
            "elm_attend")

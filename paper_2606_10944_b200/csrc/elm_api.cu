@@ -47,7 +47,7 @@ StageTimer::~StageTimer()
     if (rec_ >= 0) cudaEventRecord(profiler().ev_end[rec_], stream_);
 }
 
-int validate_params(const elm_params *p)
+int validate_params(const elm_params *p, bool allow_e4m3)
 {
     if (p->batch < 1 || p->kv_heads < 1 || p->q_heads < 1 || p->n_q < 1) return ELM_ERR_SHAPE;
     if (p->q_heads % p->kv_heads != 0) return ELM_ERR_SHAPE;
@@ -57,7 +57,8 @@ int validate_params(const elm_params *p)
     if ((int64_t)p->n_kv != ((int64_t)1 << (p->log2_nout + p->m))) return ELM_ERR_SHAPE;
     if (p->m >= 1 && p->log2_nout - p->m + 2 < 1) return ELM_ERR_SHAPE;      // level-0 groups >= 2 points
     if ((int64_t)p->batch * p->q_heads > 65535) return ELM_ERR_SHAPE;
-    if (p->dtype != ELM_F32 && p->dtype != ELM_BF16) return ELM_ERR_DTYPE;
+    if (p->dtype != ELM_F32 && p->dtype != ELM_BF16 && !(allow_e4m3 && p->dtype == ELM_E4M3)) return ELM_ERR_DTYPE;
+    if (p->dtype == ELM_E4M3 && p->d != 128) return ELM_ERR_SHAPE;
     if (p->precision != ELM_PREC_FP64_DET && p->precision != ELM_PREC_FP32) return ELM_ERR_DTYPE;
     if (!(p->delta > 0.0 && p->delta < 1.0)) return ELM_ERR_DELTA;
     if (p->delta_level)
@@ -67,13 +68,14 @@ int validate_params(const elm_params *p)
 }
 
 // The attention calls read K and V through an index list: any n_kv, and log2_nout / m are not used.
-int validate_attend_params(const elm_params *p)
+int validate_attend_params(const elm_params *p, bool allow_e4m3)
 {
     if (p->batch < 1 || p->kv_heads < 1 || p->q_heads < 1 || p->n_q < 1 || p->n_kv < 1) return ELM_ERR_SHAPE;
     if (p->q_heads % p->kv_heads != 0) return ELM_ERR_SHAPE;
     if (p->d != 64 && p->d != 128) return ELM_ERR_SHAPE;
     if ((int64_t)p->batch * p->q_heads > 65535) return ELM_ERR_SHAPE;
-    if (p->dtype != ELM_F32 && p->dtype != ELM_BF16) return ELM_ERR_DTYPE;
+    if (p->dtype != ELM_F32 && p->dtype != ELM_BF16 && !(allow_e4m3 && p->dtype == ELM_E4M3)) return ELM_ERR_DTYPE;
+    if (p->dtype == ELM_E4M3 && p->d != 128) return ELM_ERR_SHAPE;
     if (p->precision != ELM_PREC_FP64_DET && p->precision != ELM_PREC_FP32) return ELM_ERR_DTYPE;
     return ELM_OK;
 }
@@ -85,7 +87,7 @@ using namespace elm;
 extern "C" int elm_workspace_bytes(const elm_params *params, size_t *compress_bytes, size_t *attend_bytes)
 {
     if (!params) return ELM_ERR_NULL;
-    int rc = validate_params(params);
+    int rc = validate_params(params, true);
     if (rc != ELM_OK) return rc;
     if (compress_bytes) *compress_bytes = compress_layout(params).total;
     if (attend_bytes) *attend_bytes = attend_layout(params, 1 << params->log2_nout).total;
@@ -270,7 +272,7 @@ extern "C" int elm_attend_status(const void *workspace, const elm_params *params
                                  int32_t *status_host, void *stream)
 {
     if (!workspace || !params || !status_host) return ELM_ERR_NULL;
-    int rc = validate_attend_params(params);
+    int rc = validate_attend_params(params, true);
     if (rc != ELM_OK) return rc;
     if (n_core < 1 || n_core > params->n_kv) return ELM_ERR_SHAPE;
     // the status word follows the per-problem "weights differ" flags

@@ -6,6 +6,8 @@
 // fp32 mode take the tensor-core kernel in elm_attend_tc.cu.
 #include <math.h>
 
+#include <cuda_fp8.h>
+
 #include <mutex>
 #include <type_traits>
 
@@ -17,9 +19,44 @@ namespace elm {
 // ---------------------------------------------------------------------------------------------
 // Stage gather: Kc, Vc [problems][n_core][d] in the input dtype, bias [problems][n_core] fp32
 // ---------------------------------------------------------------------------------------------
-template <typename Tin>
-__global__ void __launch_bounds__(256) gather_kernel(const Tin *__restrict__ K,
-                                                     const Tin *__restrict__ V,
+// E4M3 bytes as the numbers they encode (every E4M3 value is a bf16 value)
+__device__ __forceinline__ __nv_bfloat16 widen_e4m3(unsigned char b)
+{
+    const __half_raw h = __nv_cvt_fp8_to_halfraw((__nv_fp8_storage_t)b, __NV_E4M3);
+    return __float2bfloat16_rn(__half2float(__half(h)));
+}
+__device__ __forceinline__ float gather_elt(const float *p, int e) { return p[e]; }
+__device__ __forceinline__ __nv_bfloat16 gather_elt(const __nv_bfloat16 *p, int e) { return p[e]; }
+__device__ __forceinline__ __nv_bfloat16 gather_elt(const unsigned char *p, int e) { return widen_e4m3(p[e]); }
+
+// [count] E4M3 bytes -> bf16, exactly
+__global__ void __launch_bounds__(256) widen_e4m3_kernel(const unsigned char *__restrict__ src, __nv_bfloat16 *__restrict__ dst,
+                                                        int64_t count)
+{
+    const int64_t i = ((int64_t)blockIdx.x * 256 + threadIdx.x) * 16;
+    if (i + 16 <= count) {
+        const uint4 v = __ldg(reinterpret_cast<const uint4 *>(src + i));
+        const unsigned char *b = reinterpret_cast<const unsigned char *>(&v);
+        __align__(16) __nv_bfloat16 o[16];
+#pragma unroll
+        for (int e = 0; e < 16; ++e) o[e] = widen_e4m3(b[e]);
+        reinterpret_cast<uint4 *>(dst + i)[0] = reinterpret_cast<const uint4 *>(o)[0];
+        reinterpret_cast<uint4 *>(dst + i)[1] = reinterpret_cast<const uint4 *>(o)[1];
+    } else {
+        for (int64_t e = i; e < count; ++e) dst[e] = widen_e4m3(src[e]);
+    }
+}
+int widen_e4m3(const void *src, void *dst_bf16, int64_t count, cudaStream_t st)
+{
+    const int64_t blocks = (count + 4095) / 4096;
+    widen_e4m3_kernel<<<(unsigned)blocks, 256, 0, st>>>((const unsigned char *)src, (__nv_bfloat16 *)dst_bf16, count);
+    count_launches(1);
+    return cuda_status(cudaGetLastError());
+}
+
+template <typename Tin, typename Tsrc = Tin>
+__global__ void __launch_bounds__(256) gather_kernel(const Tsrc *__restrict__ K,
+                                                     const Tsrc *__restrict__ V,
                                                      const int32_t *__restrict__ idx,
                                                      const float *__restrict__ w, int64_t n, int d,
                                                      int n_core, Tin *__restrict__ Kc,
@@ -31,13 +68,13 @@ __global__ void __launch_bounds__(256) gather_kernel(const Tin *__restrict__ K,
     const int c = blockIdx.x * 8 + warp;
     if (c >= n_core) return;
     const int64_t row = checked_row(idx[(int64_t)p * n_core + c], n, status);
-    const Tin *ks = K + ((int64_t)p * n + row) * d;
-    const Tin *vs = V + ((int64_t)p * n + row) * d;
+    const Tsrc *ks = K + ((int64_t)p * n + row) * d;
+    const Tsrc *vs = V + ((int64_t)p * n + row) * d;
     Tin *kd = Kc + ((int64_t)p * n_core + c) * d;
     Tin *vd = Vc + ((int64_t)p * n_core + c) * d;
     for (int e = lane; e < d; e += 32) {
-        kd[e] = ks[e];
-        vd[e] = vs[e];
+        kd[e] = gather_elt(ks, e);
+        vd[e] = gather_elt(vs, e);
     }
     if (lane == 0) bias[(int64_t)p * n_core + c] = log2f(w[(int64_t)p * n_core + c]);
 }
@@ -194,11 +231,15 @@ AttendLayout attend_layout(const elm_params *p, int32_t n_core)
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
     const size_t n_pad = ((size_t)n_core + 127) / 128 * 128;      // the tensor-core path pads to its block size
-    L.Kc = take(problems * n_pad * p->d * es);
-    L.Vc = take(problems * n_pad * p->d * es);
+    // E4M3 inputs: the gathered rows are kept as bf16 (exact), except the keys of the fp32-mode tensor-core path
+    const size_t ges = p->dtype == ELM_E4M3 ? 2 : es;
+    L.Kc = take(problems * n_pad * p->d * ges);
+    L.Vc = take(problems * n_pad * p->d * ges);
     L.bias = take(problems * n_pad * 4);
     L.bx = take(problems * n_pad * 32);
     L.flags = take((problems + 1) * 4);
+    L.qwide = take(p->dtype == ELM_E4M3 && p->precision == ELM_PREC_FP64_DET
+                       ? (size_t)p->batch * p->q_heads * p->n_q * p->d * 2 : 0);
     L.total = off;
     return L;
 }
@@ -219,11 +260,12 @@ static int launch_attend_simt(const Tin *Q, const Tin *Kc, const Tin *Vc, const 
     return cuda_status(cudaGetLastError());
 }
 
-template <typename Tin, typename T>
-static int attend_impl(const Tin *Q, const Tin *K, const Tin *V, const int32_t *idx, const float *w,
+// Tsrc: the type K and V are stored in (E4M3 bytes are widened by the gather; Q then is the widened copy)
+template <typename Tin, typename T, typename Tsrc = Tin>
+static int attend_impl(const Tin *Q, const Tsrc *K, const Tsrc *V, const int32_t *idx, const float *w,
                        int n_core, const elm_params *p, Tin *O, unsigned char *ws, cudaStream_t st, const AttendWindow &win)
 {
-    if constexpr (std::is_same<Tin, __nv_bfloat16>::value && std::is_same<T, float>::value)
+    if constexpr (std::is_same<Tsrc, __nv_bfloat16>::value && std::is_same<T, float>::value)
         return attend_tc(Q, K, V, idx, w, n_core, p, O, ws, st, true, win);
     const AttendLayout L = attend_layout(p, n_core);
     Tin *Kc = reinterpret_cast<Tin *>(ws + L.Kc);
@@ -234,7 +276,7 @@ static int attend_impl(const Tin *Q, const Tin *K, const Tin *V, const int32_t *
         StageTimer t(ELM_STAGE_GATHER, st, 1);
         // this path has no bounded waits: its status word reads 0
         ELM_CUDA_TRY(cudaMemsetAsync(ws + L.flags, 0, sizeof(int) * (size_t)(problems + 1), st));
-        gather_kernel<Tin><<<dim3((unsigned)((n_core + 7) / 8), (unsigned)problems), 256, 0, st>>>(
+        gather_kernel<Tin, Tsrc><<<dim3((unsigned)((n_core + 7) / 8), (unsigned)problems), 256, 0, st>>>(
             K, V, idx, w, p->n_kv, p->d, n_core, Kc, Vc, bias, reinterpret_cast<int *>(ws + L.flags) + problems);
         count_launches(1);
         ELM_CUDA_TRY(cudaGetLastError());
@@ -309,6 +351,18 @@ int attend_enqueue(const void *Q, const void *K, const void *V, const int32_t *i
     unsigned char *ws = (unsigned char *)workspace;
     const bool det = params->precision == ELM_PREC_FP64_DET;
     const bool whole = win.q_row0 == 0 && win.n_q_total == 0 && win.tail_start == 0x7fffffff && !win.birth && !win.lse;
+    if (params->dtype == ELM_E4M3) {
+        typedef __nv_bfloat16 bf;
+        if (!whole) return ELM_ERR_DTYPE;                      // no windows or lifetimes on 8-bit inputs
+        if (!det) return attend_tc_e4m3((const unsigned char *)Q, (const unsigned char *)K, (const unsigned char *)V, idx, w, n_core,
+                                        params, (bf *)O, ws, st, true);
+        // fp64 mode: the queries are widened into the workspace, the coreset rows by the gather
+        bf *Qw = reinterpret_cast<bf *>(ws + attend_layout(params, n_core).qwide);
+        const int rc = widen_e4m3(Q, Qw, (int64_t)params->batch * params->q_heads * params->n_q * params->d, st);
+        if (rc != ELM_OK) return rc;
+        return attend_impl<bf, double, unsigned char>(Qw, (const unsigned char *)K, (const unsigned char *)V, idx, w, n_core, params,
+                                                      (bf *)O, ws, st, win);
+    }
     if (whole && attend_decode_applies(params)) return attend_decode(Q, K, V, idx, w, n_core, params, O, ws, st, true);
     if (params->dtype == ELM_F32) {
         return det ? attend_impl<float, double>((const float *)Q, (const float *)K, (const float *)V, idx, w, n_core, params, (float *)O, ws, st, win)
@@ -324,7 +378,7 @@ extern "C" int elm_attend_workspace_bytes(const elm_params *params, int32_t n_co
 {
     using namespace elm;
     if (!params || !bytes) return ELM_ERR_NULL;
-    int rc = validate_attend_params(params);
+    int rc = validate_attend_params(params, true);
     if (rc != ELM_OK) return rc;
     if (n_core < 1 || n_core > params->n_kv) return ELM_ERR_SHAPE;
     *bytes = attend_layout(params, n_core).total;
@@ -337,7 +391,7 @@ extern "C" int elm_attend(const void *Q, const void *K, const void *V, const int
 {
     using namespace elm;
     if (!params) return ELM_ERR_NULL;
-    int rc = validate_attend_params(params);
+    int rc = validate_attend_params(params, true);
     if (rc != ELM_OK) return rc;
     if (!Q || !K || !V || !idx || !w || !O || !workspace) return ELM_ERR_NULL;
     if (n_core < 1 || n_core > params->n_kv) return ELM_ERR_SHAPE;

@@ -16,6 +16,7 @@ struct AttendLayout {
     size_t bias;  // [problems][n_core] log2 of the weights, fp32
     size_t bx;    // [problems][n_pad][16] bf16: the weights as an operand of the tensor-core path's bias MMA
     size_t flags; // [problems] "weights differ" flags + one device status word
+    size_t qwide; // E4M3 inputs in fp64 mode: [batch][q_heads][n_q][d] bf16, the queries widened exactly
     size_t total;
 };
 AttendLayout attend_layout(const elm_params *p, int32_t n_core);
@@ -54,6 +55,14 @@ int attend_tc(const __nv_bfloat16 *Q, const __nv_bfloat16 *K, const __nv_bfloat1
 
 // elm_debug_set for the hooks that live with the tensor-core attention
 int debug_set_attend_tc(int32_t what, int64_t value);
+
+// [count] E4M3 bytes -> bf16, exactly (every E4M3 value is a bf16 value)
+int widen_e4m3(const void *src, void *dst_bf16, int64_t count, cudaStream_t st);
+
+// Tensor-core path for E4M3 inputs (fp32 mode, d = 128, every row sees the whole list): S = Q K^T with 8-bit
+// operands, probabilities and P V in bf16 (the gather widens the coreset's value rows), O in bf16.
+int attend_tc_e4m3(const unsigned char *Q, const unsigned char *K, const unsigned char *V, const int32_t *idx, const float *w,
+                   int n_core, const elm_params *p, __nv_bfloat16 *O, unsigned char *ws, cudaStream_t st, bool timed);
 
 // A few query vectors per KV head (decode): HBM-bound kernels that read the coreset rows once through
 // the index list.  Applies to fp32 mode when (q_heads / kv_heads) * n_q <= 8.

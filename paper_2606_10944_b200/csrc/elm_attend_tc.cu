@@ -34,6 +34,7 @@
 // Every mbarrier wait is bounded; on expiry the CTA records a status word and leaves through the
 // common exit, which frees the TMEM it holds.
 #include <cuda.h>
+#include <cuda_fp8.h>
 #include <math.h>
 
 #include <atomic>
@@ -72,10 +73,11 @@ struct __align__(8) Barriers {
     float xchg[2][4][BM];        // per tile, per column quarter: row maxima / denominators being exchanged
 };
 
-template <int D> struct Smem {
-    static constexpr int KH = D / 64;                       // 64-element halves of the head dimension
-    static constexpr int Q_TILE = BM * D * 2;               // bytes
-    static constexpr int K_BLOCK = BN * D * 2;
+// QKB: bytes per element of Q and K (2: bf16; 1: E4M3, whose S = Q K^T takes the 8-bit MMA kind)
+template <int D, int QKB = 2> struct Smem {
+    static constexpr int KH = D * QKB / 128;                // 128-byte slices of a row of Q or K
+    static constexpr int Q_TILE = BM * D * QKB;             // bytes
+    static constexpr int K_BLOCK = BN * D * QKB;
     static constexpr int V_BLOCK = D * BN * 2;
     static constexpr int OFF_Q = 0;
     static constexpr int OFF_K = OFF_Q + 2 * Q_TILE;
@@ -94,7 +96,9 @@ template <int D> struct Smem {
 // the bias cancels in the ratio).
 // ---------------------------------------------------------------------------------------------
 constexpr int GATHER_COLS = 64;          // list entries per CTA of the gather
-template <int D>
+// E4M3 = true: K and V hold 8-bit floats; the key rows are copied as they are (Kc then has D bytes per row),
+// the value rows are widened to bf16 (exactly) on their way into the transposed tile.
+template <int D, bool E4M3 = false>
 __global__ void __launch_bounds__(256) gather_tc_kernel(const __nv_bfloat16 *__restrict__ K,
                                                         const __nv_bfloat16 *__restrict__ V,
                                                         const int32_t *__restrict__ idx,
@@ -118,7 +122,25 @@ __global__ void __launch_bounds__(256) gather_tc_kernel(const __nv_bfloat16 *__r
         const bool ok = c < n_core;
         const int64_t row = ok ? checked_row(idx[(int64_t)p * n_core + c], n, nonuniform + gridDim.y) : 0;
         const int chunk = lane & 15;
-        if (chunk < CH) {
+        if constexpr (E4M3) {
+            // a row is D bytes = D / 16 chunks
+            const unsigned char *K8 = reinterpret_cast<const unsigned char *>(K), *V8 = reinterpret_cast<const unsigned char *>(V);
+            if (chunk < D / 16) {
+                const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+                if (lane < 16) {
+                    const uint4 v = ok ? __ldg(reinterpret_cast<const uint4 *>(K8 + ((int64_t)p * n + row) * D) + chunk) : zero;
+                    reinterpret_cast<uint4 *>(reinterpret_cast<unsigned char *>(Kc) + ((int64_t)p * n_pad + c) * D)[chunk] = v;
+                } else {
+                    const uint4 v = ok ? __ldg(reinterpret_cast<const uint4 *>(V8 + ((int64_t)p * n + row) * D) + chunk) : zero;
+                    const unsigned char *b = reinterpret_cast<const unsigned char *>(&v);
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) {
+                        const __half_raw h = __nv_cvt_fp8_to_halfraw((__nv_fp8_storage_t)b[e], __NV_E4M3);
+                        tile[r][chunk * 16 + e] = __float2bfloat16_rn(__half2float(__half(h)));
+                    }
+                }
+            }
+        } else if (chunk < CH) {
             const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
             if (lane < 16) {
                 const uint4 v = ok ? __ldg(reinterpret_cast<const uint4 *>(K + ((int64_t)p * n + row) * D) + chunk) : zero;
@@ -320,7 +342,7 @@ __device__ __forceinline__ float exp_pass_keep(uint32_t tP, float scale_log2, fl
 // ---------------------------------------------------------------------------------------------
 // MASKED = false: every row sees the whole list (no causal tail, no lifetimes); the masked form of the
 // softmax passes is then not compiled in, which keeps the plain form's register allocation to itself.
-template <int D, bool MASKED>
+template <int D, bool MASKED, int QKB = 2>
 __global__ void __launch_bounds__(NTHREADS, 1)
 attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
                  const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapX,
@@ -333,8 +355,9 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
 {
     // every wait of this kernel is bounded by the limit the host passes (2 s unless a test shortened it)
     auto mbar_wait = [wait_limit_ns](uint64_t *b, uint32_t parity) { return sm100::mbar_wait(b, parity, wait_limit_ns); };
-    using SM = Smem<D>;
+    using SM = Smem<D, QKB>;
     constexpr int KH = SM::KH;
+    constexpr int ROW_ELTS = 128 / QKB;                            // elements of Q / K in a 128-byte slice of a row
     extern __shared__ unsigned char smem_dyn[];
     unsigned char *smem = reinterpret_cast<unsigned char *>(((uintptr_t)smem_dyn + 1023) & ~(uintptr_t)1023);
     Barriers *bar = reinterpret_cast<Barriers *>(smem + SM::OFF_BAR);
@@ -392,7 +415,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                 mbar_expect_tx(&bar->q_full, 2 * SM::Q_TILE);
                 for (int t = 0; t < 2; ++t)
                     for (int kh = 0; kh < KH; ++kh)
-                        tma_load_3d(smem + SM::OFF_Q + t * SM::Q_TILE + kh * (BM * 128), &mapQ, &bar->q_full, kh * 64, q_row0 + q0 + t * BM, bh);
+                        tma_load_3d(smem + SM::OFF_Q + t * SM::Q_TILE + kh * (BM * 128), &mapQ, &bar->q_full, kh * ROW_ELTS, q_row0 + q0 + t * BM, bh);
             };
             // Blocks are numbered G = k nblk + j along the CTA's whole stream (item k, block j).
             int flag_item = -1;
@@ -408,7 +431,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                 const bool with_bias = flag_now;
                 mbar_expect_tx(&bar->k_full[s], SM::K_BLOCK + (with_bias ? SM::X_BLOCK : 0));
                 for (int kh = 0; kh < KH; ++kh)
-                    tma_load_3d(smem + SM::OFF_K + s * SM::K_BLOCK + kh * (BN * 128), &mapK, &bar->k_full[s], kh * 64, (G % nblk) * BN, prob);
+                    tma_load_3d(smem + SM::OFF_K + s * SM::K_BLOCK + kh * (BN * 128), &mapK, &bar->k_full[s], kh * ROW_ELTS, (G % nblk) * BN, prob);
                 if (with_bias) tma_load_3d(smem + SM::OFF_X + s * SM::X_BLOCK, &mapX, &bar->k_full[s], 0, (G % nblk) * BN, prob);
             };
             auto load_v = [&](int G) {
@@ -459,7 +482,8 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
         // Each thread commits its own MMAs, so the barriers that release shared memory count two arrivals.
         if (lane == 0) {
             const int t = warp - MMA_WARP;
-            constexpr uint32_t IDESC_QK = umma_idesc_bf16(BM, BN);
+            constexpr uint32_t IDESC_QK = QKB == 1 ? umma_idesc_e4m3(BM, BN) : umma_idesc_bf16(BM, BN);
+            constexpr uint32_t IDESC_BIAS = umma_idesc_bf16(BM, BN);     // the bias operands are bf16 whatever Q and K are
             constexpr uint32_t IDESC_PV = umma_idesc_bf16(BM, D);
             // descriptors differ only in the 14-bit start-address field (address / 16)
             const uint64_t dQ = umma_desc_k128(smem_u32(smem + SM::OFF_Q));
@@ -474,10 +498,14 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                 for (int kh = 0; kh < KH; ++kh)
 #pragma unroll
                     for (int ks = 0; ks < 4; ++ks)
-                        mma_ss(tmem + t * 128, a0 + (uint64_t)(kh * (BM * 128 >> 4) + ks * 2),
-                               b0 + (uint64_t)(kh * (BN * 128 >> 4) + ks * 2), IDESC_QK, (kh | ks) != 0);
+                        if constexpr (QKB == 1)
+                            mma_ss_f8(tmem + t * 128, a0 + (uint64_t)(kh * (BM * 128 >> 4) + ks * 2),
+                                      b0 + (uint64_t)(kh * (BN * 128 >> 4) + ks * 2), IDESC_QK, (kh | ks) != 0);
+                        else
+                            mma_ss(tmem + t * 128, a0 + (uint64_t)(kh * (BM * 128 >> 4) + ks * 2),
+                                   b0 + (uint64_t)(kh * (BN * 128 >> 4) + ks * 2), IDESC_QK, (kh | ks) != 0);
                 // S += ones x (log2 w / scale_log2 in three bf16 terms)^T
-                if (with_bias) mma_ss(tmem + t * 128, dOnes, dX + (uint64_t)(s * (SM::X_BLOCK >> 4)), IDESC_QK, 1u);
+                if (with_bias) mma_ss(tmem + t * 128, dOnes, dX + (uint64_t)(s * (SM::X_BLOCK >> 4)), IDESC_BIAS, 1u);
             };
             auto issue_pv = [&](int t, int s, bool acc) {
                 const uint64_t b0 = dV + (uint64_t)(s * (SM::V_BLOCK >> 4));
@@ -821,8 +849,20 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
 // 3-D bf16 tensor [d2][d1][d0] (d0 contiguous), box {64, box_rows, 1} with the 128-byte swizzle, or
 // (narrow) box {16, box_rows, 1} with the 32-byte swizzle
 static bool make_map(CUtensorMap *map, const void *base, uint64_t d0, uint64_t d1, uint64_t d2, uint32_t box_rows,
-                     bool narrow = false)
+                     bool narrow = false, bool bytes = false)
 {
+    if (bytes) {
+        // 8-bit elements: rows of d0 bytes, boxes of 128 bytes x box_rows, 128-byte swizzle
+        sm100::EncodeTiledFn fn8 = sm100::tensor_map_encoder();
+        if (!fn8) return false;
+        cuuint64_t dims8[3] = {d0, d1, d2};
+        cuuint64_t strides8[2] = {d0, d0 * d1};
+        cuuint32_t box8[3] = {128u, box_rows, 1};
+        cuuint32_t estr8[3] = {1, 1, 1};
+        return fn8(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void *>(base), dims8, strides8, box8, estr8,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    }
     sm100::EncodeTiledFn fn = sm100::tensor_map_encoder();
     if (!fn) return false;
     cuuint64_t dims[3] = {d0, d1, d2};
@@ -889,7 +929,57 @@ static int launch(const __nv_bfloat16 *Q, const __nv_bfloat16 *K, const __nv_bfl
     return cuda_status(cudaGetLastError());
 }
 
+// E4M3 inputs, d = 128, no mask: the same kernel with 8-bit Q and K tiles
+static int launch_e4m3(const unsigned char *Q, const unsigned char *K, const unsigned char *V, const int32_t *idx, const float *w,
+                       int n_core, const elm_params *p, __nv_bfloat16 *O, unsigned char *ws, cudaStream_t st, bool timed)
+{
+    constexpr int D = 128;
+    const AttendLayout L = attend_layout(p, n_core);
+    const int n_pad = (n_core + BN - 1) / BN * BN;
+    const int problems = p->batch * p->kv_heads;
+    unsigned char *Kc = ws + L.Kc;                                  // [problems][n_pad][D] bytes
+    __nv_bfloat16 *Vt = reinterpret_cast<__nv_bfloat16 *>(ws + L.Vc);
+    __nv_bfloat16 *Bx = reinterpret_cast<__nv_bfloat16 *>(ws + L.bx);
+    int *flags = reinterpret_cast<int *>(ws + L.flags);
+    int *status = flags + problems;
+    CUtensorMap mQ, mK, mV, mX;
+    if (!make_map(&mQ, Q, D, (uint64_t)p->n_q, (uint64_t)p->batch * p->q_heads, BM, false, true) ||
+        !make_map(&mK, Kc, D, (uint64_t)n_pad, (uint64_t)problems, BN, false, true) ||
+        !make_map(&mV, Vt, (uint64_t)n_pad, D, (uint64_t)problems, D) ||
+        !make_map(&mX, Bx, 16, (uint64_t)n_pad, (uint64_t)problems, BN, true))
+        return ELM_ERR_CUDA;
+    const float scale_log2 = (float)(1.4426950408889634 / sqrt((double)D));
+    {
+        StageTimer t(timed ? ELM_STAGE_GATHER : -1, st, 1);
+        ELM_CUDA_TRY(cudaMemsetAsync(flags, 0, sizeof(int) * (size_t)(problems + 1), st));
+        gather_tc_kernel<D, true><<<dim3((unsigned)(n_pad / GATHER_COLS), (unsigned)problems), 256, 0, st>>>(
+            reinterpret_cast<const __nv_bfloat16 *>(K), reinterpret_cast<const __nv_bfloat16 *>(V), idx, w, p->n_kv, n_core, n_pad,
+            reinterpret_cast<__nv_bfloat16 *>(Kc), Vt, Bx, 1.f / scale_log2, flags);
+        count_launches(1);
+        ELM_CUDA_TRY(cudaGetLastError());
+    }
+    StageTimer t(timed ? ELM_STAGE_ATTEND : -1, st, 1);
+    auto kern = attend_tc_kernel<D, false, 1>;
+    ELM_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<D, 1>::TOTAL));
+    const int tiles_x = (p->n_q + 2 * BM - 1) / (2 * BM);
+    const int64_t items = (int64_t)tiles_x * p->batch * p->q_heads;
+    if (items > 0x7fffffff / 64) return ELM_ERR_SHAPE;
+    const int ctas = (int)(items < sm_count() ? items : sm_count());
+    kern<<<ctas, NTHREADS, Smem<D, 1>::TOTAL, st>>>(mQ, mK, mV, mX, flags, O, p->q_heads, p->kv_heads, p->n_q, n_core, n_pad,
+                                                    scale_log2, tiles_x, (int)items, 0, p->n_q, 0x7fffffff, nullptr, nullptr, nullptr,
+                                                    nullptr, nullptr, status, g_debug_extra_arrivals.exchange(0),
+                                                    g_debug_wait_limit_ns.load());
+    count_launches(1);
+    return cuda_status(cudaGetLastError());
+}
+
 }  // namespace tc
+
+int attend_tc_e4m3(const unsigned char *Q, const unsigned char *K, const unsigned char *V, const int32_t *idx, const float *w,
+                   int n_core, const elm_params *p, __nv_bfloat16 *O, unsigned char *ws, cudaStream_t st, bool timed)
+{
+    return tc::launch_e4m3(Q, K, V, idx, w, n_core, p, O, ws, st, timed);
+}
 
 int debug_set_attend_tc(int32_t what, int64_t value)
 {

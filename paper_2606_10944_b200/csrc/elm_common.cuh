@@ -47,10 +47,11 @@ inline int cuda_status(cudaError_t e) { return e == cudaSuccess ? ELM_OK : ELM_E
 // Multiprocessors of the current device (looked up once per device ordinal; 148 if the query fails).
 int device_sm_count();
 
-int validate_params(const elm_params *p);
-int validate_attend_params(const elm_params *p);
+// `allow_e4m3`: the entry point accepts 8-bit inputs (then d must be 128)
+int validate_params(const elm_params *p, bool allow_e4m3 = false);
+int validate_attend_params(const elm_params *p, bool allow_e4m3 = false);
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
-inline size_t elt_bytes(int dtype) { return dtype == ELM_BF16 ? 2 : 4; }
+inline size_t elt_bytes(int dtype) { return dtype == ELM_BF16 ? 2 : (dtype == ELM_E4M3 ? 1 : 4); }
 
 // ---------------------------------------------------------------------------------------------
 // device helpers

@@ -558,6 +558,7 @@ CompressLayout compress_layout(const elm_params *p)
     L.rdecay = take(BH * (n / 2 + 1) * ts);
     L.F_stride = n_out * n_out;
     L.F = take(p->m > 0 ? BH * L.F_stride * ts : 0);
+    L.wide = take(p->dtype == ELM_E4M3 ? 2 * BH * n * (size_t)p->d * 2 : 0);
     L.total = off;
     return L;
 }
@@ -1304,6 +1305,17 @@ int compress_enqueue(const void *K, const void *V, const elm_params *params, uin
 {
     unsigned char *ws = (unsigned char *)workspace;
     const bool det = params->precision == ELM_PREC_FP64_DET;
+    if (params->dtype == ELM_E4M3) {
+        // every E4M3 value is a bf16 value: widen K and V (exactly) and run the bf16 kernels on the copies
+        typedef __nv_bfloat16 bf;
+        const int64_t count = (int64_t)params->batch * params->kv_heads * params->n_kv * params->d;
+        bf *Kw = reinterpret_cast<bf *>(ws + compress_layout(params).wide), *Vw = Kw + count;
+        int rc = widen_e4m3(K, Kw, count, st);
+        if (rc == ELM_OK) rc = widen_e4m3(V, Vw, count, st);
+        if (rc != ELM_OK) return rc;
+        return det ? compress_impl<bf, double>(Kw, Vw, params, seed, idx_out, w_out, ws, st, pbase)
+                   : compress_impl<bf, float>(Kw, Vw, params, seed, idx_out, w_out, ws, st, pbase);
+    }
     if (params->dtype == ELM_F32) {
         return det ? compress_impl<float, double>((const float *)K, (const float *)V, params, seed, idx_out, w_out, ws, st, pbase)
                    : compress_impl<float, float>((const float *)K, (const float *)V, params, seed, idx_out, w_out, ws, st, pbase);
@@ -1319,7 +1331,7 @@ extern "C" int elm_compress(const void *K, const void *V, const elm_params *para
 {
     using namespace elm;
     if (!params) return ELM_ERR_NULL;
-    int rc = validate_params(params);
+    int rc = validate_params(params, true);
     if (rc != ELM_OK) return rc;
     if (!K || !V || !idx_out || !w_out || !workspace) return ELM_ERR_NULL;
     if (((uintptr_t)K | (uintptr_t)V | (uintptr_t)idx_out | (uintptr_t)w_out) & 15) return ELM_ERR_ALIGN;

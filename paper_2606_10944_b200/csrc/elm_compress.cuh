@@ -19,6 +19,7 @@ struct CompressLayout {
     size_t rdecay;     // [BH][n/2] exp(-(M_i - M_{i-1})/2)
     size_t F;          // [BH][n_out^2] pair Gram of the current level (all calls)
     size_t F_stride;   // elements per problem
+    size_t wide;       // E4M3 inputs: K then V widened exactly to bf16, [BH][n][d] each
     size_t total;
 };
 CompressLayout compress_layout(const elm_params *p);

@@ -24,7 +24,7 @@ class Workload:
     n: int            # keys/values per head
     n_q: int          # queries per head
     d: int
-    dtype: str        # "f32" or "bf16": storage type of Q, K, V, O
+    dtype: str        # "f32", "bf16" or "e4m3": storage type of Q, K, V (and of O, which is bf16 for "e4m3")
     g: int            # oversampling: coreset size 2^g * 2^floor(log2(n)/2)
     recipe: str
 
@@ -99,7 +99,16 @@ def _keys_values(rng, recipe: str, n: int, d: int):
 
 
 def torch_dtype(name: str):
-    return {"f32": torch.float32, "bf16": torch.bfloat16}[name]
+    return {"f32": torch.float32, "bf16": torch.bfloat16, "e4m3": torch.float8_e4m3fn}[name]
+
+
+E4M3_MAX = 448.0      # largest finite E4M3 value: the draws are clamped to it before rounding (the format has no infinity)
+
+
+def _store(x: torch.Tensor, dt):
+    if dt == torch.float8_e4m3fn:
+        return x.clamp_(-E4M3_MAX, E4M3_MAX).to(dt)
+    return x.to(dt)
 
 
 def generate(wl: Workload, seed: int = 1234, want_q: bool = True):
@@ -110,24 +119,30 @@ def generate(wl: Workload, seed: int = 1234, want_q: bool = True):
     numbers.  ``Q`` is ``None`` when ``want_q`` is false.
     """
     dt = torch_dtype(wl.dtype)
+    # drawn in the order (K, V per problem) then Q per head, whatever the storage type; 16-bit and wider types are
+    # rounded head by head, the 8-bit type (which torch cannot assign slice-wise) at the end
+    mid = torch.float32 if dt == torch.float8_e4m3fn else dt
     rng = np.random.default_rng(np.random.PCG64(seed))
-    K = torch.empty((wl.batch, wl.kv_heads, wl.n, wl.d), dtype=dt)
+    K = torch.empty((wl.batch, wl.kv_heads, wl.n, wl.d), dtype=mid)
     V = torch.empty_like(K)
     for b in range(wl.batch):
         for h in range(wl.kv_heads):
             k, v = _keys_values(rng, wl.recipe, wl.n, wl.d)
-            K[b, h] = torch.from_numpy(k).to(dt)
-            V[b, h] = torch.from_numpy(v).to(dt)
+            K[b, h] = torch.from_numpy(k).to(mid)
+            V[b, h] = torch.from_numpy(v).to(mid)
     Q = None
     if want_q:
         qstd = (1.0 / math.sqrt(wl.d)) ** 0.5
-        Q = torch.empty((wl.batch, wl.q_heads, wl.n_q, wl.d), dtype=dt)
+        Q = torch.empty((wl.batch, wl.q_heads, wl.n_q, wl.d), dtype=mid)
         for b in range(wl.batch):
             for h in range(wl.q_heads):
-                Q[b, h] = torch.from_numpy(_normal(rng, (wl.n_q, wl.d), qstd)).to(dt)
+                Q[b, h] = torch.from_numpy(_normal(rng, (wl.n_q, wl.d), qstd)).to(mid)
+    if mid != dt:
+        K, V = _store(K, dt), _store(V, dt)
+        Q = _store(Q, dt) if Q is not None else None
     return Q, K, V
 
 
 def as_f32_numpy(t: torch.Tensor) -> np.ndarray:
-    """Exact upcast of an fp32/bf16 tensor to a float32 NumPy array (for the oracle)."""
+    """Exact upcast of an fp32 / bf16 / E4M3 tensor to a float32 NumPy array (for the oracle)."""
     return t.detach().to("cpu", torch.float32).contiguous().numpy()
