@@ -277,6 +277,12 @@ int elm_stream_init(elm_stream *s, const void *K, const void *V, int64_t n_known
                     int32_t mbar, uint64_t seed, void *workspace, size_t workspace_bytes, void *stream);
 int elm_stream_step(elm_stream *s, const void *Q_t, const void *K, const void *V, const elm_params *params,
                     void *O_t, void *workspace, size_t workspace_bytes, void *stream);
+/* n_tokens calls of elm_stream_step enqueued by one call (Algorithm 4's attend, token after token): Q_T and O_T hold
+ * the tokens' queries and outputs one after the other, [n_tokens][batch][q_heads][1][d]; token i is row s->n + i of K
+ * and V when the call starts.  Stops at the first step that fails and returns its status (the steps before it stay
+ * enqueued and counted in *s). */
+int elm_stream_steps(elm_stream *s, int32_t n_tokens, const void *Q_T, const void *K, const void *V,
+                     const elm_params *params, void *O_T, void *workspace, size_t workspace_bytes, void *stream);
 /* The current cache, wtd_cache() of Algorithm 1: at most 6 n_out entries per problem, [batch][kv_heads][count]
  * row numbers and (unnormalised) weights 2^(i-q) / 1; *count_host receives the number of entries (inside a
  * stratum of a subsampled phase: of the longest list; see above for the padding of the others). */

@@ -22,7 +22,7 @@ EXPORTED_SYMBOLS = [
     "elm_workspace_bytes", "elm_default_delta_levels", "elm_compress", "elm_attend",
     "elm_attend_workspace_bytes", "elm_attend_static", "elm_attend_static_status", "elm_compress_ragged_count", "elm_compress_ragged", "elm_express_workspace_bytes", "elm_express_compress",
     "elm_express_prefill_workspace_bytes", "elm_express_prefill",
-    "elm_stream_workspace_bytes", "elm_stream_init", "elm_stream_step", "elm_stream_cache",
+    "elm_stream_workspace_bytes", "elm_stream_init", "elm_stream_step", "elm_stream_steps", "elm_stream_cache",
     "elm_host_call_scratch_bytes", "elm_compress_attend_host",
     "elm_compress_status", "elm_attend_status", "elm_debug_set", "elm_profile_enable", "elm_profile_read", "elm_launch_count", "elm_strerror", "elm_version",
 ]
@@ -87,6 +87,7 @@ def load_library():
     lib.elm_stream_workspace_bytes.argtypes = [pp, ctypes.c_int32, szp]
     lib.elm_stream_init.argtypes = [sp, vp, vp, ctypes.c_int64, pp, ctypes.c_int32, ctypes.c_uint64, vp, sz, vp]
     lib.elm_stream_step.argtypes = [sp, vp, vp, vp, pp, vp, vp, sz, vp]
+    lib.elm_stream_steps.argtypes = [sp, ctypes.c_int32, vp, vp, vp, pp, vp, vp, sz, vp]
     lib.elm_stream_cache.argtypes = [sp, pp, vp, vp, ctypes.POINTER(ctypes.c_int32), vp, sz, vp]
     lib.elm_host_call_scratch_bytes.argtypes = [pp, szp]
     lib.elm_compress_attend_host.argtypes = [vp, vp, vp, vp, vp, vp, pp, ctypes.c_uint64, vp, sz, vp]
@@ -280,6 +281,14 @@ class Stream:
         _check(load_library().elm_stream_step(ctypes.byref(self.state), q_t.data_ptr(), self.K.data_ptr(), self.V.data_ptr(),
                                               ctypes.byref(self.params), O.data_ptr(), self.ws.data_ptr(), self.ws.numel(),
                                               _stream()), "elm_stream_step")
+        return O
+
+    def steps(self, q_T, out=None):
+        """q_T [T, B, Hq, 1, d] -> O_T of the same shape: T tokens by one library call (elm_stream_steps)."""
+        O = out if out is not None else torch.empty_like(q_T)
+        _check(load_library().elm_stream_steps(ctypes.byref(self.state), q_T.shape[0], q_T.data_ptr(), self.K.data_ptr(),
+                                               self.V.data_ptr(), ctypes.byref(self.params), O.data_ptr(), self.ws.data_ptr(),
+                                               self.ws.numel(), _stream()), "elm_stream_steps")
         return O
 
     def cache(self):

@@ -53,7 +53,7 @@ def _build_one(lib: Path, extra, verbose: bool) -> Path:
     with ThreadPoolExecutor(max_workers=min(8, os.cpu_count() or 1)) as pool:
         objs = list(pool.map(compile_one, sources()))
     tmp = lib.with_suffix(f".tmp{os.getpid()}.so")
-    subprocess.run([nvcc, "-shared", "-o", str(tmp), *map(str, objs)], check=True)
+    subprocess.run([nvcc, *NVCC_FLAGS[:2], "-shared", "-o", str(tmp), *map(str, objs)], check=True)
     os.replace(tmp, lib)
     for o in objs:
         o.unlink(missing_ok=True)

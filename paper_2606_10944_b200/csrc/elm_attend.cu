@@ -17,7 +17,8 @@
 namespace elm {
 
 // ---------------------------------------------------------------------------------------------
-// Stage gather: Kc, Vc [problems][n_core][d] in the input dtype, bias [problems][n_core] fp32
+// Stage gather: Kc, Vc [problems][n_core][d] in the input dtype, bias [problems][n_core] in the arithmetic type
+// (fp64 in the deterministic mode, so that the weights enter the logits at full precision there)
 // ---------------------------------------------------------------------------------------------
 // E4M3 bytes as the numbers they encode (every E4M3 value is a bf16 value)
 __device__ __forceinline__ __nv_bfloat16 widen_e4m3(unsigned char b)
@@ -54,13 +55,16 @@ int widen_e4m3(const void *src, void *dst_bf16, int64_t count, cudaStream_t st)
     return cuda_status(cudaGetLastError());
 }
 
-template <typename Tin, typename Tsrc = Tin>
+__device__ __forceinline__ float log2_as(float w, float) { return log2f(w); }
+__device__ __forceinline__ double log2_as(float w, double) { return log2((double)w); }
+
+template <typename Tin, typename Tsrc, typename Tb>
 __global__ void __launch_bounds__(256) gather_kernel(const Tsrc *__restrict__ K,
                                                      const Tsrc *__restrict__ V,
                                                      const int32_t *__restrict__ idx,
                                                      const float *__restrict__ w, int64_t n, int d,
                                                      int n_core, Tin *__restrict__ Kc,
-                                                     Tin *__restrict__ Vc, float *__restrict__ bias,
+                                                     Tin *__restrict__ Vc, Tb *__restrict__ bias,
                                                      int *__restrict__ status)
 {
     const int p = blockIdx.y;
@@ -76,7 +80,7 @@ __global__ void __launch_bounds__(256) gather_kernel(const Tsrc *__restrict__ K,
         kd[e] = gather_elt(ks, e);
         vd[e] = gather_elt(vs, e);
     }
-    if (lane == 0) bias[(int64_t)p * n_core + c] = log2f(w[(int64_t)p * n_core + c]);
+    if (lane == 0) bias[(int64_t)p * n_core + c] = log2_as(w[(int64_t)p * n_core + c], Tb());
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -87,7 +91,7 @@ template <typename Tin, typename T, int D>
 __global__ void __launch_bounds__(128) attend_simt_kernel(const Tin *__restrict__ Q,
                                                           const Tin *__restrict__ Kc,
                                                           const Tin *__restrict__ Vc,
-                                                          const float *__restrict__ bias,
+                                                          const T *__restrict__ bias,
                                                           Tin *__restrict__ O, int q_heads,
                                                           int kv_heads, int64_t n_q, int n_core,
                                                           int64_t q_row0, int64_t n_q_total, int tail_start,
@@ -116,7 +120,7 @@ __global__ void __launch_bounds__(128) attend_simt_kernel(const Tin *__restrict_
     const Tin *Qp = Q + ((int64_t)bh * n_q_total + q_row0) * D;
     const Tin *Kp = Kc + prob * n_core * D;
     const Tin *Vp = Vc + prob * n_core * D;
-    const float *bp = bias + prob * n_core;
+    const T *bp = bias + prob * n_core;
     const T scale = (T)(1.4426950408889634 / sqrt((double)D));
 
     for (int e = tid; e < BM * D; e += 128) {
@@ -235,7 +239,7 @@ AttendLayout attend_layout(const elm_params *p, int32_t n_core)
     const size_t ges = p->dtype == ELM_E4M3 ? 2 : es;
     L.Kc = take(problems * n_pad * p->d * ges);
     L.Vc = take(problems * n_pad * p->d * ges);
-    L.bias = take(problems * n_pad * 4);
+    L.bias = take(problems * n_pad * 8);
     L.bx = take(problems * n_pad * 32);
     L.flags = take((problems + 1) * 4);
     L.qwide = take(p->dtype == ELM_E4M3 && p->precision == ELM_PREC_FP64_DET
@@ -245,7 +249,7 @@ AttendLayout attend_layout(const elm_params *p, int32_t n_core)
 }
 
 template <typename Tin, typename T, int D>
-static int launch_attend_simt(const Tin *Q, const Tin *Kc, const Tin *Vc, const float *bias, Tin *O,
+static int launch_attend_simt(const Tin *Q, const Tin *Kc, const Tin *Vc, const T *bias, Tin *O,
                               const elm_params *p, int n_core, cudaStream_t st, const AttendWindow &win = AttendWindow())
 {
     constexpr int BM = 64, BN = 32;
@@ -270,13 +274,13 @@ static int attend_impl(const Tin *Q, const Tsrc *K, const Tsrc *V, const int32_t
     const AttendLayout L = attend_layout(p, n_core);
     Tin *Kc = reinterpret_cast<Tin *>(ws + L.Kc);
     Tin *Vc = reinterpret_cast<Tin *>(ws + L.Vc);
-    float *bias = reinterpret_cast<float *>(ws + L.bias);
+    T *bias = reinterpret_cast<T *>(ws + L.bias);
     const int problems = p->batch * p->kv_heads;
     {
         StageTimer t(ELM_STAGE_GATHER, st, 1);
         // this path has no bounded waits: its status word reads 0
         ELM_CUDA_TRY(cudaMemsetAsync(ws + L.flags, 0, sizeof(int) * (size_t)(problems + 1), st));
-        gather_kernel<Tin, Tsrc><<<dim3((unsigned)((n_core + 7) / 8), (unsigned)problems), 256, 0, st>>>(
+        gather_kernel<Tin, Tsrc, T><<<dim3((unsigned)((n_core + 7) / 8), (unsigned)problems), 256, 0, st>>>(
             K, V, idx, w, p->n_kv, p->d, n_core, Kc, Vc, bias, reinterpret_cast<int *>(ws + L.flags) + problems);
         count_launches(1);
         ELM_CUDA_TRY(cudaGetLastError());
@@ -329,11 +333,11 @@ static int attend_enqueue_untimed(const Tin *Q, const Tin *K, const Tin *V, cons
     const AttendLayout L = attend_layout(p, n_core);
     Tin *Kc = reinterpret_cast<Tin *>(scratch + L.Kc);
     Tin *Vc = reinterpret_cast<Tin *>(scratch + L.Vc);
-    float *bias = reinterpret_cast<float *>(scratch + L.bias);
+    T *bias = reinterpret_cast<T *>(scratch + L.bias);
     const int problems = p->batch * p->kv_heads;
     // this path has no bounded waits: its status word reads 0
     ELM_CUDA_TRY(cudaMemsetAsync(scratch + L.flags, 0, sizeof(int) * (size_t)(problems + 1), st));
-    gather_kernel<Tin><<<dim3((unsigned)((n_core + 7) / 8), (unsigned)problems), 256, 0, st>>>(
+    gather_kernel<Tin, Tin, T><<<dim3((unsigned)((n_core + 7) / 8), (unsigned)problems), 256, 0, st>>>(
         K, V, idx, w, p->n_kv, p->d, n_core, Kc, Vc, bias, reinterpret_cast<int *>(scratch + L.flags) + problems);
     count_launches(1);
     ELM_CUDA_TRY(cudaGetLastError());

@@ -48,7 +48,8 @@ template <typename Tin, int D, int G>
 __global__ void __launch_bounds__(DEC_WARPS * 32)
 decode_partial_kernel(const Tin *__restrict__ Q, const Tin *__restrict__ K, const Tin *__restrict__ V,
                       const int32_t *__restrict__ idx, const float *__restrict__ w, int64_t n, int n_core, int q_heads,
-                      int kv_heads, int n_q, int groups /* live query vectors <= G */, int chunk, float *__restrict__ part)
+                      int kv_heads, int n_q, int groups /* live query vectors <= G */, int chunk, float *__restrict__ part,
+                      int *__restrict__ status)
 {
     constexpr int DPL = D / 32;
     __shared__ float sm_o[DEC_WARPS][G][D];
@@ -92,7 +93,7 @@ decode_partial_kernel(const Tin *__restrict__ Q, const Tin *__restrict__ K, cons
         myrow = 0;
         mylw = 0.f;
         if (lane < DEC_UNR && e0 + lane < c1) {
-            myrow = __ldg(ip + e0 + lane);
+            myrow = (int32_t)checked_row(__ldg(ip + e0 + lane), n, status);
             mylw = log2f(__ldg(wp + e0 + lane));
         }
     };
@@ -185,12 +186,12 @@ __global__ void __launch_bounds__(D) decode_merge_kernel(const float *__restrict
 
 template <typename Tin, int D, int G>
 int launch_decode(const Tin *Q, const Tin *K, const Tin *V, const int32_t *idx, const float *w, int n_core,
-                  const elm_params *p, Tin *O, float *part, int splits, int groups, cudaStream_t st)
+                  const elm_params *p, Tin *O, float *part, int *status, int splits, int groups, cudaStream_t st)
 {
     const int problems = p->batch * p->kv_heads;
     const int chunk = (n_core + splits - 1) / splits;
     decode_partial_kernel<Tin, D, G><<<dim3((unsigned)splits, (unsigned)problems), DEC_WARPS * 32, 0, st>>>(
-        Q, K, V, idx, w, p->n_kv, n_core, p->q_heads, p->kv_heads, p->n_q, groups, chunk, part);
+        Q, K, V, idx, w, p->n_kv, n_core, p->q_heads, p->kv_heads, p->n_q, groups, chunk, part, status);
     decode_merge_kernel<Tin, D, G><<<dim3((unsigned)groups, (unsigned)problems), D, 0, st>>>(part, splits, p->q_heads,
                                                                                             p->kv_heads, p->n_q, O);
     count_launches(2);
@@ -199,12 +200,12 @@ int launch_decode(const Tin *Q, const Tin *K, const Tin *V, const int32_t *idx, 
 
 template <typename Tin, int D>
 int dispatch_decode(const Tin *Q, const Tin *K, const Tin *V, const int32_t *idx, const float *w, int n_core,
-                    const elm_params *p, Tin *O, float *part, int splits, int groups, cudaStream_t st)
+                    const elm_params *p, Tin *O, float *part, int *status, int splits, int groups, cudaStream_t st)
 {
-    if (groups <= 1) return launch_decode<Tin, D, 1>(Q, K, V, idx, w, n_core, p, O, part, splits, groups, st);
-    if (groups <= 2) return launch_decode<Tin, D, 2>(Q, K, V, idx, w, n_core, p, O, part, splits, groups, st);
-    if (groups <= 4) return launch_decode<Tin, D, 4>(Q, K, V, idx, w, n_core, p, O, part, splits, groups, st);
-    return launch_decode<Tin, D, 8>(Q, K, V, idx, w, n_core, p, O, part, splits, groups, st);
+    if (groups <= 1) return launch_decode<Tin, D, 1>(Q, K, V, idx, w, n_core, p, O, part, status, splits, groups, st);
+    if (groups <= 2) return launch_decode<Tin, D, 2>(Q, K, V, idx, w, n_core, p, O, part, status, splits, groups, st);
+    if (groups <= 4) return launch_decode<Tin, D, 4>(Q, K, V, idx, w, n_core, p, O, part, status, splits, groups, st);
+    return launch_decode<Tin, D, 8>(Q, K, V, idx, w, n_core, p, O, part, status, splits, groups, st);
 }
 
 }  // namespace
@@ -236,18 +237,19 @@ int attend_decode(const void *Q, const void *K, const void *V, const int32_t *id
     if (splits > 256) splits = 256;
     if (splits < 1) return ELM_ERR_WORKSPACE;
     float *part = reinterpret_cast<float *>(ws + L.Kc);
+    int *status = reinterpret_cast<int *>(ws + L.flags) + problems;
     StageTimer t(timed ? ELM_STAGE_ATTEND : -1, st, 2);
     // this path has no bounded waits: its status word reads 0
     ELM_CUDA_TRY(cudaMemsetAsync(ws + L.flags, 0, sizeof(int) * (size_t)(problems + 1), st));
     if (p->dtype == ELM_F32) {
         const float *q = (const float *)Q, *k = (const float *)K, *v = (const float *)V;
-        return p->d == 64 ? dispatch_decode<float, 64>(q, k, v, idx, w, n_core, p, (float *)O, part, splits, groups, st)
-                          : dispatch_decode<float, 128>(q, k, v, idx, w, n_core, p, (float *)O, part, splits, groups, st);
+        return p->d == 64 ? dispatch_decode<float, 64>(q, k, v, idx, w, n_core, p, (float *)O, part, status, splits, groups, st)
+                          : dispatch_decode<float, 128>(q, k, v, idx, w, n_core, p, (float *)O, part, status, splits, groups, st);
     }
     typedef __nv_bfloat16 bf;
     const bf *q = (const bf *)Q, *k = (const bf *)K, *v = (const bf *)V;
-    return p->d == 64 ? dispatch_decode<bf, 64>(q, k, v, idx, w, n_core, p, (bf *)O, part, splits, groups, st)
-                      : dispatch_decode<bf, 128>(q, k, v, idx, w, n_core, p, (bf *)O, part, splits, groups, st);
+    return p->d == 64 ? dispatch_decode<bf, 64>(q, k, v, idx, w, n_core, p, (bf *)O, part, status, splits, groups, st)
+                      : dispatch_decode<bf, 128>(q, k, v, idx, w, n_core, p, (bf *)O, part, status, splits, groups, st);
 }
 
 }  // namespace elm

@@ -1948,6 +1948,22 @@ extern "C" int elm_stream_step(elm_stream *s, const void *Q_t, const void *K, co
                : stream_step_impl<bf, float>(s, (const bf *)Q_t, (const bf *)K, (const bf *)V, params, (bf *)O_t, ws, st);
 }
 
+extern "C" int elm_stream_steps(elm_stream *s, int32_t n_tokens, const void *Q_T, const void *K, const void *V,
+                                const elm_params *params, void *O_T, void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (!s || !params) return ELM_ERR_NULL;
+    if (n_tokens < 0) return ELM_ERR_SHAPE;
+    if (n_tokens > 0 && (!Q_T || !O_T)) return ELM_ERR_NULL;
+    const size_t per_token = (size_t)params->batch * params->q_heads * params->d * elm::elt_bytes(params->dtype);
+    if (per_token & 15) return ELM_ERR_ALIGN;
+    for (int32_t i = 0; i < n_tokens; ++i) {
+        const int rc = elm_stream_step(s, (const unsigned char *)Q_T + (size_t)i * per_token, K, V, params,
+                                       (unsigned char *)O_T + (size_t)i * per_token, workspace, workspace_bytes, stream);
+        if (rc != ELM_OK) return rc;
+    }
+    return ELM_OK;
+}
+
 extern "C" int elm_stream_cache(const elm_stream *s, const elm_params *params, int32_t *idx_out, float *w_out,
                                 int32_t *count_host, void *workspace, size_t workspace_bytes, void *stream)
 {

@@ -257,3 +257,21 @@ def test_stream_with_tokens_unknown_at_init_tracks_vmax():
     assert max_rel_err(got[0, 0, :64], ref) <= 2e-6                       # the first 4 n_out tokens are exact
     cidx, _ = st.cache()
     assert cidx.shape[-1] < 6 * 16 and len(set(cidx[0, 0].cpu().tolist())) == cidx.shape[-1]
+
+
+def test_stream_steps_in_one_call_equal_single_steps():
+    """elm_stream_steps enqueues what the same number of elm_stream_step calls would: identical outputs and cache."""
+    wl, log2_nout, n, mbar, rep = STREAM_CASES["lowrank_bf16_nout16_601_gqa_subsample"]
+    wl = wl.scaled(n=n, n_q=n, q_heads=wl.kv_heads * rep)
+    Q, K, V = generate(wl, seed=31, want_q=True)
+    Qd, Kd, Vd = Q.cuda(), K.cuda(), V.cuda()
+    a = elm.Stream(Kd, Vd, wl.q_heads, log2_nout, mbar, seed=11, precision="fp32")
+    one = torch.stack([a.step(Qd[:, :, t:t + 1, :].contiguous()) for t in range(n)])          # [T, B, Hq, 1, d]
+    b = elm.Stream(Kd, Vd, wl.q_heads, log2_nout, mbar, seed=11, precision="fp32")
+    q_T = Qd.permute(2, 0, 1, 3).unsqueeze(3).contiguous()                                     # [T, B, Hq, 1, d]
+    many = torch.cat([b.steps(q_T[:250]), b.steps(q_T[250:])])
+    torch.cuda.synchronize()
+    assert torch.equal(one, many)
+    ia, wa = a.cache()
+    ib, wb = b.cache()
+    assert torch.equal(ia, ib) and torch.equal(wa, wb)

@@ -59,7 +59,11 @@ def test_cfg5_full_size_fp32_mode_sampled_parity(cfg5):
     ref_pipe = oracle.wtd_attention_batched(Qs, Kf[None], Vf[None], ref_idx[None], ref_w[None])
     e_gpu, e_ref = e_max(Og, exact), e_max(ref_pipe, exact)
     print(f"[cfg5 full size] E_max on sampled rows: gpu {e_gpu:.4e} oracle {e_ref:.4e}")
-    assert e_gpu <= 1.05 * e_ref + 2e-2 * np.abs(exact).max()   # + the bf16 output rounding the oracle does not have
+    # the GPU's output is bf16: round the oracle's the same way before comparing (no slack beyond the 5 %)
+    ref_bf16 = torch.from_numpy(ref_pipe).to(torch.bfloat16).double().numpy()
+    e_ref_bf16 = e_max(ref_bf16, exact)
+    print(f"[cfg5 full size] E_max of the oracle pipeline rounded to bf16: {e_ref_bf16:.4e}")
+    assert e_gpu <= 1.05 * max(e_ref, e_ref_bf16)
 
 
 def test_status_words_after_generic_kernels():
