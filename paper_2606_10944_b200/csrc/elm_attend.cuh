@@ -33,6 +33,10 @@ AttendLayout attend_layout(const elm_params *p, int32_t n_core);
 // the smallest death of each block of 128 entries (a block that every row of a tile sees whole takes the
 // unmasked path).  `lse`, if set, receives log2 of each row's softmax denominator (logits in base 2,
 // weights included) at [batch * q_heads][n_q_total].
+//
+// Block lists (with lifetimes, tensor-core path only): when `tile_cnt` is set, pair x of 128-query tiles (rows
+// 256 x ... of every head) streams only the tile_cnt[x] blocks tile_blk[x * tile_cap + 0 ...] of the list; the
+// caller guarantees that every entry some row of the pair sees lies in one of them.
 struct AttendWindow {
     int64_t q_row0 = 0;
     int64_t n_q_total = 0;               // 0: params->n_q
@@ -40,6 +44,12 @@ struct AttendWindow {
     const int32_t *birth = nullptr, *death = nullptr;
     const int32_t *blk_birth = nullptr, *blk_death = nullptr;
     float *lse = nullptr;
+    const int32_t *tile_cnt = nullptr, *tile_blk = nullptr;
+    int32_t tile_cap = 0;
+    // and, since such pairs differ in length, optionally which pairs each of item_ctas persistent CTAs takes: CTA c the
+    // pairs item_tab[c * item_cap + 0 .. item_cnt[c]) (numbered head * pairs per head + x)
+    const int32_t *item_tab = nullptr, *item_cnt = nullptr;
+    int32_t item_cap = 0, item_ctas = 0;
 };
 
 // elm_attend after argument validation

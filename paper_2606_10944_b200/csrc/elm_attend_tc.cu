@@ -36,8 +36,10 @@
 #include <cuda.h>
 #include <cuda_fp8.h>
 #include <math.h>
+#include <stdlib.h>
 
 #include <atomic>
+#include <type_traits>
 
 #include "elm_attend.cuh"
 #include "elm_common.cuh"
@@ -53,15 +55,11 @@ constexpr int NTHREADS = 608;          // 16 softmax warps + TMA producer + two 
 constexpr int TMA_WARP = 16, MMA_WARP = 17;
 constexpr uint32_t TMEM_COLS = 512;
 constexpr float RESCALE_TAU = 8.0f;      // rescale the accumulator only if the max grew by > 2^8
-#ifndef ELM_EMU_PAIRS
-#define ELM_EMU_PAIRS 0
-#endif
-// Of every 16 column pairs, how many take exp2 from the FMA pipe instead of the special-function unit.
-// Measured on cfg5 (same box, alternating): 0: 4.04 ms, 1: 4.06, 2: 4.08, 3: 4.15 ... 4.25, 4: 4.25, 6: 4.26 ... 4.37,
-// 8: 4.35 ... 4.43 - since the kernel became persistent the softmax warps are short of issue slots and
-// latency, not of exp2 throughput, so the default is none.
-constexpr int EMU_PAIRS = ELM_EMU_PAIRS;
+// (Taking a share of the exponentials from the FMA pipe - a cubic for 2^f - instead of the special-function unit
+// was measured on cfg5: none 4.04 ms, 1 pair of 16: 4.06, 2: 4.08, 4: 4.25, 8: 4.35 ... 4.43 - the softmax warps are
+// short of issue slots and latency, not of exp2 throughput, so the kernel does not do it.)
 
+constexpr int EMU_PAIRS = 0;
 using namespace sm100;
 
 struct __align__(8) Barriers {
@@ -90,8 +88,8 @@ template <int D, int QKB = 2> struct Smem {
 };
 
 // ---------------------------------------------------------------------------------------------
-// gather for the tensor-core path: Kc [p][n_pad][D] (zero rows beyond n_core), Vt [p][D][n_pad]
-// (transposed, zero columns beyond n_core), Bx [p][n_pad][16]: log2 w / scale_log2 as three bf16 terms
+// gather for the tensor-core path: Kc [p][n_pad][D] (zero rows beyond n_core), Vt [p][n_pad / 128][D][128]
+// (per block of 128 entries the transposed values, 32 KB in one piece; zero columns beyond n_core), Bx [p][n_pad][16]: log2 w / scale_log2 as three bf16 terms
 // (then zeros), and a per-problem flag that says whether all weights of the problem are equal (then
 // the bias cancels in the ratio).
 // ---------------------------------------------------------------------------------------------
@@ -167,7 +165,7 @@ __global__ void __launch_bounds__(256) gather_tc_kernel(const __nv_bfloat16 *__r
     // transposed write: a warp writes the 64 entries of one dimension e, 128 contiguous bytes
     for (int e = warp; e < D; e += 8) {
         const uint32_t lo = __bfloat16_as_ushort(tile[2 * lane][e]), hi = __bfloat16_as_ushort(tile[2 * lane + 1][e]);
-        *reinterpret_cast<uint32_t *>(Vt + ((int64_t)p * D + e) * n_pad + c0 + 2 * lane) = lo | (hi << 16);
+        *reinterpret_cast<uint32_t *>(Vt + (((int64_t)p * (n_pad / 128) + c0 / 128) * D + e) * 128 + (c0 % 128) + 2 * lane) = lo | (hi << 16);
     }
 }
 
@@ -351,7 +349,9 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                  int q_row0, int n_q_total, int tail_start, const int32_t *__restrict__ birth,
                  const int32_t *__restrict__ death, const int32_t *__restrict__ blk_birth,
                  const int32_t *__restrict__ blk_death, float *__restrict__ lse, int *__restrict__ status,
-                 int extra_arrivals, unsigned long long wait_limit_ns)
+                 int extra_arrivals, unsigned long long wait_limit_ns, const int32_t *__restrict__ tile_cnt,
+                 const int32_t *__restrict__ tile_blk, int tile_cap, const int32_t *__restrict__ item_tab,
+                 const int32_t *__restrict__ item_cnt, int item_cap)
 {
     // every wait of this kernel is bounded by the limit the host passes (2 s unless a test shortened it)
     auto mbar_wait = [wait_limit_ns](uint64_t *b, uint32_t parity) { return sm100::mbar_wait(b, parity, wait_limit_ns); };
@@ -366,10 +366,44 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
     const int nblk = n_pad / BN;
     // Persistent CTA: work item k of this CTA is pair-of-query-tiles number blockIdx.x + k gridDim.x,
     // numbered with the head slowest, so that at any time the CTAs share one head's coreset in L2.
-    const int n_items = (n_items_total - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
-    const int total = n_items * nblk;                              // coreset blocks this CTA streams, over all items
-    auto item_bh = [&](int k) { return ((int)blockIdx.x + k * (int)gridDim.x) / tiles_x; };
-    auto item_q0 = [&](int k) { return (((int)blockIdx.x + k * (int)gridDim.x) % tiles_x) * (2 * BM); };
+    // (a launch with block lists may also say which items each CTA takes - item_tab[blockIdx.x][0 .. item_cnt[blockIdx.x])
+    // - because its items differ in length)
+    auto item_id = [&](int k) -> int {
+        if constexpr (MASKED) {
+            if (item_tab) return __ldg(item_tab + (int64_t)blockIdx.x * item_cap + k);
+        }
+        return (int)blockIdx.x + k * (int)gridDim.x;
+    };
+    const int n_items = (MASKED && item_tab) ? __ldg(item_cnt + blockIdx.x)
+                                             : (n_items_total - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+    // A launch with block lists (tile_cnt set; lifetimes only): pair number x of every head streams the
+    // tile_cnt[x] blocks tile_blk[x][0 ..] of the list instead of all of them - the list then holds every
+    // entry some row of the launch sees, and each pair visits the blocks that hold entries its own rows see.
+    auto item_nblk = [&](int k) -> int {
+        if constexpr (MASKED) {
+            if (tile_cnt) return __ldg(tile_cnt + item_id(k) % tiles_x);
+        }
+        return nblk;
+    };
+    auto item_blk = [&](int k, int j) -> int {
+        if constexpr (MASKED) {
+            if (tile_cnt) return __ldg(tile_blk + (int64_t)(item_id(k) % tiles_x) * tile_cap + j);
+        }
+        return j;
+    };
+    // coreset blocks this CTA streams, over all items
+    auto count_blocks = [&]() -> int {
+        if constexpr (MASKED) {
+            if (tile_cnt) {
+                int sum = 0;
+                for (int k = 0; k < n_items; ++k) sum += item_nblk(k);
+                return sum;
+            }
+        }
+        return n_items * nblk;
+    };
+    auto item_bh = [&](int k) { return item_id(k) / tiles_x; };
+    auto item_q0 = [&](int k) { return (item_id(k) % tiles_x) * (2 * BM); };
     auto prob_of = [&](int bh) { return (bh / q_heads) * kv_heads + (int)(((int64_t)(bh % q_heads) * kv_heads) / q_heads); };
     // does item k take the bias MMA?  (weights differ, or the last block is only partly filled)
     const bool ragged_end = n_core % BN != 0;
@@ -417,60 +451,128 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                     for (int kh = 0; kh < KH; ++kh)
                         tma_load_3d(smem + SM::OFF_Q + t * SM::Q_TILE + kh * (BM * 128), &mapQ, &bar->q_full, kh * ROW_ELTS, q_row0 + q0 + t * BM, bh);
             };
-            // Blocks are numbered G = k nblk + j along the CTA's whole stream (item k, block j).
-            int flag_item = -1;
-            bool flag_now = false, flag_next = n_items > 0 && item_bias(0);
-            auto load_k = [&](int G) {
-                const int s = G % STAGES, prob = prob_of(item_bh(G / nblk));
-                // the flag of an item is fetched while the item before it streams, off the critical path
-                if (G / nblk != flag_item) {
-                    flag_item = G / nblk;
-                    flag_now = flag_next;
-                    flag_next = flag_item + 1 < n_items && item_bias(flag_item + 1);
-                }
-                const bool with_bias = flag_now;
-                mbar_expect_tx(&bar->k_full[s], SM::K_BLOCK + (with_bias ? SM::X_BLOCK : 0));
-                for (int kh = 0; kh < KH; ++kh)
-                    tma_load_3d(smem + SM::OFF_K + s * SM::K_BLOCK + kh * (BN * 128), &mapK, &bar->k_full[s], kh * ROW_ELTS, (G % nblk) * BN, prob);
-                if (with_bias) tma_load_3d(smem + SM::OFF_X + s * SM::X_BLOCK, &mapX, &bar->k_full[s], 0, (G % nblk) * BN, prob);
-            };
-            auto load_v = [&](int G) {
-                const int s = G % STAGES, prob = prob_of(item_bh(G / nblk));
-                mbar_expect_tx(&bar->v_full[s], SM::V_BLOCK);
-                for (int hh = 0; hh < 2; ++hh)
-                    tma_load_3d(smem + SM::OFF_V + s * SM::V_BLOCK + hh * (D * 128), &mapV, &bar->v_full[s], (G % nblk) * BN + hh * 64, 0, prob);
-            };
             bool ok = true;
-            // The queries of item k may replace those of item k - 1 once every S = Q K^T of item k - 1
-            // has been computed (q_free); they are fetched right after the keys of the item's first block.
-            int next_q = 1, k_loaded = -1;
-            auto feed_q = [&]() {
-                while (ok && next_q < n_items && next_q * nblk <= k_loaded) {
-                    ok = mbar_wait(&bar->q_free, (uint32_t)(next_q - 1) & 1u);
-                    if (ok) load_q(next_q);
-                    ++next_q;
-                }
-            };
-            load_q(0);
-            // The issuer commits "event" i to kv_free[i % 2] after the prologue (i = 0: S = Q K^T of block
-            // 0 issued) and after iteration i - 1 (O += P V of block i - 1 and S = Q K^T of block i issued).
-            // Once event i is complete, K's stage i % 2 (block i) and V's stage (i + 1) % 2 (block i - 1)
-            // have been read, so K(i + 2) and V(i + 1) may overwrite them.
-            for (int G = 0; G < STAGES && G < total; ++G) { load_k(G); load_v(G); k_loaded = G; }
-            feed_q();
-            for (int i = 0; i + 2 < total && ok; ++i) {
-                ok = mbar_wait(&bar->kv_free[i % STAGES], (uint32_t)(i / STAGES) & 1u);
-                if (!ok) break;
-                load_k(i + 2);
-                k_loaded = i + 2;
-                if (i >= 1) load_v(i + 1);
+            if (!MASKED || !tile_cnt) {
+                // (every pair streams the whole list: block G of the stream is block G % nblk of item G / nblk)
+                // Blocks are numbered G = k nblk + j along the CTA's whole stream (item k, block j).
+                const int total = n_items * nblk;
+                int flag_item = -1;
+                bool flag_now = false, flag_next = n_items > 0 && item_bias(0);
+                auto load_k = [&](int G) {
+                    const int s = G % STAGES, prob = prob_of(item_bh(G / nblk));
+                    // the flag of an item is fetched while the item before it streams, off the critical path
+                    if (G / nblk != flag_item) {
+                        flag_item = G / nblk;
+                        flag_now = flag_next;
+                        flag_next = flag_item + 1 < n_items && item_bias(flag_item + 1);
+                    }
+                    const bool with_bias = flag_now;
+                    mbar_expect_tx(&bar->k_full[s], SM::K_BLOCK + (with_bias ? SM::X_BLOCK : 0));
+                    for (int kh = 0; kh < KH; ++kh)
+                        tma_load_3d(smem + SM::OFF_K + s * SM::K_BLOCK + kh * (BN * 128), &mapK, &bar->k_full[s], kh * ROW_ELTS, (G % nblk) * BN, prob);
+                    if (with_bias) tma_load_3d(smem + SM::OFF_X + s * SM::X_BLOCK, &mapX, &bar->k_full[s], 0, (G % nblk) * BN, prob);
+                };
+                auto load_v = [&](int G) {
+                    const int s = G % STAGES, prob = prob_of(item_bh(G / nblk));
+                    mbar_expect_tx(&bar->v_full[s], SM::V_BLOCK);
+                    for (int hh = 0; hh < 2; ++hh)
+                        tma_load_3d(smem + SM::OFF_V + s * SM::V_BLOCK + hh * (D * 128), &mapV, &bar->v_full[s], hh * 64, 0, prob * nblk + G % nblk);
+                };
+                // The queries of item k may replace those of item k - 1 once every S = Q K^T of item k - 1
+                // has been computed (q_free); they are fetched right after the keys of the item's first block.
+                int next_q = 1, k_loaded = -1;
+                auto feed_q = [&]() {
+                    while (ok && next_q < n_items && next_q * nblk <= k_loaded) {
+                        ok = mbar_wait(&bar->q_free, (uint32_t)(next_q - 1) & 1u);
+                        if (ok) load_q(next_q);
+                        ++next_q;
+                    }
+                };
+                load_q(0);
+                // The issuer commits "event" i to kv_free[i % 2] after the prologue (i = 0: S = Q K^T of block
+                // 0 issued) and after iteration i - 1 (O += P V of block i - 1 and S = Q K^T of block i issued).
+                // Once event i is complete, K's stage i % 2 (block i) and V's stage (i + 1) % 2 (block i - 1)
+                // have been read, so K(i + 2) and V(i + 1) may overwrite them.
+                for (int G = 0; G < STAGES && G < total; ++G) { load_k(G); load_v(G); k_loaded = G; }
                 feed_q();
-            }
-            // the last V block: freed by event total - 1
-            if (ok && total > STAGES) {
-                const int i = total - 2;
-                ok = mbar_wait(&bar->kv_free[i % STAGES], (uint32_t)(i / STAGES) & 1u);
-                if (ok) load_v(i + 1);
+                for (int i = 0; i + 2 < total && ok; ++i) {
+                    ok = mbar_wait(&bar->kv_free[i % STAGES], (uint32_t)(i / STAGES) & 1u);
+                    if (!ok) break;
+                    load_k(i + 2);
+                    k_loaded = i + 2;
+                    if (i >= 1) load_v(i + 1);
+                    feed_q();
+                }
+                // the last V block: freed by event total - 1
+                if (ok && total > STAGES) {
+                    const int i = total - 2;
+                    ok = mbar_wait(&bar->kv_free[i % STAGES], (uint32_t)(i / STAGES) & 1u);
+                    if (ok) load_v(i + 1);
+                }
+            } else {
+                // Blocks are numbered G = 0, 1, ... along the CTA's whole stream; a cursor (item k, block j of its
+                // nb) walks it, one for the keys and one for the values, which run a block behind.
+                struct Cursor { int k, j, nb; };
+                const int total = count_blocks();
+                auto cursor_next = [&](Cursor &c) {
+                    if (++c.j == c.nb) { c.j = 0; ++c.k; c.nb = c.k < n_items ? item_nblk(c.k) : 0; }
+                };
+                Cursor kc = {0, 0, n_items > 0 ? item_nblk(0) : 0}, vc = kc;
+                int flag_item = -1;
+                bool flag_now = false, flag_next = n_items > 0 && item_bias(0);
+                auto load_k = [&](int G) {
+                    const int s = G % STAGES, prob = prob_of(item_bh(kc.k)), blk = item_blk(kc.k, kc.j);
+                    // the flag of an item is fetched while the item before it streams, off the critical path
+                    if (kc.k != flag_item) {
+                        flag_item = kc.k;
+                        flag_now = flag_next;
+                        flag_next = flag_item + 1 < n_items && item_bias(flag_item + 1);
+                    }
+                    const bool with_bias = flag_now;
+                    mbar_expect_tx(&bar->k_full[s], SM::K_BLOCK + (with_bias ? SM::X_BLOCK : 0));
+                    for (int kh = 0; kh < KH; ++kh)
+                        tma_load_3d(smem + SM::OFF_K + s * SM::K_BLOCK + kh * (BN * 128), &mapK, &bar->k_full[s], kh * ROW_ELTS, blk * BN, prob);
+                    if (with_bias) tma_load_3d(smem + SM::OFF_X + s * SM::X_BLOCK, &mapX, &bar->k_full[s], 0, blk * BN, prob);
+                    cursor_next(kc);
+                };
+                auto load_v = [&](int G) {
+                    const int s = G % STAGES, prob = prob_of(item_bh(vc.k)), blk = item_blk(vc.k, vc.j);
+                    mbar_expect_tx(&bar->v_full[s], SM::V_BLOCK);
+                    for (int hh = 0; hh < 2; ++hh)
+                        tma_load_3d(smem + SM::OFF_V + s * SM::V_BLOCK + hh * (D * 128), &mapV, &bar->v_full[s], hh * 64, 0, prob * nblk + blk);
+                    cursor_next(vc);
+                };
+                // The queries of item k may replace those of item k - 1 once every S = Q K^T of item k - 1
+                // has been computed (q_free); they are fetched right after the keys of the item's first block
+                // (the key cursor then stands behind that block).
+                int next_q = 1;
+                auto feed_q = [&]() {
+                    while (ok && next_q < n_items && (kc.k > next_q || (kc.k == next_q && kc.j > 0))) {
+                        ok = mbar_wait(&bar->q_free, (uint32_t)(next_q - 1) & 1u);
+                        if (ok) load_q(next_q);
+                        ++next_q;
+                    }
+                };
+                load_q(0);
+                // The issuer commits "event" i to kv_free[i % 2] after the prologue (i = 0: S = Q K^T of block
+                // 0 issued) and after iteration i - 1 (O += P V of block i - 1 and S = Q K^T of block i issued).
+                // Once event i is complete, K's stage i % 2 (block i) and V's stage (i + 1) % 2 (block i - 1)
+                // have been read, so K(i + 2) and V(i + 1) may overwrite them.
+                for (int G = 0; G < STAGES && G < total; ++G) { load_k(G); load_v(G); }
+                feed_q();
+                for (int i = 0; i + 2 < total && ok; ++i) {
+                    ok = mbar_wait(&bar->kv_free[i % STAGES], (uint32_t)(i / STAGES) & 1u);
+                    if (!ok) break;
+                    load_k(i + 2);
+                    if (i >= 1) load_v(i + 1);
+                    feed_q();
+                }
+                // the last V block: freed by event total - 1
+                if (ok && total > STAGES) {
+                    const int i = total - 2;
+                    ok = mbar_wait(&bar->kv_free[i % STAGES], (uint32_t)(i / STAGES) & 1u);
+                    if (ok) load_v(i + 1);
+                }
             }
             if (!ok) { atomicExch(status, 1); bar->abort_flag = 1; }
         }
@@ -516,13 +618,15 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                         mma_ts(tmem + 256 + t * 128, tmem + t * 128 + (hh * 2 + (ks >> 1)) * 32 + (ks & 1) * 8,
                                b0 + (uint64_t)(hh * (D * 128 >> 4) + ks * 2), IDESC_PV, (acc || (hh | ks) != 0) ? 1u : 0u);
             };
+            const int total = count_blocks();
+            int nb = n_items > 0 ? item_nblk(0) : 0;                           // blocks of item k
             bool ok = mbar_wait(&bar->q_full, 0) && mbar_wait(&bar->k_full[0], 0);
             if (ok) {
                 tc_fence_after();
                 const bool b0 = item_bias(0);
                 issue_qk(t, 0, b0);
                 tc_commit(&bar->s_full[t]);
-                if (nblk == 1) tc_commit(&bar->q_free);                        // item 0 needs its queries no more
+                if (nb == 1) tc_commit(&bar->q_free);                          // item 0 needs its queries no more
                 tc_commit(&bar->kv_free[0]);                                   // event 0
             }
             // Iteration G: O += P V of block G, then S = Q K^T of block G + 1 - which may be the first
@@ -530,12 +634,16 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
             int j = 0, k = 0;                                                  // block G = item k, block j
             bool bias_next = n_items > 0 && item_bias(0);                      // of the item block G + 1 belongs to
             bool bias_after = false;
+            int nb_after = 0;                                                  // blocks of item k + 1
             for (int G = 0; G < total && ok; ++G) {
                 const int s = G % STAGES;
                 const bool more = G + 1 < total;
                 const int sn = (G + 1) % STAGES;
-                const bool last = j == nblk - 1;                               // last block of item k
-                if (j == 0) bias_after = k + 1 < n_items && item_bias(k + 1);   // fetched early, used at the item's last block
+                const bool last = j == nb - 1;                                 // last block of item k
+                if (j == 0) {                                                  // fetched early, used at the item's last block
+                    bias_after = k + 1 < n_items && item_bias(k + 1);
+                    nb_after = k + 1 < n_items ? item_nblk(k + 1) : 0;
+                }
                 if (last) bias_next = bias_after;
                 if (more) ok = mbar_wait(&bar->k_full[sn], (uint32_t)((G + 1) / STAGES) & 1u);
                 ok = ok && mbar_wait(&bar->v_full[s], (uint32_t)(G / STAGES) & 1u);
@@ -558,10 +666,10 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                 if (!ok) break;
                 // the logits just issued belong to block j + 1 of item k, or to block 0 of item k + 1
                 const int jn = last ? 0 : j + 1;
-                if (more && jn == nblk - 1) tc_commit(&bar->q_free);
+                if (more && jn == (last ? nb_after : nb) - 1) tc_commit(&bar->q_free);
                 tc_commit(&bar->kv_free[(G + 1) % STAGES]);                    // event G + 1
                 j = jn;
-                if (last) ++k;
+                if (last) { ++k; nb = nb_after; }
             }
             if (!ok) { atomicExch(status, 2); bar->abort_flag = 1; }
         }
@@ -714,7 +822,9 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
             const int64_t life0 = (int64_t)prob_of(bh) * n_pad + cq * 32;     // this thread's first entry of the lifetime arrays
             const int64_t blk0 = (int64_t)prob_of(bh) * nblk;
             float m_ref[2] = {-INFINITY, -INFINITY}, l[2] = {0.f, 0.f};
-            for (int j = 0; j < nblk && ok; ++j, ++G) {
+            const int nb = item_nblk(k);
+            for (int j = 0; j < nb && ok; ++j, ++G) {
+                const int blk = item_blk(k, j);                     // block of the list (j itself unless the launch has block lists)
 #pragma unroll
                 for (int t = 0; t < 2; ++t) {
                     // A row sees the list up to its own entry of the causal tail (if there is one), so
@@ -729,10 +839,10 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                             // lifetimes: the block is seen whole by this warp's 32 rows unless an entry is born
                             // after the first or dies before the last of them
                             const int t_first = q_row0 + q0 + t * BM + (warp & 3) * 32;
-                            special = !(__ldg(blk_birth + blk0 + j) <= t_first && __ldg(blk_death + blk0 + j) > t_first + 31);
+                            special = !(__ldg(blk_birth + blk0 + blk) <= t_first && __ldg(blk_death + blk0 + blk) > t_first + 31);
                             if (special) {
                                 const int t_row = t_first + lane;
-                                const int32_t *bp = birth + life0 + j * BN, *dp = death + life0 + j * BN;
+                                const int32_t *bp = birth + life0 + (int64_t)blk * BN, *dp = death + life0 + (int64_t)blk * BN;
                                 vmask = 0u;
                                 // 32 consecutive entries of each array, 128-byte aligned: vector loads
 #pragma unroll
@@ -746,9 +856,9 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                                 }
                             }
                         } else if (has_tail) {
-                            int valid = n_core - j * BN - cq * 32;
+                            int valid = n_core - blk * BN - cq * 32;
                             const int64_t seen = (int64_t)tail_start + q0 + t * BM + row + 1;
-                            if (seen < n_core) valid = (int)seen - j * BN - cq * 32;
+                            if (seen < n_core) valid = (int)seen - blk * BN - cq * 32;
                             special = __any_sync(0xffffffffu, valid < 32);
                             vmask = valid >= 32 ? 0xffffffffu : (valid <= 0 ? 0u : (1u << valid) - 1u);
                         }
@@ -899,7 +1009,7 @@ static int launch(const __nv_bfloat16 *Q, const __nv_bfloat16 *K, const __nv_bfl
     CUtensorMap mQ, mK, mV, mX;
     if (!make_map(&mQ, Q, D, (uint64_t)n_q_total, (uint64_t)p->batch * p->q_heads, BM) ||
         !make_map(&mK, Kc, D, (uint64_t)n_pad, (uint64_t)problems, BN) ||
-        !make_map(&mV, Vt, (uint64_t)n_pad, D, (uint64_t)problems, D) ||
+        !make_map(&mV, Vt, BN, D, (uint64_t)problems * (uint64_t)(n_pad / BN), D) ||
         !make_map(&mX, Bx, 16, (uint64_t)n_pad, (uint64_t)problems, BN, true))
         return ELM_ERR_CUDA;
     const float scale_log2 = (float)(1.4426950408889634 / sqrt((double)D));
@@ -918,13 +1028,13 @@ static int launch(const __nv_bfloat16 *Q, const __nv_bfloat16 *K, const __nv_bfl
     // one persistent CTA per SM, each taking every gridDim.x-th pair of query tiles
     const int tiles_x = (p->n_q + 2 * BM - 1) / (2 * BM);
     const int64_t items = (int64_t)tiles_x * p->batch * p->q_heads;
-    if (items > 0x7fffffff / 64) return ELM_ERR_SHAPE;
-    const int ctas = (int)(items < sm_count() ? items : sm_count());
+    if (items > 0x7fffffff / 64 || (int64_t)problems * n_pad > 0x7fffffff - 256) return ELM_ERR_SHAPE;
+    const int ctas = win.item_tab ? win.item_ctas : (int)(items < sm_count() ? items : sm_count());
     kern<<<ctas, NTHREADS, Smem<D>::TOTAL, st>>>(mQ, mK, mV, mX, flags, O, p->q_heads, p->kv_heads, p->n_q,
                                                  n_core, n_pad, scale_log2, tiles_x, (int)items, (int)win.q_row0,
                                                  (int)n_q_total, win.tail_start, win.birth, win.death, win.blk_birth,
                                                  win.blk_death, win.lse, status, g_debug_extra_arrivals.exchange(0),
-                                                 g_debug_wait_limit_ns.load());
+                                                 g_debug_wait_limit_ns.load(), win.tile_cnt, win.tile_blk, win.tile_cap, win.item_tab, win.item_cnt, win.item_cap);
     count_launches(1);
     return cuda_status(cudaGetLastError());
 }
@@ -945,7 +1055,7 @@ static int launch_e4m3(const unsigned char *Q, const unsigned char *K, const uns
     CUtensorMap mQ, mK, mV, mX;
     if (!make_map(&mQ, Q, D, (uint64_t)p->n_q, (uint64_t)p->batch * p->q_heads, BM, false, true) ||
         !make_map(&mK, Kc, D, (uint64_t)n_pad, (uint64_t)problems, BN, false, true) ||
-        !make_map(&mV, Vt, (uint64_t)n_pad, D, (uint64_t)problems, D) ||
+        !make_map(&mV, Vt, BN, D, (uint64_t)problems * (uint64_t)(n_pad / BN), D) ||
         !make_map(&mX, Bx, 16, (uint64_t)n_pad, (uint64_t)problems, BN, true))
         return ELM_ERR_CUDA;
     const float scale_log2 = (float)(1.4426950408889634 / sqrt((double)D));
@@ -968,7 +1078,7 @@ static int launch_e4m3(const unsigned char *Q, const unsigned char *K, const uns
     kern<<<ctas, NTHREADS, Smem<D, 1>::TOTAL, st>>>(mQ, mK, mV, mX, flags, O, p->q_heads, p->kv_heads, p->n_q, n_core, n_pad,
                                                     scale_log2, tiles_x, (int)items, 0, p->n_q, 0x7fffffff, nullptr, nullptr, nullptr,
                                                     nullptr, nullptr, status, g_debug_extra_arrivals.exchange(0),
-                                                    g_debug_wait_limit_ns.load());
+                                                    g_debug_wait_limit_ns.load(), nullptr, nullptr, 0, nullptr, nullptr, 0);
     count_launches(1);
     return cuda_status(cudaGetLastError());
 }

@@ -11,6 +11,7 @@
 
 #include "elm_attend.cuh"
 #include "elm_common.cuh"
+#include "elm_prefill_round.cuh"
 #include "elm_compress.cuh"
 #include "elm_walk.cuh"
 
@@ -761,28 +762,10 @@ struct ExpressLayout {
     // the softmax denominators (rounds with Subsample: the tokens that were not kept are merged in afterwards)
     size_t levels, ep_idx, ep_w, ep_birth, ep_death, ep_blk, ws_attend, ep_cap, ep_pad, ep_stride, ws_attend_stride, lse;
     int n_levels;
+    // prefill, rounds that take one attention launch: the round's universe and tile table (elm_prefill_round.cuh)
+    size_t round;
+    RoundBufferLayout rbl;
 };
-// Geometry of round r of an Express run (thinning factor m = 2r): Compress2 depth q = min(m, mbar), one
-// point kept per 2^wlog tokens (Subsample, when m > mbar), `seg` tokens and len0 kept points per sibling
-// segment, s0 kept points per level-0 Halve call.
-struct RoundGeom {
-    int m, q, wlog;
-    bool sub;
-    int64_t seg, len0, s0;
-};
-static RoundGeom round_geom(const elm_params *p, int mbar, int r)
-{
-    RoundGeom g;
-    const int64_t n_out = (int64_t)1 << p->log2_nout;
-    g.m = 2 * r;
-    g.q = g.m < mbar ? g.m : mbar;
-    g.sub = g.m > mbar;
-    g.wlog = g.m - g.q;
-    g.seg = n_out << g.m;
-    g.len0 = n_out << g.q;
-    g.s0 = g.q >= 1 ? (n_out << 2) >> g.q : g.len0;        // q = 0: no Halve call, S_0 only grows
-    return g;
-}
 // Tokens per attention launch of the prefill: windows of about 512 tokens (whole strata, at most a segment).
 static int64_t prefill_window(const RoundGeom &g)
 {
@@ -891,6 +874,8 @@ static ExpressLayout express_layout(const elm_params *p, int mbar = 0, bool pref
     L.levels = L.ep_idx = L.ep_w = L.ep_birth = L.ep_death = L.ep_blk = L.ws_attend = L.ep_cap = L.ep_pad = L.ep_stride = 0;
     L.ws_attend_stride = L.lse = 0;
     L.n_levels = 0;
+    L.round = 0;
+    L.rbl = RoundBufferLayout();
     if (prefill) {
         L.n_levels = mbar < 30 ? mbar : 30;
         L.levels = take((size_t)L.n_levels * BH * n * 4);
@@ -906,6 +891,10 @@ static ExpressLayout express_layout(const elm_params *p, int mbar = 0, bool pref
         L.lse = take((size_t)p->batch * p->q_heads * n * 4);
         L.ws_attend_stride = align_up(attend_layout(p, (int32_t)L.ep_cap).total, 256);
         L.ws_attend = take(EXPRESS_LANES * L.ws_attend_stride);
+        int R = 0;
+        for (size_t v = n_out; v < n; v *= 4) ++R;
+        L.rbl = round_buffer_layout(p, mbar, R);
+        L.round = take(L.rbl.total);
     }
     L.total = off;
     return L;
@@ -1092,6 +1081,26 @@ static PrefillLane prefill_lane(const ExpressLayout &L, unsigned char *ws, int B
     return pl;
 }
 
+static RoundBuffers round_buffers(const ExpressLayout &L, unsigned char *ws, int BH, int64_t n_univ)
+{
+    unsigned char *rw = ws + L.round;
+    RoundBuffers rb;
+    rb.idx = reinterpret_cast<int32_t *>(rw + L.rbl.idx);
+    rb.w = reinterpret_cast<float *>(rw + L.rbl.w);
+    rb.birth = reinterpret_cast<int32_t *>(rw + L.rbl.birth);
+    rb.death = reinterpret_cast<int32_t *>(rw + L.rbl.death);
+    rb.blk_birth = reinterpret_cast<int32_t *>(rw + L.rbl.blk);
+    rb.blk_death = rb.blk_birth + (size_t)BH * (n_univ / 128);
+    rb.tile_cnt = reinterpret_cast<int32_t *>(rw + L.rbl.tile_cnt);
+    rb.tile_blk = reinterpret_cast<int32_t *>(rw + L.rbl.tile_blk);
+    rb.item_tab = reinterpret_cast<int32_t *>(rw + L.rbl.item_tab);
+    rb.item_cnt = reinterpret_cast<int32_t *>(rw + L.rbl.item_cnt);
+    rb.item_cap = L.rbl.item_cap;
+    rb.item_ctas = L.rbl.item_ctas;
+    rb.ws_attend = rw + L.rbl.ws_attend;
+    return rb;
+}
+
 // The exact start of Thinformer Express (Algorithm 5) in prefill: token t < rows attends over the tokens 0 .. t.
 static int express_attend_start(const void *Q, const void *K, const void *V, void *O, const elm_params *p, const ExpressLayout &L,
                                 unsigned char *ws, int rows, cudaStream_t st)
@@ -1112,6 +1121,11 @@ static int express_attend_start(const void *Q, const void *K, const void *V, voi
     win.q_row0 = 0;
     win.n_q_total = p->n_kv;
     win.tail_start = 0;                  // the whole list is the causal tail
+    if (L.rbl.total) {
+        // (the run has the tile table of the one-launch rounds: pairs of query tiles stop at their own last token)
+        const int rc = causal_tile_table(rows, p->batch * p->q_heads, round_buffers(L, ws, BH, 0), win, st);
+        if (rc != ELM_OK) return rc;
+    }
     return attend_enqueue(Q, K, V, pl.idx, pl.w, rows, &pe, O, pl.ws_attend, st, win);
 }
 
@@ -1249,8 +1263,16 @@ static int express_impl(const Tin *K, const Tin *V, const elm_params *p, int mba
             // The launches are independent given the round's lists; they are dealt to EXPRESS_LANES
             // streams (each with its own list buffers) between two events.
             const RoundGeom g = round_geom(p, mbar, r);
-            const int64_t W = prefill_window(g), Wg = W >> g.wlog;
             float *lse = g.sub ? reinterpret_cast<float *>(ws + L.lse) : nullptr;
+            RoundUniverse u;
+            if (round_universe(p, mbar, r, u)) {
+                // one launch for the round: every entry the round's tokens ever see is gathered once, each pair of
+                // query tiles streams the blocks its own tokens see
+                const RoundBuffers rb = round_buffers(L, ws, BH, u.n_univ);
+                const int rc = express_attend_round(Q, K, V, O, p, u, E, levels, (size_t)BH * n, listA, n, rb, lse, st);
+                if (rc != ELM_OK) return rc;
+            } else {
+            const int64_t W = prefill_window(g), Wg = W >> g.wlog;
             ELM_CUDA_TRY(cudaEventRecord(fork, st));
             for (int i = 0; i < EXPRESS_LANES; ++i) ELM_CUDA_TRY(cudaStreamWaitEvent(side[i], fork, 0));
             int launch = 0;
@@ -1267,6 +1289,7 @@ static int express_impl(const Tin *K, const Tin *V, const elm_params *p, int mba
             for (int i = 0; i < EXPRESS_LANES; ++i) {
                 ELM_CUDA_TRY(cudaEventRecord(join[i], side[i]));
                 ELM_CUDA_TRY(cudaStreamWaitEvent(st, join[i], 0));             // the halvings overwrite E
+            }
             }
             if (g.sub) {
                 // the tokens Subsample dropped still attend to themselves

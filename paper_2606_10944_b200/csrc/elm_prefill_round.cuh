@@ -1,0 +1,125 @@
+// Thinformer Express (Algorithm 5) in prefill, one attention launch per round: geometry of a round and the
+// list ("universe") of every cache entry the round's tokens ever see.
+#pragma once
+#include <stddef.h>
+#include <stdint.h>
+
+#include <cuda_runtime.h>
+
+#include "../../include/elm.h"
+
+namespace elm {
+
+// Geometry of round r of an Express run (thinning factor m = 2r): Compress2 depth q = min(m, mbar), one
+// point kept per 2^wlog tokens (Subsample, when m > mbar), `seg` tokens and len0 kept points per sibling
+// segment, s0 kept points per level-0 Halve call.
+struct RoundGeom {
+    int m, q, wlog;
+    bool sub;
+    int64_t seg, len0, s0;
+};
+inline RoundGeom round_geom(const elm_params *p, int mbar, int r)
+{
+    RoundGeom g;
+    const int64_t n_out = (int64_t)1 << p->log2_nout;
+    g.m = 2 * r;
+    g.q = g.m < mbar ? g.m : mbar;
+    g.sub = g.m > mbar;
+    g.wlog = g.m - g.q;
+    g.seg = n_out << g.m;
+    g.len0 = n_out << g.q;
+    g.s0 = g.q >= 1 ? (n_out << 2) >> g.q : g.len0;        // q = 0: no Halve call, S_0 only grows
+    return g;
+}
+
+// The universe of a round, per attention problem: every entry of E and of the three siblings' point lists,
+// laid out as
+//   [0, EP)                          E and, behind it, the three siblings' outputs (4 n_out entries, padded)
+//   EP + jj SP + off(i) ...          sibling jj, piece i: i = 0 its kept points (the entries of S_0), 1 <= i < q
+//                                    the outputs of its level-(i-1) Halve calls (the entries of S_i),
+//                                    len0 / 2^i entries each, every piece padded to a multiple of 128,
+//                                    off(i) = sum over i' < i of the padded lengths
+// so that a block of 128 entries never mixes pieces.  Each entry carries the span of tokens that see it
+// (comment at round_universe_kernel); a pair of 128-query tiles streams only the blocks that hold entries
+// some of its 256 tokens see (tile_blocks).
+struct RoundUniverse {
+    int q, wlog, sub;
+    int64_t n_out, len0, s0, seg;
+    int64_t EP, SP, n_univ;
+    int tiles, cap;                  // pairs of query tiles in the round; most blocks any of them streams
+    int64_t blocks_total;            // blocks streamed by all pairs of one head
+};
+__host__ __device__ inline int64_t round_pad128(int64_t x) { return (x + 127) / 128 * 128; }
+__host__ __device__ inline int64_t round_piece_off(const RoundUniverse &u, int i)
+{
+    int64_t off = 0;
+    for (int k = 0; k < i; ++k) off += round_pad128(u.len0 >> k);
+    return off;
+}
+// Blocks of the universe that tile pair `tl` (tokens seg + 256 tl ... of every head) streams; returns their
+// number, writes them to out[] if out is not null.  With G = the number of the sibling's kept points that
+// have arrived, the pair's tokens live through G in [G0, G1]:
+//   E and the finished siblings, plus the sibling's own output once G reaches len0 (rounds with Subsample:
+//   the last kept point may come before the sibling's last token),
+//   of S_i, 1 <= i < q, the outputs of level-(i-1) calls c_lo .. c_end - 1: call c (u entries) exists from
+//   G = (c + 1) A, A = s0 4^(i-1), until the level-i call that consumes it completes at G = (c / 4 + 1) 4 A,
+//   of S_0 the kept points from the start of the running level-0 call up to the pair's last token.
+__host__ __device__ inline int tile_blocks(const RoundUniverse &u, int tl, int32_t *out)
+{
+    const int64_t t_all = (int64_t)tl * 256;
+    const int64_t jj = t_all / u.seg, t_rel = t_all % u.seg;
+    const int64_t G0 = t_rel >> u.wlog, G1 = ((t_rel + 255) >> u.wlog) + 1;
+    int n = 0;
+    auto run = [&](int64_t a, int64_t b) {
+        if (b <= a) return;
+        for (int64_t blk = a / 128; blk <= (b - 1) / 128; ++blk) {
+            if (out) out[n] = (int32_t)blk;
+            ++n;
+        }
+    };
+    run(0, (1 + jj) * u.n_out + ((u.q >= 1 && u.sub && G1 >= u.len0) ? u.n_out : 0));
+    const int64_t base = u.EP + jj * u.SP;
+    for (int i = u.q - 1; i >= 1; --i) {
+        const int64_t A = u.s0 << (2 * (i - 1)), unit = (u.s0 << (i - 1)) >> 1;
+        const int64_t c_lo = 4 * (G0 / (4 * A)), c_end = G1 / A;
+        const int64_t b0 = base + round_piece_off(u, i);
+        run(b0 + c_lo * unit, b0 + c_end * unit);
+    }
+    const int64_t g_lo = u.q >= 1 ? (G0 / u.s0) * u.s0 : 0;
+    run(base + g_lo, base + G1);
+    return n;
+}
+
+// Does round r of the prefill take the one-launch form?  (bf16 inputs in fp32 mode - the tensor-core attention
+// kernel - and segments that are whole pairs of query tiles.)  Fills `u` if so.
+bool round_universe(const elm_params *p, int mbar, int r, RoundUniverse &u);
+
+// Device buffers of the one-launch form (sized by round_buffer_bytes for the largest universe of the run)
+struct RoundBuffers {
+    int32_t *idx, *birth, *death, *blk_birth, *blk_death, *tile_cnt, *tile_blk;
+    int32_t *item_tab, *item_cnt;        // [item_ctas][item_cap], [item_ctas]: the pairs each persistent CTA takes
+    int item_cap, item_ctas;
+    float *w;
+    unsigned char *ws_attend;
+};
+struct RoundBufferLayout {
+    size_t idx, w, birth, death, blk, tile_cnt, tile_blk, item_tab, item_cnt, ws_attend, total;
+    int item_cap, item_ctas;
+};
+// Largest universe / tile table over the rounds of the run that take the one-launch form (total = 0: none does)
+RoundBufferLayout round_buffer_layout(const elm_params *p, int mbar, int rounds);
+
+// Causal attention over the first `rows` tokens of each of `heads` heads (the exact start): fills the tile table so
+// that a pair of query tiles streams the list only up to its own last token, deals the pairs to the CTAs by
+// length, and points `win` at both.
+struct AttendWindow;
+int causal_tile_table(int rows, int heads, const RoundBuffers &rb, AttendWindow &win, cudaStream_t st);
+
+// Attention of the round's 3 seg tokens over the universe: builds the universe from E (stride `stride`
+// per problem), the level lists (`levels` + (i - 1) level_stride: outputs of level i - 1) and the kept
+// points (`kept`), the tile table, then one gather and one attention launch on `st`.
+int express_attend_round(const void *Q, const void *K, const void *V, void *O, const elm_params *p, const RoundUniverse &u,
+                         const int32_t *E, const int32_t *levels, size_t level_stride, const int32_t *kept, int64_t stride,
+                         const RoundBuffers &rb, float *lse, cudaStream_t st);
+
+}  // namespace elm
