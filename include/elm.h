@@ -349,7 +349,10 @@ int elm_attend_status(const void *workspace, const elm_params *params, int32_t n
  *                                      undefined.  One launch only; later calls are normal again.
  * Environment variables read by the library (tuning aids, off the documented path): ELM_WALK_CHAIN_MIN_PAIRS
  * (default 1024: Halve calls with at least this many pairs take the cluster walk kernel; 32 .. 4096) and
- * ELM_PREFILL_WINDOW (default 512: tokens per attention launch of elm_express_prefill; a power of two >= 64).
+ * ELM_PREFILL_WINDOW (default 512: tokens per attention launch of elm_express_prefill in the rounds that are
+ * taken in windows; a power of two >= 64) and ELM_PREFILL_ROUNDS (default on; 0: every thinned round of the prefill
+ * is taken in windows - otherwise bf16 inputs in fp32 mode take one attention launch per round whenever a round's
+ * segments are multiples of 256 tokens).
  * A build with -DELM_BOUNDS_CHECK (ELM_NVCC_EXTRA of the build script) checks every caller-supplied row number
  * of elm_attend against [0, n_kv): a bad one reads row 0 instead and sets the status word to 64.
  */

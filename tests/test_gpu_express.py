@@ -115,6 +115,9 @@ PREFILL_CASES = {
     "mixture_f32_nout8_R3_mbar0": (WORKLOADS["cfg2"].scaled(batch=1, q_heads=2, kv_heads=1), 3, 3, 0, 2),
     # tensor-core path, odd mbar: round 2 keeps one token of every 2 and runs Compress2 of depth 3
     "mixture_t3_bf16_nout128_R3_subsample": (WORKLOADS["cfg5"].scaled(q_heads=4, kv_heads=2), 7, 3, 3, 2),
+    # tensor-core path, level-0 calls of 16 points in round 2 (the paper's proportions: mbar = log2 n_out - 2): most
+    # blocks a pair of query tiles streams hold entries that are born or die among its 256 tokens
+    "mixture_t3_bf16_nout64_R3_small_calls": (WORKLOADS["cfg5"].scaled(q_heads=2, kv_heads=1), 6, 3, 4, 2),
 }
 PREFILL_TOL = {("f32", "fp64"): 2e-6, ("f32", "fp32"): 1e-4, ("bf16", "fp64"): 1e-2, ("bf16", "fp32"): 2e-2}
 
