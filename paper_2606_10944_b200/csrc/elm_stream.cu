@@ -53,6 +53,22 @@ __global__ void append_kernel(int32_t *__restrict__ list, int64_t stride, int64_
     const int p = blockIdx.x * blockDim.x + threadIdx.x;
     if (p < problems) list[(int64_t)p * stride + pos] = value;
 }
+// build_list_kernel and, in the same launch, list[p][pos] = value for every problem p: the token's own entry into E
+// or S_0 (Express.update), which lies behind the entries the pieces read.  A decode step is a handful of
+// microsecond-sized launches, so each one saved shows.
+__global__ void build_list_append_kernel(ListPieces pc, int64_t src_stride, int32_t *__restrict__ idx, float *__restrict__ w,
+                                         int64_t cap, int32_t *__restrict__ list, int64_t pos, int32_t value)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t pr = blockIdx.y;
+    if (i == 0) list[pr * src_stride + pos] = value;
+    if (i >= pc.dst_off[pc.n]) return;
+    int k = 0;
+    while (i >= pc.dst_off[k + 1]) ++k;
+    const int64_t o = i - pc.dst_off[k];
+    idx[pr * cap + i] = pc.src[k] ? pc.src[k][pr * src_stride + pc.src_off[k] + o] : (int32_t)(pc.src_off[k] + o);
+    w[pr * cap + i] = pc.w[k];
+}
 
 // wtd_cache() of Algorithm 1 (+ the token t itself when t >= 0) as list pieces
 static void stream_pieces(const elm_stream *s, const int64_t *n_S, const StreamLayout &L, unsigned char *ws,
@@ -176,6 +192,7 @@ static int stream_step_impl(elm_stream *s, const Tin *Q, const Tin *K, const Tin
     bool call_due[16];
     const bool sub = stratum_state(s, n_out, dr, nS_after, call_due);
     // ---- Algorithm 5: attend over wtd_cache() plus the token ----
+    bool appended = false;
     {
         ListPieces pc = {};
         stream_pieces(s, s->n_S, L, ws, p, t, pc);
@@ -189,6 +206,12 @@ static int stream_step_impl(elm_stream *s, const Tin *Q, const Tin *K, const Tin
             if (pb.dst_off[pb.n] > total) total = pb.dst_off[pb.n];
             if ((size_t)total > L.ep_cap) return ELM_ERR_WORKSPACE;
             build_list_choice_kernel<<<dim3(blocks(total), (unsigned)BH), 256, 0, st>>>(pc, pb, dr, n, ep_idx, ep_w, total);
+        } else if (!sub) {
+            // the token's entry into E (exact phase) or S_0 rides along (the bookkeeping follows below)
+            int32_t *list = s->n + 1 <= n_out ? E : Slist(0);
+            const int64_t pos = s->n + 1 <= n_out ? s->n_E : s->n_S[0];
+            build_list_append_kernel<<<dim3(blocks(total), (unsigned)BH), 256, 0, st>>>(pc, n, ep_idx, ep_w, total, list, pos, (int32_t)t);
+            appended = true;
         } else {
             build_list_kernel<<<dim3(blocks(total), (unsigned)BH), 256, 0, st>>>(pc, n, ep_idx, ep_w, total);
         }
@@ -199,6 +222,7 @@ static int stream_step_impl(elm_stream *s, const Tin *Q, const Tin *K, const Tin
     }
     // ---- Algorithm 1: Express.update ----
     auto append = [&](int32_t *list, int64_t pos) {
+        if (appended) return (int)ELM_OK;                                  // done with the list's launch
         append_kernel<<<(BH + 127) / 128, 128, 0, st>>>(list, n, pos, (int32_t)t, BH);
         count_launches(1);
         return cuda_status(cudaGetLastError());
