@@ -336,6 +336,115 @@ __device__ __forceinline__ float exp_pass_keep(uint32_t tP, float scale_log2, fl
 }
 
 // ---------------------------------------------------------------------------------------------
+// TMA producer of a launch with block lists (one thread): the queries of each pair, and the K / V^T / bias blocks
+// of each pair's own list through the 2-stage ring.  Same protocol as the producer inside the kernel; kept out of
+// line (it is called once per CTA) so that its code does not weigh on the register allocation and scheduling of
+// the kernel's softmax warps.
+// ---------------------------------------------------------------------------------------------
+struct ProducerArgs {
+    const CUtensorMap *mapQ, *mapK, *mapV, *mapX;
+    unsigned char *smem;
+    Barriers *bar;
+    const int *nonuniform;
+    const int32_t *tile_cnt, *tile_blk, *item_tab;
+    int n_items, tiles_x, tile_cap, item_cap, q_heads, kv_heads, q_row0, nblk, ragged_end;
+    unsigned long long wait_limit_ns;
+};
+template <int D, int QKB>
+__device__ __noinline__ bool produce_block_lists(const ProducerArgs *a)
+{
+    using SM = Smem<D, QKB>;
+    constexpr int KH = SM::KH;
+    constexpr int ROW_ELTS = 128 / QKB;
+    unsigned char *smem = a->smem;
+    Barriers *bar = a->bar;
+    const int n_items = a->n_items, tiles_x = a->tiles_x, nblk = a->nblk;
+    const unsigned long long limit = a->wait_limit_ns;
+    auto item_id = [&](int k) -> int {
+        return a->item_tab ? __ldg(a->item_tab + (int64_t)blockIdx.x * a->item_cap + k) : (int)blockIdx.x + k * (int)gridDim.x;
+    };
+    auto prob_of = [&](int bh) { return (bh / a->q_heads) * a->kv_heads + (int)(((int64_t)(bh % a->q_heads) * a->kv_heads) / a->q_heads); };
+    struct Cursor { int k, j, nb, id; };
+    auto enter = [&](Cursor &c) {                                // the item the cursor has moved to
+        c.id = c.k < n_items ? item_id(c.k) : 0;
+        c.nb = c.k < n_items ? (a->tile_cnt ? __ldg(a->tile_cnt + c.id % tiles_x) : nblk) : 0;
+    };
+    auto cursor_next = [&](Cursor &c) {
+        if (++c.j == c.nb) { c.j = 0; ++c.k; enter(c); }
+    };
+    auto item_bias = [&](int id) { return a->ragged_end || __ldg(a->nonuniform + prob_of(id / tiles_x)) != 0; };
+    auto load_q = [&](int id) {
+        const int bh = id / tiles_x, q0 = (id % tiles_x) * (2 * BM);
+        mbar_expect_tx(&bar->q_full, 2 * SM::Q_TILE);
+        for (int t = 0; t < 2; ++t)
+            for (int kh = 0; kh < KH; ++kh)
+                tma_load_3d(smem + SM::OFF_Q + t * SM::Q_TILE + kh * (BM * 128), a->mapQ, &bar->q_full, kh * ROW_ELTS, a->q_row0 + q0 + t * BM, bh);
+    };
+    int total = 0;
+    if (a->tile_cnt)
+        for (int k = 0; k < n_items; ++k) total += __ldg(a->tile_cnt + item_id(k) % tiles_x);
+    else
+        total = n_items * nblk;
+    Cursor kc = {0, 0, 0, 0};
+    enter(kc);
+    Cursor vc = kc;
+    int flag_item = -1;
+    bool flag_now = false;
+    auto load_k = [&](int G) {
+        const int s = G % STAGES, prob = prob_of(kc.id / tiles_x);
+        const int blk = a->tile_blk ? __ldg(a->tile_blk + (int64_t)(kc.id % tiles_x) * a->tile_cap + kc.j) : kc.j;
+        if (kc.k != flag_item) { flag_item = kc.k; flag_now = item_bias(kc.id); }
+        const bool with_bias = flag_now;
+        mbar_expect_tx(&bar->k_full[s], SM::K_BLOCK + (with_bias ? SM::X_BLOCK : 0));
+        for (int kh = 0; kh < KH; ++kh)
+            tma_load_3d(smem + SM::OFF_K + s * SM::K_BLOCK + kh * (BN * 128), a->mapK, &bar->k_full[s], kh * ROW_ELTS, blk * BN, prob);
+        if (with_bias) tma_load_3d(smem + SM::OFF_X + s * SM::X_BLOCK, a->mapX, &bar->k_full[s], 0, blk * BN, prob);
+        cursor_next(kc);
+    };
+    auto load_v = [&](int G) {
+        const int s = G % STAGES, prob = prob_of(vc.id / tiles_x);
+        const int blk = a->tile_blk ? __ldg(a->tile_blk + (int64_t)(vc.id % tiles_x) * a->tile_cap + vc.j) : vc.j;
+        mbar_expect_tx(&bar->v_full[s], SM::V_BLOCK);
+        for (int hh = 0; hh < 2; ++hh)
+            tma_load_3d(smem + SM::OFF_V + s * SM::V_BLOCK + hh * (D * 128), a->mapV, &bar->v_full[s], hh * 64, 0, prob * nblk + blk);
+        cursor_next(vc);
+    };
+    bool ok = true;
+    // The queries of item k may replace those of item k - 1 once every S = Q K^T of item k - 1 has been computed
+    // (q_free); they are fetched right after the keys of the item's first block (the key cursor then stands
+    // behind that block).
+    int next_q = 1;
+    auto feed_q = [&]() {
+        while (ok && next_q < n_items && (kc.k > next_q || (kc.k == next_q && kc.j > 0))) {
+            ok = sm100::mbar_wait(&bar->q_free, (uint32_t)(next_q - 1) & 1u, limit);
+            if (ok) load_q(item_id(next_q));
+            ++next_q;
+        }
+    };
+    if (n_items > 0) load_q(item_id(0));
+    // The issuer commits "event" i to kv_free[i % 2] after the prologue (i = 0: S = Q K^T of block 0 issued) and
+    // after iteration i - 1 (O += P V of block i - 1 and S = Q K^T of block i issued).  Once event i is complete,
+    // K's stage i % 2 (block i) and V's stage (i + 1) % 2 (block i - 1) have been read, so K(i + 2) and V(i + 1)
+    // may overwrite them.
+    for (int G = 0; G < STAGES && G < total; ++G) { load_k(G); load_v(G); }
+    feed_q();
+    for (int i = 0; i + 2 < total && ok; ++i) {
+        ok = sm100::mbar_wait(&bar->kv_free[i % STAGES], (uint32_t)(i / STAGES) & 1u, limit);
+        if (!ok) break;
+        load_k(i + 2);
+        if (i >= 1) load_v(i + 1);
+        feed_q();
+    }
+    // the last V block: freed by event total - 1
+    if (ok && total > STAGES) {
+        const int i = total - 2;
+        ok = sm100::mbar_wait(&bar->kv_free[i % STAGES], (uint32_t)(i / STAGES) & 1u, limit);
+        if (ok) load_v(i + 1);
+    }
+    return ok;
+}
+
+// ---------------------------------------------------------------------------------------------
 // the attention kernel
 // ---------------------------------------------------------------------------------------------
 // MASKED = false: every row sees the whole list (no causal tail, no lifetimes); the masked form of the
@@ -510,69 +619,17 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                     if (ok) load_v(i + 1);
                 }
             } else {
-                // Blocks are numbered G = 0, 1, ... along the CTA's whole stream; a cursor (item k, block j of its
-                // nb) walks it, one for the keys and one for the values, which run a block behind.
-                struct Cursor { int k, j, nb; };
-                const int total = count_blocks();
-                auto cursor_next = [&](Cursor &c) {
-                    if (++c.j == c.nb) { c.j = 0; ++c.k; c.nb = c.k < n_items ? item_nblk(c.k) : 0; }
-                };
-                Cursor kc = {0, 0, n_items > 0 ? item_nblk(0) : 0}, vc = kc;
-                int flag_item = -1;
-                bool flag_now = false, flag_next = n_items > 0 && item_bias(0);
-                auto load_k = [&](int G) {
-                    const int s = G % STAGES, prob = prob_of(item_bh(kc.k)), blk = item_blk(kc.k, kc.j);
-                    // the flag of an item is fetched while the item before it streams, off the critical path
-                    if (kc.k != flag_item) {
-                        flag_item = kc.k;
-                        flag_now = flag_next;
-                        flag_next = flag_item + 1 < n_items && item_bias(flag_item + 1);
-                    }
-                    const bool with_bias = flag_now;
-                    mbar_expect_tx(&bar->k_full[s], SM::K_BLOCK + (with_bias ? SM::X_BLOCK : 0));
-                    for (int kh = 0; kh < KH; ++kh)
-                        tma_load_3d(smem + SM::OFF_K + s * SM::K_BLOCK + kh * (BN * 128), &mapK, &bar->k_full[s], kh * ROW_ELTS, blk * BN, prob);
-                    if (with_bias) tma_load_3d(smem + SM::OFF_X + s * SM::X_BLOCK, &mapX, &bar->k_full[s], 0, blk * BN, prob);
-                    cursor_next(kc);
-                };
-                auto load_v = [&](int G) {
-                    const int s = G % STAGES, prob = prob_of(item_bh(vc.k)), blk = item_blk(vc.k, vc.j);
-                    mbar_expect_tx(&bar->v_full[s], SM::V_BLOCK);
-                    for (int hh = 0; hh < 2; ++hh)
-                        tma_load_3d(smem + SM::OFF_V + s * SM::V_BLOCK + hh * (D * 128), &mapV, &bar->v_full[s], hh * 64, 0, prob * nblk + blk);
-                    cursor_next(vc);
-                };
-                // The queries of item k may replace those of item k - 1 once every S = Q K^T of item k - 1
-                // has been computed (q_free); they are fetched right after the keys of the item's first block
-                // (the key cursor then stands behind that block).
-                int next_q = 1;
-                auto feed_q = [&]() {
-                    while (ok && next_q < n_items && (kc.k > next_q || (kc.k == next_q && kc.j > 0))) {
-                        ok = mbar_wait(&bar->q_free, (uint32_t)(next_q - 1) & 1u);
-                        if (ok) load_q(next_q);
-                        ++next_q;
-                    }
-                };
-                load_q(0);
-                // The issuer commits "event" i to kv_free[i % 2] after the prologue (i = 0: S = Q K^T of block
-                // 0 issued) and after iteration i - 1 (O += P V of block i - 1 and S = Q K^T of block i issued).
-                // Once event i is complete, K's stage i % 2 (block i) and V's stage (i + 1) % 2 (block i - 1)
-                // have been read, so K(i + 2) and V(i + 1) may overwrite them.
-                for (int G = 0; G < STAGES && G < total; ++G) { load_k(G); load_v(G); }
-                feed_q();
-                for (int i = 0; i + 2 < total && ok; ++i) {
-                    ok = mbar_wait(&bar->kv_free[i % STAGES], (uint32_t)(i / STAGES) & 1u);
-                    if (!ok) break;
-                    load_k(i + 2);
-                    if (i >= 1) load_v(i + 1);
-                    feed_q();
-                }
-                // the last V block: freed by event total - 1
-                if (ok && total > STAGES) {
-                    const int i = total - 2;
-                    ok = mbar_wait(&bar->kv_free[i % STAGES], (uint32_t)(i / STAGES) & 1u);
-                    if (ok) load_v(i + 1);
-                }
+                // (launch with block lists: the producer that walks them is a function of its own, not inlined - the
+                // code of this kernel's other roles is sensitive to what is compiled in beside it)
+                ProducerArgs pa;
+                pa.mapQ = &mapQ; pa.mapK = &mapK; pa.mapV = &mapV; pa.mapX = &mapX;
+                pa.smem = smem; pa.bar = bar;
+                pa.nonuniform = nonuniform; pa.tile_cnt = tile_cnt; pa.tile_blk = tile_blk; pa.item_tab = item_tab;
+                pa.n_items = n_items; pa.tiles_x = tiles_x; pa.tile_cap = tile_cap; pa.item_cap = item_cap;
+                pa.q_heads = q_heads; pa.kv_heads = kv_heads; pa.q_row0 = q_row0; pa.nblk = nblk;
+                pa.ragged_end = ragged_end ? 1 : 0;
+                pa.wait_limit_ns = wait_limit_ns;
+                ok = produce_block_lists<D, QKB>(&pa);
             }
             if (!ok) { atomicExch(status, 1); bar->abort_flag = 1; }
         }
