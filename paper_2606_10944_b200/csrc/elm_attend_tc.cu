@@ -364,15 +364,25 @@ __device__ __noinline__ bool produce_block_lists(const ProducerArgs *a)
         return a->item_tab ? __ldg(a->item_tab + (int64_t)blockIdx.x * a->item_cap + k) : (int)blockIdx.x + k * (int)gridDim.x;
     };
     auto prob_of = [&](int bh) { return (bh / a->q_heads) * a->kv_heads + (int)(((int64_t)(bh % a->q_heads) * a->kv_heads) / a->q_heads); };
-    struct Cursor { int k, j, nb, id; };
-    auto enter = [&](Cursor &c) {                                // the item the cursor has moved to
+    // A cursor stands at block j of item k of the CTA's stream.  What the next load needs - the item's problem, the
+    // block's number in the list, whether the item takes the bias operand - is fetched when the cursor moves
+    // there, a whole block period before it is used: the ring has two stages, so whatever the producer does
+    // between "stage free" and "copy issued" delays the tensor pipe.
+    struct Cursor { int k, j, nb, id, prob, blk; bool bias; };
+    auto fetch_blk = [&](Cursor &c) {
+        c.blk = c.k < n_items ? (a->tile_blk ? __ldg(a->tile_blk + (int64_t)(c.id % tiles_x) * a->tile_cap + c.j) : c.j) : 0;
+    };
+    auto enter = [&](Cursor &c, bool want_bias) {                // the item the cursor has moved to
         c.id = c.k < n_items ? item_id(c.k) : 0;
         c.nb = c.k < n_items ? (a->tile_cnt ? __ldg(a->tile_cnt + c.id % tiles_x) : nblk) : 0;
+        c.prob = prob_of(c.id / tiles_x);
+        c.bias = want_bias && c.k < n_items && (a->ragged_end || __ldg(a->nonuniform + c.prob) != 0);
+        fetch_blk(c);
     };
-    auto cursor_next = [&](Cursor &c) {
-        if (++c.j == c.nb) { c.j = 0; ++c.k; enter(c); }
+    auto cursor_next = [&](Cursor &c, bool want_bias) {
+        if (++c.j == c.nb) { c.j = 0; ++c.k; enter(c, want_bias); }
+        else fetch_blk(c);
     };
-    auto item_bias = [&](int id) { return a->ragged_end || __ldg(a->nonuniform + prob_of(id / tiles_x)) != 0; };
     auto load_q = [&](int id) {
         const int bh = id / tiles_x, q0 = (id % tiles_x) * (2 * BM);
         mbar_expect_tx(&bar->q_full, 2 * SM::Q_TILE);
@@ -385,29 +395,23 @@ __device__ __noinline__ bool produce_block_lists(const ProducerArgs *a)
         for (int k = 0; k < n_items; ++k) total += __ldg(a->tile_cnt + item_id(k) % tiles_x);
     else
         total = n_items * nblk;
-    Cursor kc = {0, 0, 0, 0};
-    enter(kc);
+    Cursor kc = {0, 0, 0, 0, 0, 0, false};
+    enter(kc, true);
     Cursor vc = kc;
-    int flag_item = -1;
-    bool flag_now = false;
     auto load_k = [&](int G) {
-        const int s = G % STAGES, prob = prob_of(kc.id / tiles_x);
-        const int blk = a->tile_blk ? __ldg(a->tile_blk + (int64_t)(kc.id % tiles_x) * a->tile_cap + kc.j) : kc.j;
-        if (kc.k != flag_item) { flag_item = kc.k; flag_now = item_bias(kc.id); }
-        const bool with_bias = flag_now;
-        mbar_expect_tx(&bar->k_full[s], SM::K_BLOCK + (with_bias ? SM::X_BLOCK : 0));
+        const int s = G % STAGES;
+        mbar_expect_tx(&bar->k_full[s], SM::K_BLOCK + (kc.bias ? SM::X_BLOCK : 0));
         for (int kh = 0; kh < KH; ++kh)
-            tma_load_3d(smem + SM::OFF_K + s * SM::K_BLOCK + kh * (BN * 128), a->mapK, &bar->k_full[s], kh * ROW_ELTS, blk * BN, prob);
-        if (with_bias) tma_load_3d(smem + SM::OFF_X + s * SM::X_BLOCK, a->mapX, &bar->k_full[s], 0, blk * BN, prob);
-        cursor_next(kc);
+            tma_load_3d(smem + SM::OFF_K + s * SM::K_BLOCK + kh * (BN * 128), a->mapK, &bar->k_full[s], kh * ROW_ELTS, kc.blk * BN, kc.prob);
+        if (kc.bias) tma_load_3d(smem + SM::OFF_X + s * SM::X_BLOCK, a->mapX, &bar->k_full[s], 0, kc.blk * BN, kc.prob);
+        cursor_next(kc, true);
     };
     auto load_v = [&](int G) {
-        const int s = G % STAGES, prob = prob_of(vc.id / tiles_x);
-        const int blk = a->tile_blk ? __ldg(a->tile_blk + (int64_t)(vc.id % tiles_x) * a->tile_cap + vc.j) : vc.j;
+        const int s = G % STAGES;
         mbar_expect_tx(&bar->v_full[s], SM::V_BLOCK);
         for (int hh = 0; hh < 2; ++hh)
-            tma_load_3d(smem + SM::OFF_V + s * SM::V_BLOCK + hh * (D * 128), a->mapV, &bar->v_full[s], hh * 64, 0, prob * nblk + blk);
-        cursor_next(vc);
+            tma_load_3d(smem + SM::OFF_V + s * SM::V_BLOCK + hh * (D * 128), a->mapV, &bar->v_full[s], hh * 64, 0, vc.prob * nblk + vc.blk);
+        cursor_next(vc, false);
     };
     bool ok = true;
     // The queries of item k may replace those of item k - 1 once every S = Q K^T of item k - 1 has been computed
