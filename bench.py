@@ -22,9 +22,9 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one attend launch at the workload's full size, from one
-# single-pass ncu capture of that launch (read 1 083 738 880 + write 1 024 521 216 bytes); workloads without
-# a capture report null and say so
-NCU_DRAM_BYTES_PER_ATTEND_LAUNCH = {"cfg5": 1083738880 + 1024521216}
+# single-pass ncu capture of that launch (bf16: read 1 083 738 880 + write 1 024 521 216 bytes; E4M3 storage:
+# read 543 735 808 + write 1 019 808 000); workloads without a capture report null and say so
+NCU_DRAM_BYTES_PER_ATTEND_LAUNCH = {"cfg5": 1083738880 + 1024521216, "cfg5[storage=e4m3]": 543735808 + 1019808000}
 
 METRIC = "compress+attend tokens/sec per B200"
 UNIT = "tokens/s"
