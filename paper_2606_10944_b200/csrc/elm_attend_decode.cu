@@ -54,6 +54,9 @@ decode_partial_kernel(const Tin *__restrict__ Q, const Tin *__restrict__ K, cons
     constexpr int DPL = D / 32;
     __shared__ float sm_o[DEC_WARPS][G][D];
     __shared__ float sm_ml[DEC_WARPS][G][2];
+    // (launched with programmatic stream serialization: resident before the kernel in front of it has finished;
+    // nothing is read before this point)
+    cudaGridDependencySynchronize();
     const int prob = blockIdx.y, split = blockIdx.x, splits = gridDim.x;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int b = prob / kv_heads, kvh = prob % kv_heads, rep = q_heads / kv_heads;
@@ -182,6 +185,9 @@ __global__ void __launch_bounds__(D) decode_merge_kernel(const float *__restrict
 #endif
     const int b = prob / kv_heads, kvh = prob % kv_heads, rep = q_heads / kv_heads;
     const float *p = part + ((int64_t)prob * splits * G + g) * (D + 2);
+    // launched with programmatic stream serialization: the CTAs of this kernel are resident while the partial
+    // kernel still runs and wait here for its results, so the gap between the two launches is not on the path
+    cudaGridDependencySynchronize();
     // thread s (and s + D, ...) fetches split s's maximum and denominator
     float M = -INFINITY;
     float ms[(DEC_MAX_SPLITS + D - 1) / D], ls[(DEC_MAX_SPLITS + D - 1) / D];
@@ -240,10 +246,33 @@ int launch_decode(const Tin *Q, const Tin *K, const Tin *V, const int32_t *idx, 
 {
     const int problems = p->batch * p->kv_heads;
     const int chunk = (n_core + splits - 1) / splits;
-    decode_partial_kernel<Tin, D, G><<<dim3((unsigned)splits, (unsigned)problems), DEC_WARPS * 32, 0, st>>>(
-        Q, K, V, idx, w, p->n_kv, n_core, p->q_heads, p->kv_heads, p->n_q, groups, chunk, part, status);
-    decode_merge_kernel<Tin, D, G><<<dim3((unsigned)groups, (unsigned)problems), D, 0, st>>>(part, splits, p->q_heads,
-                                                                                            p->kv_heads, p->n_q, O, status);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)splits, (unsigned)problems);
+        cfg.blockDim = dim3(DEC_WARPS * 32);
+        cfg.stream = st;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        int64_t n_kv = p->n_kv;
+        int q_heads = p->q_heads, kv_heads = p->kv_heads, n_q = p->n_q;
+        ELM_CUDA_TRY(cudaLaunchKernelEx(&cfg, decode_partial_kernel<Tin, D, G>, Q, K, V, idx, w, n_kv, n_core, q_heads, kv_heads,
+                                        n_q, groups, chunk, part, status));
+    }
+    {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)groups, (unsigned)problems);
+        cfg.blockDim = dim3(D);
+        cfg.dynamicSmemBytes = 0;
+        cfg.stream = st;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        const float *part_c = part;
+        int q_heads = p->q_heads, kv_heads = p->kv_heads, n_q = p->n_q;
+        ELM_CUDA_TRY(cudaLaunchKernelEx(&cfg, decode_merge_kernel<Tin, D, G>, part_c, splits, q_heads, kv_heads, n_q, O, status));
+    }
     count_launches(2);
     return cuda_status(cudaGetLastError());
 }

@@ -59,6 +59,8 @@ __global__ void append_kernel(int32_t *__restrict__ list, int64_t stride, int64_
 __global__ void build_list_append_kernel(ListPieces pc, int64_t src_stride, int32_t *__restrict__ idx, float *__restrict__ w,
                                          int64_t cap, int32_t *__restrict__ list, int64_t pos, int32_t value)
 {
+    // (launched with programmatic stream serialization; nothing is read or written before this point)
+    cudaGridDependencySynchronize();
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     const int64_t pr = blockIdx.y;
     if (i == 0) list[pr * src_stride + pos] = value;
@@ -210,7 +212,18 @@ static int stream_step_impl(elm_stream *s, const Tin *Q, const Tin *K, const Tin
             // the token's entry into E (exact phase) or S_0 rides along (the bookkeeping follows below)
             int32_t *list = s->n + 1 <= n_out ? E : Slist(0);
             const int64_t pos = s->n + 1 <= n_out ? s->n_E : s->n_S[0];
-            build_list_append_kernel<<<dim3(blocks(total), (unsigned)BH), 256, 0, st>>>(pc, n, ep_idx, ep_w, total, list, pos, (int32_t)t);
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+            attr[0].val.programmaticStreamSerializationAllowed = 1;
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3(blocks(total), (unsigned)BH);
+            cfg.blockDim = dim3(256);
+            cfg.stream = st;
+            cfg.attrs = attr;
+            cfg.numAttrs = 1;
+            const int64_t cap = total;
+            const int32_t value = (int32_t)t;
+            ELM_CUDA_TRY(cudaLaunchKernelEx(&cfg, build_list_append_kernel, pc, n, ep_idx, ep_w, cap, list, pos, value));
             appended = true;
         } else {
             build_list_kernel<<<dim3(blocks(total), (unsigned)BH), 256, 0, st>>>(pc, n, ep_idx, ep_w, total);
