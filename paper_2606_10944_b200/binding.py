@@ -429,7 +429,8 @@ def attend_status(workspace, params: ElmParams, n_core: int) -> int:
     return int(out.value)
 
 
-def profile_enable(on: bool = True):
+def profile_enable(on=True):
+    """0 / False: off; 1 / True: every stage; 2: the attention stage only (see include/elm.h)."""
     _check(load_library().elm_profile_enable(int(on)), "elm_profile_enable")
 
 

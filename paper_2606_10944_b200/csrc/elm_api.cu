@@ -31,6 +31,7 @@ StageTimer::StageTimer(int stage, cudaStream_t stream, int launches) : stream_(s
     Profiler &pr = profiler();
     g_stage_launches[stage] += launches;
     if (!pr.enabled || pr.n_records >= Profiler::kMaxRecords) return;
+    if (pr.attend_only && stage != ELM_STAGE_ATTEND) return;
     rec_ = pr.n_records++;
     if (rec_ >= pr.events_created) {
         cudaEventCreate(&pr.ev_begin[rec_]);
@@ -289,6 +290,7 @@ extern "C" int elm_profile_enable(int on)
 {
     Profiler &pr = profiler();
     pr.enabled = on != 0;
+    pr.attend_only = on == 2;
     pr.n_records = 0;
     for (int s = 0; s < ELM_N_STAGES; ++s) g_stage_launches[s] = 0;
     return ELM_OK;

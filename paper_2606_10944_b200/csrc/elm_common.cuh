@@ -14,6 +14,7 @@ namespace elm {
 // ---------------------------------------------------------------------------------------------
 struct Profiler {
     bool enabled = false;
+    bool attend_only = false;     // events around the attention stage only (elm_profile_enable(2))
     static constexpr int kMaxRecords = 4096;
     int n_records = 0;
     cudaEvent_t ev_begin[kMaxRecords];
@@ -43,6 +44,25 @@ inline int cuda_status(cudaError_t e) { return e == cudaSuccess ? ELM_OK : ELM_E
         cudaError_t _e = (expr);                          \
         if (_e != cudaSuccess) return ELM_ERR_CUDA;       \
     } while (0)
+
+// Launch with programmatic stream serialization: the grid may become resident before the kernel in front of it in
+// the stream has finished, which takes the launch latency off a chain of short dependent kernels.  The kernel must
+// call cudaGridDependencySynchronize() before it reads or writes global memory.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_after(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args &&...args)
+{
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
 
 // Multiprocessors of the current device (looked up once per device ordinal; 148 if the query fails).
 int device_sm_count();

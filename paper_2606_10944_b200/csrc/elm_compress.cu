@@ -59,7 +59,7 @@ static int compress_impl(const Tin *K, const Tin *V, const elm_params *p, uint64
         StageTimer t(ELM_STAGE_PREPASS, st, 1);
         ELM_CUDA_TRY(cudaMemsetAsync(c.vmax_bits, 0, (size_t)(BH + 1) * 4, st));
         dim3 grid((unsigned)((n + 255) / 256), (unsigned)BH);
-        prepass_kernel<Tin, T><<<grid, 256, 0, st>>>(K, V, n, p->d, c.cnorm, c.vmax_bits, cur);
+        ELM_CUDA_TRY(launch_after(prepass_kernel<Tin, T>, grid, dim3(256), 0, st, K, V, n, p->d, c.cnorm, c.vmax_bits, cur, (int64_t)0, (int64_t)-1));
         count_launches(1);
         ELM_CUDA_TRY(cudaGetLastError());
     }
@@ -75,7 +75,7 @@ static int compress_impl(const Tin *K, const Tin *V, const elm_params *p, uint64
     {
         StageTimer t(ELM_STAGE_EMIT, st, 1);
         const int64_t total = (int64_t)BH * n_out;
-        emit_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(w_out, idx_out, total, n_out, m == 0);
+        ELM_CUDA_TRY(launch_after(emit_kernel, dim3((unsigned)((total + 255) / 256)), dim3(256), 0, st, w_out, idx_out, total, n_out, m == 0));
         count_launches(1);
         ELM_CUDA_TRY(cudaGetLastError());
     }

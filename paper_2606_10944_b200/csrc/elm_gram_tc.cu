@@ -104,6 +104,7 @@ gram_tc_kernel(const __nv_bfloat16 *__restrict__ K, const __nv_bfloat16 *__restr
                const unsigned *__restrict__ vmax_bits, int64_t n, int P, int64_t Ptotal,
                float *__restrict__ F, int64_t F_stride, int *__restrict__ status, WalkArgs wk)
 {
+    cudaGridDependencySynchronize();           // launched with programmatic stream serialization (launch_after)
     using SM = Smem<D>;
     constexpr int KH = SM::KH;
     extern __shared__ unsigned char smem_dyn[];
@@ -324,6 +325,7 @@ gram_tc_persistent_kernel(const __nv_bfloat16 *__restrict__ K, const __nv_bfloat
                           const unsigned *__restrict__ vmax_bits, int64_t n, int P, int tiles_per_problem,
                           int total_items, float *__restrict__ F, int64_t F_stride, int *__restrict__ status)
 {
+    cudaGridDependencySynchronize();           // launched with programmatic stream serialization (launch_after)
     using SM = PSmem<D>;
     constexpr int KH = D / 64;
     constexpr int CHUNKS = D / 8;                             // 16-byte chunks per row
@@ -540,15 +542,15 @@ static int launch(const __nv_bfloat16 *K, const __nv_bfloat16 *V, const elm_para
         const int grid = (int)(total < sm_count ? total : sm_count);
         auto pk = gram_tc_persistent_kernel<D>;
         ELM_CUDA_TRY(cudaFuncSetAttribute(pk, cudaFuncAttributeMaxDynamicSharedMemorySize, PSmem<D>::TOTAL));
-        pk<<<grid, PTHREADS, PSmem<D>::TOTAL, st>>>(K, V, cur, Mpair, vmax_bits, p->n_kv, P, (int)tiles, (int)total, F,
-                                                   F_stride, status);
+        ELM_CUDA_TRY(launch_after(pk, dim3((unsigned)grid), dim3(PTHREADS), (size_t)PSmem<D>::TOTAL, st, K, V, cur, Mpair, vmax_bits,
+                                  p->n_kv, P, (int)tiles, (int)total, F, F_stride, status));
         count_launches(1);
         return cuda_status(cudaGetLastError());
     }
     auto kern = gram_tc_kernel<D>;
     ELM_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<D>::TOTAL));
-    kern<<<dim3((unsigned)tiles, (unsigned)BH), NTHREADS, Smem<D>::TOTAL, st>>>(K, V, cur, Mpair, vmax_bits, p->n_kv, P,
-                                                                                 Ptotal, F, F_stride, status, wk);
+    ELM_CUDA_TRY(launch_after(kern, dim3((unsigned)tiles, (unsigned)BH), dim3(NTHREADS), (size_t)Smem<D>::TOTAL, st, K, V, cur, Mpair, vmax_bits,
+                              p->n_kv, P, Ptotal, F, F_stride, status, wk));
     count_launches(1);
     return cuda_status(cudaGetLastError());
 }

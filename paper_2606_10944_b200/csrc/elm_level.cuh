@@ -57,6 +57,7 @@ static __global__ void __launch_bounds__(256) prepass_kernel(const Tin *__restri
                                                       int32_t *__restrict__ cur, int64_t first = 0,
                                                       int64_t last = -1 /* rows [first, last); -1: n */)
 {
+    cudaGridDependencySynchronize();           // launched with programmatic stream serialization (launch_after)
     if (last < 0) last = n;
     constexpr int EPC = 16 / sizeof(Tin);                 // elements per 16-byte chunk
     const int p = blockIdx.y;
@@ -94,6 +95,7 @@ static __global__ void __launch_bounds__(1024) level_prep_kernel(const T *__rest
                                                          int P, T *__restrict__ Mpair,
                                                          T *__restrict__ rdecay)
 {
+    cudaGridDependencySynchronize();           // launched with programmatic stream serialization (launch_after)
     __shared__ T warp_tot[32];
     const int p = blockIdx.y, g = blockIdx.x;
     const int nthr = blockDim.x, nwarp = nthr >> 5;
@@ -150,6 +152,7 @@ static __global__ void __launch_bounds__(256) gram_simt_kernel(const Tin *__rest
                                                         int64_t n, int P, int64_t Ptotal,
                                                         T *__restrict__ F, int64_t F_stride)
 {
+    cudaGridDependencySynchronize();           // launched with programmatic stream serialization (launch_after)
     constexpr int DC = 16, LD = 68;
     __shared__ T Ak[DC][LD], Bk[DC][LD], Av[DC][LD], Bv[DC][LD];
     __shared__ int32_t rowsA[64], rowsB[64];
@@ -333,6 +336,7 @@ static __global__ void __launch_bounds__(576) walk_cta_kernel(const T *__restric
                                                        int64_t n, int P, int64_t lvl, uint64_t seed,
                                                        T logfac, uint32_t pbase)
 {
+    cudaGridDependencySynchronize();           // launched with programmatic stream serialization (launch_after)
     constexpr int PW = 2048 / sizeof(T);                             // panel width in columns (64 KB / 2 buffers... per 32 rows)
     extern __shared__ __align__(16) unsigned char smem_raw[];
     T *tiles = reinterpret_cast<T *>(smem_raw);                      // [2][2][32][32]: buffer, (diag, cross)
@@ -511,6 +515,7 @@ static __global__ void __launch_bounds__(256) walk_warp_kernel(const T *__restri
                                                         int64_t n, int P, int groups, int64_t lvl,
                                                         uint64_t seed, T logfac, uint32_t pbase)
 {
+    cudaGridDependencySynchronize();           // launched with programmatic stream serialization (launch_after)
     const int p = blockIdx.y;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = blockIdx.x * 8 + warp;
@@ -536,6 +541,7 @@ static __global__ void __launch_bounds__(256) walk_warp_kernel(const T *__restri
 static __global__ void emit_kernel(float *__restrict__ w, int32_t *__restrict__ idx, int64_t total,
                             int64_t n_out, int write_identity)
 {
+    cudaGridDependencySynchronize();           // launched with programmatic stream serialization (launch_after)
     int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= total) return;
     w[i] = 1.0f / (float)n_out;
@@ -560,9 +566,9 @@ static int run_gram_simt(const Tin *K, const Tin *V, const elm_params *p, const 
     }
     dim3 grid((unsigned)tiles, (unsigned)BH);
     if (p->d == 64)
-        gram_simt_kernel<Tin, T, 64><<<grid, 256, 0, st>>>(K, V, cur, Mpair, vmax_bits, p->n_kv, P, Ptotal, F, F_stride);
+        ELM_CUDA_TRY(launch_after(gram_simt_kernel<Tin, T, 64>, grid, dim3(256), 0, st, K, V, cur, Mpair, vmax_bits, p->n_kv, P, Ptotal, F, F_stride));
     else
-        gram_simt_kernel<Tin, T, 128><<<grid, 256, 0, st>>>(K, V, cur, Mpair, vmax_bits, p->n_kv, P, Ptotal, F, F_stride);
+        ELM_CUDA_TRY(launch_after(gram_simt_kernel<Tin, T, 128>, grid, dim3(256), 0, st, K, V, cur, Mpair, vmax_bits, p->n_kv, P, Ptotal, F, F_stride));
     count_launches(1);
     return cuda_status(cudaGetLastError());
 }
@@ -599,7 +605,7 @@ static int run_halve_level(const LevelCtx<Tin, T> &c, const int32_t *cur, int32_
     {
         StageTimer t(ELM_STAGE_LEVEL_PREP, st, 1);
         const int lp_threads = P >= 1024 ? 1024 : (P <= 32 ? 32 : (P + 31) / 32 * 32);
-        level_prep_kernel<T><<<dim3((unsigned)groups, (unsigned)BH), lp_threads, 0, st>>>(c.cnorm, cur, n, P, c.Mpair, c.rdecay);
+        ELM_CUDA_TRY(launch_after(level_prep_kernel<T>, dim3((unsigned)groups, (unsigned)BH), dim3(lp_threads), 0, st, c.cnorm, cur, n, P, c.Mpair, c.rdecay));
         count_launches(1);
         ELM_CUDA_TRY(cudaGetLastError());
     }
@@ -654,11 +660,11 @@ static int run_halve_level(const LevelCtx<Tin, T> &c, const int32_t *cur, int32_
             if (smem > 227 * 1024) return ELM_ERR_SHAPE;               // a call this long needs the chain kernel
             auto kern = walk_cta_kernel<T>;
             ELM_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-            kern<<<dim3((unsigned)groups, (unsigned)BH), threads, smem, st>>>(
-                c.F, c.F_stride, c.rdecay, cur, out, out_stride, n, P, lvl, c.seed, logfac, c.pbase);
+            ELM_CUDA_TRY(launch_after(kern, dim3((unsigned)groups, (unsigned)BH), dim3(threads), smem, st,
+                                      c.F, c.F_stride, c.rdecay, cur, out, out_stride, n, P, lvl, c.seed, logfac, c.pbase));
         } else {
-            walk_warp_kernel<T><<<dim3((unsigned)((groups + 7) / 8), (unsigned)BH), 256, 0, st>>>(
-                c.F, c.F_stride, c.rdecay, cur, out, out_stride, n, P, groups, lvl, c.seed, logfac, c.pbase);
+            ELM_CUDA_TRY(launch_after(walk_warp_kernel<T>, dim3((unsigned)((groups + 7) / 8), (unsigned)BH), dim3(256), 0, st,
+                                      c.F, c.F_stride, c.rdecay, cur, out, out_stride, n, P, groups, lvl, c.seed, logfac, c.pbase));
         }
         count_launches(1);
         ELM_CUDA_TRY(cudaGetLastError());

@@ -158,6 +158,7 @@ walk_chain_kernel(const __grid_constant__ CUtensorMap mapF, const T *__restrict_
                   int64_t n, int P, int64_t lvl, uint64_t seed, T logfac, uint32_t pbase, int nb_cap, int *status)
 {
     using namespace sm100;
+    cudaGridDependencySynchronize();           // launched with programmatic stream serialization
     constexpr bool EAGER = std::is_same<T, float>::value;            // the fp32 walker also scores the next block
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const int C = (int)cluster_nctarank(), k = (int)cluster_ctarank();
@@ -418,13 +419,16 @@ int walk_chain(const T *F, int64_t F_stride, const T *rdecay, const int32_t *cur
     cfg.blockDim = dim3((unsigned)threads, 1, 1);
     cfg.dynamicSmemBytes = S.total;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = (unsigned)C;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    // (the grid may become resident while the Gram kernel in front of it drains; the kernel waits on the device)
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     if (C > 8) {
         // clusters of 16 CTAs need the opt-in and a GPC with 16 free SMs; if none can be resident
         // the caller falls back to one CTA per call
