@@ -276,3 +276,23 @@ def test_launch_counter_and_stage_profile():
     launched = elm.launch_count() - before
     assert launched == sum(v[1] for v in prof.values()) and launched >= 3 * wl.m + 3
     assert prof["attend"][0] > 0 and prof["walk"][1] == wl.m
+
+
+def test_stage_profile_of_the_attention_stage_only():
+    """elm_profile_enable(2): events around the attention stage alone, launches counted for every stage, and the
+    results of the step are those of an unprofiled one (the compression's launches then keep their device-side
+    ordering without events between them)."""
+    wl = SMALL_CASES["cfg3_four_heads"]
+    Q, K, V = generate(wl, seed=8)
+    Qd, Kd, Vd = _dev(Q, K, V)
+    idx0, w0 = elm.compress(Kd, Vd, wl.log2_nout, wl.m, seed=4)
+    O0 = elm.attend(Qd, Kd, Vd, idx0, w0)
+    elm.profile_enable(2)
+    idx, w = elm.compress(Kd, Vd, wl.log2_nout, wl.m, seed=4)
+    O = elm.attend(Qd, Kd, Vd, idx, w)
+    prof = elm.profile_read()
+    elm.profile_enable(False)
+    assert prof["attend"][0] > 0 and prof["attend"][1] >= 1
+    for stage in ("prepass", "level_prep", "gram", "walk", "emit"):
+        assert prof[stage][0] == 0.0 and prof[stage][1] >= 1
+    assert torch.equal(idx, idx0) and torch.equal(w, w0) and torch.equal(O, O0)
