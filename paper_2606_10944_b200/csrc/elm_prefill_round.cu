@@ -29,7 +29,7 @@ constexpr int32_t NEVER = 0x7fffffff;
 // not any more (death); per block of 128 entries the largest birth and the smallest death.  With G = the
 // number of a sibling's kept points that have arrived - G = X is reached right after the X-th kept point, at
 // token kept[X - 1] + 1:
-//   E                       always;  the output of sibling j: from G_j = len0 on
+//   E                       always;  the output of sibling j: from G_j = len0 on (q = 0: from the end of its segment)
 //   S_i entry of call c     from G = (c + 1) A until G = (c / 4 + 1) 4 A          (A = s0 4^(i-1))
 //   S_0 entry g             from its own token (which sees itself) until G = (g / s0 + 1) s0   (q = 0: for good)
 // Padding entries are never seen.
@@ -52,7 +52,9 @@ __global__ void __launch_bounds__(256) round_universe_kernel(RoundUniverse u, co
             if (pos < 4 * u.n_out) {
                 const int64_t part = pos / u.n_out;
                 row = E[pr * stride + pos];
-                bt = part == 0 ? 0 : token_after(part - 1, u.len0);
+                // (q = 0: no Halve call - the sibling's kept points stay in S_0 to the end of its segment and only
+                // then join E, so their copy in E must not be seen before the next sibling begins)
+                bt = part == 0 ? 0 : (u.q >= 1 ? token_after(part - 1, u.len0) : (int32_t)((part + 1) * u.seg));
             }
         } else {
             const int64_t jj = (pos - u.EP) / u.SP;

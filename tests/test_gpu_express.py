@@ -118,6 +118,9 @@ PREFILL_CASES = {
     # tensor-core path, level-0 calls of 16 points in round 2 (the paper's proportions: mbar = log2 n_out - 2): most
     # blocks a pair of query tiles streams hold entries that are born or die among its 256 tokens
     "mixture_t3_bf16_nout64_R3_small_calls": (WORKLOADS["cfg5"].scaled(q_heads=2, kv_heads=1), 6, 3, 4, 2),
+    # tensor-core path, mbar = 0: the kept points of a sibling stay in S_0 to the end of its segment (their copy in E
+    # shares a block of 128 list entries with entries the sibling's tokens do see)
+    "mixture_t3_bf16_nout64_R3_mbar0": (WORKLOADS["cfg5"].scaled(q_heads=2, kv_heads=1), 6, 3, 0, 2),
 }
 PREFILL_TOL = {("f32", "fp64"): 2e-6, ("f32", "fp32"): 1e-4, ("bf16", "fp64"): 1e-2, ("bf16", "fp32"): 2e-2}
 
