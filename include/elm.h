@@ -228,8 +228,12 @@ int elm_express_workspace_bytes(const elm_params *params, int32_t mbar, size_t *
  *   workspace  at least elm_express_prefill_workspace_bytes(params, mbar) bytes, 256-byte aligned.
  * In a round whose thinning factor exceeds mbar (Subsample active) the kept points differ from problem to
  * problem; a token that is not kept still attends to itself with the weight of a point of S_0.
- * One attention launch per window of about 512 tokens, over every cache entry that some token of the
- * window sees; each entry carries the span of tokens that see it.
+ * Every cache entry carries the span of tokens that see it.  bf16 inputs in fp32 mode, in rounds whose segments
+ * are multiples of 256 tokens: the entries of a whole round are gathered once and one attention launch serves the
+ * round, each pair of 128-query tiles streaming the blocks of 128 entries that hold something its tokens see.
+ * Otherwise: one attention launch per window of about 512 tokens over every entry some token of the window sees.
+ * The call copies a table of a few hundred KB from pageable host memory to the device per round (which pairs of
+ * query tiles each persistent CTA takes) - it enqueues, but is not capturable into a CUDA graph.
  */
 int elm_express_prefill_workspace_bytes(const elm_params *params, int32_t mbar, size_t *bytes);
 int elm_express_prefill(const void *Q, const void *K, const void *V, const elm_params *params, int32_t mbar,
