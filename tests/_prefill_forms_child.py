@@ -9,9 +9,9 @@ import torch
 SHAPES = [
     (6, 4, 3, 64, 2, 4, 2),       # d = 64, two batch entries, level-0 calls of 16 points
     (7, 5, 3, 128, 1, 8, 2),      # grouped queries
-    (8, 2, 3, 128, 1, 4, 4),      # Subsample in round 2 (one token kept of 4)
+    (8, 2, 3, 128, 1, 4, 4),      # Subsample in Express round r = 2 (one token kept of 4)
     (6, 0, 3, 128, 1, 2, 1),      # mbar = 0: no Halve call inside a segment
-    (6, 1, 4, 64, 1, 4, 2),       # strata of 32 tokens in round 3
+    (6, 1, 4, 64, 1, 4, 2),       # strata of 32 tokens in Express round r = 3
     (6, 0, 6, 64, 1, 2, 1),       # strata of 1024 tokens: a pair of query tiles lies inside one stratum
     (7, 3, 4, 128, 2, 2, 2),
 ]

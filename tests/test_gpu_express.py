@@ -109,13 +109,13 @@ PREFILL_CASES = {
     "lowrank_bf16_nout32_R3": (WORKLOADS["cfg3"].scaled(batch=1, q_heads=2, kv_heads=2), 5, 3, 4, 1),
     # tensor-core path with blocks of 128 list entries, grouped queries
     "mixture_t3_bf16_nout256_R2": (WORKLOADS["cfg5"].scaled(q_heads=4, kv_heads=2), 8, 2, 6, 2),
-    # Subsample active in round 2 (m = 4 > mbar = 2: one token kept per 4, a different one in every head)
+    # Subsample active in Express round r = 2 (m = 4 > mbar = 2: one token kept per 4, a different one in every head)
     "iid_f32_nout16_R3_subsample": (WORKLOADS["cfg1"].scaled(q_heads=2, kv_heads=2), 4, 3, 2, 1),
     # mbar = 0: no Halve call inside a segment, strata of 4 and of 16 tokens
     "mixture_f32_nout8_R3_mbar0": (WORKLOADS["cfg2"].scaled(batch=1, q_heads=2, kv_heads=1), 3, 3, 0, 2),
-    # tensor-core path, odd mbar: round 2 keeps one token of every 2 and runs Compress2 of depth 3
+    # tensor-core path, odd mbar: Express round r = 2 keeps one token of every 2 and runs Compress2 of depth 3
     "mixture_t3_bf16_nout128_R3_subsample": (WORKLOADS["cfg5"].scaled(q_heads=4, kv_heads=2), 7, 3, 3, 2),
-    # tensor-core path, level-0 calls of 16 points in round 2 (the paper's proportions: mbar = log2 n_out - 2): most
+    # tensor-core path, level-0 calls of 16 points in Express round r = 2 (the paper's proportions: mbar = log2 n_out - 2): most
     # blocks a pair of query tiles streams hold entries that are born or die among its 256 tokens
     "mixture_t3_bf16_nout64_R3_small_calls": (WORKLOADS["cfg5"].scaled(q_heads=2, kv_heads=1), 6, 3, 4, 2),
     # tensor-core path, mbar = 0: the kept points of a sibling stay in S_0 to the end of its segment (their copy in E
@@ -186,18 +186,18 @@ def test_express_prefill_rejects_level0_calls_below_one_pair():
 # ----------------------------------------------------------------------------------------------
 # name -> (workload, log2_nout, tokens, mbar, q heads per KV head): token counts that stop mid-round
 STREAM_CASES = {
-    # stops in the third segment of round 2 (m = 4): S_1 .. S_3 partly filled
+    # stops in the third segment of Express round r = 2 (m = 4): S_1 .. S_3 partly filled
     "iid_f32_nout16_300": (WORKLOADS["cfg1"].scaled(q_heads=1, kv_heads=1), 4, 300, 4, 1),
-    # stops just before the end of round 2
+    # stops just before the end of Express round r = 2
     "mixture_f32_nout8_500": (WORKLOADS["cfg2"].scaled(batch=1, q_heads=2, kv_heads=2), 3, 500, 4, 1),
-    # grouped queries, stops early in round 2
+    # grouped queries, stops early in Express round r = 2
     "lowrank_bf16_nout32_600_gqa": (WORKLOADS["cfg3"].scaled(batch=1, q_heads=2, kv_heads=1), 5, 600, 4, 2),
     # Subsample active from token 128 on (m = 4 > mbar = 2): every head keeps another token of each stratum of 4 and
     # takes its Halve calls at another token; stops inside a stratum
     "iid_f32_nout8_302_subsample": (WORKLOADS["cfg1"].scaled(q_heads=2, kv_heads=2), 3, 302, 2, 1),
     # mbar = 0: strata of 4, then of 16 tokens, no Halve call inside a segment; stops inside a stratum
     "mixture_f32_nout8_200_mbar0": (WORKLOADS["cfg2"].scaled(batch=1, q_heads=3, kv_heads=3), 3, 200, 0, 1),
-    # bf16 storage, grouped queries, Subsample in round 2
+    # bf16 storage, grouped queries, Subsample in Express round r = 2
     "lowrank_bf16_nout16_601_gqa_subsample": (WORKLOADS["cfg3"].scaled(batch=1, q_heads=2, kv_heads=2), 4, 601, 2, 2),
 }
 
