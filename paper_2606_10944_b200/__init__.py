@@ -7,7 +7,7 @@ CUDA library in ``csrc/``; they are loaded on first use so that the input genera
 _BINDING_NAMES = {
     "compress", "compress_ragged", "compress_ragged_count", "express_compress", "express_prefill", "attend_workspace_bytes", "Stream", "ElmStream", "attend", "compress_status", "attend_status", "attend_static", "attend_static_status", "ATTEND_STATIC_SCRATCH_BYTES", "compress_attend_host", "workspace_bytes", "default_delta_levels",
     "ElmParams", "ElmError", "library_path", "load_library", "make_params", "profile_enable",
-    "profile_read", "version", "EXPORTED_SYMBOLS", "STAGE_NAMES", "launch_count", "host_call_scratch_bytes",
+    "profile_read", "version", "debug_round_check", "EXPORTED_SYMBOLS", "STAGE_NAMES", "launch_count", "host_call_scratch_bytes",
 }
 
 

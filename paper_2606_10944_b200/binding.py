@@ -24,7 +24,7 @@ EXPORTED_SYMBOLS = [
     "elm_express_prefill_workspace_bytes", "elm_express_prefill",
     "elm_stream_workspace_bytes", "elm_stream_init", "elm_stream_step", "elm_stream_steps", "elm_stream_cache",
     "elm_host_call_scratch_bytes", "elm_compress_attend_host",
-    "elm_compress_status", "elm_attend_status", "elm_debug_set", "elm_profile_enable", "elm_profile_read", "elm_launch_count", "elm_strerror", "elm_version",
+    "elm_compress_status", "elm_attend_status", "elm_debug_set", "elm_debug_round_check", "elm_profile_enable", "elm_profile_read", "elm_launch_count", "elm_strerror", "elm_version",
 ]
 
 
@@ -94,6 +94,9 @@ def load_library():
     lib.elm_compress_status.argtypes = [vp, pp, ctypes.POINTER(ctypes.c_int32), vp]
     lib.elm_attend_status.argtypes = [vp, pp, ctypes.c_int32, ctypes.POINTER(ctypes.c_int32), vp]
     lib.elm_debug_set.argtypes = [ctypes.c_int32, ctypes.c_int64]
+    lib.elm_debug_round_check.argtypes = [ctypes.POINTER(ElmParams), ctypes.c_int32, ctypes.c_int32, ctypes.c_uint64,
+                                          ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_int64),
+                                          ctypes.POINTER(ctypes.c_int64)]
     lib.elm_profile_enable.argtypes = [ctypes.c_int]
     lib.elm_profile_read.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int64), ctypes.c_int32]
     lib.elm_launch_count.argtypes = []
@@ -427,6 +430,19 @@ def attend_status(workspace, params: ElmParams, n_core: int) -> int:
     _check(load_library().elm_attend_status(workspace.data_ptr(), ctypes.byref(params), n_core, ctypes.byref(out),
                                             _stream()), "elm_attend_status")
     return int(out.value)
+
+
+def debug_round_check(B, Hq, Hkv, n, d, log2_nout, mbar, r, seed=1, dtype_code=None, precision="fp32"):
+    """elm_debug_round_check (host only): (missing, listed_blocks, needed_blocks) for Express round r of a prefill, or
+    None when that round does not take the one-launch form."""
+    lib = load_library()
+    p, _ = make_params(B, Hq, Hkv, n, n, d, log2_nout, 0, ELM_BF16 if dtype_code is None else dtype_code, precision)
+    out = [ctypes.c_int64(0) for _ in range(3)]
+    rc = lib.elm_debug_round_check(ctypes.byref(p), mbar, r, seed, *[ctypes.byref(o) for o in out])
+    if rc == -2:                     # ELM_ERR_SHAPE: the round is taken in windows
+        return None
+    _check(rc, "elm_debug_round_check")
+    return tuple(int(o.value) for o in out)
 
 
 def profile_enable(on=True):

@@ -23,16 +23,10 @@
 namespace elm {
 namespace {
 
-constexpr int32_t NEVER = 0x7fffffff;
+constexpr int32_t NEVER = ROUND_NEVER;
 
-// One thread per universe entry: row number, weight, first token that sees it (birth) and first that does
-// not any more (death); per block of 128 entries the largest birth and the smallest death.  With G = the
-// number of a sibling's kept points that have arrived - G = X is reached right after the X-th kept point, at
-// token kept[X - 1] + 1:
-//   E                       always;  the output of sibling j: from G_j = len0 on (q = 0: from the end of its segment)
-//   S_i entry of call c     from G = (c + 1) A until G = (c / 4 + 1) 4 A          (A = s0 4^(i-1))
-//   S_0 entry g             from its own token (which sees itself) until G = (g / s0 + 1) s0   (q = 0: for good)
-// Padding entries are never seen.
+// One thread per universe entry (universe_entry in the header): row number, weight, lifetime; per block of 128
+// entries the largest birth and the smallest death.
 __global__ void __launch_bounds__(256) round_universe_kernel(RoundUniverse u, const int32_t *__restrict__ E,
                                                              const int32_t *__restrict__ levels, int64_t level_stride,
                                                              const int32_t *__restrict__ kept_all, int64_t stride,
@@ -47,34 +41,13 @@ __global__ void __launch_bounds__(256) round_universe_kernel(RoundUniverse u, co
     float wt = 1.f;
     if (pos < u.n_univ) {
         const int32_t *kept = kept_all + pr * stride;
-        auto token_after = [&](int64_t jj, int64_t X) { return X > u.len0 ? NEVER : kept[jj * u.len0 + X - 1] + 1; };
-        if (pos < u.EP) {
-            if (pos < 4 * u.n_out) {
-                const int64_t part = pos / u.n_out;
-                row = E[pr * stride + pos];
-                // (q = 0: no Halve call - the sibling's kept points stay in S_0 to the end of its segment and only
-                // then join E, so their copy in E must not be seen before the next sibling begins)
-                bt = part == 0 ? 0 : (u.q >= 1 ? token_after(part - 1, u.len0) : (int32_t)((part + 1) * u.seg));
-            }
-        } else {
-            const int64_t jj = (pos - u.EP) / u.SP;
-            int64_t o = (pos - u.EP) % u.SP;
-            int i = 0;
-            while (o >= round_pad128(u.len0 >> i)) { o -= round_pad128(u.len0 >> i); ++i; }
-            if (o < (u.len0 >> i)) {
-                wt = ldexpf(1.f, i - u.q);
-                if (i == 0) {
-                    row = kept[jj * u.len0 + o];
-                    bt = row;
-                    if (u.q >= 1) dt = token_after(jj, (o / u.s0 + 1) * u.s0);
-                } else {
-                    const int64_t A = u.s0 << (2 * (i - 1)), unit = (u.s0 << (i - 1)) >> 1, c = o / unit;
-                    row = levels[(int64_t)(i - 1) * level_stride + pr * stride + jj * (u.len0 >> i) + o];
-                    bt = token_after(jj, (c + 1) * A);
-                    dt = token_after(jj, (c / 4 + 1) * 4 * A);
-                }
-            }
-        }
+        const UniverseEntry e = universe_entry(u, pos, KeptArray{kept, u.len0});
+        bt = e.birth;
+        dt = e.death;
+        wt = e.w;
+        if (e.piece == -1) row = E[pr * stride + e.off];
+        else if (e.piece == 0) row = kept[e.jj * u.len0 + e.off];
+        else if (e.piece > 0) row = levels[(int64_t)(e.piece - 1) * level_stride + pr * stride + e.jj * (u.len0 >> e.piece) + e.off];
         idx[pr * u.n_univ + pos] = row;
         w[pr * u.n_univ + pos] = wt;
         birth[pr * u.n_univ + pos] = bt;
@@ -300,3 +273,51 @@ int express_attend_round(const void *Q, const void *K, const void *V, void *O, c
 }
 
 }  // namespace elm
+
+// Host-only consistency check of the one-launch form's two descriptions of a round (test hook, no CUDA call): the
+// lifetimes say which tokens see an entry, the block lists say which blocks a pair of query tiles streams - every
+// entry that some token of a pair sees must lie in a block of the pair's list.  Kept points: the segment's own
+// tokens, or (rounds with Subsample) one pseudo-random token per stratum drawn from `seed`.
+extern "C" int elm_debug_round_check(const elm_params *params, int32_t mbar, int32_t r, uint64_t seed, int64_t *missing,
+                                     int64_t *listed_blocks, int64_t *needed_blocks)
+{
+    using namespace elm;
+    if (!params || !missing || !listed_blocks || !needed_blocks) return ELM_ERR_NULL;
+    RoundUniverse u;
+    if (!round_universe(params, mbar, r, u)) return ELM_ERR_SHAPE;
+    std::vector<int32_t> kept((size_t)3 * u.len0);
+    uint64_t state = seed * 6364136223846793005ull + 1442695040888963407ull;
+    for (int64_t jj = 0; jj < 3; ++jj)
+        for (int64_t g = 0; g < u.len0; ++g) {
+            state = state * 6364136223846793005ull + 1442695040888963407ull;
+            const int64_t within = u.wlog ? (int64_t)((state >> 33) % ((uint64_t)1 << u.wlog)) : 0;
+            kept[(size_t)(jj * u.len0 + g)] = (int32_t)((jj + 1) * u.seg + (g << u.wlog) + within);
+        }
+    const KeptArray kept_of = {kept.data(), u.len0};
+    std::vector<UniverseEntry> entries((size_t)u.n_univ);
+    for (int64_t pos = 0; pos < u.n_univ; ++pos) entries[(size_t)pos] = universe_entry(u, pos, kept_of);
+    *missing = *listed_blocks = *needed_blocks = 0;
+    std::vector<int32_t> list((size_t)u.cap);
+    std::vector<char> in_list((size_t)(u.n_univ / 128)), needed((size_t)(u.n_univ / 128));
+    for (int tl = 0; tl < u.tiles; ++tl) {
+        const int cnt = tile_blocks(u, tl, list.data());
+        if (cnt > u.cap) return ELM_ERR_WORKSPACE;
+        std::fill(in_list.begin(), in_list.end(), 0);
+        std::fill(needed.begin(), needed.end(), 0);
+        for (int j = 0; j < cnt; ++j) {
+            if (list[(size_t)j] < 0 || list[(size_t)j] >= u.n_univ / 128 || in_list[(size_t)list[(size_t)j]]) return ELM_ERR_SHAPE;   // out of range or twice
+            in_list[(size_t)list[(size_t)j]] = 1;
+        }
+        const int64_t T0 = u.seg + (int64_t)tl * 256, T1 = T0 + 256;       // the pair's tokens
+        for (int64_t pos = 0; pos < u.n_univ; ++pos) {
+            const UniverseEntry &e = entries[(size_t)pos];
+            if (e.birth < e.death && e.birth < T1 && e.death > T0) {
+                needed[(size_t)(pos / 128)] = 1;
+                if (!in_list[(size_t)(pos / 128)]) ++*missing;
+            }
+        }
+        *listed_blocks += cnt;
+        for (size_t b = 0; b < needed.size(); ++b) *needed_blocks += needed[b];
+    }
+    return ELM_OK;
+}

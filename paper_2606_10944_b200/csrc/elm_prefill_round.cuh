@@ -81,13 +81,74 @@ __host__ __device__ inline int tile_blocks(const RoundUniverse &u, int tl, int32
     const int64_t base = u.EP + jj * u.SP;
     for (int i = u.q - 1; i >= 1; --i) {
         const int64_t A = u.s0 << (2 * (i - 1)), unit = (u.s0 << (i - 1)) >> 1;
-        const int64_t c_lo = 4 * (G0 / (4 * A)), c_end = G1 / A;
+        // call c's output is born when G reaches (c + 1) A, right after that kept point: without Subsample the
+        // G1-th kept point is the pair's last token, so what is born there belongs to the next pair
+        const int64_t c_lo = 4 * (G0 / (4 * A)), c_end = (u.sub ? G1 : G1 - 1) / A;
         const int64_t b0 = base + round_piece_off(u, i);
         run(b0 + c_lo * unit, b0 + c_end * unit);
     }
     const int64_t g_lo = u.q >= 1 ? (G0 / u.s0) * u.s0 : 0;
     run(base + g_lo, base + G1);
     return n;
+}
+
+// Entry `pos` of the universe: which row of K / V it is (through `row_of`), its weight, the first token that sees it
+// (birth) and the first that does not any more (death).  With G = the number of a sibling's kept points that have
+// arrived - G = X is reached right after the X-th kept point, at token kept(jj, X - 1) + 1:
+//   E                       always;  the output of sibling j: from G_j = len0 on (q = 0: from the end of its segment)
+//   S_i entry of call c     from G = (c + 1) A until G = (c / 4 + 1) 4 A          (A = s0 4^(i-1))
+//   S_0 entry g             from its own token (which sees itself) until G = (g / s0 + 1) s0   (q = 0: until the
+//                           sibling's segment ends)
+// Padding entries are never seen.  `kept(jj, g)` is the token of kept point g of sibling jj; piece = -1 for E,
+// -2 for padding, else the level i, with `off` the entry's index within the sibling's piece (within E for piece -1).
+constexpr int32_t ROUND_NEVER = 0x7fffffff;
+// kept(jj, g) over an array that holds the three siblings' kept points one after the other
+struct KeptArray {
+    const int32_t *kept;
+    int64_t len0;
+    __host__ __device__ int32_t operator()(int64_t jj, int64_t g) const { return kept[jj * len0 + g]; }
+};
+struct UniverseEntry {
+    int piece;
+    int64_t jj, off;
+    int32_t birth, death;
+    float w;
+};
+template <class Kept>
+__host__ __device__ inline UniverseEntry universe_entry(const RoundUniverse &u, int64_t pos, Kept kept)
+{
+    UniverseEntry e = {-2, 0, 0, ROUND_NEVER, ROUND_NEVER, 1.f};
+    auto token_after = [&](int64_t jj, int64_t X) { return X > u.len0 ? ROUND_NEVER : (int32_t)(kept(jj, X - 1) + 1); };
+    if (pos < u.EP) {
+        if (pos < 4 * u.n_out) {
+            const int64_t part = pos / u.n_out;
+            e.piece = -1;
+            e.off = pos;
+            // (q = 0: no Halve call - the sibling's kept points stay in S_0 to the end of its segment and only then
+            // join E, so their copy in E must not be seen before the next sibling begins)
+            e.birth = part == 0 ? 0 : (u.q >= 1 ? token_after(part - 1, u.len0) : (int32_t)((part + 1) * u.seg));
+        }
+        return e;
+    }
+    e.jj = (pos - u.EP) / u.SP;
+    int64_t o = (pos - u.EP) % u.SP;
+    int i = 0;
+    while (o >= round_pad128(u.len0 >> i)) { o -= round_pad128(u.len0 >> i); ++i; }
+    if (o >= (u.len0 >> i)) return e;                         // padding behind the piece
+    e.piece = i;
+    e.off = o;
+    e.w = 1.f;
+    for (int k = 0; k < u.q - i; ++k) e.w *= 0.5f;           // 2^(i - q)
+    if (i == 0) {
+        e.birth = (int32_t)kept(e.jj, o);
+        // (q = 0: no Halve call; the points leave S_0 for E when the sibling's segment ends)
+        e.death = u.q >= 1 ? token_after(e.jj, (o / u.s0 + 1) * u.s0) : (int32_t)((e.jj + 2) * u.seg);
+    } else {
+        const int64_t A = u.s0 << (2 * (i - 1)), unit = (u.s0 << (i - 1)) >> 1, c = o / unit;
+        e.birth = token_after(e.jj, (c + 1) * A);
+        e.death = token_after(e.jj, (c / 4 + 1) * 4 * A);
+    }
+    return e;
 }
 
 // Does round r of the prefill take the one-launch form?  (bf16 inputs in fp32 mode - the tensor-core attention
