@@ -20,6 +20,9 @@ namespace elm {
 constexpr int EXPRESS_LANES = 6;       // side streams of the prefill: two per sibling segment
 struct ExpressLayout {
     size_t vmax_bits, cnorm, listA, listB, E, T1, Mpair, rdecay, F, F_stride, total;
+    // the halvings of E run beside the next round's compression, on a stream and with scratch of their own; E itself
+    // alternates between two buffers (round r reads one, its halvings write the other)
+    size_t E2, Mpair2, rdecay2, F2;
     // prefill only: the output lists of every Compress2 level of a round; per side stream the cache list
     // of one launch with its weights and lifetimes and the workspace of elm_attend for that list; log2 of
     // the softmax denominators (rounds with Subsample: the tokens that were not kept are merged in afterwards)
@@ -134,6 +137,10 @@ static ExpressLayout express_layout(const elm_params *p, int mbar = 0, bool pref
     L.rdecay = take(BH * (n / 2 + 1) * ts);
     L.F_stride = 4 * n_out * n_out;        // the first halving of E is one call of 2 n_out pairs
     L.F = take(BH * L.F_stride * ts);
+    L.E2 = take(BH * n * 4);
+    L.Mpair2 = take(BH * (n / 2 + 1) * ts);       // (indexed with the problem stride n / 2, like Mpair)
+    L.rdecay2 = take(BH * (n / 2 + 1) * ts);
+    L.F2 = take(BH * L.F_stride * ts);
     L.levels = L.ep_idx = L.ep_w = L.ep_birth = L.ep_death = L.ep_blk = L.ws_attend = L.ep_cap = L.ep_pad = L.ep_stride = 0;
     L.ws_attend_stride = L.lse = 0;
     L.n_levels = 0;
@@ -381,6 +388,8 @@ static int express_impl(const Tin *K, const Tin *V, const elm_params *p, int mba
     struct SideStreams {                                             // released on every return path
         cudaStream_t s[EXPRESS_LANES] = {};
         cudaEvent_t fork = nullptr, join[EXPRESS_LANES] = {};
+        cudaStream_t halve = nullptr;                                // the halvings of E
+        cudaEvent_t ready[16] = {}, halved[16] = {};                 // per round: E and the siblings' outputs complete; E halved
         ~SideStreams()
         {
             for (int i = 0; i < EXPRESS_LANES; ++i) {
@@ -388,6 +397,11 @@ static int express_impl(const Tin *K, const Tin *V, const elm_params *p, int mba
                 if (join[i]) cudaEventDestroy(join[i]);
             }
             if (fork) cudaEventDestroy(fork);
+            if (halve) cudaStreamDestroy(halve);
+            for (int i = 0; i < 16; ++i) {
+                if (ready[i]) cudaEventDestroy(ready[i]);
+                if (halved[i]) cudaEventDestroy(halved[i]);
+            }
         }
     } sides;
     cudaStream_t *side = sides.s;
@@ -400,6 +414,22 @@ static int express_impl(const Tin *K, const Tin *V, const elm_params *p, int mba
             ELM_CUDA_TRY(cudaEventCreateWithFlags(&join[i], cudaEventDisableTiming));
         }
     }
+    // The two halvings of E that end round r (serial chains that keep at most a few dozen SMs busy) run on a stream of
+    // their own beside the compression of round r + 1's segments, which does not depend on E; E alternates between
+    // two buffers so that round r + 1's segments can deliver their outputs while round r's E is still being read.
+    int32_t *Ebuf[2] = {E, reinterpret_cast<int32_t *>(ws + L.E2)};
+    LevelCtx<Tin, T> ch = c;
+    ch.Mpair = reinterpret_cast<T *>(ws + L.Mpair2);
+    ch.rdecay = reinterpret_cast<T *>(ws + L.rdecay2);
+    ch.F = reinterpret_cast<T *>(ws + L.F2);
+    if (R >= 1) {
+        ELM_CUDA_TRY(cudaStreamCreateWithFlags(&sides.halve, cudaStreamNonBlocking));
+        for (int r = 0; r < R && r < 16; ++r) {
+            ELM_CUDA_TRY(cudaEventCreateWithFlags(&sides.ready[r], cudaEventDisableTiming));
+            ELM_CUDA_TRY(cudaEventCreateWithFlags(&sides.halved[r], cudaEventDisableTiming));
+        }
+    }
+    ch.st = sides.halve;
     if (prefill) {
         // Exact phase and round 0 (thinning factor 1: nothing is dropped): each of the first 4 n_out
         // tokens attends over all tokens up to itself (Theorem 3's exact regime).
@@ -407,6 +437,7 @@ static int express_impl(const Tin *K, const Tin *V, const elm_params *p, int mba
         if (rc != ELM_OK) return rc;
     }
     for (int r = 0; r < R; ++r) {
+        int32_t *const Er = Ebuf[r & 1], *const Enext = Ebuf[(r + 1) & 1];   // this round's E; where its halvings put the next
         const int m = 2 * r, q = m < mbar ? m : mbar;
         const int64_t seg = n_out << m, len0 = n_out << q;
         const double dm = kh_express_delta(p->delta, m);
@@ -422,7 +453,7 @@ static int express_impl(const Tin *K, const Tin *V, const elm_params *p, int mba
         count_launches(1);
         ELM_CUDA_TRY(cudaGetLastError());
         if (q == 0) {
-            copy_list_kernel<<<dim3(blocks(3 * n_out), (unsigned)BH), 256, 0, st>>>(E, n_out, listA, n, 3 * n_out);
+            copy_list_kernel<<<dim3(blocks(3 * n_out), (unsigned)BH), 256, 0, st>>>(Er, n_out, listA, n, 3 * n_out);
             count_launches(1);
             ELM_CUDA_TRY(cudaGetLastError());
         } else {
@@ -434,12 +465,13 @@ static int express_impl(const Tin *K, const Tin *V, const elm_params *p, int mba
                 const int P = (int)((len0 >> i) / per / 2);
                 const double dlt = ldexp(dm, 2 * (i + 1 - q)) / (3.0 * (double)q);
                 if (prefill) nxt = levels + (size_t)i * BH * n;
-                const int rc = run_halve_level<Tin, T>(c, cur, i == q - 1 ? E + n_out : nxt, n, 3 * per, P, i + code1, dlt, per);
+                const int rc = run_halve_level<Tin, T>(c, cur, i == q - 1 ? Er + n_out : nxt, n, 3 * per, P, i + code1, dlt, per);
                 if (rc != ELM_OK) return rc;
                 int32_t *tmp = cur; cur = nxt; nxt = tmp;
             }
         }
         if (prefill && r >= 1) {
+            ELM_CUDA_TRY(cudaStreamWaitEvent(st, sides.halved[r - 1], 0));        // this round's E
             // Thinformer Express (Algorithm 5) for the 3 n_out 2^m tokens of this round.  The cache a token
             // sees is E with the finished siblings (weight 1), in every S_i the outputs of level-(i-1)
             // Halve calls that level i has not consumed yet (weight 2^(i-q)), and in S_0 the kept points
@@ -455,7 +487,7 @@ static int express_impl(const Tin *K, const Tin *V, const elm_params *p, int mba
                 // one launch for the round: every entry the round's tokens ever see is gathered once, each pair of
                 // query tiles streams the blocks its own tokens see
                 const RoundBuffers rb = round_buffers(L, ws, BH, u.n_univ);
-                const int rc = express_attend_round(Q, K, V, O, p, u, E, levels, (size_t)BH * n, listA, n, rb, lse, st);
+                const int rc = express_attend_round(Q, K, V, O, p, u, Er, levels, (size_t)BH * n, listA, n, rb, lse, st);
                 if (rc != ELM_OK) return rc;
             } else {
             const int64_t W = prefill_window(g), Wg = W >> g.wlog;
@@ -466,7 +498,7 @@ static int express_impl(const Tin *K, const Tin *V, const elm_params *p, int mba
                 for (int64_t G0 = 0; G0 < g.len0; G0 += Wg, ++launch) {
                     const int lane_id = launch % EXPRESS_LANES;
                     WindowPieces pc;
-                    window_pieces(g, n_out, jj, G0, G0 + Wg, E, levels, (size_t)BH * n, listA, pc);
+                    window_pieces(g, n_out, jj, G0, G0 + Wg, Er, levels, (size_t)BH * n, listA, pc);
                     const int64_t t0 = (jj + 1) * seg + (G0 << g.wlog);
                     const int rc = express_attend_window(Q, K, V, O, p, L, ws, pc, t0, (int)W, lse, side[lane_id], lane_id);
                     if (rc != ELM_OK) return rc;
@@ -486,14 +518,19 @@ static int express_impl(const Tin *K, const Tin *V, const elm_params *p, int mba
                 ELM_CUDA_TRY(cudaGetLastError());
             }
         }
-        // halve phase: 4 n_out -> 2 n_out -> n_out
+        // halve phase: 4 n_out -> 2 n_out -> n_out, on the halving stream: it starts when this round's E (the
+        // halvings of the round before, same stream) and the three outputs are there and, in the prefill, read
         const bool last_round = r == R - 1;
-        int rc = run_halve_level<Tin, T>(c, E, T1, n, 1, (int)(2 * n_out), (int)(62 + 64 * 4 * r), 0.5 * dm);
+        ELM_CUDA_TRY(cudaEventRecord(sides.ready[r], st));
+        ELM_CUDA_TRY(cudaStreamWaitEvent(sides.halve, sides.ready[r], 0));
+        int rc = run_halve_level<Tin, T>(ch, Er, T1, n, 1, (int)(2 * n_out), (int)(62 + 64 * 4 * r), 0.5 * dm);
         if (rc != ELM_OK) return rc;
-        rc = run_halve_level<Tin, T>(c, T1, last_round ? idx_out : E, last_round ? n_out : n, 1, (int)n_out,
+        rc = run_halve_level<Tin, T>(ch, T1, last_round ? idx_out : Enext, last_round ? n_out : n, 1, (int)n_out,
                                      (int)(63 + 64 * 4 * r), 0.5 * dm);
         if (rc != ELM_OK) return rc;
+        ELM_CUDA_TRY(cudaEventRecord(sides.halved[r], sides.halve));
     }
+    if (R >= 1) ELM_CUDA_TRY(cudaStreamWaitEvent(st, sides.halved[R - 1], 0));
     {
         StageTimer t(ELM_STAGE_EMIT, st, 1);
         const int64_t total = (int64_t)BH * n_out;
