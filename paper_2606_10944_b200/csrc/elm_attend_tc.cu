@@ -55,11 +55,15 @@ constexpr int NTHREADS = 608;          // 16 softmax warps + TMA producer + two 
 constexpr int TMA_WARP = 16, MMA_WARP = 17;
 constexpr uint32_t TMEM_COLS = 512;
 constexpr float RESCALE_TAU = 8.0f;      // rescale the accumulator only if the max grew by > 2^8
-// (Taking a share of the exponentials from the FMA pipe - a cubic for 2^f - instead of the special-function unit
-// was measured on cfg5: none 4.04 ms, 1 pair of 16: 4.06, 2: 4.08, 4: 4.25, 8: 4.35 ... 4.43 - the softmax warps are
-// short of issue slots and latency, not of exp2 throughput, so the kernel does not do it.)
-
-constexpr int EMU_PAIRS = 0;
+// Of every 16 column pairs, how many take 2^x from the FMA pipe (a cubic for 2^f, relative error 1e-4 - below the
+// bf16 rounding of the probabilities) instead of the special-function unit.  Launches with a mask only: there all
+// 16 softmax warps work on one query tile at a time, and a device timeline shows 1350 of a block's 2150 cycles in
+// the pass that exponentiates - 16384 exp2 and 8192 conversions through a unit that does 16 a cycle.  A quarter of
+// the exponentials on the FMA pipe: prefill of cfg5 21.3 -> 20.8 ms, 524288 tokens in the paper's setting
+// 34.7 -> 34.0 ms; half of them: 20.9 and 34.7 ms.  The launches without a mask run their two query tiles out of
+// phase and are short of issue slots and latency instead: none 4.04 ms, 1 pair of 16: 4.06, 2: 4.08, 4: 4.25,
+// 8: 4.35 ... 4.43 - they do not use it.
+constexpr int EMU_PAIRS = 4;
 using namespace sm100;
 
 struct __align__(8) Barriers {
