@@ -372,12 +372,14 @@ int elm_debug_set(int32_t what, int64_t value);
  * round r >= 1 of the run described by (params, mbar) it rebuilds, on the host, the lifetime of every entry of the
  * round's list and the blocks of 128 entries each pair of 128-query tiles streams, with the kept points of
  * subsampled rounds drawn from `seed`, and counts in *missing the (pair, entry) combinations where a token of the
- * pair sees the entry but the entry's block is not in the pair's list (must be 0).  *listed_blocks / *needed_blocks:
- * blocks streamed over all pairs, and how many of them hold an entry the pair sees.  ELM_ERR_SHAPE when the round
- * does not take that form (other storage or precision, segments that are not multiples of 256 tokens).
+ * pair sees the entry but the entry's block is not in the pair's list, plus the entries of blocks listed as "seen
+ * whole by the pair" that some token of the pair does not see (must be 0).  *listed_blocks / *needed_blocks:
+ * blocks streamed over all pairs, and how many of them hold an entry the pair sees; *partly_blocks: how many are
+ * listed as possibly partly visible (the attention kernel looks at lifetimes only there).  ELM_ERR_SHAPE when the
+ * round does not take that form (other storage or precision, segments that are not multiples of 256 tokens).
  */
 int elm_debug_round_check(const elm_params *params, int32_t mbar, int32_t r, uint64_t seed, int64_t *missing,
-                          int64_t *listed_blocks, int64_t *needed_blocks);
+                          int64_t *listed_blocks, int64_t *needed_blocks, int64_t *partly_blocks);
 
 /* Kernels launched by this library since it was loaded (all calls, all stages). */
 int64_t elm_launch_count(void);

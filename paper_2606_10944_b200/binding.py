@@ -96,7 +96,7 @@ def load_library():
     lib.elm_debug_set.argtypes = [ctypes.c_int32, ctypes.c_int64]
     lib.elm_debug_round_check.argtypes = [ctypes.POINTER(ElmParams), ctypes.c_int32, ctypes.c_int32, ctypes.c_uint64,
                                           ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_int64),
-                                          ctypes.POINTER(ctypes.c_int64)]
+                                          ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_int64)]
     lib.elm_profile_enable.argtypes = [ctypes.c_int]
     lib.elm_profile_read.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int64), ctypes.c_int32]
     lib.elm_launch_count.argtypes = []
@@ -433,11 +433,11 @@ def attend_status(workspace, params: ElmParams, n_core: int) -> int:
 
 
 def debug_round_check(B, Hq, Hkv, n, d, log2_nout, mbar, r, seed=1, dtype_code=None, precision="fp32"):
-    """elm_debug_round_check (host only): (missing, listed_blocks, needed_blocks) for Express round r of a prefill, or
+    """elm_debug_round_check (host only): (missing, listed_blocks, needed_blocks, partly_blocks) for Express round r of a prefill, or
     None when that round does not take the one-launch form."""
     lib = load_library()
     p, _ = make_params(B, Hq, Hkv, n, n, d, log2_nout, 0, ELM_BF16 if dtype_code is None else dtype_code, precision)
-    out = [ctypes.c_int64(0) for _ in range(3)]
+    out = [ctypes.c_int64(0) for _ in range(4)]
     rc = lib.elm_debug_round_check(ctypes.byref(p), mbar, r, seed, *[ctypes.byref(o) for o in out])
     if rc == -2:                     # ELM_ERR_SHAPE: the round is taken in windows
         return None

@@ -345,6 +345,9 @@ __device__ __forceinline__ float exp_pass_keep(uint32_t tP, float scale_log2, fl
 // line (it is called once per CTA) so that its code does not weigh on the register allocation and scheduling of
 // the kernel's softmax warps.
 // ---------------------------------------------------------------------------------------------
+// An entry of a block list: the block's number, and bit 30 set unless every row of the pair sees the block whole
+// (then no lifetime is looked at).
+constexpr int BLK_NUMBER = 0x3fffffff, BLK_PARTLY = 1 << 30;
 struct ProducerArgs {
     const CUtensorMap *mapQ, *mapK, *mapV, *mapX;
     unsigned char *smem;
@@ -374,7 +377,7 @@ __device__ __noinline__ bool produce_block_lists(const ProducerArgs *a)
     // between "stage free" and "copy issued" delays the tensor pipe.
     struct Cursor { int k, j, nb, id, prob, blk; bool bias; };
     auto fetch_blk = [&](Cursor &c) {
-        c.blk = c.k < n_items ? (a->tile_blk ? __ldg(a->tile_blk + (int64_t)(c.id % tiles_x) * a->tile_cap + c.j) : c.j) : 0;
+        c.blk = c.k < n_items ? (a->tile_blk ? (__ldg(a->tile_blk + (int64_t)(c.id % tiles_x) * a->tile_cap + c.j) & BLK_NUMBER) : c.j) : 0;
     };
     auto enter = [&](Cursor &c, bool want_bias) {                // the item the cursor has moved to
         c.id = c.k < n_items ? item_id(c.k) : 0;
@@ -504,7 +507,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
     };
     auto item_blk = [&](int k, int j) -> int {
         if constexpr (MASKED) {
-            if (tile_cnt) return __ldg(tile_blk + (int64_t)(item_id(k) % tiles_x) * tile_cap + j);
+            if (tile_cnt) return __ldg(tile_blk + (int64_t)(item_id(k) % tiles_x) * tile_cap + j);      // number | BLK_PARTLY
         }
         return j;
     };
@@ -889,7 +892,11 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
             float m_ref[2] = {-INFINITY, -INFINITY}, l[2] = {0.f, 0.f};
             const int nb = item_nblk(k);
             for (int j = 0; j < nb && ok; ++j, ++G) {
-                const int blk = item_blk(k, j);                     // block of the list (j itself unless the launch has block lists)
+                // block of the list (j itself unless the launch has block lists); a list may say that the pair sees the
+                // block whole - then no lifetime is looked at
+                const int blk_entry = item_blk(k, j);
+                const int blk = MASKED && tile_cnt ? (blk_entry & BLK_NUMBER) : blk_entry;
+                const bool maybe_partly = !(MASKED && tile_cnt) || (blk_entry & BLK_PARTLY) != 0;
 #pragma unroll
                 for (int t = 0; t < 2; ++t) {
                     // A row sees the list up to its own entry of the causal tail (if there is one), so
@@ -900,7 +907,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                     uint32_t vmask = 0xffffffffu;
                     bool special = false;
                     if constexpr (MASKED) {
-                        if (birth) {
+                        if (birth && maybe_partly) {
                             // lifetimes: the block is seen whole by this warp's 32 rows unless an entry is born
                             // after the first or dies before the last of them
                             const int t_first = q_row0 + q0 + t * BM + (warp & 3) * 32;

@@ -276,13 +276,14 @@ int express_attend_round(const void *Q, const void *K, const void *V, void *O, c
 
 // Host-only consistency check of the one-launch form's two descriptions of a round (test hook, no CUDA call): the
 // lifetimes say which tokens see an entry, the block lists say which blocks a pair of query tiles streams - every
-// entry that some token of a pair sees must lie in a block of the pair's list.  Kept points: the segment's own
+// entry that some token of a pair sees must lie in a block of the pair's list, and a block listed as seen whole must
+// hold only entries that every token of the pair sees.  Kept points: the segment's own
 // tokens, or (rounds with Subsample) one pseudo-random token per stratum drawn from `seed`.
 extern "C" int elm_debug_round_check(const elm_params *params, int32_t mbar, int32_t r, uint64_t seed, int64_t *missing,
-                                     int64_t *listed_blocks, int64_t *needed_blocks)
+                                     int64_t *listed_blocks, int64_t *needed_blocks, int64_t *partly_blocks)
 {
     using namespace elm;
-    if (!params || !missing || !listed_blocks || !needed_blocks) return ELM_ERR_NULL;
+    if (!params || !missing || !listed_blocks || !needed_blocks || !partly_blocks) return ELM_ERR_NULL;
     RoundUniverse u;
     if (!round_universe(params, mbar, r, u)) return ELM_ERR_SHAPE;
     std::vector<int32_t> kept((size_t)3 * u.len0);
@@ -296,7 +297,7 @@ extern "C" int elm_debug_round_check(const elm_params *params, int32_t mbar, int
     const KeptArray kept_of = {kept.data(), u.len0};
     std::vector<UniverseEntry> entries((size_t)u.n_univ);
     for (int64_t pos = 0; pos < u.n_univ; ++pos) entries[(size_t)pos] = universe_entry(u, pos, kept_of);
-    *missing = *listed_blocks = *needed_blocks = 0;
+    *missing = *listed_blocks = *needed_blocks = *partly_blocks = 0;
     std::vector<int32_t> list((size_t)u.cap);
     std::vector<char> in_list((size_t)(u.n_univ / 128)), needed((size_t)(u.n_univ / 128));
     for (int tl = 0; tl < u.tiles; ++tl) {
@@ -304,11 +305,21 @@ extern "C" int elm_debug_round_check(const elm_params *params, int32_t mbar, int
         if (cnt > u.cap) return ELM_ERR_WORKSPACE;
         std::fill(in_list.begin(), in_list.end(), 0);
         std::fill(needed.begin(), needed.end(), 0);
-        for (int j = 0; j < cnt; ++j) {
-            if (list[(size_t)j] < 0 || list[(size_t)j] >= u.n_univ / 128 || in_list[(size_t)list[(size_t)j]]) return ELM_ERR_SHAPE;   // out of range or twice
-            in_list[(size_t)list[(size_t)j]] = 1;
-        }
         const int64_t T0 = u.seg + (int64_t)tl * 256, T1 = T0 + 256;       // the pair's tokens
+        for (int j = 0; j < cnt; ++j) {
+            const int32_t b = list[(size_t)j] & ~TILE_BLK_PARTLY;
+            if (b < 0 || b >= u.n_univ / 128 || in_list[(size_t)b]) return ELM_ERR_SHAPE;   // out of range or twice
+            in_list[(size_t)b] = 1;
+            if (!(list[(size_t)j] & TILE_BLK_PARTLY)) {
+                // said to be seen whole: every one of its entries must be seen by every token of the pair
+                for (int64_t pos = (int64_t)b * 128; pos < (int64_t)b * 128 + 128; ++pos) {
+                    const UniverseEntry &e = entries[(size_t)pos];
+                    if (!(e.birth <= T0 && e.death >= T1)) ++*missing;
+                }
+            } else {
+                ++*partly_blocks;
+            }
+        }
         for (int64_t pos = 0; pos < u.n_univ; ++pos) {
             const UniverseEntry &e = entries[(size_t)pos];
             if (e.birth < e.death && e.birth < T1 && e.death > T0) {

@@ -64,20 +64,39 @@ __host__ __device__ inline int64_t round_piece_off(const RoundUniverse &u, int i
 //   of S_i, 1 <= i < q, the outputs of level-(i-1) calls c_lo .. c_end - 1: call c (u entries) exists from
 //   G = (c + 1) A, A = s0 4^(i-1), until the level-i call that consumes it completes at G = (c / 4 + 1) 4 A,
 //   of S_0 the kept points from the start of the running level-0 call up to the pair's last token.
+// A listed block carries TILE_BLK_PARTLY unless all of its 128 entries are seen by every token of the pair, whatever
+// the problem (with Subsample the kept points differ between problems: the test is then conservative) - the
+// attention kernel takes such a block without looking at any lifetime.
+constexpr int32_t TILE_BLK_PARTLY = 1 << 30;
 __host__ __device__ inline int tile_blocks(const RoundUniverse &u, int tl, int32_t *out)
 {
     const int64_t t_all = (int64_t)tl * 256;
     const int64_t jj = t_all / u.seg, t_rel = t_all % u.seg;
     const int64_t G0 = t_rel >> u.wlog, G1 = ((t_rel + 255) >> u.wlog) + 1;
+    // an entry born when G reaches X is seen by the pair's first token iff X <= G0; one that dies when G reaches Y is
+    // seen by the pair's last token iff Y >= G_keep (the G1-th kept point is the last token itself without Subsample,
+    // and may come earlier with it)
+    const int64_t G_keep = u.sub ? G1 + 1 : G1;
     int n = 0;
-    auto run = [&](int64_t a, int64_t b) {
+    // blocks of the universe entries [a, b), which belong to the piece that starts at `base` and has `len` entries;
+    // born(e) / dies(e): the G at which entry e of the piece appears / disappears (dies < 0: never)
+    auto run = [&](int64_t a, int64_t b, int64_t base, int64_t len, auto born, auto dies) {
         if (b <= a) return;
         for (int64_t blk = a / 128; blk <= (b - 1) / 128; ++blk) {
-            if (out) out[n] = (int32_t)blk;
+            const int64_t lo = blk * 128 - base, hi = lo + 127;
+            bool whole = lo >= 0 && hi < len && born(hi) <= G0;
+            if (whole) {
+                const int64_t d = dies(lo);
+                whole = d < 0 || d >= G_keep;
+            }
+            if (out) out[n] = (int32_t)blk | (whole ? 0 : TILE_BLK_PARTLY);
             ++n;
         }
     };
-    run(0, (1 + jj) * u.n_out + ((u.q >= 1 && u.sub && G1 >= u.len0) ? u.n_out : 0));
+    // E and the finished siblings (always there for this sibling's tokens); its own output only behind its last kept point
+    const int64_t e_seen = (1 + jj) * u.n_out;
+    run(0, e_seen + ((u.q >= 1 && u.sub && G1 >= u.len0) ? u.n_out : 0), 0, e_seen,
+        [&](int64_t) { return (int64_t)0; }, [&](int64_t) { return (int64_t)-1; });
     const int64_t base = u.EP + jj * u.SP;
     for (int i = u.q - 1; i >= 1; --i) {
         const int64_t A = u.s0 << (2 * (i - 1)), unit = (u.s0 << (i - 1)) >> 1;
@@ -85,10 +104,13 @@ __host__ __device__ inline int tile_blocks(const RoundUniverse &u, int tl, int32
         // G1-th kept point is the pair's last token, so what is born there belongs to the next pair
         const int64_t c_lo = 4 * (G0 / (4 * A)), c_end = (u.sub ? G1 : G1 - 1) / A;
         const int64_t b0 = base + round_piece_off(u, i);
-        run(b0 + c_lo * unit, b0 + c_end * unit);
+        run(b0 + c_lo * unit, b0 + c_end * unit, b0, u.len0 >> i,
+            [&](int64_t e) { return (e / unit + 1) * A; }, [&](int64_t e) { return (e / unit / 4 + 1) * 4 * A; });
     }
     const int64_t g_lo = u.q >= 1 ? (G0 / u.s0) * u.s0 : 0;
-    run(base + g_lo, base + G1);
+    // kept point g is born at its own token: before the pair iff its stratum lies before the pair's first
+    run(base + g_lo, base + G1, base, u.len0, [&](int64_t e) { return e + 1; },
+        [&](int64_t e) { return u.q >= 1 ? (e / u.s0 + 1) * u.s0 : (int64_t)-1; });
     return n;
 }
 

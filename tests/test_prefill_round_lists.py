@@ -29,12 +29,22 @@ def test_every_visible_entry_lies_in_a_listed_block(log2_nout, mbar, R, d):
             if res is None:                      # segments shorter than a pair of query tiles: taken in windows
                 assert (1 << log2_nout) * 4 ** r % 256 != 0
                 continue
-            missing, listed, needed = res
+            missing, listed, needed, partly = res
             assert missing == 0, (r, seed, res)
             # the lists are tight: at most one block in twenty holds nothing the pair sees
             assert needed <= listed <= needed * 1.05 + 1, (r, seed, res)
+            assert 0 < partly <= listed
             checked += 1
     assert checked >= 2
+
+
+def test_most_blocks_of_cfg5_are_listed_as_seen_whole():
+    """cfg5's prefill (level-0 calls of 512 and 2048 points): only the blocks around a pair's own tokens can be partly
+    visible - the kernel looks at lifetimes for about one block in twenty."""
+    n = 2048 * 4 ** 3
+    for r in (1, 2):
+        missing, listed, needed, partly = elm.debug_round_check(1, 32, 8, n, 128, 11, 9, r)
+        assert missing == 0 and partly <= 0.08 * listed
 
 
 def test_rounds_of_other_storage_or_precision_are_taken_in_windows():
