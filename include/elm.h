@@ -373,7 +373,8 @@ int elm_debug_set(int32_t what, int64_t value);
  * round's list and the blocks of 128 entries each pair of 128-query tiles streams, with the kept points of
  * subsampled rounds drawn from `seed`, and counts in *missing the (pair, entry) combinations where a token of the
  * pair sees the entry but the entry's block is not in the pair's list, plus the entries of blocks listed as "seen
- * whole by the pair" that some token of the pair does not see (must be 0).  *listed_blocks / *needed_blocks:
+ * whole by the pair" that some token of the pair does not see, plus the places where a birth or a death decreases
+ * within a block (must be 0).  *listed_blocks / *needed_blocks:
  * blocks streamed over all pairs, and how many of them hold an entry the pair sees; *partly_blocks: how many are
  * listed as possibly partly visible (the attention kernel looks at lifetimes only there).  ELM_ERR_SHAPE when the
  * round does not take that form (other storage or precision, segments that are not multiples of 256 tokens).

@@ -911,6 +911,30 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                             // lifetimes: the block is seen whole by this warp's 32 rows unless an entry is born
                             // after the first or dies before the last of them
                             const int t_first = q_row0 + q0 + t * BM + (warp & 3) * 32;
+                            // (with block lists, a block that comes here is one the list marks as possibly partly visible:
+                            // its entries are fetched at once rather than behind the block's summaries)
+                            if (tile_cnt) {
+                                // Births and deaths do not decrease along a block of such a list (every piece of the
+                                // round's list is in order of arrival and no block mixes pieces), so a row sees an
+                                // interval of the columns: [entries that died by its token, entries born by it).  Lane c
+                                // fetches entry c of this warp's 32 columns and each lane finds its row's two bounds by
+                                // bisection over the lanes.
+                                const int t_row = t_first + lane;
+                                const int32_t b_mine = __ldg(birth + life0 + (int64_t)blk * BN + lane);
+                                const int32_t d_mine = __ldg(death + life0 + (int64_t)blk * BN + lane);
+                                int hi = 0, lo = 0;
+#pragma unroll
+                                for (int step = 16; step > 0; step >>= 1) {
+                                    if (__shfl_sync(0xffffffffu, b_mine, hi + step - 1) <= t_row) hi += step;
+                                    if (__shfl_sync(0xffffffffu, d_mine, lo + step - 1) <= t_row) lo += step;
+                                }
+                                if (__shfl_sync(0xffffffffu, b_mine, hi) <= t_row) ++hi;          // hi, lo <= 31 here
+                                if (__shfl_sync(0xffffffffu, d_mine, lo) <= t_row) ++lo;
+                                const uint32_t below_hi = hi >= 32 ? 0xffffffffu : (1u << hi) - 1u;
+                                const uint32_t below_lo = lo >= 32 ? 0xffffffffu : (1u << lo) - 1u;
+                                vmask = below_hi & ~below_lo;
+                                special = __any_sync(0xffffffffu, vmask != 0xffffffffu);          // this warp's rows may see it whole
+                            } else {
                             special = !(__ldg(blk_birth + blk0 + blk) <= t_first && __ldg(blk_death + blk0 + blk) > t_first + 31);
                             if (special) {
                                 const int t_row = t_first + lane;
@@ -926,6 +950,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                                     vmask |= (uint32_t)(b4.z <= t_row && t_row < d4.z) << (c + 2);
                                     vmask |= (uint32_t)(b4.w <= t_row && t_row < d4.w) << (c + 3);
                                 }
+                            }
                             }
                         } else if (has_tail) {
                             int valid = n_core - blk * BN - cq * 32;

@@ -298,6 +298,11 @@ extern "C" int elm_debug_round_check(const elm_params *params, int32_t mbar, int
     std::vector<UniverseEntry> entries((size_t)u.n_univ);
     for (int64_t pos = 0; pos < u.n_univ; ++pos) entries[(size_t)pos] = universe_entry(u, pos, kept_of);
     *missing = *listed_blocks = *needed_blocks = *partly_blocks = 0;
+    // (the attention kernel finds a row's visible columns by bisection: births and deaths must not decrease within a block)
+    for (int64_t pos = 1; pos < u.n_univ; ++pos)
+        if (pos % 128 != 0 && (entries[(size_t)pos].birth < entries[(size_t)pos - 1].birth ||
+                               entries[(size_t)pos].death < entries[(size_t)pos - 1].death))
+            ++*missing;
     std::vector<int32_t> list((size_t)u.cap);
     std::vector<char> in_list((size_t)(u.n_univ / 128)), needed((size_t)(u.n_univ / 128));
     for (int tl = 0; tl < u.tiles; ++tl) {
